@@ -1,0 +1,206 @@
+"""CPU oracle for the LoQT quantized low-rank linear layer (arXiv 2405.16528).
+
+TEST INFRASTRUCTURE ONLY.  This file is the slow, plain, obviously-correct
+statement of what the GPU library must compute.  It is imported by the tests,
+by the smoke check and by the benchmark's CPU-baseline leg, and by nothing
+else; the product path never routes through it.  It shares no code, table or
+helper with the CUDA sources: the NF4 level table below is this file's own
+copy.
+
+Everything is numpy.  Floating-point contractions run in float64 (numpy's
+matmul serves as the library primitive); no blocking, fusion or reordering is
+applied beyond what the definitions state.
+
+Conventions (PyTorch nn.Linear style: W is out x in):
+
+    W_q : NF4 codes + one fp32 absmax per block of 64 consecutive elements of
+          a row (Section 5.1 "Neural Network Quantization and NF4")
+    P_q : NF4, out x r        B : r x in (16-bit)        s : scalar (Alg. 1)
+    W_eff = deq(W_q) + s * deq(P_q) @ B          (Section 2, Alg. 1 merge line)
+
+Parity pins (tests/test_oracle_*.py): level table vs. the closed-form quantile
+construction; quantiser vs. pure-Python brute force, exact round trip of the
+16 levels, +-1 at the block maximum, idempotence; bf16 rounding vs. torch's
+conversion; forward/backward vs. the dense W_eff route, torch fp64 autograd and
+central finite differences; merge vs. zero-B identity and the dense product.
+No function here is "parity unpinned".
+"""
+from __future__ import annotations
+
+import numpy as np
+
+BLOCK = 64  # Section 5.1: "blocks of 64 weights"
+
+# NF4 levels q_1..q_16 (ascending).  The paper defers to QLoRA for the values
+# (Section 5.1); these are the 16 fp32 numbers published there: 8 positive and
+# 7 negative equal-probability N(0,1) quantiles plus an exact zero, divided by
+# the largest.  tests/test_oracle_nf4.py rebuilds them from that closed form.
+NF4_LEVELS = np.array(
+    [
+        -1.0,
+        -0.6961928009986877,
+        -0.5250730514526367,
+        -0.39491748809814453,
+        -0.28444138169288635,
+        -0.18477343022823334,
+        -0.09105003625154495,
+        0.0,
+        0.07958029955625534,
+        0.16093020141124725,
+        0.24611230194568634,
+        0.33791524171829224,
+        0.44070982933044434,
+        0.5626170039176941,
+        0.7229568362236023,
+        1.0,
+    ],
+    dtype=np.float32,
+)
+ZERO_CODE = 7  # index of the exact 0.0 level; used for padding and all-zero blocks
+
+
+# ----------------------------------------------------------------------------
+# bf16 helpers (the 16-bit format of B, x, dy and of the dequantised operands)
+# ----------------------------------------------------------------------------
+def bf16_round(a: np.ndarray) -> np.ndarray:
+    """Round fp32 values to the nearest bf16 (ties to even); returns fp32 holding
+    bf16-representable values.  bf16 keeps the top 16 bits of an fp32."""
+    a32 = np.ascontiguousarray(a, dtype=np.float32)
+    u = a32.view(np.uint32).astype(np.uint64)
+    lsb = (u >> np.uint64(16)) & np.uint64(1)
+    r = ((u + np.uint64(0x7FFF) + lsb) >> np.uint64(16)) << np.uint64(16)
+    return (r & np.uint64(0xFFFFFFFF)).astype(np.uint32).view(np.float32).reshape(a32.shape)
+
+
+# ----------------------------------------------------------------------------
+# Storage layout (ABI-visible, not arithmetic): rows padded to a multiple of 64
+# ----------------------------------------------------------------------------
+def padded_cols(cols: int) -> int:
+    return (cols + BLOCK - 1) // BLOCK * BLOCK
+
+
+def pack_codes(codes: np.ndarray) -> np.ndarray:
+    """[rows, ld] codes 0..15 -> [rows, ld/2] bytes; element 2j is the low nibble
+    of byte j, element 2j+1 the high nibble."""
+    c = codes.astype(np.uint8)
+    return (c[:, 0::2] | (c[:, 1::2] << 4)).astype(np.uint8)
+
+
+def unpack_codes(packed: np.ndarray) -> np.ndarray:
+    rows, half = packed.shape
+    out = np.empty((rows, half * 2), dtype=np.uint8)
+    out[:, 0::2] = packed & 0x0F
+    out[:, 1::2] = packed >> 4
+    return out
+
+
+# ----------------------------------------------------------------------------
+# NF4 quantise / dequantise  (Section 5.1, the four displayed equations)
+# ----------------------------------------------------------------------------
+def nf4_quantize(w: np.ndarray):
+    """q_NF4 applied to a 2-D fp32 matrix.
+
+    Blocks are 64 consecutive elements along a row; a row whose length is not a
+    multiple of 64 ends in a short block whose scale is taken over its real
+    elements, and the storage is padded with the zero level.
+
+    Per block: M = max |w| (fp32, exact).  Per element: n = w / M rounded to
+    fp32 (so the block's largest-magnitude element maps to exactly +-1), and
+    the code is argmin_i |n - q_i| over the 16 levels, evaluated in float64,
+    first index on ties.  A block of zeros gets M = 0 and the zero level.
+
+    Returns (codes uint8 [rows, ld] with values 0..15, absmax fp32 [rows, ld/64]).
+    """
+    w = np.asarray(w)
+    assert w.ndim == 2 and w.dtype == np.float32
+    rows, cols = w.shape
+    ld = padded_cols(cols)
+    nb = ld // BLOCK
+    codes = np.full((rows, ld), ZERO_CODE, dtype=np.uint8)
+    absmax = np.zeros((rows, nb), dtype=np.float32)
+    levels64 = NF4_LEVELS.astype(np.float64)
+    for b in range(nb):
+        c0, c1 = b * BLOCK, min((b + 1) * BLOCK, cols)
+        blk = w[:, c0:c1]
+        m = np.max(np.abs(blk), axis=1).astype(np.float32)
+        absmax[:, b] = m
+        nz = m > 0
+        if not np.any(nz):
+            continue
+        with np.errstate(divide="ignore", invalid="ignore"):
+            n = (blk / m[:, None]).astype(np.float32)  # fp32 IEEE division
+        dist = np.abs(n.astype(np.float64)[:, :, None] - levels64[None, None, :])
+        idx = np.argmin(dist, axis=2).astype(np.uint8)  # first occurrence on ties
+        idx[~nz, :] = ZERO_CODE
+        codes[:, c0:c1] = idx
+    return codes, absmax
+
+
+def nf4_dequantize(codes: np.ndarray, absmax: np.ndarray, cols: int | None = None) -> np.ndarray:
+    """q_NF4^{-1}: w = M_beta * q[code], one fp32 multiply.  Returns fp32 [rows, cols]."""
+    rows, ld = codes.shape
+    cols = ld if cols is None else cols
+    m = np.repeat(absmax.astype(np.float32), BLOCK, axis=1)[:, :ld]
+    w = (m * NF4_LEVELS[codes]).astype(np.float32)
+    return w[:, :cols]
+
+
+def nf4_dequantize_bf16(codes, absmax, cols=None) -> np.ndarray:
+    """The 16-bit operand the matrix products see (Section 2.4: W_BF16, P_BF16):
+    the fp32 dequantised value rounded once to bf16."""
+    return bf16_round(nf4_dequantize(codes, absmax, cols))
+
+
+# ----------------------------------------------------------------------------
+# Forward, backward  (Section 2, "Equivalence of Gradient Updates"; Alg. 1)
+# ----------------------------------------------------------------------------
+def _operands(wq, pq, B, out_in_r):
+    out, inn, r = out_in_r
+    W = nf4_dequantize_bf16(wq[0], wq[1], inn).astype(np.float64)  # out x in
+    P = nf4_dequantize_bf16(pq[0], pq[1], r).astype(np.float64)  # out x r
+    Bm = np.asarray(B, dtype=np.float64)
+    assert W.shape == (out, inn) and P.shape == (out, r) and Bm.shape == (r, inn)
+    return W, P, Bm
+
+
+def loqt_forward(wq, pq, B, s, x, shape):
+    """y = x W^T + s (x B^T) P^T with W = deq(W_q), P = deq(P_q); float64, the
+    factored order the method states.  `wq`, `pq` are (codes, absmax) pairs,
+    `shape` = (out, in, r).  x is T x in (bf16-representable values)."""
+    W, P, Bm = _operands(wq, pq, B, shape)
+    x = np.asarray(x, dtype=np.float64)
+    u = x @ Bm.T  # T x r
+    return x @ W.T + float(s) * (u @ P.T)
+
+
+def loqt_backward(wq, pq, B, s, x, dy, shape):
+    """Gradients of L = <y, dy>:  v = dy P;  dx = dy W + s v B;
+    dB = s v^T x  (= s P^T G^W with G^W = dy^T x).  W and P are frozen, so no
+    other gradient exists.  Returns (dx [T, in], dB [r, in]) in float64."""
+    W, P, Bm = _operands(wq, pq, B, shape)
+    x = np.asarray(x, dtype=np.float64)
+    dy = np.asarray(dy, dtype=np.float64)
+    v = dy @ P  # T x r
+    dx = dy @ W + float(s) * (v @ Bm)
+    dB = float(s) * (v.T @ x)
+    return dx, dB
+
+
+# ----------------------------------------------------------------------------
+# Periodic merge + requantise  (Section 2.4; Alg. 1 merge line; Section 2.5)
+# ----------------------------------------------------------------------------
+def loqt_merge_values(wq, pq, B, s, shape) -> np.ndarray:
+    """The fp32 matrix handed to the quantiser at a merge:
+    fl32( deq32(W_q) + s * P_BF16 @ B ), the sum formed in float64 and rounded
+    once.  The quantiser's input is 32-bit (Section 5.1), so W enters with its
+    unrounded fp32 dequantised value; P enters as the 16-bit matmul operand."""
+    out, inn, r = shape
+    W32 = nf4_dequantize(wq[0], wq[1], inn).astype(np.float64)
+    P = nf4_dequantize_bf16(pq[0], pq[1], r).astype(np.float64)
+    delta = P @ np.asarray(B, dtype=np.float64)
+    return (W32 + float(s) * delta).astype(np.float32)
+
+
+def loqt_merge_requant(wq, pq, B, s, shape):
+    """W_q <- q_NF4( deq(W_q) + s deq(P_q) B ).  Returns (codes, absmax)."""
+    return nf4_quantize(loqt_merge_values(wq, pq, B, s, shape))

@@ -1,0 +1,181 @@
+"""Pins for the oracle's forward, backward and merge.
+
+Independent routes: the explicit dense matrix W_eff = W + s P B formed on the
+CPU (Section 2 update rule / Alg. 1 merge line), the identity G^B = P^T G^W
+("Equivalence of Gradient Updates"), torch float64 autograd on the dense layer,
+and central finite differences of L = <y, dy>.
+"""
+import numpy as np
+import pytest
+import torch
+
+from oracle import loqt_oracle as O
+from paper_2405_16528_b200 import synth
+
+
+def _layer(seed, out, inn, r, T, sigma_B=1e-2):
+    d = synth.make_layer(seed, "t", out, inn, r, sigma_B, T)
+    wq = O.nf4_quantize(d["W"].numpy())
+    pq = O.nf4_quantize(d["P"].numpy())
+    f = lambda t: t.to(torch.float32).numpy()
+    return wq, pq, f(d["B"]), f(d["x"]), f(d["dy"])
+
+
+def _dense(wq, pq, B, s, shape):
+    """W_eff built entry by entry from the stored codes; no oracle GEMM code."""
+    out, inn, r = shape
+    lv = O.NF4_LEVELS
+    W = np.zeros((out, inn))
+    P = np.zeros((out, r))
+    bf = lambda v: float(torch.tensor(float(v), dtype=torch.float32).to(torch.bfloat16))
+    for o in range(out):
+        for i in range(inn):
+            W[o, i] = bf(np.float32(wq[1][o, i // 64]) * lv[wq[0][o, i]])
+        for k in range(r):
+            P[o, k] = bf(np.float32(pq[1][o, k // 64]) * lv[pq[0][o, k]])
+    return W, P, W + s * (P @ B.astype(np.float64))
+
+
+SHAPES = [(48, 80, 8, 5), (64, 64, 16, 9), (70, 130, 24, 3)]
+
+
+@pytest.mark.parametrize("shape", SHAPES)
+@pytest.mark.parametrize("s", [1.0, 0.5])
+def test_forward_equals_dense_layer(shape, s):
+    out, inn, r, T = shape
+    wq, pq, B, x, dy = _layer(1, out, inn, r, T)
+    _, _, Weff = _dense(wq, pq, B, s, (out, inn, r))
+    y = O.loqt_forward(wq, pq, B, s, x, (out, inn, r))
+    ref = x.astype(np.float64) @ Weff.T
+    assert np.max(np.abs(y - ref)) <= 1e-12 * np.max(np.abs(ref))
+
+
+@pytest.mark.parametrize("shape", SHAPES)
+@pytest.mark.parametrize("s", [1.0, 0.25])
+def test_backward_dense_route_and_projection_identity(shape, s):
+    out, inn, r, T = shape
+    wq, pq, B, x, dy = _layer(2, out, inn, r, T)
+    W, P, Weff = _dense(wq, pq, B, s, (out, inn, r))
+    dx, dB = O.loqt_backward(wq, pq, B, s, x, dy, (out, inn, r))
+    x64, dy64 = x.astype(np.float64), dy.astype(np.float64)
+    GW = dy64.T @ x64  # out x in, the full-rank gradient
+    assert np.allclose(dx, dy64 @ Weff, rtol=0, atol=1e-11 * np.max(np.abs(dx)))
+    assert np.allclose(dB, s * (P.T @ GW), rtol=0, atol=1e-11 * np.max(np.abs(dB)))
+
+
+def test_backward_matches_torch_autograd():
+    out, inn, r, T, s = 40, 72, 8, 6, 0.5
+    wq, pq, B, x, dy = _layer(3, out, inn, r, T)
+    W, P, _ = _dense(wq, pq, B, s, (out, inn, r))
+    tW, tP = torch.tensor(W), torch.tensor(P)
+    tB = torch.tensor(B, dtype=torch.float64, requires_grad=True)
+    tx = torch.tensor(x, dtype=torch.float64, requires_grad=True)
+    y = torch.nn.functional.linear(tx, tW + s * tP @ tB)
+    (y * torch.tensor(dy, dtype=torch.float64)).sum().backward()
+    dx, dB = O.loqt_backward(wq, pq, B, s, x, dy, (out, inn, r))
+    assert np.allclose(y.detach().numpy(), O.loqt_forward(wq, pq, B, s, x, (out, inn, r)), rtol=1e-11, atol=1e-12)
+    assert np.allclose(dx, tx.grad.numpy(), rtol=1e-10, atol=1e-12)
+    assert np.allclose(dB, tB.grad.numpy(), rtol=1e-10, atol=1e-12)
+
+
+def test_backward_finite_differences():
+    out, inn, r, T, s = 24, 64, 4, 3, 0.5
+    wq, pq, B, x, dy = _layer(4, out, inn, r, T)
+    shape = (out, inn, r)
+    L = lambda B_, x_: float(np.sum(O.loqt_forward(wq, pq, B_, s, x_, shape) * dy))
+    dx, dB = O.loqt_backward(wq, pq, B, s, x, dy, shape)
+    rng = np.random.default_rng(0)
+    B64, x64 = B.astype(np.float64), x.astype(np.float64)
+    h = 1e-4
+    for _ in range(10):
+        k, i = rng.integers(r), rng.integers(inn)
+        Bp, Bm = B64.copy(), B64.copy()
+        Bp[k, i] += h
+        Bm[k, i] -= h
+        assert abs((L(Bp, x64) - L(Bm, x64)) / (2 * h) - dB[k, i]) <= 1e-6 * (1 + abs(dB[k, i]))
+        t, j = rng.integers(T), rng.integers(inn)
+        xp, xm = x64.copy(), x64.copy()
+        xp[t, j] += h
+        xm[t, j] -= h
+        assert abs((L(B64, xp) - L(B64, xm)) / (2 * h) - dx[t, j]) <= 1e-6 * (1 + abs(dx[t, j]))
+
+
+def test_forward_special_cases():
+    out, inn, r, T = 64, 128, 16, 4
+    wq, pq, B, x, dy = _layer(5, out, inn, r, T)
+    shape = (out, inn, r)
+    # B = 0: a plain weight-only-quantised linear
+    y0 = O.loqt_forward(wq, pq, np.zeros_like(B), 1.0, x, shape)
+    W = O.nf4_dequantize_bf16(*wq).astype(np.float64)
+    assert np.allclose(y0, x.astype(np.float64) @ W.T, rtol=1e-13)
+    # W_q = 0: pure low-rank adapter
+    z = (np.full_like(wq[0], 7), np.zeros_like(wq[1]))
+    P = O.nf4_dequantize_bf16(*pq, r).astype(np.float64)
+    y1 = O.loqt_forward(z, pq, B, 0.5, x, shape)
+    assert np.allclose(y1, 0.5 * x.astype(np.float64) @ (P @ B.astype(np.float64)).T, rtol=1e-11, atol=1e-13)
+    # the scale is linear in the adapter term
+    ya = O.loqt_forward(wq, pq, B, 1.0, x, shape)
+    yb = O.loqt_forward(wq, pq, B, 0.5, x, shape)
+    assert np.allclose(ya - y0, 2 * (yb - y0), rtol=1e-9, atol=1e-12)
+
+
+def test_merge_zero_B_is_identity():
+    out, inn, r, T = 64, 192, 16, 2
+    wq, pq, B, x, dy = _layer(6, out, inn, r, T)
+    c, m = O.loqt_merge_requant(wq, pq, np.zeros_like(B), 1.0, (out, inn, r))
+    assert np.array_equal(c, wq[0]) and np.array_equal(m, wq[1])
+
+
+@pytest.mark.parametrize("shape", [(64, 128, 16), (40, 100, 8)])
+def test_merge_equals_quantised_dense_sum(shape):
+    out, inn, r = shape
+    s = 0.5
+    wq, pq, B, x, dy = _layer(7, out, inn, r, 2, sigma_B=3e-2)
+    W, P, _ = _dense(wq, pq, B, s, shape)  # W here is bf16-rounded; rebuild the fp32 one
+    W32 = np.zeros((out, inn))
+    for o in range(out):
+        for i in range(inn):
+            W32[o, i] = float(np.float32(wq[1][o, i // 64]) * O.NF4_LEVELS[wq[0][o, i]])
+    tP = torch.tensor(P, dtype=torch.float64)
+    tB = torch.tensor(B, dtype=torch.float64)
+    vw = (W32 + s * (tP @ tB).numpy()).astype(np.float32)
+    assert np.array_equal(O.loqt_merge_values(wq, pq, B, s, shape), vw)
+    # brute-force quantisation of that matrix, block by block
+    from tests.test_oracle_nf4 import _brute_quantize_block
+
+    c, m = O.loqt_merge_requant(wq, pq, B, s, shape)
+    for o in range(0, out, 7):
+        for b in range(O.padded_cols(inn) // 64):
+            c0, c1 = b * 64, min(b * 64 + 64, inn)
+            bc, bm = _brute_quantize_block(list(vw[o, c0:c1]))
+            assert list(c[o, c0:c1]) == bc and m[o, b] == bm
+
+
+def test_merge_changes_more_codes_for_larger_B():
+    """Section 2.5: small P B leaves the quantised state (almost) unchanged, a
+    larger one moves it."""
+    out, inn, r = 128, 256, 32
+    frac = []
+    for sig in (1e-4, 1e-3, 1e-2, 1e-1):
+        wq, pq, B, _, _ = _layer(8, out, inn, r, 2, sigma_B=sig)
+        c, _ = O.loqt_merge_requant(wq, pq, B, 1.0, (out, inn, r))
+        frac.append(float(np.mean(c != wq[0])))
+    assert frac[0] <= frac[1] <= frac[2] <= frac[3]
+    assert frac[0] < 0.01 and frac[3] > 0.3
+
+
+def test_merged_weight_reproduces_adapter_output():
+    """After a merge, the plain quantised layer approximates the adapted one to
+    within NF4's quantisation error (half the widest level gap times absmax)."""
+    out, inn, r, T, s = 64, 128, 16, 8, 1.0
+    wq, pq, B, x, dy = _layer(9, out, inn, r, T, sigma_B=2e-2)
+    shape = (out, inn, r)
+    vw = O.loqt_merge_values(wq, pq, B, s, shape).astype(np.float64)
+    c, m = O.loqt_merge_requant(wq, pq, B, s, shape)
+    half_gap = float(np.max(np.diff(O.NF4_LEVELS.astype(np.float64)))) / 2
+    err = np.abs(O.nf4_dequantize(c, m).astype(np.float64) - vw)
+    assert np.all(err <= np.repeat(m.astype(np.float64), 64, axis=1)[:, :inn] * half_gap * (1 + 1e-6))
+    y_adapt = O.loqt_forward(wq, pq, B, s, x, shape)
+    y_merged = O.loqt_forward((c, m), pq, np.zeros_like(B), s, x, shape)
+    bound = np.abs(x.astype(np.float64)) @ (np.repeat(m.astype(np.float64), 64, axis=1)[:, :inn] * (half_gap + 2 ** -8)).T
+    assert np.all(np.abs(y_adapt - y_merged) <= bound + 1e-9)
