@@ -1,0 +1,157 @@
+/*
+ * loqt.h - C ABI of the B200 (sm_100a) LoQT quantized low-rank linear layer.
+ *
+ * The layer (LoQT, arXiv 2405.16528, Section 2 and Algorithm 1) is
+ *
+ *     W_eff = deq(W_q) + s * deq(P_q) * B            (out x in)
+ *
+ * with W_q (out x in) and P_q (out x r) frozen and stored in NF4 (Section 5.1:
+ * blocks of 64 weights, one fp32 scale M = max|w| per block, 16 levels), B
+ * (r x in) the only trained matrix, kept in bf16, and s the adapter scale of
+ * Algorithm 1's merge line.
+ *
+ * General rules for every entry point
+ *   - All data pointers are DEVICE pointers owned by the caller; the library
+ *     allocates no device memory and keeps no reference after the call's
+ *     kernels have run.  `stream` is a cudaStream_t passed as void* (NULL =
+ *     default stream).  Work is enqueued asynchronously on that stream.
+ *   - Matrices are row-major with an explicit leading dimension in ELEMENTS.
+ *     bf16 matrices: base 16-byte aligned, leading dimension a multiple of 8.
+ *   - Return value: LOQT_OK or an error code; argument checking is synchronous
+ *     and happens before anything is enqueued.  The library never aborts and
+ *     never falls back to the CPU; on a device that is not sm_100 every compute
+ *     entry point returns LOQT_ERR_ARCH.
+ *   - Workspaces are caller-allocated, 256-byte aligned scratch.  Their first
+ *     256 bytes hold a sticky device status word: zero it once after
+ *     allocation.  Device-side waits are bounded; if one expires the kernel
+ *     sets that word and returns.  Read it with loqt_device_status().
+ */
+#ifndef LOQT_H_
+#define LOQT_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  LOQT_OK = 0,
+  LOQT_ERR_INVALID_ARG = 1, /* null pointer, non-positive size, ld too small      */
+  LOQT_ERR_ALIGNMENT = 2,   /* pointer or leading dimension violates alignment    */
+  LOQT_ERR_UNSUPPORTED = 3, /* block size other than 64                            */
+  LOQT_ERR_WORKSPACE = 4,   /* workspace missing or smaller than required          */
+  LOQT_ERR_CUDA = 5,        /* a CUDA runtime / driver call failed                 */
+  LOQT_ERR_TIMEOUT = 6,     /* a bounded device-side wait expired                  */
+  LOQT_ERR_ARCH = 7         /* current device is not compute capability 10.x       */
+} loqt_status;
+
+/*
+ * View of an NF4 matrix (Section 5.1).  DEVICE pointers, caller-owned.
+ *   codes  : [rows][ld/2] bytes.  Element k of a row lives in byte k/2: low
+ *            nibble when k is even, high nibble when k is odd.  Code c stands
+ *            for the c-th NF4 level in ascending order (0 -> -1, 7 -> 0, 15 -> +1).
+ *   absmax : [rows][ld/64] fp32, the scale M of each block.
+ *   rows, cols : logical shape.   ld : padded row length, ld >= cols,
+ *            ld % 64 == 0.  Blocks are 64 consecutive elements of one row; a
+ *            row whose length is not a multiple of 64 ends in a short block
+ *            whose scale covers its real elements only, and the padding
+ *            elements hold code 7 (the exact zero level).
+ *   block  : must be 64.
+ * codes must be 16-byte aligned, absmax 4-byte aligned.
+ */
+typedef struct {
+  uint8_t *codes;
+  float *absmax;
+  int32_t rows, cols, ld;
+  int32_t block;
+} loqt_nf4_mat;
+
+/* Operation selector for loqt_workspace_bytes(). */
+enum { LOQT_OP_FWD = 0, LOQT_OP_BWD = 1, LOQT_OP_MERGE = 2 };
+
+/*
+ * q_NF4 (Section 5.1, first two displayed equations): per block M = max|w|,
+ * per element code = argmin_i |w / M - q_i| (fp32 division, lower index on a
+ * tie; an all-zero block gets M = 0 and code 7).
+ *   src : fp32 [dst.rows][ld_src] on the device, ld_src >= dst.cols.
+ *   dst : receives codes and absmax, padding included.
+ */
+loqt_status loqt_nf4_quantize(const float *src, int64_t ld_src, loqt_nf4_mat dst, void *stream);
+
+/*
+ * q_NF4^{-1} (Section 5.1, last two displayed equations): w = M * q[code],
+ * one fp32 multiply.  Writes src.rows x src.cols elements to `dst` (row-major,
+ * ld_dst elements per row), as fp32 when dst_is_bf16 == 0, else rounded once
+ * to bf16 (nearest even).
+ */
+loqt_status loqt_nf4_dequantize(loqt_nf4_mat src, void *dst, int64_t ld_dst, int dst_is_bf16,
+                                void *stream);
+
+/*
+ * Forward (Section 2 "Equivalence of Gradient Updates"; Section 2.4 weight-only
+ * quantisation; Algorithm 1 merge line for the scale):
+ *     y = x deq(W_q)^T + s (x B^T) deq(P_q)^T
+ *   Wq : out x in,  Pq : out x r,  B : bf16 [r][ldb] (r x in)
+ *   x  : bf16 [T][ldx] (T x in)    y : bf16 [T][ldy] (T x out), overwritten
+ * Dequantised operands are bf16 (one rounding of M*q); products accumulate in
+ * fp32; the intermediate s*(x B^T) is rounded to bf16.  ws: workspace of at
+ * least loqt_workspace_bytes(LOQT_OP_FWD, ...) bytes.
+ */
+loqt_status loqt_linear_fwd(loqt_nf4_mat Wq, loqt_nf4_mat Pq, const void *B, int64_t ldb, float s,
+                            const void *x, int64_t ldx, int32_t T, void *y, int64_t ldy, void *ws,
+                            size_t ws_bytes, void *stream);
+
+/*
+ * Backward (same section: G^B = P^T G^W, evaluated factored):
+ *     v  = dy deq(P_q)                 (T x r, scratch, kept as bf16 s*v)
+ *     dx = dy deq(W_q) + s v B         (bf16 [T][lddx])
+ *     dB = s v^T x                     (fp32 [r][lddb])
+ * W_q and P_q are frozen: no other gradient is produced.  dB is overwritten,
+ * or added to when accumulate_dB != 0 (gradient accumulation).  The split-K
+ * reduction of dB is done in a fixed order, so results are reproducible.
+ * dx may be NULL to skip the input gradient.
+ */
+loqt_status loqt_linear_bwd(loqt_nf4_mat Wq, loqt_nf4_mat Pq, const void *B, int64_t ldb, float s,
+                            const void *x, int64_t ldx, const void *dy, int64_t lddy, int32_t T,
+                            void *dx, int64_t lddx, float *dB, int64_t lddb, int accumulate_dB,
+                            void *ws, size_t ws_bytes, void *stream);
+
+/*
+ * Periodic merge + requantise (Section 2.4; Algorithm 1 merge line; Section 2.5):
+ *     W_q <- q_NF4( deq(W_q) + s deq(P_q) B )        in place
+ * deq(W_q) enters as the unrounded fp32 product M*q, deq(P_q) as the bf16
+ * operand of the tensor-core product, the sum is formed in fp32.  Each block of
+ * W_q depends only on its own previous contents, so the update is in place.
+ */
+loqt_status loqt_merge_requant(loqt_nf4_mat Wq, loqt_nf4_mat Pq, const void *B, int64_t ldb,
+                               float s, void *ws, size_t ws_bytes, void *stream);
+
+/*
+ * The same merge for n independent matrices in one call (a whole model at a
+ * merge step).  Wq, Pq, B, ldb are HOST arrays of length n; the workspace is
+ * shared and must satisfy the largest matrix.
+ */
+loqt_status loqt_merge_requant_many(int32_t n, const loqt_nf4_mat *Wq, const loqt_nf4_mat *Pq,
+                                    const void *const *B, const int64_t *ldb, float s, void *ws,
+                                    size_t ws_bytes, void *stream);
+
+/* Bytes of workspace `op` needs for the given shape (never less than 256: the
+ * first 256 bytes always hold the device status word). */
+size_t loqt_workspace_bytes(int op, int32_t out, int32_t in, int32_t r, int32_t T);
+
+/* Copies the status word at the start of a workspace back to the host
+ * (synchronises `stream`) and maps it to LOQT_OK / LOQT_ERR_TIMEOUT. */
+loqt_status loqt_device_status(const void *ws, void *stream);
+
+/* Number of kernels this library has launched in this process (all entry
+ * points, all streams); monotone, for instrumentation. */
+uint64_t loqt_launch_count(void);
+
+const char *loqt_status_string(loqt_status st);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LOQT_H_ */

@@ -1,0 +1,213 @@
+"""ctypes binding of libloqt.so: argument marshalling only.
+
+Every function here has the name and the argument order of the C entry point it
+wraps (include/loqt.h); torch supplies device memory and the current stream,
+all arithmetic runs in the library's CUDA kernels.  There is no fallback: if
+the library is missing or a call fails, an exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from dataclasses import dataclass
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libloqt.so")
+
+LOQT_OP_FWD, LOQT_OP_BWD, LOQT_OP_MERGE = 0, 1, 2
+BLOCK = 64
+
+EXPORTS = (
+    "loqt_nf4_quantize", "loqt_nf4_dequantize", "loqt_linear_fwd", "loqt_linear_bwd",
+    "loqt_merge_requant", "loqt_merge_requant_many", "loqt_workspace_bytes",
+    "loqt_device_status", "loqt_launch_count", "loqt_status_string",
+)
+
+
+class LoqtError(RuntimeError):
+    pass
+
+
+class loqt_nf4_mat(ctypes.Structure):
+    _fields_ = [
+        ("codes", ctypes.c_void_p),
+        ("absmax", ctypes.c_void_p),
+        ("rows", ctypes.c_int32),
+        ("cols", ctypes.c_int32),
+        ("ld", ctypes.c_int32),
+        ("block", ctypes.c_int32),
+    ]
+
+
+_lib = None
+
+
+def lib():
+    """Loads libloqt.so (once).  Raises if it has not been built."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise LoqtError(
+            f"{LIB_PATH} is missing: build it with `python -m paper_2405_16528_b200.build`; "
+            "there is no CPU or PyTorch fallback"
+        )
+    L = ctypes.CDLL(LIB_PATH)
+    vp, i64, i32, f32, sz = ctypes.c_void_p, ctypes.c_int64, ctypes.c_int32, ctypes.c_float, ctypes.c_size_t
+    M = loqt_nf4_mat
+    L.loqt_nf4_quantize.argtypes = [vp, i64, M, vp]
+    L.loqt_nf4_dequantize.argtypes = [M, vp, i64, ctypes.c_int, vp]
+    L.loqt_linear_fwd.argtypes = [M, M, vp, i64, f32, vp, i64, i32, vp, i64, vp, sz, vp]
+    L.loqt_linear_bwd.argtypes = [M, M, vp, i64, f32, vp, i64, vp, i64, i32, vp, i64, vp, i64, ctypes.c_int, vp, sz, vp]
+    L.loqt_merge_requant.argtypes = [M, M, vp, i64, f32, vp, sz, vp]
+    L.loqt_merge_requant_many.argtypes = [i32, ctypes.POINTER(M), ctypes.POINTER(M), ctypes.POINTER(vp), ctypes.POINTER(i64), f32, vp, sz, vp]
+    L.loqt_workspace_bytes.argtypes = [ctypes.c_int, i32, i32, i32, i32]
+    L.loqt_workspace_bytes.restype = sz
+    L.loqt_device_status.argtypes = [vp, vp]
+    L.loqt_launch_count.argtypes = []
+    L.loqt_launch_count.restype = ctypes.c_uint64
+    L.loqt_status_string.argtypes = [ctypes.c_int]
+    L.loqt_status_string.restype = ctypes.c_char_p
+    for name in ("loqt_nf4_quantize", "loqt_nf4_dequantize", "loqt_linear_fwd", "loqt_linear_bwd",
+                 "loqt_merge_requant", "loqt_merge_requant_many", "loqt_device_status"):
+        getattr(L, name).restype = ctypes.c_int
+    _lib = L
+    return L
+
+
+def _check(st: int, what: str):
+    if st != 0:
+        raise LoqtError(f"{what} failed: {lib().loqt_status_string(st).decode()} (status {st})")
+
+
+def _stream() -> int:
+    return torch.cuda.current_stream().cuda_stream
+
+
+def _dev(t: torch.Tensor, dtype=None) -> int:
+    if not t.is_cuda:
+        raise LoqtError("the LoQT library works on CUDA tensors only")
+    if dtype is not None and t.dtype != dtype:
+        raise LoqtError(f"expected {dtype}, got {t.dtype}")
+    if t.dim() == 2 and t.stride(1) != 1:
+        raise LoqtError("matrices must be row-major with unit inner stride")
+    return t.data_ptr()
+
+
+@dataclass
+class NF4Tensor:
+    """Device storage of one NF4 matrix in the library's layout."""
+    codes: torch.Tensor   # uint8 [rows, ld/2]
+    absmax: torch.Tensor  # fp32  [rows, ld/64]
+    rows: int
+    cols: int
+
+    @property
+    def ld(self) -> int:
+        return self.codes.shape[1] * 2
+
+    def view(self) -> loqt_nf4_mat:
+        return loqt_nf4_mat(self.codes.data_ptr(), self.absmax.data_ptr(), self.rows, self.cols, self.ld, BLOCK)
+
+    @staticmethod
+    def empty(rows: int, cols: int, device="cuda") -> "NF4Tensor":
+        ld = (cols + BLOCK - 1) // BLOCK * BLOCK
+        return NF4Tensor(
+            torch.empty((rows, ld // 2), dtype=torch.uint8, device=device),
+            torch.empty((rows, ld // BLOCK), dtype=torch.float32, device=device),
+            rows, cols,
+        )
+
+    def clone(self) -> "NF4Tensor":
+        return NF4Tensor(self.codes.clone(), self.absmax.clone(), self.rows, self.cols)
+
+    def nbytes(self) -> int:
+        return self.codes.numel() + 4 * self.absmax.numel()
+
+
+def loqt_workspace_bytes(op: int, out: int, inn: int, r: int, T: int) -> int:
+    return int(lib().loqt_workspace_bytes(op, out, inn, r, T))
+
+
+def new_workspace(nbytes: int, device="cuda") -> torch.Tensor:
+    """Zeroed uint8 workspace (the first word is the sticky device status)."""
+    return torch.zeros((max(int(nbytes), 256),), dtype=torch.uint8, device=device)
+
+
+def loqt_nf4_quantize(src: torch.Tensor, dst: NF4Tensor | None = None) -> NF4Tensor:
+    rows, cols = src.shape
+    dst = dst if dst is not None else NF4Tensor.empty(rows, cols, src.device)
+    _check(lib().loqt_nf4_quantize(_dev(src, torch.float32), src.stride(0), dst.view(), _stream()), "loqt_nf4_quantize")
+    return dst
+
+
+def loqt_nf4_dequantize(src: NF4Tensor, dtype=torch.float32, dst: torch.Tensor | None = None) -> torch.Tensor:
+    if dst is None:
+        dst = torch.empty((src.rows, src.cols), dtype=dtype, device=src.codes.device)
+    is_bf16 = {torch.float32: 0, torch.bfloat16: 1}[dst.dtype]
+    _check(lib().loqt_nf4_dequantize(src.view(), _dev(dst), dst.stride(0), is_bf16, _stream()), "loqt_nf4_dequantize")
+    return dst
+
+
+def loqt_linear_fwd(Wq: NF4Tensor, Pq: NF4Tensor, B: torch.Tensor, s: float, x: torch.Tensor,
+                    y: torch.Tensor | None = None, ws: torch.Tensor | None = None) -> torch.Tensor:
+    T = x.shape[0]
+    if y is None:
+        y = torch.empty((T, Wq.rows), dtype=torch.bfloat16, device=x.device)
+    if ws is None:
+        ws = new_workspace(loqt_workspace_bytes(LOQT_OP_FWD, Wq.rows, Wq.cols, Pq.cols, T), x.device)
+    _check(lib().loqt_linear_fwd(Wq.view(), Pq.view(), _dev(B, torch.bfloat16), B.stride(0), float(s),
+                                 _dev(x, torch.bfloat16), x.stride(0), T, _dev(y, torch.bfloat16), y.stride(0),
+                                 ws.data_ptr(), ws.numel(), _stream()), "loqt_linear_fwd")
+    return y
+
+
+def loqt_linear_bwd(Wq: NF4Tensor, Pq: NF4Tensor, B: torch.Tensor, s: float, x: torch.Tensor, dy: torch.Tensor,
+                    dx: torch.Tensor | None = None, dB: torch.Tensor | None = None, accumulate_dB: bool = False,
+                    ws: torch.Tensor | None = None, need_dx: bool = True):
+    T = x.shape[0]
+    if dx is None and need_dx:
+        dx = torch.empty((T, Wq.cols), dtype=torch.bfloat16, device=x.device)
+    if dB is None:
+        dB = torch.zeros((Pq.cols, Wq.cols), dtype=torch.float32, device=x.device)
+    if ws is None:
+        ws = new_workspace(loqt_workspace_bytes(LOQT_OP_BWD, Wq.rows, Wq.cols, Pq.cols, T), x.device)
+    _check(lib().loqt_linear_bwd(Wq.view(), Pq.view(), _dev(B, torch.bfloat16), B.stride(0), float(s),
+                                 _dev(x, torch.bfloat16), x.stride(0), _dev(dy, torch.bfloat16), dy.stride(0), T,
+                                 _dev(dx, torch.bfloat16) if dx is not None else None,
+                                 dx.stride(0) if dx is not None else 0,
+                                 _dev(dB, torch.float32), dB.stride(0), int(bool(accumulate_dB)),
+                                 ws.data_ptr(), ws.numel(), _stream()), "loqt_linear_bwd")
+    return dx, dB
+
+
+def loqt_merge_requant(Wq: NF4Tensor, Pq: NF4Tensor, B: torch.Tensor, s: float, ws: torch.Tensor | None = None) -> NF4Tensor:
+    if ws is None:
+        ws = new_workspace(loqt_workspace_bytes(LOQT_OP_MERGE, Wq.rows, Wq.cols, Pq.cols, 0), B.device)
+    _check(lib().loqt_merge_requant(Wq.view(), Pq.view(), _dev(B, torch.bfloat16), B.stride(0), float(s),
+                                    ws.data_ptr(), ws.numel(), _stream()), "loqt_merge_requant")
+    return Wq
+
+
+def loqt_merge_requant_many(Wqs, Pqs, Bs, s: float, ws: torch.Tensor | None = None):
+    n = len(Wqs)
+    if ws is None:
+        need = max(loqt_workspace_bytes(LOQT_OP_MERGE, w.rows, w.cols, p.cols, 0) for w, p in zip(Wqs, Pqs))
+        ws = new_workspace(need, Bs[0].device)
+    aW = (loqt_nf4_mat * n)(*[w.view() for w in Wqs])
+    aP = (loqt_nf4_mat * n)(*[p.view() for p in Pqs])
+    aB = (ctypes.c_void_p * n)(*[_dev(b, torch.bfloat16) for b in Bs])
+    aL = (ctypes.c_int64 * n)(*[b.stride(0) for b in Bs])
+    _check(lib().loqt_merge_requant_many(n, aW, aP, aB, aL, float(s), ws.data_ptr(), ws.numel(), _stream()),
+           "loqt_merge_requant_many")
+    return Wqs
+
+
+def loqt_device_status(ws: torch.Tensor) -> None:
+    _check(lib().loqt_device_status(ws.data_ptr(), _stream()), "device status")
+
+
+def loqt_launch_count() -> int:
+    return int(lib().loqt_launch_count())
