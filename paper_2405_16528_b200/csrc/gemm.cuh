@@ -1,0 +1,555 @@
+// Warp-specialised persistent tcgen05 GEMM engine of the LoQT linear layer.
+//
+//   D[M x N] = sum over up to two K-segments of  A_seg[M x K_seg] * B_seg[N x K_seg]^T
+//
+// Each operand of each segment is either a bf16 matrix brought in by TMA (stored
+// K-major or MN-major) or an NF4 matrix (paper Section 5.1) whose 4-bit codes are
+// unpacked and scaled by dedicated warps straight into the 128-byte-swizzled
+// shared-memory layout the tensor core reads, so a dequantised weight never
+// exists in global memory.  Accumulators live in TMEM (two buffers, so the
+// epilogue of one tile overlaps the main loop of the next).
+//
+// Warp roles (448 threads): warp 0 TMA producer, warp 1 MMA issuer + TMEM
+// owner, warps 2-5 epilogue (one per TMEM lane quarter), warps 6-13 NF4
+// dequantisation.  One CTA per SM; tiles are 128 x BN with 64-deep K stages.
+#pragma once
+#include "nf4_dequant.cuh"
+#include "ptx.cuh"
+
+namespace loqt {
+
+constexpr int kBM = 128;      // tile rows (MMA M)
+constexpr int kBK = 64;       // K elements per pipeline stage (one 128-byte swizzle row of bf16)
+constexpr int kUmmaK = 16;    // K of one tcgen05.mma for 16-bit inputs
+constexpr int kStages = 4;
+constexpr int kNumThreads = 448;
+constexpr int kEpiWarp0 = 2;  // warps 2..5
+constexpr int kDeqWarp0 = 6;  // warps 6..13
+constexpr int kDeqWarps = 8;
+constexpr int kDeqThreads = kDeqWarps * 32;
+
+// Operand kinds
+enum : int {
+  OP_TMA_K = 0,   // bf16 [rows][K], K contiguous
+  OP_TMA_MN = 1,  // bf16 [K][rows], rows (M or N index) contiguous
+  OP_NF4_K = 2,   // NF4 [rows][K], blocks run along K
+  OP_NF4_MN = 3,  // NF4 [K][rows], blocks run along the M/N index
+};
+
+// Epilogue kinds
+enum : int {
+  EPI_BF16 = 0,     // out bf16 = alpha * D
+  EPI_F32 = 1,      // out fp32 = (accumulate ? out : 0) + D          (splits == 1)
+  EPI_PARTIAL = 2,  // partial[split] fp32 = D                        (splits > 1)
+  EPI_REQUANT = 3,  // W_q <- q_NF4(deq32(W_q) + alpha * D), in place (merge)
+};
+
+struct Nf4Src {
+  const uint8_t *codes;
+  const float *absmax;
+  int rows, cols, ld;
+};
+
+struct Segment {
+  int K;
+  int a_kind, b_kind;
+  Nf4Src a_nf4, b_nf4;
+};
+
+struct GemmParams {
+  int M, N;
+  int num_segs;
+  Segment seg[2];
+  int splits;       // split-K factor (single-segment GEMMs only)
+  int kb_per_split; // k-blocks per split when splits > 1
+  int epi;
+  void *out;        // bf16 / fp32 output, or split-K partials
+  int64_t ld_out;   // elements
+  float alpha;
+  int accumulate;
+  uint8_t *wq_codes;  // EPI_REQUANT: W_q updated in place ([M][wq_ld/2], [M][wq_ld/64])
+  float *wq_absmax;
+  int wq_ld;
+  uint32_t *status;  // device status word
+  int has_nf4;       // any NF4 operand in any segment
+};
+
+struct TensorMaps {
+  CUtensorMap a[2];
+  CUtensorMap b[2];
+};
+
+template <int BN>
+struct SmemLayout {
+  static constexpr int kABytes = kBM * kBK * 2;  // 16 KiB
+  static constexpr int kBBytes = BN * kBK * 2;
+  static constexpr int kStageBytes = kABytes + kBBytes;
+  static constexpr int kBarOffset = kStages * kStageBytes;
+  // full[kStages], empty[kStages], tfull[2], tempty[2], drain
+  static constexpr int kNumBars = 2 * kStages + 5;
+  static constexpr int kMiscOffset = kBarOffset + kNumBars * 8;
+  static constexpr int kTablesOffset = kMiscOffset + 16;
+  static constexpr int kTotal = kTablesOffset + static_cast<int>(sizeof(Nf4Tables));
+  static constexpr int kDynamicBytes = kTotal + 1024;  // slack for 1024-byte alignment
+};
+
+// Shared-memory matrix descriptor (tcgen05), 128-byte swizzle.
+//   K-major : rows of 128 bytes (64 bf16 of K), 8-row groups 1024 bytes apart.
+//   MN-major: 64-element (128-byte) runs along M/N, 8 K-rows per 1024-byte group,
+//             groups consecutive along K, 64-element column chunks 8192 bytes apart.
+__device__ __forceinline__ uint64_t make_smem_desc(uint32_t saddr, bool mn_major) {
+  const uint64_t start = (saddr & 0x3FFFFu) >> 4;
+  const uint64_t lbo = mn_major ? (8192u >> 4) : 1u;
+  const uint64_t sbo = 1024u >> 4;
+  return start | (lbo << 16) | (sbo << 32) | (1ull << 46) | (2ull << 61);
+}
+
+__device__ __forceinline__ uint32_t make_idesc(int bn, bool a_mn, bool b_mn) {
+  return (1u << 4)                                  // D format fp32
+         | (1u << 7) | (1u << 10)                   // A, B format bf16
+         | (a_mn ? (1u << 15) : 0u) | (b_mn ? (1u << 16) : 0u)
+         | (static_cast<uint32_t>(bn >> 3) << 17)   // N
+         | (static_cast<uint32_t>(kBM >> 4) << 24); // M
+}
+
+// Work decomposition shared by all roles.
+struct Sched {
+  int mt, nt, units;
+  int kb_seg0, kb_total, splits, kb_per_split;
+  __device__ __forceinline__ Sched(const GemmParams &p, int bn) {
+    mt = (p.M + kBM - 1) / kBM;
+    nt = (p.N + bn - 1) / bn;
+    splits = p.splits;
+    kb_per_split = p.kb_per_split;
+    units = mt * nt * splits;
+    kb_seg0 = (p.seg[0].K + kBK - 1) / kBK;
+    kb_total = kb_seg0 + (p.num_segs > 1 ? (p.seg[1].K + kBK - 1) / kBK : 0);
+  }
+  __device__ __forceinline__ void unit(int u, int &m_blk, int &n_blk, int &split, int &kb_lo, int &kb_hi) const {
+    m_blk = u % mt;
+    const int t = u / mt;
+    n_blk = t % nt;
+    split = t / nt;
+    if (splits > 1) {
+      kb_lo = split * kb_per_split;
+      kb_hi = min(kb_lo + kb_per_split, kb_total);
+    } else {
+      kb_lo = 0;
+      kb_hi = kb_total;
+    }
+  }
+};
+
+// One NF4 block (64 codes + scale) fetched ahead of its use.
+struct DeqTask {
+  uint4 c0, c1;
+  float M;
+  int mode;  // 0: nothing to do, 1: dequantise, 2: write zeros
+  uint32_t dst;  // shared-memory byte address of the 128-byte row
+  uint32_t sw;   // row index & 7 (swizzle key)
+};
+
+template <int BN>
+__device__ __forceinline__ DeqTask deq_fetch(const GemmParams &p, int seg_idx, int kb_in_seg, int m_blk, int n_blk,
+                                             uint32_t stage_base, int t) {
+  DeqTask task;
+  task.mode = 0;
+  const Segment &sg = p.seg[seg_idx];
+  const bool a_nf4 = sg.a_kind >= OP_NF4_K;
+  const bool b_nf4 = sg.b_kind >= OP_NF4_K;
+  if (!a_nf4 && !b_nf4) return task;
+  const int kind = a_nf4 ? sg.a_kind : sg.b_kind;
+  const Nf4Src &src = a_nf4 ? sg.a_nf4 : sg.b_nf4;
+  const int rows_tile = a_nf4 ? kBM : BN;
+  if (t >= rows_tile) return task;
+  const uint32_t base = stage_base + (a_nf4 ? 0u : static_cast<uint32_t>(SmemLayout<BN>::kABytes));
+  const int mn0 = a_nf4 ? m_blk * kBM : n_blk * BN;
+  const int k0 = kb_in_seg * kBK;
+  int row, col0, r8;
+  if (kind == OP_NF4_K) {
+    // tile row t <- matrix row mn0 + t, codes k0 .. k0+63
+    row = mn0 + t;
+    col0 = k0;
+    r8 = t & 7;
+    task.dst = base + static_cast<uint32_t>((t >> 3) * 1024 + r8 * 128);
+    if (row >= src.rows) return task;  // feeds only discarded outputs
+  } else {
+    // chunk j = t / 64 of 64 tile columns, K-row kk = t % 64 <- matrix row k0 + kk
+    const int j = t >> 6, kk = t & 63;
+    row = k0 + kk;
+    col0 = mn0 + 64 * j;
+    r8 = kk & 7;
+    task.dst = base + static_cast<uint32_t>(j * 8192 + (kk >> 3) * 1024 + r8 * 128);
+    if (col0 >= src.ld) return task;  // beyond the matrix: discarded outputs
+    if (row >= src.rows) {            // K tail: must contribute zero
+      task.mode = 2;
+      task.sw = static_cast<uint32_t>(r8);
+      return task;
+    }
+  }
+  task.sw = static_cast<uint32_t>(r8);
+  task.mode = 1;
+  const uint4 *cp = reinterpret_cast<const uint4 *>(src.codes + static_cast<int64_t>(row) * (src.ld >> 1) + (col0 >> 1));
+  task.c0 = __ldg(cp);
+  task.c1 = __ldg(cp + 1);
+  task.M = __ldg(src.absmax + static_cast<int64_t>(row) * (src.ld >> 6) + (col0 >> 6));
+  return task;
+}
+
+__device__ __forceinline__ void st_shared_v4(uint32_t addr, uint4 v) {
+  asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w)
+               : "memory");
+}
+
+__device__ __forceinline__ void deq_store(const DeqTask &task) {
+  if (task.mode == 0) return;
+  if (task.mode == 2) {
+#pragma unroll
+    for (uint32_t c = 0; c < 8; ++c) st_shared_v4(task.dst + ((c ^ task.sw) << 4), make_uint4(0, 0, 0, 0));
+    return;
+  }
+  Nf4BlockTable tab;
+  nf4_block_table(task.M, tab);
+  const uint32_t w[8] = {task.c0.x, task.c0.y, task.c0.z, task.c0.w, task.c1.x, task.c1.y, task.c1.z, task.c1.w};
+#pragma unroll
+  for (uint32_t c = 0; c < 8; ++c) st_shared_v4(task.dst + ((c ^ task.sw) << 4), nf4_dequant8(tab, w[c]));
+}
+
+// ---------------------------------------------------------------------------
+// The kernel
+// ---------------------------------------------------------------------------
+template <int BN>
+__global__ void __launch_bounds__(kNumThreads, 1)
+loqt_gemm_kernel(const __grid_constant__ TensorMaps maps, const GemmParams p) {
+  using L = SmemLayout<BN>;
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t *smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
+
+  const uint32_t bar0 = smem_base + L::kBarOffset;
+  auto full_bar = [&](int s) { return bar0 + 8u * s; };
+  auto empty_bar = [&](int s) { return bar0 + 8u * (kStages + s); };
+  auto tfull_bar = [&](int a) { return bar0 + 8u * (2 * kStages + a); };
+  auto tempty_bar = [&](int a) { return bar0 + 8u * (2 * kStages + 2 + a); };
+  const uint32_t drain_bar = bar0 + 8u * (2 * kStages + 4);
+  volatile uint32_t *misc = reinterpret_cast<volatile uint32_t *>(smem_gen + L::kMiscOffset);
+  volatile uint32_t *tmem_slot = misc;       // written by tcgen05.alloc
+  volatile uint32_t *abort_flag = misc + 1;  // raised by any role whose wait expired
+  Nf4Tables &tables = *reinterpret_cast<Nf4Tables *>(smem_gen + L::kTablesOffset);
+
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+  const Sched sched(p, BN);
+  constexpr uint32_t kTmemCols = 2 * BN;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kStages; ++s) {
+      ptx::mbar_init(full_bar(s), 1 + (p.has_nf4 ? kDeqWarps : 0));
+      ptx::mbar_init(empty_bar(s), 1);
+    }
+    for (int a = 0; a < 2; ++a) {
+      ptx::mbar_init(tfull_bar(a), 1);
+      ptx::mbar_init(tempty_bar(a), 4);
+    }
+    ptx::mbar_init(drain_bar, 1);
+    *abort_flag = 0;
+    ptx::fence_barrier_init();
+  }
+  if (p.epi == EPI_REQUANT) nf4_tables_init(tables, threadIdx.x);
+  if (warp == 1) {
+    ptx::tmem_alloc(smem_u32(const_cast<uint32_t *>(tmem_slot)), kTmemCols);
+    ptx::tmem_relinquish();
+  }
+  ptx::tc_fence_before();
+  __syncthreads();
+  ptx::tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  // =========================================================== TMA producer
+  if (warp == 0) {
+    if (lane == 0) {
+      for (int s = 0; s < p.num_segs; ++s) {
+        if (p.seg[s].a_kind <= OP_TMA_MN) ptx::prefetch_tensormap(&maps.a[s]);
+        if (p.seg[s].b_kind <= OP_TMA_MN) ptx::prefetch_tensormap(&maps.b[s]);
+      }
+      uint32_t it = 0;
+      bool ok = true;
+      for (int u = blockIdx.x; ok && u < sched.units; u += gridDim.x) {
+        int m_blk, n_blk, split, kb_lo, kb_hi;
+        sched.unit(u, m_blk, n_blk, split, kb_lo, kb_hi);
+        for (int kb = kb_lo; kb < kb_hi; ++kb, ++it) {
+          const int s = it % kStages;
+          const uint32_t ph = (it / kStages) & 1u;
+          if (!(ok = ptx::mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, p.status))) break;
+          const int sidx = kb < sched.kb_seg0 ? 0 : 1;
+          const int k0 = (sidx == 0 ? kb : kb - sched.kb_seg0) * kBK;
+          const Segment &sg = p.seg[sidx];
+          const uint32_t a_dst = smem_base + s * L::kStageBytes;
+          const uint32_t b_dst = a_dst + L::kABytes;
+          uint32_t bytes = 0;
+          if (sg.a_kind <= OP_TMA_MN) bytes += L::kABytes;
+          if (sg.b_kind <= OP_TMA_MN) bytes += L::kBBytes;
+          ptx::mbar_arrive_expect_tx(full_bar(s), bytes);
+          if (sg.a_kind == OP_TMA_K) {
+            ptx::tma_load_2d(a_dst, &maps.a[sidx], full_bar(s), k0, m_blk * kBM);
+          } else if (sg.a_kind == OP_TMA_MN) {
+#pragma unroll
+            for (int j = 0; j < kBM / 64; ++j)
+              ptx::tma_load_2d(a_dst + j * 8192, &maps.a[sidx], full_bar(s), m_blk * kBM + 64 * j, k0);
+          }
+          if (sg.b_kind == OP_TMA_K) {
+            ptx::tma_load_2d(b_dst, &maps.b[sidx], full_bar(s), k0, n_blk * BN);
+          } else if (sg.b_kind == OP_TMA_MN) {
+#pragma unroll
+            for (int j = 0; j < BN / 64; ++j)
+              ptx::tma_load_2d(b_dst + j * 8192, &maps.b[sidx], full_bar(s), n_blk * BN + 64 * j, k0);
+          }
+        }
+      }
+      if (!ok) {
+        // Give copies already in flight time to land before the CTA's shared
+        // memory is released.
+        const uint64_t t0 = ptx::globaltimer_ns();
+        while (ptx::globaltimer_ns() - t0 < 200000ull) {
+        }
+      }
+    }
+  }
+  // =========================================================== MMA issuer
+  else if (warp == 1) {
+    if (lane == 0) {
+      uint32_t it = 0, tile = 0;
+      bool ok = true;
+      for (int u = blockIdx.x; ok && u < sched.units; u += gridDim.x, ++tile) {
+        int m_blk, n_blk, split, kb_lo, kb_hi;
+        sched.unit(u, m_blk, n_blk, split, kb_lo, kb_hi);
+        const uint32_t acc = tile & 1u;
+        const uint32_t acc_ph = (tile >> 1) & 1u;
+        if (!(ok = ptx::mbar_wait(tempty_bar(acc), acc_ph ^ 1u, abort_flag, p.status))) break;
+        ptx::tc_fence_after();
+        const uint32_t d_tmem = tmem_base + acc * BN;
+        for (int kb = kb_lo; kb < kb_hi; ++kb, ++it) {
+          const int s = it % kStages;
+          const uint32_t ph = (it / kStages) & 1u;
+          if (!(ok = ptx::mbar_wait(full_bar(s), ph, abort_flag, p.status))) break;
+          ptx::tc_fence_after();
+          const Segment &sg = p.seg[kb < sched.kb_seg0 ? 0 : 1];
+          const bool a_mn = (sg.a_kind == OP_TMA_MN);  // NF4_MN is never an A operand
+          const bool b_mn = (sg.b_kind == OP_TMA_MN) || (sg.b_kind == OP_NF4_MN);
+          const uint32_t idesc = make_idesc(BN, a_mn, b_mn);
+          const uint32_t a_addr = smem_base + s * L::kStageBytes;
+          const uint32_t b_addr = a_addr + L::kABytes;
+          const uint64_t a_desc = make_smem_desc(a_addr, a_mn);
+          const uint64_t b_desc = make_smem_desc(b_addr, b_mn);
+          const uint32_t a_step = a_mn ? (2048u >> 4) : (32u >> 4);
+          const uint32_t b_step = b_mn ? (2048u >> 4) : (32u >> 4);
+#pragma unroll
+          for (uint32_t k = 0; k < kBK / kUmmaK; ++k)
+            ptx::mma_bf16_ss(d_tmem, a_desc + k * a_step, b_desc + k * b_step, idesc, (kb > kb_lo || k > 0) ? 1u : 0u);
+          ptx::mma_commit(empty_bar(s));  // stage reusable once these MMAs have read it
+        }
+        if (ok) ptx::mma_commit(tfull_bar(acc));
+      }
+      // Every MMA issued above must have finished before TMEM is freed.
+      ptx::mma_commit(drain_bar);
+      ptx::mbar_wait(drain_bar, 0, abort_flag, p.status);
+    }
+  }
+  // =========================================================== epilogue
+  else if (warp < kDeqWarp0) {
+    const int q = warp & 3;  // TMEM lane quarter this warp may access
+    uint32_t tile = 0;
+    bool ok = true;
+    for (int u = blockIdx.x; ok && u < sched.units; u += gridDim.x, ++tile) {
+      int m_blk, n_blk, split, kb_lo, kb_hi;
+      sched.unit(u, m_blk, n_blk, split, kb_lo, kb_hi);
+      const uint32_t acc = tile & 1u;
+      const uint32_t acc_ph = (tile >> 1) & 1u;
+      if (!(ok = ptx::mbar_wait(tfull_bar(acc), acc_ph, abort_flag, p.status))) break;
+      ptx::tc_fence_after();
+      const int row = m_blk * kBM + q * 32 + lane;
+      const bool row_ok = row < p.M;
+      const uint32_t t_row = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + acc * BN;
+      const int n_base = n_blk * BN;
+
+      if (p.epi == EPI_REQUANT) {
+        // One NF4 block of W_q per 64 accumulator columns of this thread's row.
+#pragma unroll 1
+        for (int jb = 0; jb < BN / 64; ++jb) {
+          uint32_t d0[32], d1[32];
+          ptx::tmem_ld32(t_row + jb * 64, d0);
+          ptx::tmem_ld32(t_row + jb * 64 + 32, d1);
+          ptx::tmem_ld_wait();
+          const int c0 = n_base + jb * 64;
+          if (row_ok && c0 < p.wq_ld) {
+            uint4 *cp = reinterpret_cast<uint4 *>(p.wq_codes + static_cast<int64_t>(row) * (p.wq_ld >> 1) + (c0 >> 1));
+            float *mp = p.wq_absmax + static_cast<int64_t>(row) * (p.wq_ld >> 6) + (c0 >> 6);
+            const uint4 ca = *cp, cb = *(cp + 1);
+            const float Mold = *mp;
+            const uint32_t w[8] = {ca.x, ca.y, ca.z, ca.w, cb.x, cb.y, cb.z, cb.w};
+            float v[64];
+            float Mnew = 0.0f;
+#pragma unroll
+            for (int e = 0; e < 64; ++e) {
+              const float deq = Mold * tables.level[(w[e >> 3] >> (4 * (e & 7))) & 15u];
+              const float delta = __uint_as_float(e < 32 ? d0[e] : d1[e - 32]);
+              v[e] = fmaf(p.alpha, delta, deq);
+              Mnew = fmaxf(Mnew, fabsf(v[e]));
+            }
+            uint32_t o[8];
+#pragma unroll
+            for (int g = 0; g < 8; ++g) {
+              if (Mnew > 0.0f) {
+                const float vv[8] = {v[8 * g], v[8 * g + 1], v[8 * g + 2], v[8 * g + 3],
+                                     v[8 * g + 4], v[8 * g + 5], v[8 * g + 6], v[8 * g + 7]};
+                o[g] = nf4_quantize8(tables, vv, Mnew);
+              } else {
+                o[g] = kZeroWord;
+              }
+            }
+            *cp = make_uint4(o[0], o[1], o[2], o[3]);
+            *(cp + 1) = make_uint4(o[4], o[5], o[6], o[7]);
+            *mp = Mnew;
+          }
+          __syncwarp();
+        }
+      } else {
+#pragma unroll 1
+        for (int cb = 0; cb < BN / 32; ++cb) {
+          uint32_t d[32];
+          ptx::tmem_ld32(t_row + cb * 32, d);
+          ptx::tmem_ld_wait();
+          const int c0 = n_base + cb * 32;
+          const bool full = (c0 + 32 <= p.N);
+          if (!row_ok || c0 >= p.N) {
+            // nothing to store for this thread
+          } else if (p.epi == EPI_BF16) {
+            __nv_bfloat16 *o = reinterpret_cast<__nv_bfloat16 *>(p.out) + static_cast<int64_t>(row) * p.ld_out + c0;
+            if (full && (p.ld_out & 7) == 0) {
+#pragma unroll
+              for (int g = 0; g < 4; ++g) {
+                uint4 qv;
+                qv.x = pack_bf16x2(p.alpha * __uint_as_float(d[8 * g + 0]), p.alpha * __uint_as_float(d[8 * g + 1]));
+                qv.y = pack_bf16x2(p.alpha * __uint_as_float(d[8 * g + 2]), p.alpha * __uint_as_float(d[8 * g + 3]));
+                qv.z = pack_bf16x2(p.alpha * __uint_as_float(d[8 * g + 4]), p.alpha * __uint_as_float(d[8 * g + 5]));
+                qv.w = pack_bf16x2(p.alpha * __uint_as_float(d[8 * g + 6]), p.alpha * __uint_as_float(d[8 * g + 7]));
+                reinterpret_cast<uint4 *>(o)[g] = qv;
+              }
+            } else {
+#pragma unroll
+              for (int e = 0; e < 32; ++e)
+                if (c0 + e < p.N) o[e] = __float2bfloat16_rn(p.alpha * __uint_as_float(d[e]));
+            }
+          } else {
+            float *o;
+            int64_t ldo;
+            bool acc_out = false;
+            if (p.epi == EPI_PARTIAL) {
+              ldo = p.ld_out;
+              o = reinterpret_cast<float *>(p.out) + (static_cast<int64_t>(split) * p.M + row) * ldo + c0;
+            } else {
+              ldo = p.ld_out;
+              o = reinterpret_cast<float *>(p.out) + static_cast<int64_t>(row) * ldo + c0;
+              acc_out = p.accumulate != 0;
+            }
+            if (full && (ldo & 3) == 0) {
+#pragma unroll
+              for (int g = 0; g < 8; ++g) {
+                float4 f = make_float4(__uint_as_float(d[4 * g]), __uint_as_float(d[4 * g + 1]),
+                                       __uint_as_float(d[4 * g + 2]), __uint_as_float(d[4 * g + 3]));
+                if (acc_out) {
+                  const float4 old = reinterpret_cast<float4 *>(o)[g];
+                  f.x += old.x; f.y += old.y; f.z += old.z; f.w += old.w;
+                }
+                reinterpret_cast<float4 *>(o)[g] = f;
+              }
+            } else {
+#pragma unroll
+              for (int e = 0; e < 32; ++e)
+                if (c0 + e < p.N) o[e] = (acc_out ? o[e] : 0.0f) + __uint_as_float(d[e]);
+            }
+          }
+          __syncwarp();
+        }
+      }
+      // Accumulator fully read: hand the TMEM buffer back to the MMA warp.
+      ptx::tc_fence_before();
+      __syncwarp();
+      if (lane == 0) ptx::mbar_arrive(tempty_bar(acc));
+    }
+  }
+  // =========================================================== NF4 dequant
+  else {
+    if (p.has_nf4) {
+      const int t = threadIdx.x - kDeqWarp0 * 32;
+      // Position of the k-block being staged and of the one being fetched ahead.
+      int u = blockIdx.x, kb = 0, kb_hi = 0, m_blk = 0, n_blk = 0, split = 0;
+      bool have = false;
+      auto open_unit = [&]() {
+        while (u < sched.units) {
+          int lo;
+          sched.unit(u, m_blk, n_blk, split, lo, kb_hi);
+          kb = lo;
+          if (kb < kb_hi) return true;
+          u += gridDim.x;
+        }
+        return false;
+      };
+      auto fetch = [&](uint32_t it_) {
+        const int sidx = kb < sched.kb_seg0 ? 0 : 1;
+        const int kb_in = sidx == 0 ? kb : kb - sched.kb_seg0;
+        const uint32_t stage_base = smem_base + (it_ % kStages) * L::kStageBytes;
+        return deq_fetch<BN>(p, sidx, kb_in, m_blk, n_blk, stage_base, t);
+      };
+      uint32_t it = 0;
+      DeqTask next;
+      next.mode = 0;
+      have = open_unit();
+      if (have) next = fetch(0);
+      bool ok = true;
+      while (have && ok) {
+        const DeqTask cur = next;
+        // advance to the following k-block and start its loads
+        ++kb;
+        if (kb >= kb_hi) {
+          u += gridDim.x;
+          have = open_unit();
+        }
+        if (have) next = fetch(it + 1);
+        const int s = it % kStages;
+        const uint32_t ph = (it / kStages) & 1u;
+        if (!(ok = ptx::mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, p.status))) break;
+        deq_store(cur);
+        ptx::fence_proxy_async_smem();
+        __syncwarp();
+        if (lane == 0) ptx::mbar_arrive(full_bar(s));
+        ++it;
+      }
+    }
+  }
+
+  // =========================================================== teardown
+  ptx::tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    ptx::tc_fence_after();
+    ptx::tmem_dealloc(tmem_base, kTmemCols);
+  }
+}
+
+// Deterministic split-K reduction: out = (accumulate ? out : 0) + sum_s partial[s].
+__global__ void __launch_bounds__(256)
+splitk_reduce_kernel(const float *__restrict__ partial, int splits, int M, int N, int64_t ld_partial,
+                     float *__restrict__ out, int64_t ld_out, int accumulate) {
+  const int64_t total = static_cast<int64_t>(M) * N;
+  const int64_t stride = static_cast<int64_t>(gridDim.x) * blockDim.x;
+  for (int64_t i = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x; i < total; i += stride) {
+    const int m = static_cast<int>(i / N);
+    const int n = static_cast<int>(i - static_cast<int64_t>(m) * N);
+    float acc = accumulate ? out[static_cast<int64_t>(m) * ld_out + n] : 0.0f;
+    for (int s = 0; s < splits; ++s) acc += partial[(static_cast<int64_t>(s) * M + m) * ld_partial + n];
+    out[static_cast<int64_t>(m) * ld_out + n] = acc;
+  }
+}
+
+}  // namespace loqt

@@ -1,0 +1,290 @@
+// Host side of the LoQT linear layer: argument checks, TMA descriptors, kernel
+// launches for forward, backward and merge (paper Section 2, Algorithm 1).
+#include <mutex>
+
+#include "gemm.cuh"
+
+namespace loqt {
+
+// ---------------------------------------------------------------------------
+// TMA descriptor construction (driver entry point resolved at run time, so the
+// library does not link against libcuda)
+// ---------------------------------------------------------------------------
+using EncodeTiledFn = CUresult (*)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                   const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  static std::once_flag once;
+  std::call_once(once, [] {
+    void *ptr = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) == cudaSuccess &&
+        qres == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(ptr);
+  });
+  return fn;
+}
+
+// bf16 row-major matrix [outer][inner] with `ld` elements per row; box
+// box_inner x box_outer, 128-byte swizzle, out-of-range elements read as zero.
+static bool make_map(CUtensorMap *map, const void *base, int64_t inner, int64_t outer, int64_t ld, int box_inner,
+                     int box_outer) {
+  EncodeTiledFn fn = encode_fn();
+  if (fn == nullptr) return false;
+  const cuuint64_t dims[2] = {static_cast<cuuint64_t>(inner), static_cast<cuuint64_t>(outer)};
+  const cuuint64_t strides[1] = {static_cast<cuuint64_t>(ld) * 2};
+  const cuuint32_t box[2] = {static_cast<cuuint32_t>(box_inner), static_cast<cuuint32_t>(box_outer)};
+  const cuuint32_t estr[2] = {1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// A bf16 operand of the engine.  K-major: stored [rows][K]; MN-major: stored [K][rows].
+struct Bf16Operand {
+  const void *ptr;
+  int64_t ld;
+};
+
+static bool map_operand(CUtensorMap *map, int kind, const Bf16Operand &op, int rows, int K, int rows_tile) {
+  if (kind == OP_TMA_K) return make_map(map, op.ptr, K, rows, op.ld, kBK, rows_tile);
+  return make_map(map, op.ptr, rows, K, op.ld, 64, kBK);
+}
+
+static Nf4Src nf4_src(const loqt_nf4_mat &m) { return Nf4Src{m.codes, m.absmax, m.rows, m.cols, m.ld}; }
+
+static loqt_status check_bf16(const void *p, int64_t ld, int64_t cols) {
+  if (p == nullptr || ld < cols) return LOQT_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(p) & 15u) != 0 || (ld & 7) != 0) return LOQT_ERR_ALIGNMENT;
+  return LOQT_OK;
+}
+
+// ---------------------------------------------------------------------------
+// One GEMM launch
+// ---------------------------------------------------------------------------
+struct GemmCall {
+  GemmParams p;
+  Bf16Operand a[2], b[2];
+};
+
+template <int BN>
+static loqt_status launch_bn(const GemmCall &c, cudaStream_t stream) {
+  using L = SmemLayout<BN>;
+  TensorMaps maps;
+  memset(&maps, 0, sizeof(maps));
+  for (int s = 0; s < c.p.num_segs; ++s) {
+    const Segment &sg = c.p.seg[s];
+    if (sg.a_kind <= OP_TMA_MN && !map_operand(&maps.a[s], sg.a_kind, c.a[s], c.p.M, sg.K, kBM)) return LOQT_ERR_CUDA;
+    if (sg.b_kind <= OP_TMA_MN && !map_operand(&maps.b[s], sg.b_kind, c.b[s], c.p.N, sg.K, BN)) return LOQT_ERR_CUDA;
+  }
+  if (cudaFuncSetAttribute(loqt_gemm_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kDynamicBytes) !=
+      cudaSuccess)
+    return LOQT_ERR_CUDA;
+  const int mt = (c.p.M + kBM - 1) / kBM, nt = (c.p.N + BN - 1) / BN;
+  const int units = mt * nt * c.p.splits;
+  const int grid = units < sm_count() ? units : sm_count();
+  loqt_gemm_kernel<BN><<<grid, kNumThreads, L::kDynamicBytes, stream>>>(maps, c.p);
+  count_launch();
+  return cudaGetLastError() == cudaSuccess ? LOQT_OK : LOQT_ERR_CUDA;
+}
+
+static loqt_status launch(GemmCall &c, cudaStream_t stream) {
+  c.p.has_nf4 = 0;
+  for (int s = 0; s < c.p.num_segs; ++s)
+    if (c.p.seg[s].a_kind >= OP_NF4_K || c.p.seg[s].b_kind >= OP_NF4_K) c.p.has_nf4 = 1;
+  if (c.p.N > 128) return launch_bn<256>(c, stream);
+  return launch_bn<128>(c, stream);
+}
+
+// ---------------------------------------------------------------------------
+// Workspace layout: [0,256) status word | region 1 | region 2
+// ---------------------------------------------------------------------------
+static size_t align256(size_t v) { return (v + 255) & ~static_cast<size_t>(255); }
+static int64_t ld_lowrank(int r) { return (static_cast<int64_t>(r) + 63) / 64 * 64; }  // bf16 T x r scratch
+
+// Split-K factor of the dB product (M = r, N = in, K = T), for a 148-SM part.
+static void db_splits(int r, int in, int T, int &splits, int &kb_per_split) {
+  const int tiles = ((r + kBM - 1) / kBM) * ((in + (in > 128 ? 255 : 127)) / (in > 128 ? 256 : 128));
+  const int kb_total = (T + kBK - 1) / kBK;
+  int want = 148 / (tiles > 0 ? tiles : 1);
+  if (want < 1) want = 1;
+  if (want > 16) want = 16;
+  const int max_by_k = kb_total / 4 > 0 ? kb_total / 4 : 1;  // at least 4 k-blocks per split
+  if (want > max_by_k) want = max_by_k;
+  kb_per_split = (kb_total + want - 1) / want;
+  splits = (kb_total + kb_per_split - 1) / kb_per_split;
+}
+
+}  // namespace loqt
+
+using namespace loqt;
+
+extern "C" size_t loqt_workspace_bytes(int op, int32_t out, int32_t in, int32_t r, int32_t T) {
+  size_t total = 256;
+  if (op == LOQT_OP_FWD || op == LOQT_OP_BWD) total += align256(static_cast<size_t>(T > 0 ? T : 0) * ld_lowrank(r) * 2);
+  if (op == LOQT_OP_BWD) {
+    int splits = 1, kbps = 1;
+    db_splits(r, in, T > 0 ? T : 1, splits, kbps);
+    if (splits > 1) total += align256(static_cast<size_t>(splits) * r * ((static_cast<size_t>(in) + 3) / 4 * 4) * 4);
+  }
+  (void)out;
+  return total;
+}
+
+static loqt_status check_layer(const loqt_nf4_mat &Wq, const loqt_nf4_mat &Pq, const void *B, int64_t ldb) {
+  loqt_status st;
+  if ((st = validate_nf4(Wq)) != LOQT_OK) return st;
+  if ((st = validate_nf4(Pq)) != LOQT_OK) return st;
+  if (Pq.rows != Wq.rows) return LOQT_ERR_INVALID_ARG;
+  return check_bf16(B, ldb, Wq.cols);
+}
+
+static loqt_status check_ws(const void *ws, size_t ws_bytes, size_t need) {
+  if (ws == nullptr || ws_bytes < need) return LOQT_ERR_WORKSPACE;
+  if ((reinterpret_cast<uintptr_t>(ws) & 255u) != 0) return LOQT_ERR_ALIGNMENT;
+  return LOQT_OK;
+}
+
+extern "C" loqt_status loqt_linear_fwd(loqt_nf4_mat Wq, loqt_nf4_mat Pq, const void *B, int64_t ldb, float s,
+                                       const void *x, int64_t ldx, int32_t T, void *y, int64_t ldy, void *ws,
+                                       size_t ws_bytes, void *stream) {
+  loqt_status st;
+  if ((st = check_layer(Wq, Pq, B, ldb)) != LOQT_OK) return st;
+  if (T <= 0) return LOQT_ERR_INVALID_ARG;
+  const int out = Wq.rows, in = Wq.cols, r = Pq.cols;
+  if ((st = check_bf16(x, ldx, in)) != LOQT_OK) return st;
+  if ((st = check_bf16(y, ldy, out)) != LOQT_OK) return st;
+  if ((st = check_ws(ws, ws_bytes, loqt_workspace_bytes(LOQT_OP_FWD, out, in, r, T))) != LOQT_OK) return st;
+  if ((st = check_arch()) != LOQT_OK) return st;
+  cudaStream_t stm = static_cast<cudaStream_t>(stream);
+  uint32_t *status = static_cast<uint32_t *>(ws);
+  void *u = static_cast<uint8_t *>(ws) + 256;
+  const int64_t ldu = ld_lowrank(r);
+
+  // u = s * x B^T            (T x r; both operands K-major over `in`)
+  GemmCall c1{};
+  c1.p.M = T; c1.p.N = r; c1.p.num_segs = 1;
+  c1.p.seg[0].K = in; c1.p.seg[0].a_kind = OP_TMA_K; c1.p.seg[0].b_kind = OP_TMA_K;
+  c1.a[0] = {x, ldx}; c1.b[0] = {B, ldb};
+  c1.p.splits = 1; c1.p.kb_per_split = 0;
+  c1.p.epi = EPI_BF16; c1.p.out = u; c1.p.ld_out = ldu; c1.p.alpha = s; c1.p.status = status;
+  if ((st = launch(c1, stm)) != LOQT_OK) return st;
+
+  // y = x deq(W_q)^T + u deq(P_q)^T    (K = in, then K = r, one accumulator)
+  GemmCall c2{};
+  c2.p.M = T; c2.p.N = out; c2.p.num_segs = 2;
+  c2.p.seg[0].K = in; c2.p.seg[0].a_kind = OP_TMA_K; c2.p.seg[0].b_kind = OP_NF4_K; c2.p.seg[0].b_nf4 = nf4_src(Wq);
+  c2.p.seg[1].K = r; c2.p.seg[1].a_kind = OP_TMA_K; c2.p.seg[1].b_kind = OP_NF4_K; c2.p.seg[1].b_nf4 = nf4_src(Pq);
+  c2.a[0] = {x, ldx}; c2.a[1] = {u, ldu};
+  c2.p.splits = 1;
+  c2.p.epi = EPI_BF16; c2.p.out = y; c2.p.ld_out = ldy; c2.p.alpha = 1.0f; c2.p.status = status;
+  return launch(c2, stm);
+}
+
+extern "C" loqt_status loqt_linear_bwd(loqt_nf4_mat Wq, loqt_nf4_mat Pq, const void *B, int64_t ldb, float s,
+                                       const void *x, int64_t ldx, const void *dy, int64_t lddy, int32_t T, void *dx,
+                                       int64_t lddx, float *dB, int64_t lddb, int accumulate_dB, void *ws,
+                                       size_t ws_bytes, void *stream) {
+  loqt_status st;
+  if ((st = check_layer(Wq, Pq, B, ldb)) != LOQT_OK) return st;
+  if (T <= 0) return LOQT_ERR_INVALID_ARG;
+  const int out = Wq.rows, in = Wq.cols, r = Pq.cols;
+  if ((st = check_bf16(x, ldx, in)) != LOQT_OK) return st;
+  if ((st = check_bf16(dy, lddy, out)) != LOQT_OK) return st;
+  if (dx != nullptr && (st = check_bf16(dx, lddx, in)) != LOQT_OK) return st;
+  if (dB == nullptr || lddb < in) return LOQT_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(dB) & 15u) != 0) return LOQT_ERR_ALIGNMENT;
+  if ((st = check_ws(ws, ws_bytes, loqt_workspace_bytes(LOQT_OP_BWD, out, in, r, T))) != LOQT_OK) return st;
+  if ((st = check_arch()) != LOQT_OK) return st;
+  cudaStream_t stm = static_cast<cudaStream_t>(stream);
+  uint32_t *status = static_cast<uint32_t *>(ws);
+  const int64_t ldv = ld_lowrank(r);
+  void *v = static_cast<uint8_t *>(ws) + 256;
+  float *partial = reinterpret_cast<float *>(static_cast<uint8_t *>(v) + align256(static_cast<size_t>(T) * ldv * 2));
+
+  // v' = s * dy deq(P_q)      (T x r; K = out; P_q read with its blocks along N = r)
+  GemmCall c1{};
+  c1.p.M = T; c1.p.N = r; c1.p.num_segs = 1;
+  c1.p.seg[0].K = out; c1.p.seg[0].a_kind = OP_TMA_K; c1.p.seg[0].b_kind = OP_NF4_MN; c1.p.seg[0].b_nf4 = nf4_src(Pq);
+  c1.a[0] = {dy, lddy};
+  c1.p.splits = 1;
+  c1.p.epi = EPI_BF16; c1.p.out = v; c1.p.ld_out = ldv; c1.p.alpha = s; c1.p.status = status;
+  if ((st = launch(c1, stm)) != LOQT_OK) return st;
+
+  // dx = dy deq(W_q) + v' B   (T x in; K = out with W_q blocks along N = in, then K = r)
+  if (dx != nullptr) {
+    GemmCall c2{};
+    c2.p.M = T; c2.p.N = in; c2.p.num_segs = 2;
+    c2.p.seg[0].K = out; c2.p.seg[0].a_kind = OP_TMA_K; c2.p.seg[0].b_kind = OP_NF4_MN; c2.p.seg[0].b_nf4 = nf4_src(Wq);
+    c2.p.seg[1].K = r; c2.p.seg[1].a_kind = OP_TMA_K; c2.p.seg[1].b_kind = OP_TMA_MN;
+    c2.a[0] = {dy, lddy}; c2.a[1] = {v, ldv}; c2.b[1] = {B, ldb};
+    c2.p.splits = 1;
+    c2.p.epi = EPI_BF16; c2.p.out = dx; c2.p.ld_out = lddx; c2.p.alpha = 1.0f; c2.p.status = status;
+    if ((st = launch(c2, stm)) != LOQT_OK) return st;
+  }
+
+  // dB = v'^T x               (r x in; K = T; both operands stored K-outermost)
+  GemmCall c3{};
+  c3.p.M = r; c3.p.N = in; c3.p.num_segs = 1;
+  c3.p.seg[0].K = T; c3.p.seg[0].a_kind = OP_TMA_MN; c3.p.seg[0].b_kind = OP_TMA_MN;
+  c3.a[0] = {v, ldv}; c3.b[0] = {x, ldx};
+  int splits = 1, kbps = 1;
+  db_splits(r, in, T, splits, kbps);
+  c3.p.splits = splits; c3.p.kb_per_split = kbps; c3.p.status = status; c3.p.alpha = 1.0f;
+  const int64_t ldp = (static_cast<int64_t>(in) + 3) / 4 * 4;
+  if (splits == 1) {
+    c3.p.epi = EPI_F32; c3.p.out = dB; c3.p.ld_out = lddb; c3.p.accumulate = accumulate_dB;
+  } else {
+    c3.p.epi = EPI_PARTIAL; c3.p.out = partial; c3.p.ld_out = ldp;
+  }
+  if ((st = launch(c3, stm)) != LOQT_OK) return st;
+  if (splits > 1) {
+    const int64_t total = static_cast<int64_t>(r) * in;
+    int64_t blocks = (total + 255) / 256;
+    const int64_t cap = static_cast<int64_t>(sm_count()) * 8;
+    if (blocks > cap) blocks = cap;
+    splitk_reduce_kernel<<<static_cast<int>(blocks), 256, 0, stm>>>(partial, splits, r, in, ldp, dB, lddb, accumulate_dB);
+    count_launch();
+    if (cudaGetLastError() != cudaSuccess) return LOQT_ERR_CUDA;
+  }
+  return LOQT_OK;
+}
+
+static loqt_status merge_one(const loqt_nf4_mat &Wq, const loqt_nf4_mat &Pq, const void *B, int64_t ldb, float s,
+                             uint32_t *status, cudaStream_t stm) {
+  // Delta = deq(P_q) B  (out x in; K = r; P_q blocks along K), requantised in the epilogue.
+  GemmCall c{};
+  c.p.M = Wq.rows; c.p.N = Wq.cols; c.p.num_segs = 1;
+  c.p.seg[0].K = Pq.cols; c.p.seg[0].a_kind = OP_NF4_K; c.p.seg[0].a_nf4 = nf4_src(Pq); c.p.seg[0].b_kind = OP_TMA_MN;
+  c.b[0] = {B, ldb};
+  c.p.splits = 1;
+  c.p.epi = EPI_REQUANT; c.p.alpha = s; c.p.status = status;
+  c.p.wq_codes = Wq.codes; c.p.wq_absmax = Wq.absmax; c.p.wq_ld = Wq.ld;
+  return launch(c, stm);
+}
+
+extern "C" loqt_status loqt_merge_requant(loqt_nf4_mat Wq, loqt_nf4_mat Pq, const void *B, int64_t ldb, float s,
+                                          void *ws, size_t ws_bytes, void *stream) {
+  loqt_status st;
+  if ((st = check_layer(Wq, Pq, B, ldb)) != LOQT_OK) return st;
+  if ((st = check_ws(ws, ws_bytes, 256)) != LOQT_OK) return st;
+  if ((st = check_arch()) != LOQT_OK) return st;
+  return merge_one(Wq, Pq, B, ldb, s, static_cast<uint32_t *>(ws), static_cast<cudaStream_t>(stream));
+}
+
+extern "C" loqt_status loqt_merge_requant_many(int32_t n, const loqt_nf4_mat *Wq, const loqt_nf4_mat *Pq,
+                                               const void *const *B, const int64_t *ldb, float s, void *ws,
+                                               size_t ws_bytes, void *stream) {
+  if (n < 0 || (n > 0 && (Wq == nullptr || Pq == nullptr || B == nullptr || ldb == nullptr))) return LOQT_ERR_INVALID_ARG;
+  loqt_status st;
+  for (int i = 0; i < n; ++i)
+    if ((st = check_layer(Wq[i], Pq[i], B[i], ldb[i])) != LOQT_OK) return st;
+  if ((st = check_ws(ws, ws_bytes, 256)) != LOQT_OK) return st;
+  if ((st = check_arch()) != LOQT_OK) return st;
+  for (int i = 0; i < n; ++i)
+    if ((st = merge_one(Wq[i], Pq[i], B[i], ldb[i], s, static_cast<uint32_t *>(ws), static_cast<cudaStream_t>(stream))) != LOQT_OK)
+      return st;
+  return LOQT_OK;
+}

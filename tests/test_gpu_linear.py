@@ -1,0 +1,126 @@
+"""GPU parity: loqt_linear_fwd / loqt_linear_bwd / loqt_merge_requant against
+the CPU oracle on the same seeded inputs, through the C ABI."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import loqt_oracle as O
+from paper_2405_16528_b200 import binding as L
+from paper_2405_16528_b200 import synth
+from tests.gpu_util import check_close, check_merge, f32, from_dev_nf4, padded, to_dev_nf4
+
+pytestmark = pytest.mark.gpu
+
+# (out, in, r, T): config 0 of the benchmark, then shapes that span several
+# tiles with ragged edges in every dimension (1376 and 5461 are the paper's MLP
+# widths; r = 32 is below one K stage).
+SHAPES = [
+    (256, 256, 32, 512),
+    (384, 320, 64, 200),
+    (512, 1376, 128, 300),
+    (1376, 512, 128, 257),
+    (200, 136, 24, 130),
+    (640, 5461, 96, 140),
+    (5461, 256, 40, 133),
+]
+
+
+def _setup(seed, out, inn, r, T, sigma_B=1e-2):
+    d = synth.make_layer(seed, "g", out, inn, r, sigma_B, T)
+    wq = O.nf4_quantize(d["W"].numpy())
+    pq = O.nf4_quantize(d["P"].numpy())
+    dev = {
+        "Wq": to_dev_nf4(*wq, inn),
+        "Pq": to_dev_nf4(*pq, r),
+        "B": padded(d["B"]),
+        "x": padded(d["x"]),
+        "dy": padded(d["dy"]),
+    }
+    host = {"wq": wq, "pq": pq, "B": f32(d["B"]), "x": f32(d["x"]), "dy": f32(d["dy"])}
+    return host, dev
+
+
+@pytest.mark.parametrize("shape", SHAPES)
+@pytest.mark.parametrize("s", [1.0, 0.5])
+def test_forward(shape, s):
+    out, inn, r, T = shape
+    h, d = _setup(10, out, inn, r, T)
+    ref = O.loqt_forward(h["wq"], h["pq"], h["B"], s, h["x"], (out, inn, r))
+    y = padded(torch.zeros((T, out), dtype=torch.bfloat16))
+    ws = L.new_workspace(L.loqt_workspace_bytes(L.LOQT_OP_FWD, out, inn, r, T))
+    L.loqt_linear_fwd(d["Wq"], d["Pq"], d["B"], s, d["x"], y=y, ws=ws)
+    L.loqt_device_status(ws)
+    check_close(f32(y), ref, f"y {shape}")
+
+
+@pytest.mark.parametrize("shape", SHAPES)
+def test_backward(shape):
+    out, inn, r, T = shape
+    s = 0.5
+    h, d = _setup(11, out, inn, r, T)
+    ref_dx, ref_dB = O.loqt_backward(h["wq"], h["pq"], h["B"], s, h["x"], h["dy"], (out, inn, r))
+    dx = padded(torch.zeros((T, inn), dtype=torch.bfloat16))
+    dB = torch.full((r, inn), 7.0, dtype=torch.float32, device="cuda")
+    ws = L.new_workspace(L.loqt_workspace_bytes(L.LOQT_OP_BWD, out, inn, r, T))
+    L.loqt_linear_bwd(d["Wq"], d["Pq"], d["B"], s, d["x"], d["dy"], dx=dx, dB=dB, ws=ws)
+    L.loqt_device_status(ws)
+    check_close(f32(dx), ref_dx, f"dx {shape}")
+    check_close(f32(dB), ref_dB, f"dB {shape}")
+    # gradient accumulation adds to what is there, and the result is reproducible
+    first = dB.clone()
+    L.loqt_linear_bwd(d["Wq"], d["Pq"], d["B"], s, d["x"], d["dy"], dx=dx, dB=dB, accumulate_dB=True, ws=ws)
+    check_close(f32(dB), 2 * ref_dB, f"dB accumulated {shape}")
+    dB2 = torch.empty_like(dB)
+    L.loqt_linear_bwd(d["Wq"], d["Pq"], d["B"], s, d["x"], d["dy"], dx=None, dB=dB2, ws=ws, need_dx=False)
+    assert torch.equal(dB2, first)
+
+
+@pytest.mark.parametrize("shape", SHAPES)
+@pytest.mark.parametrize("sigma_B", [1e-3, 1e-2])
+def test_merge(shape, sigma_B):
+    out, inn, r, _ = shape
+    s = 1.0
+    h, d = _setup(12, out, inn, r, 8, sigma_B)
+    vw = O.loqt_merge_values(h["wq"], h["pq"], h["B"], s, (out, inn, r))
+    ref_c, ref_m = O.nf4_quantize(vw)
+    L.loqt_merge_requant(d["Wq"], d["Pq"], d["B"], s)
+    got_c, got_m = from_dev_nf4(d["Wq"])
+    check_merge(got_c, got_m, ref_c, ref_m, vw, inn, f"merge {shape}")
+    assert np.all(got_c[:, inn:] == 7)
+
+
+def test_merge_zero_B_leaves_weights_untouched():
+    out, inn, r = 256, 320, 32
+    h, d = _setup(13, out, inn, r, 8)
+    before = d["Wq"].clone()
+    L.loqt_merge_requant(d["Wq"], d["Pq"], torch.zeros_like(d["B"]), 1.0)
+    assert torch.equal(before.codes, d["Wq"].codes) and torch.equal(before.absmax, d["Wq"].absmax)
+
+
+def test_merge_many_matches_single():
+    shapes = [(256, 256, 32), (384, 320, 64), (200, 136, 24)]
+    sets = [_setup(14 + i, o, n, r, 8)[1] for i, (o, n, r) in enumerate(shapes)]
+    singles = [L.loqt_merge_requant(x["Wq"].clone(), x["Pq"], x["B"], 0.5) for x in sets]
+    L.loqt_merge_requant_many([x["Wq"] for x in sets], [x["Pq"] for x in sets], [x["B"] for x in sets], 0.5)
+    for one, x in zip(singles, sets):
+        assert torch.equal(one.codes, x["Wq"].codes) and torch.equal(one.absmax, x["Wq"].absmax)
+
+
+def test_forward_special_cases_on_device():
+    out, inn, r, T = 256, 256, 32, 128
+    h, d = _setup(15, out, inn, r, T)
+    # B = 0: plain quantised linear
+    y0 = L.loqt_linear_fwd(d["Wq"], d["Pq"], torch.zeros_like(d["B"]), 1.0, d["x"])
+    W = O.nf4_dequantize_bf16(*h["wq"]).astype(np.float64)
+    check_close(f32(y0), h["x"].astype(np.float64) @ W.T, "B=0")
+
+
+def test_argument_errors():
+    out, inn, r, T = 256, 256, 32, 128
+    h, d = _setup(16, out, inn, r, T)
+    y = torch.empty((T, out), dtype=torch.bfloat16, device="cuda")
+    small = L.new_workspace(256)
+    with pytest.raises(L.LoqtError, match="workspace"):
+        L.loqt_linear_fwd(d["Wq"], d["Pq"], d["B"], 1.0, d["x"], y=y, ws=small)
+    with pytest.raises(L.LoqtError, match="misaligned"):
+        L.loqt_linear_fwd(d["Wq"], d["Pq"], d["B"], 1.0, d["x"][:, 1:], y=y)
