@@ -1,0 +1,455 @@
+#!/usr/bin/env python
+"""Benchmark of the LoQT quantized low-rank linear hot path on B200.
+
+One step = one pass of the whole hot path over one batch of synthetic input:
+forward + backward of every projection matrix of a Llama-shaped layer set, then
+one merge + requantise of all of them.  Prints one JSON line (rank 0).
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--config 0..4]
+  python bench.py --impl reference ...      # times the CPU oracle instead
+
+With N > 1 (launched by torch.distributed.run) every rank runs an independent
+replica of the layer set (the path has no exchange step); the reported value is
+the sum over ranks divided by the slowest rank's time.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "LoQT linear fwd+bwd TFLOP/s & % bf16 tensor peak; merge_requant GB/s % HBM"
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return {
+            "hbm_gbs": float(p["hbm_gbs"]),
+            "bf16_tflops": float(p["bf16_tflops"]),
+            "bf16_tflops_sustained": float(p.get("bf16_tflops_sustained", p["bf16_tflops"])),
+            "source": "measured",
+        }
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+# --------------------------------------------------------------------------- clocks
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while a region runs."""
+
+    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+             "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu = gpu_index
+        self.proc = None
+        self.path = None
+
+    def start(self):
+        try:
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            os.close(fd)
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.gpu}", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": []}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        try:
+            rows = [l.strip().split(", ") for l in open(self.path) if l.strip()]
+            os.unlink(self.path)
+            sm = sorted(float(r[1]) for r in rows if len(r) >= 9)
+            if sm:
+                out["sm_mhz"] = sm[len(sm) // 2]
+                out["sm_max_mhz"] = float(rows[0][2])
+                out["power_w_max"] = max(float(r[3]) for r in rows if len(r) >= 9)
+                names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+                for i, n in enumerate(names):
+                    if any(r[5 + i].strip().lower() == "active" for r in rows if len(r) >= 9):
+                        out["reasons"].append(n)
+                out["samples"] = len(sm)
+        except Exception:
+            pass
+        return out
+
+
+# --------------------------------------------------------------------------- workload
+def build_model(cfg, seed, device):
+    """All projection matrices of the layer set, quantised on the device, plus
+    per-matrix activations.  Returns a list of dicts (one per matrix)."""
+    import torch
+
+    from paper_2405_16528_b200 import binding as L
+    from paper_2405_16528_b200 import synth
+
+    mats = []
+    for layer in range(cfg.layers):
+        for label, out, inn, count in cfg.shapes():
+            for j in range(count):
+                name = (cfg.name, layer, label, j)
+                W = synth.normal(seed, name + ("W",), (out, inn), 0.02, torch.float32, device)
+                P = synth.orthonormal(seed, name + ("P",), out, cfg.r, device)
+                m = {
+                    "out": out, "in": inn, "label": label,
+                    "Wq": L.loqt_nf4_quantize(W), "Pq": L.loqt_nf4_quantize(P),
+                    "B": synth.normal(seed, name + ("B",), (cfg.r, inn), cfg.sigma_B, torch.bfloat16, device),
+                    "x": synth.normal(seed, name + ("x",), (cfg.T, inn), 1.0, torch.bfloat16, device),
+                    "dy": synth.normal(seed, name + ("dy",), (cfg.T, out), 1.0, torch.bfloat16, device),
+                }
+                del W, P
+                mats.append(m)
+    return mats
+
+
+def pad8(n):
+    return (n + 7) // 8 * 8
+
+
+def alloc_outputs(cfg, mats, device):
+    """Output buffers shared by all matrices of a shape (overwritten every call)."""
+    import torch
+
+    from paper_2405_16528_b200 import binding as L
+
+    bufs = {}
+    ws_bytes = 256
+    for m in mats:
+        key = (m["out"], m["in"])
+        if key not in bufs:
+            bufs[key] = {
+                "y": torch.empty((cfg.T, pad8(m["out"])), dtype=torch.bfloat16, device=device)[:, : m["out"]],
+                "dx": torch.empty((cfg.T, pad8(m["in"])), dtype=torch.bfloat16, device=device)[:, : m["in"]],
+                "dB": torch.empty((cfg.r, m["in"]), dtype=torch.float32, device=device),
+            }
+        ws_bytes = max(ws_bytes, L.loqt_workspace_bytes(L.LOQT_OP_FWD, m["out"], m["in"], cfg.r, cfg.T),
+                       L.loqt_workspace_bytes(L.LOQT_OP_BWD, m["out"], m["in"], cfg.r, cfg.T))
+    return bufs, L.new_workspace(ws_bytes, device)
+
+
+def pad_rows(t):
+    """Row stride a multiple of 8 elements (16 bytes), as the library requires."""
+    import torch
+
+    rows, cols = t.shape
+    if cols % 8 == 0:
+        return t
+    buf = torch.zeros((rows, pad8(cols)), dtype=t.dtype, device=t.device)
+    buf[:, :cols] = t
+    return buf[:, :cols]
+
+
+def run_ours(args, rank, world, local_rank):
+    import torch
+
+    from paper_2405_16528_b200 import binding as L
+    from paper_2405_16528_b200 import build, synth
+
+    build.build()
+    L.lib()  # fails loudly when the CUDA library is missing
+    torch.cuda.set_device(local_rank)
+    device = torch.device("cuda", local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+
+        dist = dist_mod
+        dist.init_process_group("nccl", device_id=device)
+
+    cfg = synth.CONFIGS[args.config]
+    s = 1.0
+    mats = build_model(cfg, args.seed + rank, device)
+    for m in mats:
+        for k in ("B", "x", "dy"):
+            m[k] = pad_rows(m[k])
+    bufs, ws = alloc_outputs(cfg, mats, device)
+    flops_step = sum(synth.fwd_bwd_flops(m["out"], m["in"], cfg.r, cfg.T) for m in mats)
+    merge_bytes_step = sum(synth.merge_bytes(m["out"], m["in"], cfg.r) for m in mats)
+    merge_flops_step = sum(2 * m["out"] * m["in"] * cfg.r for m in mats)
+
+    def fwd_bwd():
+        for m in mats:
+            b = bufs[(m["out"], m["in"])]
+            L.loqt_linear_fwd(m["Wq"], m["Pq"], m["B"], s, m["x"], y=b["y"], ws=ws)
+            L.loqt_linear_bwd(m["Wq"], m["Pq"], m["B"], s, m["x"], m["dy"], dx=b["dx"], dB=b["dB"], ws=ws)
+
+    Wqs, Pqs, Bs = [m["Wq"] for m in mats], [m["Pq"] for m in mats], [m["B"] for m in mats]
+
+    def merge():
+        L.loqt_merge_requant_many(Wqs, Pqs, Bs, s, ws=ws)
+
+    def sync():
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        fwd_bwd()
+        merge()
+    sync()
+    L.loqt_device_status(ws)
+
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
+    launches0 = L.loqt_launch_count()
+    sync()
+    t_wall0 = time.perf_counter()
+    for k in range(args.steps):
+        ev[k][0].record()
+        fwd_bwd()
+        ev[k][1].record()
+        merge()
+        ev[k][2].record()
+    sync()
+    t_wall = time.perf_counter() - t_wall0
+    launches = L.loqt_launch_count() - launches0
+    clocks = sampler.stop() if rank == 0 else None
+    L.loqt_device_status(ws)
+
+    ms_fb = sum(e[0].elapsed_time(e[1]) for e in ev) / args.steps
+    ms_mg = sum(e[1].elapsed_time(e[2]) for e in ev) / args.steps
+    ms_step = sum(e[0].elapsed_time(e[2]) for e in ev) / args.steps
+
+    # ---- end to end: activations come from pinned host memory every step, the
+    # gradient of the trained matrix goes back to the host
+    e2e_steps = max(1, min(args.steps, 2))
+    shapes = {}
+    for m in mats:
+        key = (m["out"], m["in"])
+        if key not in shapes:
+            shapes[key] = {
+                "hx": torch.empty((cfg.T, m["x"].stride(0)), dtype=torch.bfloat16).pin_memory(),
+                "hdy": torch.empty((cfg.T, m["dy"].stride(0)), dtype=torch.bfloat16).pin_memory(),
+                "hdB": torch.empty((cfg.r, m["in"]), dtype=torch.float32).pin_memory(),
+                "dxin": torch.empty((cfg.T, m["x"].stride(0)), dtype=torch.bfloat16, device=device),
+                "ddy": torch.empty((cfg.T, m["dy"].stride(0)), dtype=torch.bfloat16, device=device),
+            }
+            shapes[key]["hx"].normal_()
+            shapes[key]["hdy"].normal_()
+    h2d = d2h = 0
+    for m in mats:
+        sh = shapes[(m["out"], m["in"])]
+        h2d += sh["hx"].numel() * 2 + sh["hdy"].numel() * 2
+        d2h += sh["hdB"].numel() * 4
+
+    def e2e_step():
+        for m in mats:
+            sh = shapes[(m["out"], m["in"])]
+            b = bufs[(m["out"], m["in"])]
+            sh["dxin"].copy_(sh["hx"], non_blocking=True)
+            sh["ddy"].copy_(sh["hdy"], non_blocking=True)
+            xin = sh["dxin"][:, : m["in"]]
+            dyin = sh["ddy"][:, : m["out"]]
+            L.loqt_linear_fwd(m["Wq"], m["Pq"], m["B"], s, xin, y=b["y"], ws=ws)
+            L.loqt_linear_bwd(m["Wq"], m["Pq"], m["B"], s, xin, dyin, dx=b["dx"], dB=b["dB"], ws=ws)
+            sh["hdB"].copy_(b["dB"], non_blocking=True)
+
+    e2e_step()
+    sync()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(e2e_steps):
+        e2e_step()
+    e1.record()
+    sync()
+    ms_e2e = e0.elapsed_time(e1) / e2e_steps
+
+    times = torch.tensor([ms_fb, ms_mg, ms_step, ms_e2e], dtype=torch.float64, device=device)
+    if dist is not None:
+        dist.all_reduce(times, op=dist.ReduceOp.MAX)
+    ms_fb, ms_mg, ms_step, ms_e2e = [float(v) for v in times.cpu()]
+
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    peaks = load_peaks()
+    tflops = world * flops_step / (ms_fb * 1e-3) / 1e12
+    merge_gbs = world * merge_bytes_step / (ms_mg * 1e-3) / 1e9
+    merge_tflops = world * merge_flops_step / (ms_mg * 1e-3) / 1e12
+    per_gpu_tflops = tflops / world
+    result = {
+        "metric": METRIC,
+        "value": round(tflops, 2),
+        "unit": "TFLOP/s (fwd+bwd, algorithmic flops of the factored layer)",
+        "n_gpus": world,
+        "steps": args.steps,
+        "warmup": args.warmup,
+        "ms_per_step": round(ms_step, 3),
+        "ms_fwd_bwd": round(ms_fb, 3),
+        "ms_merge": round(ms_mg, 3),
+        "higher_is_better": True,
+        "scaling": "weak",
+        "vs_baseline": None,
+        "dtype": "bf16 x bf16 -> fp32 (NF4 weights)",
+        "data": "synthetic",
+        "config": {
+            "workload": f"configs[{args.config}] {cfg.name}: {len(mats)} projection matrices, r={cfg.r}, T={cfg.T}",
+            "step": "fwd+bwd of every matrix, then merge_requant of all",
+            "l2": "inputs larger than L2: every matrix has its own weights and activations",
+            "replicas": world,
+            "s": s,
+        },
+        "pct_bf16_peak": {
+            "burst": round(100 * per_gpu_tflops / peaks["bf16_tflops"], 2),
+            "sustained": round(100 * per_gpu_tflops / peaks["bf16_tflops_sustained"], 2),
+            "of": peaks["source"],
+        },
+        "merge_requant": {
+            "gb_s": round(merge_gbs, 1),
+            "pct_hbm": round(100 * merge_gbs / world / peaks["hbm_gbs"], 2),
+            "gemm_tflops": round(merge_tflops, 1),
+            "pct_of_binding_roof": round(
+                100 * max(merge_flops_step / (peaks["bf16_tflops_sustained"] * 1e12), merge_bytes_step / (peaks["hbm_gbs"] * 1e9))
+                / (ms_mg * 1e-3), 2),
+            "bytes_per_step": merge_bytes_step,
+        },
+        "roofline": {
+            "kernel": "loqt_gemm_kernel (fused NF4-dequant tcgen05 GEMM; all fwd+bwd launches)",
+            "bound": "tensor",
+            "achieved": round(per_gpu_tflops, 2),
+            "peak": peaks["bf16_tflops_sustained"],
+            "unit": "TFLOP/s",
+            "frac": round(per_gpu_tflops / peaks["bf16_tflops_sustained"], 4),
+            "peak_kind": f"sustained, of {peaks['source']}",
+            "traffic": None,
+        },
+        "e2e": {
+            "value": round(world * flops_step / (ms_e2e * 1e-3) / 1e12, 2),
+            "unit": "TFLOP/s",
+            "h2d_bytes_per_step": h2d,
+            "d2h_bytes_per_step": d2h,
+            "steps": e2e_steps,
+        },
+        "gpu_launches": int(launches),
+        "clocks": clocks,
+        "wall_s_timed": round(t_wall, 3),
+    }
+    if not args.no_cpu_baseline and world == 1:
+        result["cpu_baseline"] = cpu_baseline(cfg, args.seed)
+    print(json.dumps(result), flush=True)
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+# --------------------------------------------------------------------------- oracle timing
+def oracle_sample(cfg, seed, T_sample):
+    """One forward + backward of the attention-shaped matrix of `cfg` through the
+    CPU oracle on T_sample tokens.  Returns (seconds, algorithmic flops)."""
+    import numpy as np
+    import torch
+
+    from oracle import loqt_oracle as O
+    from paper_2405_16528_b200 import synth
+
+    out = inn = cfg.hidden
+    d = synth.make_layer(seed, "cpu", out, inn, cfg.r, cfg.sigma_B, T_sample)
+    wq, pq = O.nf4_quantize(d["W"].numpy()), O.nf4_quantize(d["P"].numpy())
+    f = lambda t: t.to(torch.float32).numpy()
+    B, x, dy = f(d["B"]), f(d["x"]), f(d["dy"])
+    t0 = time.perf_counter()
+    O.loqt_forward(wq, pq, B, 1.0, x, (out, inn, cfg.r))
+    O.loqt_backward(wq, pq, B, 1.0, x, dy, (out, inn, cfg.r))
+    dt = time.perf_counter() - t0
+    return dt, synth.fwd_bwd_flops(out, inn, cfg.r, T_sample)
+
+
+def blas_threads():
+    try:
+        from threadpoolctl import threadpool_info
+
+        n = [p.get("num_threads", 0) for p in threadpool_info() if p.get("user_api") == "blas"]
+        if n:
+            return max(n)
+    except Exception:
+        pass
+    return os.cpu_count() or 1
+
+
+def cpu_baseline(cfg, seed):
+    T_sample = min(cfg.T, 1024)
+    dt, flops = oracle_sample(cfg, seed, T_sample)
+    return {
+        "value": round(flops / dt / 1e12, 5),
+        "unit": "TFLOP/s",
+        "cores": blas_threads(),
+        "kind": "oracle",
+        "sample": f"fwd+bwd of one {cfg.hidden}x{cfg.hidden} r={cfg.r} matrix on {T_sample} of {cfg.T} tokens, fp64, {dt:.2f} s",
+    }
+
+
+def run_reference(args, rank, world):
+    if rank != 0:
+        return
+    from paper_2405_16528_b200 import synth
+
+    cfg = synth.CONFIGS[args.config]
+    T_sample = min(cfg.T, 512)
+    for _ in range(args.warmup):
+        oracle_sample(cfg, args.seed, T_sample)
+    tot_t = tot_f = 0.0
+    for _ in range(args.steps):
+        dt, fl = oracle_sample(cfg, args.seed, T_sample)
+        tot_t += dt
+        tot_f += fl
+    val = tot_f / tot_t / 1e12
+    sample = f"per step: fwd+bwd of one {cfg.hidden}x{cfg.hidden} r={cfg.r} matrix on {T_sample} of {cfg.T} tokens, fp64"
+    print(json.dumps({
+        "impl": "reference",
+        "metric": METRIC,
+        "value": round(val, 5),
+        "unit": "TFLOP/s (fwd+bwd, algorithmic flops of the factored layer)",
+        "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": round(1e3 * tot_t / args.steps, 3),
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f64", "data": "synthetic",
+        "config": {"workload": f"configs[{args.config}] {cfg.name} (bounded sample)", "sample": sample},
+        "cpu_baseline": {"value": round(val, 5), "unit": "TFLOP/s", "cores": blas_threads(), "kind": "oracle", "sample": sample},
+        "e2e": {"value": round(val, 5), "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", type=int, default=4)
+    ap.add_argument("--seed", type=int, default=0)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.impl == "reference":
+        run_reference(args, rank, world)
+    else:
+        run_ours(args, rank, world, local_rank)
+
+
+if __name__ == "__main__":
+    main()
