@@ -356,25 +356,29 @@ def run_ours(args, rank, world, local_rank):
 
 
 # --------------------------------------------------------------------------- oracle timing
-def oracle_sample(cfg, seed, T_sample):
-    """One forward + backward of the attention-shaped matrix of `cfg` through the
-    CPU oracle on T_sample tokens.  Returns (seconds, algorithmic flops)."""
-    import numpy as np
+def oracle_sample(cfg, seed, T_sample, shapes=None):
+    """Forward + backward of one matrix per listed (out, in) shape of `cfg`
+    (default: the attention shape) through the CPU oracle on T_sample tokens.
+    Returns (seconds, algorithmic flops)."""
     import torch
 
     from oracle import loqt_oracle as O
     from paper_2405_16528_b200 import synth
 
-    out = inn = cfg.hidden
-    d = synth.make_layer(seed, "cpu", out, inn, cfg.r, cfg.sigma_B, T_sample)
-    wq, pq = O.nf4_quantize(d["W"].numpy()), O.nf4_quantize(d["P"].numpy())
-    f = lambda t: t.to(torch.float32).numpy()
-    B, x, dy = f(d["B"]), f(d["x"]), f(d["dy"])
-    t0 = time.perf_counter()
-    O.loqt_forward(wq, pq, B, 1.0, x, (out, inn, cfg.r))
-    O.loqt_backward(wq, pq, B, 1.0, x, dy, (out, inn, cfg.r))
-    dt = time.perf_counter() - t0
-    return dt, synth.fwd_bwd_flops(out, inn, cfg.r, T_sample)
+    shapes = shapes or [(cfg.hidden, cfg.hidden)]
+    dt = 0.0
+    flops = 0
+    for out, inn in shapes:
+        d = synth.make_layer(seed, ("cpu", out, inn), out, inn, cfg.r, cfg.sigma_B, T_sample)
+        wq, pq = O.nf4_quantize(d["W"].numpy()), O.nf4_quantize(d["P"].numpy())
+        f = lambda t: t.to(torch.float32).numpy()
+        B, x, dy = f(d["B"]), f(d["x"]), f(d["dy"])
+        t0 = time.perf_counter()
+        O.loqt_forward(wq, pq, B, 1.0, x, (out, inn, cfg.r))
+        O.loqt_backward(wq, pq, B, 1.0, x, dy, (out, inn, cfg.r))
+        dt += time.perf_counter() - t0
+        flops += synth.fwd_bwd_flops(out, inn, cfg.r, T_sample)
+    return dt, flops
 
 
 def blas_threads():
@@ -390,14 +394,14 @@ def blas_threads():
 
 
 def cpu_baseline(cfg, seed):
-    T_sample = min(cfg.T, 1024)
-    dt, flops = oracle_sample(cfg, seed, T_sample)
+    shapes = [(o, i) for _, o, i, _ in cfg.shapes()]
+    dt, flops = oracle_sample(cfg, seed, cfg.T, shapes)
     return {
         "value": round(flops / dt / 1e12, 5),
         "unit": "TFLOP/s",
         "cores": blas_threads(),
         "kind": "oracle",
-        "sample": f"fwd+bwd of one {cfg.hidden}x{cfg.hidden} r={cfg.r} matrix on {T_sample} of {cfg.T} tokens, fp64, {dt:.2f} s",
+        "sample": f"fwd+bwd of one matrix of each of the {len(shapes)} distinct shapes of a layer, all {cfg.T} tokens, fp64, {dt:.2f} s",
     }
 
 
