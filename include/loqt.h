@@ -137,6 +137,44 @@ loqt_status loqt_merge_requant_many(int32_t n, const loqt_nf4_mat *Wq, const loq
                                     const void *const *B, const int64_t *ldb, float s, void *ws,
                                     size_t ws_bytes, void *stream);
 
+/*
+ * Forward for callers that cannot allocate device memory.  (The paper has no
+ * counterpart: this is a convenience of this library, not part of the method.)
+ *
+ * Some code that wants to run a LoQT layer has no way to obtain a workspace:
+ * a plug-in that is handed tensors by a host framework whose allocator it must
+ * not call, code running where cudaMalloc is forbidden because it would
+ * synchronise the device (inside a latency-critical serving loop, between the
+ * nodes of a pre-planned memory budget), or a small C program that simply owns
+ * no allocator.  For them this entry point computes exactly what
+ * loqt_linear_fwd computes - same arguments for W_q, P_q, B, s, x, y - but the
+ * intermediate s*(x B^T) and the status word live in a fixed array compiled
+ * into the library instead of a caller workspace.
+ *
+ *   - Limit: T * roundup(r, 64) * 2 bytes must not exceed
+ *     LOQT_STATIC_FWD_MAX_SCRATCH (8 MiB: e.g. T = 4096 tokens at r = 1024, or
+ *     16384 tokens at r = 256).  Larger problems return LOQT_ERR_WORKSPACE and
+ *     enqueue nothing; split the tokens or use loqt_linear_fwd.
+ *   - Cost: every GPU on which the library is loaded holds the 8 MiB + 256 B
+ *     array until the process exits, whether or not this function is called.
+ *   - It calls no cudaMalloc / cudaFree and no allocating library routine.
+ *   - The first call on each device looks up the array's device address
+ *     (once per device, with that device current).  Make that first call
+ *     outside any stream capture.
+ *   - All calls on a device share the one array.  Two calls whose kernels can
+ *     overlap on the GPU (different streams without an ordering between them)
+ *     race on it and produce garbage; calls on one stream are safe.  The array
+ *     keeps the previous call's contents; the status word is cleared at the
+ *     start of every call, nothing else needs clearing.
+ *   - check_device_status != 0: after enqueuing, wait for `stream` and return
+ *     LOQT_ERR_TIMEOUT if a bounded device-side wait expired; 0: return as
+ *     soon as the work is enqueued (a device-side timeout then goes unreported).
+ */
+#define LOQT_STATIC_FWD_MAX_SCRATCH (8u * 1024u * 1024u)
+loqt_status loqt_linear_fwd_static(loqt_nf4_mat Wq, loqt_nf4_mat Pq, const void *B, int64_t ldb,
+                                   float s, const void *x, int64_t ldx, int32_t T, void *y,
+                                   int64_t ldy, int check_device_status, void *stream);
+
 /* Bytes of workspace `op` needs for the given shape (never less than 256: the
  * first 256 bytes always hold the device status word). */
 size_t loqt_workspace_bytes(int op, int32_t out, int32_t in, int32_t r, int32_t T);

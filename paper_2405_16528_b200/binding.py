@@ -21,7 +21,7 @@ BLOCK = 64
 
 EXPORTS = (
     "loqt_nf4_quantize", "loqt_nf4_dequantize", "loqt_linear_fwd", "loqt_linear_bwd",
-    "loqt_merge_requant", "loqt_merge_requant_many", "loqt_workspace_bytes",
+    "loqt_merge_requant", "loqt_merge_requant_many", "loqt_linear_fwd_static", "loqt_workspace_bytes",
     "loqt_device_status", "loqt_launch_count", "loqt_status_string",
 )
 
@@ -61,6 +61,8 @@ def lib():
     L.loqt_nf4_dequantize.argtypes = [M, vp, i64, ctypes.c_int, vp]
     L.loqt_linear_fwd.argtypes = [M, M, vp, i64, f32, vp, i64, i32, vp, i64, vp, sz, vp]
     L.loqt_linear_bwd.argtypes = [M, M, vp, i64, f32, vp, i64, vp, i64, i32, vp, i64, vp, i64, ctypes.c_int, vp, sz, vp]
+    L.loqt_linear_fwd_static.argtypes = [M, M, vp, i64, f32, vp, i64, i32, vp, i64, ctypes.c_int, vp]
+    L.loqt_linear_fwd_static.restype = ctypes.c_int
     L.loqt_merge_requant.argtypes = [M, M, vp, i64, f32, vp, sz, vp]
     L.loqt_merge_requant_many.argtypes = [i32, ctypes.POINTER(M), ctypes.POINTER(M), ctypes.POINTER(vp), ctypes.POINTER(i64), f32, vp, sz, vp]
     L.loqt_workspace_bytes.argtypes = [ctypes.c_int, i32, i32, i32, i32]
@@ -161,6 +163,17 @@ def loqt_linear_fwd(Wq: NF4Tensor, Pq: NF4Tensor, B: torch.Tensor, s: float, x: 
     _check(lib().loqt_linear_fwd(Wq.view(), Pq.view(), _dev(B, torch.bfloat16), B.stride(0), float(s),
                                  _dev(x, torch.bfloat16), x.stride(0), T, _dev(y, torch.bfloat16), y.stride(0),
                                  ws.data_ptr(), ws.numel(), _stream()), "loqt_linear_fwd")
+    return y
+
+
+def loqt_linear_fwd_static(Wq: NF4Tensor, Pq: NF4Tensor, B: torch.Tensor, s: float, x: torch.Tensor,
+                           y: torch.Tensor, check_device_status: bool = True) -> torch.Tensor:
+    """Forward through the entry point that needs no workspace: the caller passes
+    only inputs and the output `y`; scratch is a fixed array inside the library."""
+    T = x.shape[0]
+    _check(lib().loqt_linear_fwd_static(Wq.view(), Pq.view(), _dev(B, torch.bfloat16), B.stride(0), float(s),
+                                        _dev(x, torch.bfloat16), x.stride(0), T, _dev(y, torch.bfloat16), y.stride(0),
+                                        int(bool(check_device_status)), _stream()), "loqt_linear_fwd_static")
     return y
 
 

@@ -288,3 +288,54 @@ extern "C" loqt_status loqt_merge_requant_many(int32_t n, const loqt_nf4_mat *Wq
       return st;
   return LOQT_OK;
 }
+
+// ---------------------------------------------------------------------------
+// Forward without any caller-provided scratch (see loqt_linear_fwd_static in loqt.h)
+// ---------------------------------------------------------------------------
+namespace loqt {
+
+// Status word (first 256 bytes) + the T x r intermediate of the forward.  Lives
+// in every GPU context that loads this library, until the process exits.
+constexpr size_t kStaticScratchBytes = 256 + LOQT_STATIC_FWD_MAX_SCRATCH;
+static __device__ __align__(256) unsigned char g_static_fwd_scratch[kStaticScratchBytes];
+
+constexpr int kMaxDevices = 64;
+static void *g_static_scratch_addr[kMaxDevices] = {nullptr};
+static std::mutex g_static_scratch_mutex;
+
+// Device address of the scratch array on the current device.  In host code the
+// symbol's name is only a handle; the address a kernel can use comes from
+// cudaGetSymbolAddress, asked once per device with that device current.
+static loqt_status static_scratch_for_current_device(void **out) {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return LOQT_ERR_CUDA;
+  if (dev < 0 || dev >= kMaxDevices) return LOQT_ERR_UNSUPPORTED;
+  std::lock_guard<std::mutex> lock(g_static_scratch_mutex);
+  if (g_static_scratch_addr[dev] == nullptr) {
+    void *ptr = nullptr;
+    if (cudaGetSymbolAddress(&ptr, g_static_fwd_scratch) != cudaSuccess || ptr == nullptr) return LOQT_ERR_CUDA;
+    g_static_scratch_addr[dev] = ptr;
+  }
+  *out = g_static_scratch_addr[dev];
+  return LOQT_OK;
+}
+
+}  // namespace loqt
+
+extern "C" loqt_status loqt_linear_fwd_static(loqt_nf4_mat Wq, loqt_nf4_mat Pq, const void *B, int64_t ldb, float s,
+                                              const void *x, int64_t ldx, int32_t T, void *y, int64_t ldy,
+                                              int check_device_status, void *stream) {
+  if (T <= 0 || Pq.cols <= 0) return LOQT_ERR_INVALID_ARG;
+  const size_t need = loqt_workspace_bytes(LOQT_OP_FWD, Wq.rows, Wq.cols, Pq.cols, T);
+  if (need > kStaticScratchBytes) return LOQT_ERR_WORKSPACE;  // T * roundup(r, 64) * 2 bytes exceeds the built-in scratch
+  loqt_status st;
+  if ((st = check_arch()) != LOQT_OK) return st;
+  void *scratch = nullptr;
+  if ((st = static_scratch_for_current_device(&scratch)) != LOQT_OK) return st;
+  cudaStream_t stm = static_cast<cudaStream_t>(stream);
+  // The array keeps whatever the previous call left; only the status word has to start at zero.
+  if (cudaMemsetAsync(scratch, 0, 256, stm) != cudaSuccess) return LOQT_ERR_CUDA;
+  if ((st = loqt_linear_fwd(Wq, Pq, B, ldb, s, x, ldx, T, y, ldy, scratch, kStaticScratchBytes, stream)) != LOQT_OK)
+    return st;
+  return check_device_status ? loqt_device_status(scratch, stream) : LOQT_OK;
+}
