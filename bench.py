@@ -176,6 +176,10 @@ def run_ours(args, rank, world, local_rank):
         dist.init_process_group("nccl", device_id=device)
 
     cfg = synth.CONFIGS[args.config]
+    if args.layers > 0:
+        import dataclasses
+
+        cfg = dataclasses.replace(cfg, layers=args.layers, name=f"{cfg.name}[{args.layers} layer(s)]")
     s = 1.0
     mats = build_model(cfg, args.seed + rank, device)
     for m in mats:
@@ -445,6 +449,7 @@ def main():
     ap.add_argument("--config", type=int, default=4)
     ap.add_argument("--seed", type=int, default=0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--layers", type=int, default=0, help="override the layer count (small cases for profiling)")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
