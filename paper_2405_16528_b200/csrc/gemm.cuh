@@ -3,37 +3,39 @@
 //   D[M x N] = sum over up to two K-segments of  A_seg[M x K_seg] * B_seg[N x K_seg]^T
 //
 // Each operand of each segment is either a bf16 matrix brought in by TMA (stored
-// K-major or MN-major) or an NF4 matrix (paper Section 5.1) whose 4-bit codes are
-// unpacked and scaled by dedicated warps straight into the 128-byte-swizzled
-// shared-memory layout the tensor core reads, so a dequantised weight never
-// exists in global memory.  Accumulators live in TMEM (two buffers, so the
-// epilogue of one tile overlaps the main loop of the next).
+// K-major or MN-major) or an NF4 matrix (paper Section 5.1).  For an NF4 operand
+// TMA brings the packed 4-bit codes into shared memory and dedicated warps
+// unpack and scale them straight into the 128-byte-swizzled layout the tensor
+// core reads, so a dequantised weight never exists in global memory.
+//
+// Tile: (MH * 128) x BN outputs per CTA, K staged 64 deep.  MH = 1 keeps two
+// TMEM accumulators so the epilogue of one tile overlaps the main loop of the
+// next; MH = 2 computes two 128-row halves against the same B tile (each
+// dequantised weight is then reused by 256 rows), filling TMEM with one tile.
 //
 // Warp roles (448 threads): warp 0 TMA producer, warp 1 MMA issuer + TMEM
 // owner, warps 2-5 epilogue (one per TMEM lane quarter), warps 6-13 NF4
-// dequantisation.  One CTA per SM; tiles are 128 x BN with 64-deep K stages.
+// dequantisation.  One CTA per SM.
 #pragma once
 #include "nf4_dequant.cuh"
 #include "ptx.cuh"
 
 namespace loqt {
 
-constexpr int kBM = 128;      // tile rows (MMA M)
+constexpr int kHM = 128;      // rows of one MMA (M of tcgen05.mma)
 constexpr int kBK = 64;       // K elements per pipeline stage (one 128-byte swizzle row of bf16)
 constexpr int kUmmaK = 16;    // K of one tcgen05.mma for 16-bit inputs
-constexpr int kStages = 4;
 constexpr int kNumThreads = 448;
 constexpr int kEpiWarp0 = 2;  // warps 2..5
 constexpr int kDeqWarp0 = 6;  // warps 6..13
 constexpr int kDeqWarps = 8;
-constexpr int kDeqThreads = kDeqWarps * 32;
 
 // Operand kinds
 enum : int {
   OP_TMA_K = 0,   // bf16 [rows][K], K contiguous
   OP_TMA_MN = 1,  // bf16 [K][rows], rows (M or N index) contiguous
   OP_NF4_K = 2,   // NF4 [rows][K], blocks run along K
-  OP_NF4_MN = 3,  // NF4 [K][rows], blocks run along the M/N index
+  OP_NF4_MN = 3,  // NF4 [K][rows], blocks run along the M/N index (B operand only)
 };
 
 // Epilogue kinds
@@ -74,23 +76,31 @@ struct GemmParams {
   int has_nf4;       // any NF4 operand in any segment
 };
 
+// a/b: bf16 operands; ca/cb: packed NF4 codes viewed as a byte matrix.
 struct TensorMaps {
   CUtensorMap a[2];
   CUtensorMap b[2];
+  CUtensorMap ca[2];
+  CUtensorMap cb[2];
 };
 
-template <int BN>
+template <int BN, int MH>
 struct SmemLayout {
-  static constexpr int kABytes = kBM * kBK * 2;  // 16 KiB
+  static constexpr int kStages = (MH == 1) ? 4 : 3;
+  static constexpr int kBM = MH * kHM;
+  static constexpr int kABytes = kBM * kBK * 2;
   static constexpr int kBBytes = BN * kBK * 2;
-  static constexpr int kStageBytes = kABytes + kBBytes;
+  static constexpr int kCodeBytes = 8192;  // 256 blocks x 32 bytes
+  static constexpr int kStageBytes = kABytes + kBBytes + kCodeBytes;
   static constexpr int kBarOffset = kStages * kStageBytes;
-  // full[kStages], empty[kStages], tfull[2], tempty[2], drain
-  static constexpr int kNumBars = 2 * kStages + 5;
+  // full[S], empty[S], codes[S], tfull[2], tempty[2], drain
+  static constexpr int kNumBars = 3 * kStages + 5;
   static constexpr int kMiscOffset = kBarOffset + kNumBars * 8;
   static constexpr int kTablesOffset = kMiscOffset + 16;
   static constexpr int kTotal = kTablesOffset + static_cast<int>(sizeof(Nf4Tables));
   static constexpr int kDynamicBytes = kTotal + 1024;  // slack for 1024-byte alignment
+  static_assert(kDynamicBytes <= 232448, "exceeds the 227 KiB shared memory of one CTA");
+  static_assert(kBM * 32 <= kCodeBytes && BN * 32 <= kCodeBytes, "code tile too large");
 };
 
 // Shared-memory matrix descriptor (tcgen05), 128-byte swizzle.
@@ -109,15 +119,15 @@ __device__ __forceinline__ uint32_t make_idesc(int bn, bool a_mn, bool b_mn) {
          | (1u << 7) | (1u << 10)                   // A, B format bf16
          | (a_mn ? (1u << 15) : 0u) | (b_mn ? (1u << 16) : 0u)
          | (static_cast<uint32_t>(bn >> 3) << 17)   // N
-         | (static_cast<uint32_t>(kBM >> 4) << 24); // M
+         | (static_cast<uint32_t>(kHM >> 4) << 24); // M
 }
 
 // Work decomposition shared by all roles.
 struct Sched {
   int mt, nt, units;
   int kb_seg0, kb_total, splits, kb_per_split;
-  __device__ __forceinline__ Sched(const GemmParams &p, int bn) {
-    mt = (p.M + kBM - 1) / kBM;
+  __device__ __forceinline__ Sched(const GemmParams &p, int bm, int bn) {
+    mt = (p.M + bm - 1) / bm;
     nt = (p.N + bn - 1) / bn;
     splits = p.splits;
     kb_per_split = p.kb_per_split;
@@ -140,46 +150,67 @@ struct Sched {
   }
 };
 
-// One NF4 block (64 codes + scale) fetched ahead of its use.
+// What one dequant thread does for one stage: where its 32 bytes of codes sit in
+// the stage's code tile, where its 128-byte operand row goes, and the block
+// scale (fetched from global memory one stage ahead).
 struct DeqTask {
-  uint4 c0, c1;
   float M;
-  int mode;  // 0: nothing to do, 1: dequantise, 2: write zeros
-  uint32_t dst;  // shared-memory byte address of the 128-byte row
-  uint32_t sw;   // row index & 7 (swizzle key)
+  int mode;      // 0: nothing to do, 1: dequantise, 2: write zeros
+  uint32_t src;  // byte offsets of the two 16-byte code chunks inside the code tile
+  uint32_t src2;
+  uint32_t dst;  // byte offset of the 128-byte operand row inside the stage
+  uint32_t sw;   // row index & 7 (swizzle key of the operand row)
 };
 
-template <int BN>
-__device__ __forceinline__ DeqTask deq_fetch(const GemmParams &p, int seg_idx, int kb_in_seg, int m_blk, int n_blk,
-                                             uint32_t stage_base, int t) {
+template <int BN, int MH>
+__device__ __forceinline__ DeqTask deq_plan(const GemmParams &p, int seg_idx, int kb_in_seg, int m_blk, int n_blk,
+                                            int t) {
+  using L = SmemLayout<BN, MH>;
   DeqTask task;
   task.mode = 0;
+  task.M = 0.0f;
+  task.src = task.src2 = task.dst = task.sw = 0;
   const Segment &sg = p.seg[seg_idx];
   const bool a_nf4 = sg.a_kind >= OP_NF4_K;
   const bool b_nf4 = sg.b_kind >= OP_NF4_K;
   if (!a_nf4 && !b_nf4) return task;
   const int kind = a_nf4 ? sg.a_kind : sg.b_kind;
   const Nf4Src &src = a_nf4 ? sg.a_nf4 : sg.b_nf4;
-  const int rows_tile = a_nf4 ? kBM : BN;
+  const int rows_tile = a_nf4 ? L::kBM : BN;
   if (t >= rows_tile) return task;
-  const uint32_t base = stage_base + (a_nf4 ? 0u : static_cast<uint32_t>(SmemLayout<BN>::kABytes));
-  const int mn0 = a_nf4 ? m_blk * kBM : n_blk * BN;
+  const uint32_t base = a_nf4 ? 0u : static_cast<uint32_t>(L::kABytes);
+  const int mn0 = a_nf4 ? m_blk * L::kBM : n_blk * BN;
   const int k0 = kb_in_seg * kBK;
   int row, col0, r8;
   if (kind == OP_NF4_K) {
-    // tile row t <- matrix row mn0 + t, codes k0 .. k0+63
+    // tile row t <- matrix row mn0 + t, codes k0 .. k0+63; code tile is [rows][32 B]
     row = mn0 + t;
     col0 = k0;
     r8 = t & 7;
     task.dst = base + static_cast<uint32_t>((t >> 3) * 1024 + r8 * 128);
+    task.src = static_cast<uint32_t>(t * 32);
+    task.src2 = task.src + 16;
     if (row >= src.rows) return task;  // feeds only discarded outputs
   } else {
-    // chunk j = t / 64 of 64 tile columns, K-row kk = t % 64 <- matrix row k0 + kk
-    const int j = t >> 6, kk = t & 63;
+    // 64-column chunk j, K-row kk <- matrix row k0 + kk, codes of columns mn0 + 64 j ..
+    // A warp takes 8 consecutive K-rows of every chunk, so that its operand-row
+    // stores and its code-tile loads each touch 8 different swizzle positions.
+    constexpr int JB = BN / 64;
+    constexpr int jbits = (JB == 4) ? 2 : 1;
+    const int j = (t >> 3) & (JB - 1);
+    const int kk = (t & 7) | ((t >> (3 + jbits)) << 3);
     row = k0 + kk;
     col0 = mn0 + 64 * j;
     r8 = kk & 7;
     task.dst = base + static_cast<uint32_t>(j * 8192 + (kk >> 3) * 1024 + r8 * 128);
+    // code tile is [64 K-rows][BN/2 bytes], TMA-swizzled (128 B rows: 128-byte
+    // swizzle, 64 B rows: 64-byte swizzle): chunk ^= (offset >> 7) & mask
+    constexpr uint32_t RB = BN / 2;
+    constexpr uint32_t mask = (RB == 128) ? 7u : 3u;
+    const uint32_t o0 = static_cast<uint32_t>(kk) * RB + static_cast<uint32_t>(j) * 32u;
+    const uint32_t o1 = o0 + 16u;
+    task.src = o0 ^ (((o0 >> 7) & mask) << 4);
+    task.src2 = o1 ^ (((o1 >> 7) & mask) << 4);
     if (col0 >= src.ld) return task;  // beyond the matrix: discarded outputs
     if (row >= src.rows) {            // K tail: must contribute zero
       task.mode = 2;
@@ -189,9 +220,6 @@ __device__ __forceinline__ DeqTask deq_fetch(const GemmParams &p, int seg_idx, i
   }
   task.sw = static_cast<uint32_t>(r8);
   task.mode = 1;
-  const uint4 *cp = reinterpret_cast<const uint4 *>(src.codes + static_cast<int64_t>(row) * (src.ld >> 1) + (col0 >> 1));
-  task.c0 = __ldg(cp);
-  task.c1 = __ldg(cp + 1);
   task.M = __ldg(src.absmax + static_cast<int64_t>(row) * (src.ld >> 6) + (col0 >> 6));
   return task;
 }
@@ -200,28 +228,40 @@ __device__ __forceinline__ void st_shared_v4(uint32_t addr, uint4 v) {
   asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w)
                : "memory");
 }
+__device__ __forceinline__ uint4 ld_shared_v4(uint32_t addr) {
+  uint4 v;
+  asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr)
+               : "memory");
+  return v;
+}
 
-__device__ __forceinline__ void deq_store(const DeqTask &task) {
+__device__ __forceinline__ void deq_store(const DeqTask &task, uint32_t stage_base, uint32_t code_base) {
   if (task.mode == 0) return;
+  const uint32_t dst = stage_base + task.dst;
   if (task.mode == 2) {
 #pragma unroll
-    for (uint32_t c = 0; c < 8; ++c) st_shared_v4(task.dst + ((c ^ task.sw) << 4), make_uint4(0, 0, 0, 0));
+    for (uint32_t c = 0; c < 8; ++c) st_shared_v4(dst + ((c ^ task.sw) << 4), make_uint4(0, 0, 0, 0));
     return;
   }
+  const uint4 c0 = ld_shared_v4(code_base + task.src);
+  const uint4 c1 = ld_shared_v4(code_base + task.src2);
   Nf4BlockTable tab;
   nf4_block_table(task.M, tab);
-  const uint32_t w[8] = {task.c0.x, task.c0.y, task.c0.z, task.c0.w, task.c1.x, task.c1.y, task.c1.z, task.c1.w};
+  const uint32_t w[8] = {c0.x, c0.y, c0.z, c0.w, c1.x, c1.y, c1.z, c1.w};
 #pragma unroll
-  for (uint32_t c = 0; c < 8; ++c) st_shared_v4(task.dst + ((c ^ task.sw) << 4), nf4_dequant8(tab, w[c]));
+  for (uint32_t c = 0; c < 8; ++c) st_shared_v4(dst + ((c ^ task.sw) << 4), nf4_dequant8(tab, w[c]));
 }
 
 // ---------------------------------------------------------------------------
 // The kernel
 // ---------------------------------------------------------------------------
-template <int BN>
+template <int BN, int MH>
 __global__ void __launch_bounds__(kNumThreads, 1)
 loqt_gemm_kernel(const __grid_constant__ TensorMaps maps, const GemmParams p) {
-  using L = SmemLayout<BN>;
+  using L = SmemLayout<BN, MH>;
+  constexpr int kStages = L::kStages;
+  constexpr int kBM = L::kBM;
+  constexpr int kAccBufs = (MH == 1) ? 2 : 1;  // TMEM accumulator buffers (each MH * BN columns)
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t *smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
@@ -229,9 +269,10 @@ loqt_gemm_kernel(const __grid_constant__ TensorMaps maps, const GemmParams p) {
   const uint32_t bar0 = smem_base + L::kBarOffset;
   auto full_bar = [&](int s) { return bar0 + 8u * s; };
   auto empty_bar = [&](int s) { return bar0 + 8u * (kStages + s); };
-  auto tfull_bar = [&](int a) { return bar0 + 8u * (2 * kStages + a); };
-  auto tempty_bar = [&](int a) { return bar0 + 8u * (2 * kStages + 2 + a); };
-  const uint32_t drain_bar = bar0 + 8u * (2 * kStages + 4);
+  auto codes_bar = [&](int s) { return bar0 + 8u * (2 * kStages + s); };
+  auto tfull_bar = [&](int a) { return bar0 + 8u * (3 * kStages + a); };
+  auto tempty_bar = [&](int a) { return bar0 + 8u * (3 * kStages + 2 + a); };
+  const uint32_t drain_bar = bar0 + 8u * (3 * kStages + 4);
   volatile uint32_t *misc = reinterpret_cast<volatile uint32_t *>(smem_gen + L::kMiscOffset);
   volatile uint32_t *tmem_slot = misc;       // written by tcgen05.alloc
   volatile uint32_t *abort_flag = misc + 1;  // raised by any role whose wait expired
@@ -239,13 +280,14 @@ loqt_gemm_kernel(const __grid_constant__ TensorMaps maps, const GemmParams p) {
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
-  const Sched sched(p, BN);
+  const Sched sched(p, kBM, BN);
   constexpr uint32_t kTmemCols = 2 * BN;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) {
       ptx::mbar_init(full_bar(s), 1 + (p.has_nf4 ? kDeqWarps : 0));
       ptx::mbar_init(empty_bar(s), 1);
+      ptx::mbar_init(codes_bar(s), 1);
     }
     for (int a = 0; a < 2; ++a) {
       ptx::mbar_init(tfull_bar(a), 1);
@@ -269,8 +311,8 @@ loqt_gemm_kernel(const __grid_constant__ TensorMaps maps, const GemmParams p) {
   if (warp == 0) {
     if (lane == 0) {
       for (int s = 0; s < p.num_segs; ++s) {
-        if (p.seg[s].a_kind <= OP_TMA_MN) ptx::prefetch_tensormap(&maps.a[s]);
-        if (p.seg[s].b_kind <= OP_TMA_MN) ptx::prefetch_tensormap(&maps.b[s]);
+        ptx::prefetch_tensormap(p.seg[s].a_kind <= OP_TMA_MN ? &maps.a[s] : &maps.ca[s]);
+        ptx::prefetch_tensormap(p.seg[s].b_kind <= OP_TMA_MN ? &maps.b[s] : &maps.cb[s]);
       }
       uint32_t it = 0;
       bool ok = true;
@@ -286,6 +328,22 @@ loqt_gemm_kernel(const __grid_constant__ TensorMaps maps, const GemmParams p) {
           const Segment &sg = p.seg[sidx];
           const uint32_t a_dst = smem_base + s * L::kStageBytes;
           const uint32_t b_dst = a_dst + L::kABytes;
+          const uint32_t c_dst = b_dst + L::kBBytes;
+          // packed codes of the stage's NF4 operand (if any) -> code tile
+          if (p.has_nf4) {
+            if (sg.a_kind == OP_NF4_K) {
+              ptx::mbar_arrive_expect_tx(codes_bar(s), kBM * 32);
+              ptx::tma_load_2d(c_dst, &maps.ca[sidx], codes_bar(s), k0 >> 1, m_blk * kBM);
+            } else if (sg.b_kind == OP_NF4_K) {
+              ptx::mbar_arrive_expect_tx(codes_bar(s), BN * 32);
+              ptx::tma_load_2d(c_dst, &maps.cb[sidx], codes_bar(s), k0 >> 1, n_blk * BN);
+            } else if (sg.b_kind == OP_NF4_MN) {
+              ptx::mbar_arrive_expect_tx(codes_bar(s), BN * 32);
+              ptx::tma_load_2d(c_dst, &maps.cb[sidx], codes_bar(s), (n_blk * BN) >> 1, k0);
+            } else {
+              ptx::mbar_arrive(codes_bar(s));  // nothing to dequantise in this stage
+            }
+          }
           uint32_t bytes = 0;
           if (sg.a_kind <= OP_TMA_MN) bytes += L::kABytes;
           if (sg.b_kind <= OP_TMA_MN) bytes += L::kBBytes;
@@ -323,29 +381,34 @@ loqt_gemm_kernel(const __grid_constant__ TensorMaps maps, const GemmParams p) {
       for (int u = blockIdx.x; ok && u < sched.units; u += gridDim.x, ++tile) {
         int m_blk, n_blk, split, kb_lo, kb_hi;
         sched.unit(u, m_blk, n_blk, split, kb_lo, kb_hi);
-        const uint32_t acc = tile & 1u;
-        const uint32_t acc_ph = (tile >> 1) & 1u;
+        const uint32_t acc = tile % kAccBufs;
+        const uint32_t acc_ph = (tile / kAccBufs) & 1u;
         if (!(ok = ptx::mbar_wait(tempty_bar(acc), acc_ph ^ 1u, abort_flag, p.status))) break;
         ptx::tc_fence_after();
-        const uint32_t d_tmem = tmem_base + acc * BN;
+        const uint32_t d_tmem = tmem_base + acc * (MH * BN);
         for (int kb = kb_lo; kb < kb_hi; ++kb, ++it) {
           const int s = it % kStages;
           const uint32_t ph = (it / kStages) & 1u;
           if (!(ok = ptx::mbar_wait(full_bar(s), ph, abort_flag, p.status))) break;
           ptx::tc_fence_after();
           const Segment &sg = p.seg[kb < sched.kb_seg0 ? 0 : 1];
-          const bool a_mn = (sg.a_kind == OP_TMA_MN);  // NF4_MN is never an A operand
+          const bool a_mn = (sg.a_kind == OP_TMA_MN);
           const bool b_mn = (sg.b_kind == OP_TMA_MN) || (sg.b_kind == OP_NF4_MN);
           const uint32_t idesc = make_idesc(BN, a_mn, b_mn);
           const uint32_t a_addr = smem_base + s * L::kStageBytes;
           const uint32_t b_addr = a_addr + L::kABytes;
-          const uint64_t a_desc = make_smem_desc(a_addr, a_mn);
           const uint64_t b_desc = make_smem_desc(b_addr, b_mn);
           const uint32_t a_step = a_mn ? (2048u >> 4) : (32u >> 4);
           const uint32_t b_step = b_mn ? (2048u >> 4) : (32u >> 4);
 #pragma unroll
-          for (uint32_t k = 0; k < kBK / kUmmaK; ++k)
-            ptx::mma_bf16_ss(d_tmem, a_desc + k * a_step, b_desc + k * b_step, idesc, (kb > kb_lo || k > 0) ? 1u : 0u);
+          for (int h = 0; h < MH; ++h) {
+            // half h: rows 128 h .. 128 h + 127 of the A tile (16 KiB further in either layout)
+            const uint64_t a_desc = make_smem_desc(a_addr + h * (kHM * kBK * 2), a_mn);
+#pragma unroll
+            for (uint32_t k = 0; k < kBK / kUmmaK; ++k)
+              ptx::mma_bf16_ss(d_tmem + h * BN, a_desc + k * a_step, b_desc + k * b_step, idesc,
+                               (kb > kb_lo || k > 0) ? 1u : 0u);
+          }
           ptx::mma_commit(empty_bar(s));  // stage reusable once these MMAs have read it
         }
         if (ok) ptx::mma_commit(tfull_bar(acc));
@@ -363,113 +426,114 @@ loqt_gemm_kernel(const __grid_constant__ TensorMaps maps, const GemmParams p) {
     for (int u = blockIdx.x; ok && u < sched.units; u += gridDim.x, ++tile) {
       int m_blk, n_blk, split, kb_lo, kb_hi;
       sched.unit(u, m_blk, n_blk, split, kb_lo, kb_hi);
-      const uint32_t acc = tile & 1u;
-      const uint32_t acc_ph = (tile >> 1) & 1u;
+      const uint32_t acc = tile % kAccBufs;
+      const uint32_t acc_ph = (tile / kAccBufs) & 1u;
       if (!(ok = ptx::mbar_wait(tfull_bar(acc), acc_ph, abort_flag, p.status))) break;
       ptx::tc_fence_after();
-      const int row = m_blk * kBM + q * 32 + lane;
-      const bool row_ok = row < p.M;
-      const uint32_t t_row = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + acc * BN;
       const int n_base = n_blk * BN;
+#pragma unroll 1
+      for (int h = 0; h < MH; ++h) {
+        const int row = m_blk * kBM + h * kHM + q * 32 + lane;
+        const bool row_ok = row < p.M;
+        const uint32_t t_row = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + acc * (MH * BN) + h * BN;
 
-      if (p.epi == EPI_REQUANT) {
-        // One NF4 block of W_q per 64 accumulator columns of this thread's row.
+        if (p.epi == EPI_REQUANT) {
+          // One NF4 block of W_q per 64 accumulator columns of this thread's row.
 #pragma unroll 1
-        for (int jb = 0; jb < BN / 64; ++jb) {
-          uint32_t d0[32], d1[32];
-          ptx::tmem_ld32(t_row + jb * 64, d0);
-          ptx::tmem_ld32(t_row + jb * 64 + 32, d1);
-          ptx::tmem_ld_wait();
-          const int c0 = n_base + jb * 64;
-          if (row_ok && c0 < p.wq_ld) {
-            uint4 *cp = reinterpret_cast<uint4 *>(p.wq_codes + static_cast<int64_t>(row) * (p.wq_ld >> 1) + (c0 >> 1));
-            float *mp = p.wq_absmax + static_cast<int64_t>(row) * (p.wq_ld >> 6) + (c0 >> 6);
-            const uint4 ca = *cp, cb = *(cp + 1);
-            const float Mold = *mp;
-            const uint32_t w[8] = {ca.x, ca.y, ca.z, ca.w, cb.x, cb.y, cb.z, cb.w};
-            float v[64];
-            float Mnew = 0.0f;
+          for (int jb = 0; jb < BN / 64; ++jb) {
+            uint32_t d0[32], d1[32];
+            ptx::tmem_ld32(t_row + jb * 64, d0);
+            ptx::tmem_ld32(t_row + jb * 64 + 32, d1);
+            ptx::tmem_ld_wait();
+            const int c0 = n_base + jb * 64;
+            if (row_ok && c0 < p.wq_ld) {
+              uint4 *cp = reinterpret_cast<uint4 *>(p.wq_codes + static_cast<int64_t>(row) * (p.wq_ld >> 1) + (c0 >> 1));
+              float *mp = p.wq_absmax + static_cast<int64_t>(row) * (p.wq_ld >> 6) + (c0 >> 6);
+              const uint4 ca = *cp, cb = *(cp + 1);
+              const float Mold = *mp;
+              const uint32_t w[8] = {ca.x, ca.y, ca.z, ca.w, cb.x, cb.y, cb.z, cb.w};
+              float v[64];
+              float Mnew = 0.0f;
 #pragma unroll
-            for (int e = 0; e < 64; ++e) {
-              const float deq = Mold * tables.level[(w[e >> 3] >> (4 * (e & 7))) & 15u];
-              const float delta = __uint_as_float(e < 32 ? d0[e] : d1[e - 32]);
-              v[e] = fmaf(p.alpha, delta, deq);
-              Mnew = fmaxf(Mnew, fabsf(v[e]));
-            }
-            uint32_t o[8];
-#pragma unroll
-            for (int g = 0; g < 8; ++g) {
-              if (Mnew > 0.0f) {
-                const float vv[8] = {v[8 * g], v[8 * g + 1], v[8 * g + 2], v[8 * g + 3],
-                                     v[8 * g + 4], v[8 * g + 5], v[8 * g + 6], v[8 * g + 7]};
-                o[g] = nf4_quantize8(tables, vv, Mnew);
-              } else {
-                o[g] = kZeroWord;
+              for (int e = 0; e < 64; ++e) {
+                const float deq = Mold * tables.level[(w[e >> 3] >> (4 * (e & 7))) & 15u];
+                const float delta = __uint_as_float(e < 32 ? d0[e] : d1[e - 32]);
+                v[e] = fmaf(p.alpha, delta, deq);
+                Mnew = fmaxf(Mnew, fabsf(v[e]));
               }
-            }
-            *cp = make_uint4(o[0], o[1], o[2], o[3]);
-            *(cp + 1) = make_uint4(o[4], o[5], o[6], o[7]);
-            *mp = Mnew;
-          }
-          __syncwarp();
-        }
-      } else {
-#pragma unroll 1
-        for (int cb = 0; cb < BN / 32; ++cb) {
-          uint32_t d[32];
-          ptx::tmem_ld32(t_row + cb * 32, d);
-          ptx::tmem_ld_wait();
-          const int c0 = n_base + cb * 32;
-          const bool full = (c0 + 32 <= p.N);
-          if (!row_ok || c0 >= p.N) {
-            // nothing to store for this thread
-          } else if (p.epi == EPI_BF16) {
-            __nv_bfloat16 *o = reinterpret_cast<__nv_bfloat16 *>(p.out) + static_cast<int64_t>(row) * p.ld_out + c0;
-            if (full && (p.ld_out & 7) == 0) {
-#pragma unroll
-              for (int g = 0; g < 4; ++g) {
-                uint4 qv;
-                qv.x = pack_bf16x2(p.alpha * __uint_as_float(d[8 * g + 0]), p.alpha * __uint_as_float(d[8 * g + 1]));
-                qv.y = pack_bf16x2(p.alpha * __uint_as_float(d[8 * g + 2]), p.alpha * __uint_as_float(d[8 * g + 3]));
-                qv.z = pack_bf16x2(p.alpha * __uint_as_float(d[8 * g + 4]), p.alpha * __uint_as_float(d[8 * g + 5]));
-                qv.w = pack_bf16x2(p.alpha * __uint_as_float(d[8 * g + 6]), p.alpha * __uint_as_float(d[8 * g + 7]));
-                reinterpret_cast<uint4 *>(o)[g] = qv;
-              }
-            } else {
-#pragma unroll
-              for (int e = 0; e < 32; ++e)
-                if (c0 + e < p.N) o[e] = __float2bfloat16_rn(p.alpha * __uint_as_float(d[e]));
-            }
-          } else {
-            float *o;
-            int64_t ldo;
-            bool acc_out = false;
-            if (p.epi == EPI_PARTIAL) {
-              ldo = p.ld_out;
-              o = reinterpret_cast<float *>(p.out) + (static_cast<int64_t>(split) * p.M + row) * ldo + c0;
-            } else {
-              ldo = p.ld_out;
-              o = reinterpret_cast<float *>(p.out) + static_cast<int64_t>(row) * ldo + c0;
-              acc_out = p.accumulate != 0;
-            }
-            if (full && (ldo & 3) == 0) {
+              uint32_t o[8];
 #pragma unroll
               for (int g = 0; g < 8; ++g) {
-                float4 f = make_float4(__uint_as_float(d[4 * g]), __uint_as_float(d[4 * g + 1]),
-                                       __uint_as_float(d[4 * g + 2]), __uint_as_float(d[4 * g + 3]));
-                if (acc_out) {
-                  const float4 old = reinterpret_cast<float4 *>(o)[g];
-                  f.x += old.x; f.y += old.y; f.z += old.z; f.w += old.w;
+                if (Mnew > 0.0f) {
+                  const float vv[8] = {v[8 * g], v[8 * g + 1], v[8 * g + 2], v[8 * g + 3],
+                                       v[8 * g + 4], v[8 * g + 5], v[8 * g + 6], v[8 * g + 7]};
+                  o[g] = nf4_quantize8(tables, vv, Mnew);
+                } else {
+                  o[g] = kZeroWord;
                 }
-                reinterpret_cast<float4 *>(o)[g] = f;
+              }
+              *cp = make_uint4(o[0], o[1], o[2], o[3]);
+              *(cp + 1) = make_uint4(o[4], o[5], o[6], o[7]);
+              *mp = Mnew;
+            }
+            __syncwarp();
+          }
+        } else {
+#pragma unroll 1
+          for (int cb = 0; cb < BN / 32; ++cb) {
+            uint32_t d[32];
+            ptx::tmem_ld32(t_row + cb * 32, d);
+            ptx::tmem_ld_wait();
+            const int c0 = n_base + cb * 32;
+            const bool full = (c0 + 32 <= p.N);
+            if (!row_ok || c0 >= p.N) {
+              // nothing to store for this thread
+            } else if (p.epi == EPI_BF16) {
+              __nv_bfloat16 *o = reinterpret_cast<__nv_bfloat16 *>(p.out) + static_cast<int64_t>(row) * p.ld_out + c0;
+              if (full && (p.ld_out & 7) == 0) {
+#pragma unroll
+                for (int g = 0; g < 4; ++g) {
+                  uint4 qv;
+                  qv.x = pack_bf16x2(p.alpha * __uint_as_float(d[8 * g + 0]), p.alpha * __uint_as_float(d[8 * g + 1]));
+                  qv.y = pack_bf16x2(p.alpha * __uint_as_float(d[8 * g + 2]), p.alpha * __uint_as_float(d[8 * g + 3]));
+                  qv.z = pack_bf16x2(p.alpha * __uint_as_float(d[8 * g + 4]), p.alpha * __uint_as_float(d[8 * g + 5]));
+                  qv.w = pack_bf16x2(p.alpha * __uint_as_float(d[8 * g + 6]), p.alpha * __uint_as_float(d[8 * g + 7]));
+                  reinterpret_cast<uint4 *>(o)[g] = qv;
+                }
+              } else {
+#pragma unroll
+                for (int e = 0; e < 32; ++e)
+                  if (c0 + e < p.N) o[e] = __float2bfloat16_rn(p.alpha * __uint_as_float(d[e]));
               }
             } else {
+              float *o;
+              const int64_t ldo = p.ld_out;
+              bool acc_out = false;
+              if (p.epi == EPI_PARTIAL) {
+                o = reinterpret_cast<float *>(p.out) + (static_cast<int64_t>(split) * p.M + row) * ldo + c0;
+              } else {
+                o = reinterpret_cast<float *>(p.out) + static_cast<int64_t>(row) * ldo + c0;
+                acc_out = p.accumulate != 0;
+              }
+              if (full && (ldo & 3) == 0) {
 #pragma unroll
-              for (int e = 0; e < 32; ++e)
-                if (c0 + e < p.N) o[e] = (acc_out ? o[e] : 0.0f) + __uint_as_float(d[e]);
+                for (int g = 0; g < 8; ++g) {
+                  float4 f = make_float4(__uint_as_float(d[4 * g]), __uint_as_float(d[4 * g + 1]),
+                                         __uint_as_float(d[4 * g + 2]), __uint_as_float(d[4 * g + 3]));
+                  if (acc_out) {
+                    const float4 old = reinterpret_cast<float4 *>(o)[g];
+                    f.x += old.x; f.y += old.y; f.z += old.z; f.w += old.w;
+                  }
+                  reinterpret_cast<float4 *>(o)[g] = f;
+                }
+              } else {
+#pragma unroll
+                for (int e = 0; e < 32; ++e)
+                  if (c0 + e < p.N) o[e] = (acc_out ? o[e] : 0.0f) + __uint_as_float(d[e]);
+              }
             }
+            __syncwarp();
           }
-          __syncwarp();
         }
       }
       // Accumulator fully read: hand the TMEM buffer back to the MMA warp.
@@ -482,9 +546,8 @@ loqt_gemm_kernel(const __grid_constant__ TensorMaps maps, const GemmParams p) {
   else {
     if (p.has_nf4) {
       const int t = threadIdx.x - kDeqWarp0 * 32;
-      // Position of the k-block being staged and of the one being fetched ahead.
+      // Position of the k-block being staged and of the one whose scale is fetched ahead.
       int u = blockIdx.x, kb = 0, kb_hi = 0, m_blk = 0, n_blk = 0, split = 0;
-      bool have = false;
       auto open_unit = [&]() {
         while (u < sched.units) {
           int lo;
@@ -495,31 +558,31 @@ loqt_gemm_kernel(const __grid_constant__ TensorMaps maps, const GemmParams p) {
         }
         return false;
       };
-      auto fetch = [&](uint32_t it_) {
+      auto plan = [&]() {
         const int sidx = kb < sched.kb_seg0 ? 0 : 1;
         const int kb_in = sidx == 0 ? kb : kb - sched.kb_seg0;
-        const uint32_t stage_base = smem_base + (it_ % kStages) * L::kStageBytes;
-        return deq_fetch<BN>(p, sidx, kb_in, m_blk, n_blk, stage_base, t);
+        return deq_plan<BN, MH>(p, sidx, kb_in, m_blk, n_blk, t);
       };
       uint32_t it = 0;
       DeqTask next;
       next.mode = 0;
-      have = open_unit();
-      if (have) next = fetch(0);
+      bool have = open_unit();
+      if (have) next = plan();
       bool ok = true;
       while (have && ok) {
         const DeqTask cur = next;
-        // advance to the following k-block and start its loads
         ++kb;
         if (kb >= kb_hi) {
           u += gridDim.x;
           have = open_unit();
         }
-        if (have) next = fetch(it + 1);
+        if (have) next = plan();
         const int s = it % kStages;
         const uint32_t ph = (it / kStages) & 1u;
-        if (!(ok = ptx::mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, p.status))) break;
-        deq_store(cur);
+        // The code tile landing implies the stage's previous contents were consumed.
+        if (!(ok = ptx::mbar_wait(codes_bar(s), ph, abort_flag, p.status))) break;
+        const uint32_t stage_base = smem_base + s * L::kStageBytes;
+        deq_store(cur, stage_base, stage_base + L::kABytes + L::kBBytes);
         ptx::fence_proxy_async_smem();
         __syncwarp();
         if (lane == 0) ptx::mbar_arrive(full_bar(s));

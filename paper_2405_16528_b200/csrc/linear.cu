@@ -42,6 +42,19 @@ static bool make_map(CUtensorMap *map, const void *base, int64_t inner, int64_t 
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// Packed NF4 codes as a byte matrix [rows][ld/2]; box in bytes x rows.
+static bool make_code_map(CUtensorMap *map, const Nf4Src &m, int box_bytes, int box_rows, CUtensorMapSwizzle swz) {
+  EncodeTiledFn fn = encode_fn();
+  if (fn == nullptr) return false;
+  const cuuint64_t dims[2] = {static_cast<cuuint64_t>(m.ld / 2), static_cast<cuuint64_t>(m.rows)};
+  const cuuint64_t strides[1] = {static_cast<cuuint64_t>(m.ld / 2)};
+  const cuuint32_t box[2] = {static_cast<cuuint32_t>(box_bytes), static_cast<cuuint32_t>(box_rows)};
+  const cuuint32_t estr[2] = {1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<uint8_t *>(m.codes), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, swz, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 // A bf16 operand of the engine.  K-major: stored [rows][K]; MN-major: stored [K][rows].
 struct Bf16Operand {
   const void *ptr;
@@ -69,33 +82,70 @@ struct GemmCall {
   Bf16Operand a[2], b[2];
 };
 
-template <int BN>
-static loqt_status launch_bn(const GemmCall &c, cudaStream_t stream) {
-  using L = SmemLayout<BN>;
+// Relative cost of a 128-row pass that has to dequantise its B tile (1.0 = a
+// pass over an already staged tile), and the penalty of the single-buffered
+// 256-row tile whose epilogue does not overlap the next main loop.
+constexpr double kCostDequantPass = 2.0;
+constexpr double kCostSingleBuffer = 1.05;
+
+template <int BN, int MH>
+static loqt_status launch_cfg(const GemmCall &c, cudaStream_t stream) {
+  using L = SmemLayout<BN, MH>;
   TensorMaps maps;
   memset(&maps, 0, sizeof(maps));
   for (int s = 0; s < c.p.num_segs; ++s) {
     const Segment &sg = c.p.seg[s];
-    if (sg.a_kind <= OP_TMA_MN && !map_operand(&maps.a[s], sg.a_kind, c.a[s], c.p.M, sg.K, kBM)) return LOQT_ERR_CUDA;
-    if (sg.b_kind <= OP_TMA_MN && !map_operand(&maps.b[s], sg.b_kind, c.b[s], c.p.N, sg.K, BN)) return LOQT_ERR_CUDA;
+    if (sg.a_kind <= OP_TMA_MN) {
+      if (!map_operand(&maps.a[s], sg.a_kind, c.a[s], c.p.M, sg.K, L::kBM)) return LOQT_ERR_CUDA;
+    } else if (sg.a_kind == OP_NF4_K) {
+      if (!make_code_map(&maps.ca[s], sg.a_nf4, 32, L::kBM, CU_TENSOR_MAP_SWIZZLE_NONE)) return LOQT_ERR_CUDA;
+    } else {
+      return LOQT_ERR_UNSUPPORTED;
+    }
+    if (sg.b_kind <= OP_TMA_MN) {
+      if (!map_operand(&maps.b[s], sg.b_kind, c.b[s], c.p.N, sg.K, BN)) return LOQT_ERR_CUDA;
+    } else if (sg.b_kind == OP_NF4_K) {
+      if (!make_code_map(&maps.cb[s], sg.b_nf4, 32, BN, CU_TENSOR_MAP_SWIZZLE_NONE)) return LOQT_ERR_CUDA;
+    } else {
+      if (!make_code_map(&maps.cb[s], sg.b_nf4, BN / 2, kBK,
+                         BN == 256 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B))
+        return LOQT_ERR_CUDA;
+    }
   }
-  if (cudaFuncSetAttribute(loqt_gemm_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kDynamicBytes) !=
+  if (cudaFuncSetAttribute(loqt_gemm_kernel<BN, MH>, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kDynamicBytes) !=
       cudaSuccess)
     return LOQT_ERR_CUDA;
-  const int mt = (c.p.M + kBM - 1) / kBM, nt = (c.p.N + BN - 1) / BN;
+  const int mt = (c.p.M + L::kBM - 1) / L::kBM, nt = (c.p.N + BN - 1) / BN;
   const int units = mt * nt * c.p.splits;
   const int grid = units < sm_count() ? units : sm_count();
-  loqt_gemm_kernel<BN><<<grid, kNumThreads, L::kDynamicBytes, stream>>>(maps, c.p);
+  loqt_gemm_kernel<BN, MH><<<grid, kNumThreads, L::kDynamicBytes, stream>>>(maps, c.p);
   count_launch();
   return cudaGetLastError() == cudaSuccess ? LOQT_OK : LOQT_ERR_CUDA;
+}
+
+// Rows per CTA tile: 128 (two TMEM buffers, overlapped epilogue) or 256 (one
+// buffer, every staged B tile used twice).  Estimated time = waves x rows x cost
+// per 128-row pass; with an NF4 operand the second pass over a staged tile is
+// cheaper because it needs no dequantisation.
+static int pick_mh(const GemmCall &c, int bn) {
+  if (c.p.M <= kHM) return 1;
+  const int sms = sm_count();
+  const int nt = (c.p.N + bn - 1) / bn;
+  const int u1 = ((c.p.M + 127) / 128) * nt * c.p.splits, u2 = ((c.p.M + 255) / 256) * nt * c.p.splits;
+  const double w1 = (u1 + sms - 1) / sms, w2 = (u2 + sms - 1) / sms;
+  const bool b_nf4 = c.p.seg[0].b_kind >= OP_NF4_K;
+  const double t1 = w1 * (b_nf4 ? kCostDequantPass : 1.0);
+  const double t2 = w2 * ((b_nf4 ? kCostDequantPass : 1.0) + 1.0) * kCostSingleBuffer;
+  return t2 < t1 ? 2 : 1;
 }
 
 static loqt_status launch(GemmCall &c, cudaStream_t stream) {
   c.p.has_nf4 = 0;
   for (int s = 0; s < c.p.num_segs; ++s)
     if (c.p.seg[s].a_kind >= OP_NF4_K || c.p.seg[s].b_kind >= OP_NF4_K) c.p.has_nf4 = 1;
-  if (c.p.N > 128) return launch_bn<256>(c, stream);
-  return launch_bn<128>(c, stream);
+  // The 128-wide tile is only for N <= 128 (a single column of tiles).
+  if (c.p.N > 128) return pick_mh(c, 256) == 2 ? launch_cfg<256, 2>(c, stream) : launch_cfg<256, 1>(c, stream);
+  return pick_mh(c, 128) == 2 ? launch_cfg<128, 2>(c, stream) : launch_cfg<128, 1>(c, stream);
 }
 
 // ---------------------------------------------------------------------------
@@ -106,7 +156,7 @@ static int64_t ld_lowrank(int r) { return (static_cast<int64_t>(r) + 63) / 64 * 
 
 // Split-K factor of the dB product (M = r, N = in, K = T), for a 148-SM part.
 static void db_splits(int r, int in, int T, int &splits, int &kb_per_split) {
-  const int tiles = ((r + kBM - 1) / kBM) * ((in + (in > 128 ? 255 : 127)) / (in > 128 ? 256 : 128));
+  const int tiles = ((r + kHM - 1) / kHM) * ((in + (in > 128 ? 255 : 127)) / (in > 128 ? 256 : 128));
   const int kb_total = (T + kBK - 1) / kBK;
   int want = 148 / (tiles > 0 ? tiles : 1);
   if (want < 1) want = 1;
