@@ -82,11 +82,14 @@ struct GemmCall {
   Bf16Operand a[2], b[2];
 };
 
-// Relative cost of a 128-row pass that has to dequantise its B tile (1.0 = a
-// pass over an already staged tile), and the penalty of the single-buffered
-// 256-row tile whose epilogue does not overlap the next main loop.
-constexpr double kCostDequantPass = 2.0;
-constexpr double kCostSingleBuffer = 1.05;
+// Cost model of pick_tile(), in SM cycles (measured on B200): one K stage of a
+// 128 x 256 MMA pass, dequantising one 64-weight block, the epilogue per 32
+// output columns of a 128-row half, and the per-tile fixed cost.
+constexpr double kCyclesMma256 = 700.0;
+constexpr double kNarrowTilePenalty = 1.15;  // N = 128 passes move more operand bytes per flop
+constexpr double kCyclesDequantRow = 3.3;
+constexpr double kCyclesEpilogueRow = 400.0;
+constexpr double kCyclesFixed = 3000.0;
 
 template <int BN, int MH>
 static loqt_status launch_cfg(const GemmCall &c, cudaStream_t stream) {
@@ -123,29 +126,50 @@ static loqt_status launch_cfg(const GemmCall &c, cudaStream_t stream) {
   return cudaGetLastError() == cudaSuccess ? LOQT_OK : LOQT_ERR_CUDA;
 }
 
-// Rows per CTA tile: 128 (two TMEM buffers, overlapped epilogue) or 256 (one
-// buffer, every staged B tile used twice).  Estimated time = waves x rows x cost
-// per 128-row pass; with an NF4 operand the second pass over a staged tile is
-// cheaper because it needs no dequantisation.
-static int pick_mh(const GemmCall &c, int bn) {
-  if (c.p.M <= kHM) return 1;
+// Tile selection.  Candidates: BN in {256, 128}, rows per CTA 128 (two TMEM
+// buffers, overlapped epilogue) or 256 (one buffer, every staged B tile used by
+// two MMA passes).  A stage costs the larger of its tensor time and - when the B
+// operand is NF4 - its dequantisation time (one pass over BN blocks per stage,
+// whatever the tile height); the single-buffered tile adds an exposed epilogue.
+// Estimated time = waves x (stages x stage cost + exposed epilogue); smallest wins.
+struct TileCfg {
+  int bn, mh;
+};
+
+static TileCfg pick_tile(const GemmCall &c) {
   const int sms = sm_count();
-  const int nt = (c.p.N + bn - 1) / bn;
-  const int u1 = ((c.p.M + 127) / 128) * nt * c.p.splits, u2 = ((c.p.M + 255) / 256) * nt * c.p.splits;
-  const double w1 = (u1 + sms - 1) / sms, w2 = (u2 + sms - 1) / sms;
   const bool b_nf4 = c.p.seg[0].b_kind >= OP_NF4_K;
-  const double t1 = w1 * (b_nf4 ? kCostDequantPass : 1.0);
-  const double t2 = w2 * ((b_nf4 ? kCostDequantPass : 1.0) + 1.0) * kCostSingleBuffer;
-  return t2 < t1 ? 2 : 1;
+  int kb = 0;
+  for (int s = 0; s < c.p.num_segs; ++s) kb += (c.p.seg[s].K + kBK - 1) / kBK;
+  if (c.p.splits > 1) kb = c.p.kb_per_split;
+  const TileCfg cands[4] = {{256, 1}, {256, 2}, {128, 1}, {128, 2}};
+  TileCfg best = {256, 1};
+  double best_t = 1e300;
+  for (const TileCfg &t : cands) {
+    if (t.mh == 2 && c.p.M <= kHM) continue;
+    if (t.bn == 256 && c.p.N <= 128) continue;
+    const int units = ((c.p.M + t.mh * kHM - 1) / (t.mh * kHM)) * ((c.p.N + t.bn - 1) / t.bn) * c.p.splits;
+    const double waves = (units + sms - 1) / sms;
+    const double mma = kCyclesMma256 * t.mh * (t.bn == 256 ? 1.0 : 0.5 * kNarrowTilePenalty);
+    const double deq = b_nf4 ? kCyclesDequantRow * t.bn : 0.0;
+    const double stage = mma > deq ? mma : deq;
+    const double epi = (t.mh == 2 ? 1.0 : 0.25) * kCyclesEpilogueRow * t.mh * t.bn / 32.0;
+    const double cost = waves * (kb * stage + epi + kCyclesFixed);
+    if (cost < best_t) {
+      best_t = cost;
+      best = t;
+    }
+  }
+  return best;
 }
 
 static loqt_status launch(GemmCall &c, cudaStream_t stream) {
   c.p.has_nf4 = 0;
   for (int s = 0; s < c.p.num_segs; ++s)
     if (c.p.seg[s].a_kind >= OP_NF4_K || c.p.seg[s].b_kind >= OP_NF4_K) c.p.has_nf4 = 1;
-  // The 128-wide tile is only for N <= 128 (a single column of tiles).
-  if (c.p.N > 128) return pick_mh(c, 256) == 2 ? launch_cfg<256, 2>(c, stream) : launch_cfg<256, 1>(c, stream);
-  return pick_mh(c, 128) == 2 ? launch_cfg<128, 2>(c, stream) : launch_cfg<128, 1>(c, stream);
+  const TileCfg t = pick_tile(c);
+  if (t.bn == 256) return t.mh == 2 ? launch_cfg<256, 2>(c, stream) : launch_cfg<256, 1>(c, stream);
+  return t.mh == 2 ? launch_cfg<128, 2>(c, stream) : launch_cfg<128, 1>(c, stream);
 }
 
 // ---------------------------------------------------------------------------
