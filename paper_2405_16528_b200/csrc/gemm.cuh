@@ -281,17 +281,22 @@ loqt_gemm_kernel(const __grid_constant__ TensorMaps maps, const GemmParams p) {
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
   const Sched sched(p, kBM, BN);
+  // In the merge kernel (128-row tiles) only four dequant warps have rows to
+  // stage; the other four (warps 10-13, TMEM lane quarters 2,3,0,1) join the
+  // requantising epilogue and take every second 64-column block.
+  const bool helpers = (MH == 1) && (p.epi == EPI_REQUANT);
+  const int epi_groups = helpers ? 2 : 1;
   constexpr uint32_t kTmemCols = 2 * BN;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) {
-      ptx::mbar_init(full_bar(s), 1 + (p.has_nf4 ? kDeqWarps : 0));
+      ptx::mbar_init(full_bar(s), 1 + (p.has_nf4 ? (helpers ? kDeqWarps / 2 : kDeqWarps) : 0));
       ptx::mbar_init(empty_bar(s), 1);
       ptx::mbar_init(codes_bar(s), 1);
     }
     for (int a = 0; a < 2; ++a) {
       ptx::mbar_init(tfull_bar(a), 1);
-      ptx::mbar_init(tempty_bar(a), 4);
+      ptx::mbar_init(tempty_bar(a), 4 * epi_groups);
     }
     ptx::mbar_init(drain_bar, 1);
     *abort_flag = 0;
@@ -419,8 +424,9 @@ loqt_gemm_kernel(const __grid_constant__ TensorMaps maps, const GemmParams p) {
     }
   }
   // =========================================================== epilogue
-  else if (warp < kDeqWarp0) {
+  else if (warp < kDeqWarp0 || (helpers && warp >= kDeqWarp0 + kDeqWarps / 2)) {
     const int q = warp & 3;  // TMEM lane quarter this warp may access
+    const int grp = warp < kDeqWarp0 ? 0 : 1;
     uint32_t tile = 0;
     bool ok = true;
     for (int u = blockIdx.x; ok && u < sched.units; u += gridDim.x, ++tile) {
@@ -440,7 +446,7 @@ loqt_gemm_kernel(const __grid_constant__ TensorMaps maps, const GemmParams p) {
         if (p.epi == EPI_REQUANT) {
           // One NF4 block of W_q per 64 accumulator columns of this thread's row.
 #pragma unroll 1
-          for (int jb = 0; jb < BN / 64; ++jb) {
+          for (int jb = grp; jb < BN / 64; jb += epi_groups) {
             uint32_t d0[32], d1[32];
             ptx::tmem_ld32(t_row + jb * 64, d0);
             ptx::tmem_ld32(t_row + jb * 64 + 32, d1);
@@ -462,12 +468,13 @@ loqt_gemm_kernel(const __grid_constant__ TensorMaps maps, const GemmParams p) {
                 Mnew = fmaxf(Mnew, fabsf(v[e]));
               }
               uint32_t o[8];
+              const Nf4Divisor dv = nf4_divisor(Mnew);
 #pragma unroll
               for (int g = 0; g < 8; ++g) {
                 if (Mnew > 0.0f) {
                   const float vv[8] = {v[8 * g], v[8 * g + 1], v[8 * g + 2], v[8 * g + 3],
                                        v[8 * g + 4], v[8 * g + 5], v[8 * g + 6], v[8 * g + 7]};
-                  o[g] = nf4_quantize8(tables, vv, Mnew);
+                  o[g] = nf4_quantize8_tree(vv, dv);
                 } else {
                   o[g] = kZeroWord;
                 }

@@ -146,7 +146,7 @@ static TileCfg pick_tile(const GemmCall &c) {
   TileCfg best = {256, 1};
   double best_t = 1e300;
   for (const TileCfg &t : cands) {
-    if (t.mh == 2 && c.p.M <= kHM) continue;
+    if (t.mh == 2 && (c.p.M <= kHM || c.p.epi == EPI_REQUANT)) continue;  // the merge epilogue wants 128-row tiles
     if (t.bn == 256 && c.p.N <= 128) continue;
     const int units = ((c.p.M + t.mh * kHM - 1) / (t.mh * kHM)) * ((c.p.N + t.bn - 1) / t.bn) * c.p.splits;
     const double waves = (units + sms - 1) / sms;

@@ -59,7 +59,7 @@ nf4_quantize_kernel(const float *__restrict__ src, int64_t ld_src, uint8_t *__re
     if (!live) continue;
 
     uint32_t w = kZeroWord;
-    if (m > 0.0f) w = nf4_quantize8(tab, v, m);
+    if (m > 0.0f) w = nf4_quantize8(tab, v, nf4_divisor(m));
     uint8_t *crow = codes + static_cast<int64_t>(row) * (ld / 2) + c0 / 2;
     *reinterpret_cast<uint16_t *>(crow + 2 * l) = static_cast<uint16_t>(w & 0xffffu);
     *reinterpret_cast<uint16_t *>(crow + 16 + 2 * l) = static_cast<uint16_t>(w >> 16);

@@ -43,7 +43,9 @@ def test_quantize_decision_boundaries_and_special_values():
         pts += [m, np.nextafter(m, np.float32(-2)), np.nextafter(m, np.float32(2))]
     pts += list(O.NF4_LEVELS)
     rows = []
-    for scale in (1.0, 0.03125, 3.0, 1.7e-3, 2.5e30, 1e-38):
+    # 0x1.fffffep-5 has an all-ones significand; 2.5e30 and 1e-38 lie outside the
+    # range of the reciprocal-based division: all three take the IEEE-divide path
+    for scale in (1.0, 0.03125, 3.0, 0.75, 1.7e-3, 0.0523, float(np.nextafter(np.float32(0.0625), np.float32(0))), 2.5e30, 1e-38, 7e17, 3e-18):
         blk = np.zeros(64, dtype=np.float32)
         blk[: len(pts)] = np.array(pts, dtype=np.float32) * np.float32(scale)
         blk[63] = np.float32(scale)  # pins the block scale
