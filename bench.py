@@ -158,6 +158,42 @@ def pad_rows(t):
     return buf[:, :cols]
 
 
+def time_nf4_kernels(device, peaks, rows=8192, cols=8192, iters=10):
+    """The two streaming kernels on a matrix larger than L2 (fp32 source 268 MB):
+    achieved GB/s on their algorithmic bytes (quantise 4 + 0.5625 B/element,
+    dequantise to bf16 0.5625 + 2 B/element) against the measured HBM copy rate."""
+    import torch
+
+    from paper_2405_16528_b200 import binding as L
+
+    w = torch.randn((rows, cols), device=device, dtype=torch.float32) * 0.02
+    q = L.NF4Tensor.empty(rows, cols, device)
+    out = torch.empty((rows, cols), device=device, dtype=torch.bfloat16)
+
+    def timed(fn):
+        for _ in range(3):
+            fn()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(iters):
+            fn()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / iters
+
+    n = rows * cols
+    ms_q = timed(lambda: L.loqt_nf4_quantize(w, q))
+    ms_d = timed(lambda: L.loqt_nf4_dequantize(q, dst=out))
+    gq = n * 4.5625 / (ms_q * 1e-3) / 1e9
+    gd = n * 2.5625 / (ms_d * 1e-3) / 1e9
+    return {
+        "shape": [rows, cols],
+        "quantize_gb_s": round(gq, 1), "quantize_pct_hbm": round(100 * gq / peaks["hbm_gbs"], 1),
+        "dequantize_bf16_gb_s": round(gd, 1), "dequantize_pct_hbm": round(100 * gd / peaks["hbm_gbs"], 1),
+        "of": peaks["source"],
+    }
+
+
 def run_ours(args, rank, world, local_rank):
     import torch
 
@@ -291,6 +327,7 @@ def run_ours(args, rank, world, local_rank):
         return
 
     peaks = load_peaks()
+    nf4 = time_nf4_kernels(device, peaks)
     tflops = world * flops_step / (ms_fb * 1e-3) / 1e12
     merge_gbs = world * merge_bytes_step / (ms_mg * 1e-3) / 1e9
     merge_tflops = world * merge_flops_step / (ms_mg * 1e-3) / 1e12
@@ -348,6 +385,7 @@ def run_ours(args, rank, world, local_rank):
             "d2h_bytes_per_step": d2h,
             "steps": e2e_steps,
         },
+        "nf4_stream": nf4,
         "gpu_launches": int(launches),
         "clocks": clocks,
         "wall_s_timed": round(t_wall, 3),
