@@ -13,9 +13,16 @@
 // next; MH = 2 computes two 128-row halves against the same B tile (each
 // dequantised weight is then reused by 256 rows), filling TMEM with one tile.
 //
-// Warp roles (448 threads): warp 0 TMA producer, warp 1 MMA issuer + TMEM
-// owner, warps 2-5 epilogue (one per TMEM lane quarter), warps 6-13 NF4
-// dequantisation.  One CTA per SM.
+// Packed codes travel through a ring of their own (kCodeSlots tiles of 8 KiB,
+// deeper than the operand ring): a code tile is requested as soon as the
+// dequant warps have read the one it replaces, several stages before its
+// operand slot frees, so the codes are already in shared memory when the
+// dequant warps get the slot.
+//
+// Warp roles (480 threads): warp 0 TMA producer of the operand stages, warp 1
+// MMA issuer + TMEM owner, warps 2-5 epilogue (one per TMEM lane quarter),
+// warps 6-13 NF4 dequantisation, warp 14 TMA producer of the code ring.  One
+// CTA per SM.
 #pragma once
 #include "nf4_dequant.cuh"
 #include "ptx.cuh"
@@ -25,7 +32,8 @@ namespace loqt {
 constexpr int kHM = 128;      // rows of one MMA (M of tcgen05.mma)
 constexpr int kBK = 64;       // K elements per pipeline stage (one 128-byte swizzle row of bf16)
 constexpr int kUmmaK = 16;    // K of one tcgen05.mma for 16-bit inputs
-constexpr int kNumThreads = 448;
+constexpr int kNumThreads = 480;
+constexpr int kCodeWarp = 14;  // TMA producer of the code ring
 constexpr int kEpiWarp0 = 2;  // warps 2..5
 constexpr int kDeqWarp0 = 6;  // warps 6..13
 constexpr int kDeqWarps = 8;
@@ -91,10 +99,12 @@ struct SmemLayout {
   static constexpr int kABytes = kBM * kBK * 2;
   static constexpr int kBBytes = BN * kBK * 2;
   static constexpr int kCodeBytes = 8192;  // 256 blocks x 32 bytes
-  static constexpr int kStageBytes = kABytes + kBBytes + kCodeBytes;
-  static constexpr int kBarOffset = kStages * kStageBytes;
-  // full[S], empty[S], codes[S], tfull[2], tempty[2], drain
-  static constexpr int kNumBars = 3 * kStages + 5;
+  static constexpr int kCodeSlots = 4;
+  static constexpr int kStageBytes = kABytes + kBBytes;
+  static constexpr int kCodeOffset = kStages * kStageBytes;
+  static constexpr int kBarOffset = kCodeOffset + kCodeSlots * kCodeBytes;
+  // full[S], empty[S], cfull[C], cempty[C], tfull[2], tempty[2], drain
+  static constexpr int kNumBars = 2 * kStages + 2 * kCodeSlots + 5;
   static constexpr int kMiscOffset = kBarOffset + kNumBars * 8;
   static constexpr int kTablesOffset = kMiscOffset + 16;
   static constexpr int kTotal = kTablesOffset + static_cast<int>(sizeof(Nf4Tables));
@@ -269,10 +279,13 @@ loqt_gemm_kernel(const __grid_constant__ TensorMaps maps, const GemmParams p) {
   const uint32_t bar0 = smem_base + L::kBarOffset;
   auto full_bar = [&](int s) { return bar0 + 8u * s; };
   auto empty_bar = [&](int s) { return bar0 + 8u * (kStages + s); };
-  auto codes_bar = [&](int s) { return bar0 + 8u * (2 * kStages + s); };
-  auto tfull_bar = [&](int a) { return bar0 + 8u * (3 * kStages + a); };
-  auto tempty_bar = [&](int a) { return bar0 + 8u * (3 * kStages + 2 + a); };
-  const uint32_t drain_bar = bar0 + 8u * (3 * kStages + 4);
+  constexpr int kCS = L::kCodeSlots;
+  auto cfull_bar = [&](int s) { return bar0 + 8u * (2 * kStages + s); };
+  auto cempty_bar = [&](int s) { return bar0 + 8u * (2 * kStages + kCS + s); };
+  auto tfull_bar = [&](int a) { return bar0 + 8u * (2 * kStages + 2 * kCS + a); };
+  auto tempty_bar = [&](int a) { return bar0 + 8u * (2 * kStages + 2 * kCS + 2 + a); };
+  const uint32_t drain_bar = bar0 + 8u * (2 * kStages + 2 * kCS + 4);
+  auto code_tile = [&](int s) { return smem_base + L::kCodeOffset + s * L::kCodeBytes; };
   volatile uint32_t *misc = reinterpret_cast<volatile uint32_t *>(smem_gen + L::kMiscOffset);
   volatile uint32_t *tmem_slot = misc;       // written by tcgen05.alloc
   volatile uint32_t *abort_flag = misc + 1;  // raised by any role whose wait expired
@@ -292,7 +305,10 @@ loqt_gemm_kernel(const __grid_constant__ TensorMaps maps, const GemmParams p) {
     for (int s = 0; s < kStages; ++s) {
       ptx::mbar_init(full_bar(s), 1 + (p.has_nf4 ? (helpers ? kDeqWarps / 2 : kDeqWarps) : 0));
       ptx::mbar_init(empty_bar(s), 1);
-      ptx::mbar_init(codes_bar(s), 1);
+    }
+    for (int s = 0; s < kCS; ++s) {
+      ptx::mbar_init(cfull_bar(s), 1);
+      ptx::mbar_init(cempty_bar(s), helpers ? kDeqWarps / 2 : kDeqWarps);
     }
     for (int a = 0; a < 2; ++a) {
       ptx::mbar_init(tfull_bar(a), 1);
@@ -316,8 +332,8 @@ loqt_gemm_kernel(const __grid_constant__ TensorMaps maps, const GemmParams p) {
   if (warp == 0) {
     if (lane == 0) {
       for (int s = 0; s < p.num_segs; ++s) {
-        ptx::prefetch_tensormap(p.seg[s].a_kind <= OP_TMA_MN ? &maps.a[s] : &maps.ca[s]);
-        ptx::prefetch_tensormap(p.seg[s].b_kind <= OP_TMA_MN ? &maps.b[s] : &maps.cb[s]);
+        if (p.seg[s].a_kind <= OP_TMA_MN) ptx::prefetch_tensormap(&maps.a[s]);
+        if (p.seg[s].b_kind <= OP_TMA_MN) ptx::prefetch_tensormap(&maps.b[s]);
       }
       uint32_t it = 0;
       bool ok = true;
@@ -333,22 +349,6 @@ loqt_gemm_kernel(const __grid_constant__ TensorMaps maps, const GemmParams p) {
           const Segment &sg = p.seg[sidx];
           const uint32_t a_dst = smem_base + s * L::kStageBytes;
           const uint32_t b_dst = a_dst + L::kABytes;
-          const uint32_t c_dst = b_dst + L::kBBytes;
-          // packed codes of the stage's NF4 operand (if any) -> code tile
-          if (p.has_nf4) {
-            if (sg.a_kind == OP_NF4_K) {
-              ptx::mbar_arrive_expect_tx(codes_bar(s), kBM * 32);
-              ptx::tma_load_2d(c_dst, &maps.ca[sidx], codes_bar(s), k0 >> 1, m_blk * kBM);
-            } else if (sg.b_kind == OP_NF4_K) {
-              ptx::mbar_arrive_expect_tx(codes_bar(s), BN * 32);
-              ptx::tma_load_2d(c_dst, &maps.cb[sidx], codes_bar(s), k0 >> 1, n_blk * BN);
-            } else if (sg.b_kind == OP_NF4_MN) {
-              ptx::mbar_arrive_expect_tx(codes_bar(s), BN * 32);
-              ptx::tma_load_2d(c_dst, &maps.cb[sidx], codes_bar(s), (n_blk * BN) >> 1, k0);
-            } else {
-              ptx::mbar_arrive(codes_bar(s));  // nothing to dequantise in this stage
-            }
-          }
           uint32_t bytes = 0;
           if (sg.a_kind <= OP_TMA_MN) bytes += L::kABytes;
           if (sg.b_kind <= OP_TMA_MN) bytes += L::kBBytes;
@@ -372,6 +372,46 @@ loqt_gemm_kernel(const __grid_constant__ TensorMaps maps, const GemmParams p) {
       if (!ok) {
         // Give copies already in flight time to land before the CTA's shared
         // memory is released.
+        const uint64_t t0 = ptx::globaltimer_ns();
+        while (ptx::globaltimer_ns() - t0 < 200000ull) {
+        }
+      }
+    }
+  }
+  // =========================================================== code-ring producer
+  else if (warp == kCodeWarp) {
+    if (lane == 0 && p.has_nf4) {
+      for (int s = 0; s < p.num_segs; ++s) {
+        if (p.seg[s].a_kind >= OP_NF4_K) ptx::prefetch_tensormap(&maps.ca[s]);
+        if (p.seg[s].b_kind >= OP_NF4_K) ptx::prefetch_tensormap(&maps.cb[s]);
+      }
+      uint32_t it = 0;
+      bool ok = true;
+      for (int u = blockIdx.x; ok && u < sched.units; u += gridDim.x) {
+        int m_blk, n_blk, split, kb_lo, kb_hi;
+        sched.unit(u, m_blk, n_blk, split, kb_lo, kb_hi);
+        for (int kb = kb_lo; kb < kb_hi; ++kb, ++it) {
+          const int sc = it % kCS;
+          const uint32_t ph = (it / kCS) & 1u;
+          if (!(ok = ptx::mbar_wait(cempty_bar(sc), ph ^ 1u, abort_flag, p.status))) break;
+          const int sidx = kb < sched.kb_seg0 ? 0 : 1;
+          const int k0 = (sidx == 0 ? kb : kb - sched.kb_seg0) * kBK;
+          const Segment &sg = p.seg[sidx];
+          if (sg.a_kind == OP_NF4_K) {
+            ptx::mbar_arrive_expect_tx(cfull_bar(sc), kBM * 32);
+            ptx::tma_load_2d(code_tile(sc), &maps.ca[sidx], cfull_bar(sc), k0 >> 1, m_blk * kBM);
+          } else if (sg.b_kind == OP_NF4_K) {
+            ptx::mbar_arrive_expect_tx(cfull_bar(sc), BN * 32);
+            ptx::tma_load_2d(code_tile(sc), &maps.cb[sidx], cfull_bar(sc), k0 >> 1, n_blk * BN);
+          } else if (sg.b_kind == OP_NF4_MN) {
+            ptx::mbar_arrive_expect_tx(cfull_bar(sc), BN * 32);
+            ptx::tma_load_2d(code_tile(sc), &maps.cb[sidx], cfull_bar(sc), (n_blk * BN) >> 1, k0);
+          } else {
+            ptx::mbar_arrive(cfull_bar(sc));  // nothing to dequantise in this stage
+          }
+        }
+      }
+      if (!ok) {
         const uint64_t t0 = ptx::globaltimer_ns();
         while (ptx::globaltimer_ns() - t0 < 200000ull) {
         }
@@ -424,7 +464,7 @@ loqt_gemm_kernel(const __grid_constant__ TensorMaps maps, const GemmParams p) {
     }
   }
   // =========================================================== epilogue
-  else if (warp < kDeqWarp0 || (helpers && warp >= kDeqWarp0 + kDeqWarps / 2)) {
+  else if (warp < kDeqWarp0 || (helpers && warp >= kDeqWarp0 + kDeqWarps / 2 && warp < kDeqWarp0 + kDeqWarps)) {
     const int q = warp & 3;  // TMEM lane quarter this warp may access
     const int grp = warp < kDeqWarp0 ? 0 : 1;
     uint32_t tile = 0;
@@ -584,15 +624,17 @@ loqt_gemm_kernel(const __grid_constant__ TensorMaps maps, const GemmParams p) {
           have = open_unit();
         }
         if (have) next = plan();
-        const int s = it % kStages;
-        const uint32_t ph = (it / kStages) & 1u;
-        // The code tile landing implies the stage's previous contents were consumed.
-        if (!(ok = ptx::mbar_wait(codes_bar(s), ph, abort_flag, p.status))) break;
-        const uint32_t stage_base = smem_base + s * L::kStageBytes;
-        deq_store(cur, stage_base, stage_base + L::kABytes + L::kBBytes);
+        const int s = it % kStages, sc = it % kCS;
+        // codes landed (requested several stages ago), then the operand slot is free
+        if (!(ok = ptx::mbar_wait(cfull_bar(sc), (it / kCS) & 1u, abort_flag, p.status))) break;
+        if (!(ok = ptx::mbar_wait(empty_bar(s), ((it / kStages) & 1u) ^ 1u, abort_flag, p.status))) break;
+        deq_store(cur, smem_base + s * L::kStageBytes, code_tile(sc));
         ptx::fence_proxy_async_smem();
         __syncwarp();
-        if (lane == 0) ptx::mbar_arrive(full_bar(s));
+        if (lane == 0) {
+          ptx::mbar_arrive(full_bar(s));
+          ptx::mbar_arrive(cempty_bar(sc));  // this warp has read its codes
+        }
         ++it;
       }
     }
