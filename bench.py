@@ -194,6 +194,55 @@ def time_nf4_kernels(device, peaks, rows=8192, cols=8192, iters=10):
     }
 
 
+def run_per_shape(args):
+    """Diagnostic: median time of forward, backward and merge for one matrix of
+    each distinct shape of the configuration, L2 flushed between calls."""
+    import torch
+
+    from paper_2405_16528_b200 import binding as L
+    from paper_2405_16528_b200 import build, synth
+
+    build.build()
+    torch.cuda.set_device(0)
+    cfg = synth.CONFIGS[args.config]
+    r, T = cfg.r, cfg.T
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+
+    def timeit(fn, n=7):
+        ts = []
+        for i in range(n + 2):
+            flush.zero_()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            fn()
+            e1.record()
+            torch.cuda.synchronize()
+            if i >= 2:
+                ts.append(e0.elapsed_time(e1))
+        return sorted(ts)[len(ts) // 2]
+
+    res = {}
+    for _, out, inn, _ in cfg.shapes():
+        d = synth.make_layer(args.seed, ("shape", out, inn), out, inn, r, cfg.sigma_B, T, device="cuda")
+        Wq, Pq = L.loqt_nf4_quantize(d["W"]), L.loqt_nf4_quantize(d["P"])
+        B, x, dy = pad_rows(d["B"]), pad_rows(d["x"]), pad_rows(d["dy"])
+        y = torch.empty((T, pad8(out)), dtype=torch.bfloat16, device="cuda")[:, :out]
+        dx = torch.empty((T, pad8(inn)), dtype=torch.bfloat16, device="cuda")[:, :inn]
+        dB = torch.empty((r, inn), dtype=torch.float32, device="cuda")
+        ws = L.new_workspace(L.loqt_workspace_bytes(L.LOQT_OP_BWD, out, inn, r, T))
+        tf = timeit(lambda: L.loqt_linear_fwd(Wq, Pq, B, 1.0, x, y=y, ws=ws))
+        tb = timeit(lambda: L.loqt_linear_bwd(Wq, Pq, B, 1.0, x, dy, dx=dx, dB=dB, ws=ws))
+        Wc = Wq.clone()
+        tm = timeit(lambda: L.loqt_merge_requant(Wc, Pq, B, 1.0, ws=ws))
+        L.loqt_device_status(ws)
+        res[f"{out}x{inn}"] = {
+            "fwd_ms": round(tf, 4), "bwd_ms": round(tb, 4), "merge_ms": round(tm, 4),
+            "fwdbwd_tflops": round(synth.fwd_bwd_flops(out, inn, r, T) / (tf + tb) / 1e9, 1),
+            "merge_gb_s": round(synth.merge_bytes(out, inn, r) / tm / 1e6, 1),
+        }
+    print(json.dumps({"per_shape": res, "config": cfg.name}), flush=True)
+
+
 def run_ours(args, rank, world, local_rank):
     import torch
 
@@ -488,11 +537,15 @@ def main():
     ap.add_argument("--seed", type=int, default=0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--layers", type=int, default=0, help="override the layer count (small cases for profiling)")
+    ap.add_argument("--per-shape", action="store_true", help="diagnostic: time one matrix of each distinct shape and exit")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
-    if args.impl == "reference":
+    if args.per_shape:
+        if rank == 0:
+            run_per_shape(args)
+    elif args.impl == "reference":
         run_reference(args, rank, world)
     else:
         run_ours(args, rank, world, local_rank)
