@@ -19,6 +19,13 @@
 // operand slot frees, so the codes are already in shared memory when the
 // dequant warps get the slot.
 //
+// PAIR mode (NF4 B operand): two CTAs on neighbouring M tiles form a cluster and
+// share the dequantisation of every B tile.  Each dequantises half of the
+// tile's blocks and writes its rows into both CTAs' shared memory (a local
+// store and a distributed-shared-memory store), then arrives on both CTAs'
+// full barriers; each CTA still issues its own MMAs.  This halves the ALU work
+// per flop, which is what bounds the fused products.
+//
 // Warp roles (480 threads): warp 0 TMA producer of the operand stages, warp 1
 // MMA issuer + TMEM owner, warps 2-5 epilogue (one per TMEM lane quarter),
 // warps 6-13 NF4 dequantisation, warp 14 TMA producer of the code ring.  One
@@ -103,8 +110,8 @@ struct SmemLayout {
   static constexpr int kStageBytes = kABytes + kBBytes;
   static constexpr int kCodeOffset = kStages * kStageBytes;
   static constexpr int kBarOffset = kCodeOffset + kCodeSlots * kCodeBytes;
-  // full[S], empty[S], cfull[C], cempty[C], tfull[2], tempty[2], drain
-  static constexpr int kNumBars = 2 * kStages + 2 * kCodeSlots + 5;
+  // full[S], empty[S], cfull[C], cempty[C], tfull[2], tempty[2], drain, pempty[S]
+  static constexpr int kNumBars = 3 * kStages + 2 * kCodeSlots + 5;
   static constexpr int kMiscOffset = kBarOffset + kNumBars * 8;
   static constexpr int kTablesOffset = kMiscOffset + 16;
   static constexpr int kTotal = kTablesOffset + static_cast<int>(sizeof(Nf4Tables));
@@ -245,12 +252,18 @@ __device__ __forceinline__ uint4 ld_shared_v4(uint32_t addr) {
   return v;
 }
 
-__device__ __forceinline__ void deq_store(const DeqTask &task, uint32_t stage_base, uint32_t code_base) {
+// PAIR: every row is also written to the same place in the partner CTA.
+template <bool PAIR>
+__device__ __forceinline__ void deq_store(const DeqTask &task, uint32_t stage_base, uint32_t code_base, uint32_t peer) {
   if (task.mode == 0) return;
   const uint32_t dst = stage_base + task.dst;
+  const uint32_t rdst = PAIR ? ptx::map_to_cta(dst, peer) : 0u;
   if (task.mode == 2) {
 #pragma unroll
-    for (uint32_t c = 0; c < 8; ++c) st_shared_v4(dst + ((c ^ task.sw) << 4), make_uint4(0, 0, 0, 0));
+    for (uint32_t c = 0; c < 8; ++c) {
+      st_shared_v4(dst + ((c ^ task.sw) << 4), make_uint4(0, 0, 0, 0));
+      if (PAIR) ptx::st_cluster_v4(rdst + ((c ^ task.sw) << 4), make_uint4(0, 0, 0, 0));
+    }
     return;
   }
   const uint4 c0 = ld_shared_v4(code_base + task.src);
@@ -259,13 +272,19 @@ __device__ __forceinline__ void deq_store(const DeqTask &task, uint32_t stage_ba
   nf4_block_table(task.M, tab);
   const uint32_t w[8] = {c0.x, c0.y, c0.z, c0.w, c1.x, c1.y, c1.z, c1.w};
 #pragma unroll
-  for (uint32_t c = 0; c < 8; ++c) st_shared_v4(dst + ((c ^ task.sw) << 4), nf4_dequant8(tab, w[c]));
+  for (uint32_t c = 0; c < 8; ++c) {
+    const uint4 v = nf4_dequant8(tab, w[c]);
+    st_shared_v4(dst + ((c ^ task.sw) << 4), v);
+    if (PAIR) ptx::st_cluster_v4(rdst + ((c ^ task.sw) << 4), v);
+  }
 }
+
+__device__ __forceinline__ bool helpers_of(const GemmParams &p, int mh) { return mh == 1 && p.epi == EPI_REQUANT; }
 
 // ---------------------------------------------------------------------------
 // The kernel
 // ---------------------------------------------------------------------------
-template <int BN, int MH>
+template <int BN, int MH, bool PAIR>
 __global__ void __launch_bounds__(kNumThreads, 1)
 loqt_gemm_kernel(const __grid_constant__ TensorMaps maps, const GemmParams p) {
   using L = SmemLayout<BN, MH>;
@@ -285,6 +304,11 @@ loqt_gemm_kernel(const __grid_constant__ TensorMaps maps, const GemmParams p) {
   auto tfull_bar = [&](int a) { return bar0 + 8u * (2 * kStages + 2 * kCS + a); };
   auto tempty_bar = [&](int a) { return bar0 + 8u * (2 * kStages + 2 * kCS + 2 + a); };
   const uint32_t drain_bar = bar0 + 8u * (2 * kStages + 2 * kCS + 4);
+  auto pempty_bar = [&](int s) { return bar0 + 8u * (2 * kStages + 2 * kCS + 5 + s); };  // partner released slot s
+  const uint32_t peer = PAIR ? (ptx::cluster_ctarank() ^ 1u) : 0u;
+  // dequant warps that take part: all eight, four in the merge kernel (the rest
+  // help its epilogue), four per CTA in PAIR mode (each CTA does half the tile)
+  const int deq_local = (helpers_of(p, MH) || PAIR) ? kDeqWarps / 2 : kDeqWarps;
   auto code_tile = [&](int s) { return smem_base + L::kCodeOffset + s * L::kCodeBytes; };
   volatile uint32_t *misc = reinterpret_cast<volatile uint32_t *>(smem_gen + L::kMiscOffset);
   volatile uint32_t *tmem_slot = misc;       // written by tcgen05.alloc
@@ -303,12 +327,14 @@ loqt_gemm_kernel(const __grid_constant__ TensorMaps maps, const GemmParams p) {
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) {
-      ptx::mbar_init(full_bar(s), 1 + (p.has_nf4 ? (helpers ? kDeqWarps / 2 : kDeqWarps) : 0));
+      // arrivals: the TMA producer, the local dequant warps, and in PAIR mode the partner's
+      ptx::mbar_init(full_bar(s), 1 + (p.has_nf4 ? deq_local * (PAIR ? 2 : 1) : 0));
       ptx::mbar_init(empty_bar(s), 1);
+      ptx::mbar_init(pempty_bar(s), 1);
     }
     for (int s = 0; s < kCS; ++s) {
       ptx::mbar_init(cfull_bar(s), 1);
-      ptx::mbar_init(cempty_bar(s), helpers ? kDeqWarps / 2 : kDeqWarps);
+      ptx::mbar_init(cempty_bar(s), deq_local);
     }
     for (int a = 0; a < 2; ++a) {
       ptx::mbar_init(tfull_bar(a), 1);
@@ -325,6 +351,7 @@ loqt_gemm_kernel(const __grid_constant__ TensorMaps maps, const GemmParams p) {
   }
   ptx::tc_fence_before();
   __syncthreads();
+  if (PAIR) ptx::cluster_sync_all();  // the partner's barriers exist before anything arrives on them
   ptx::tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
@@ -344,6 +371,8 @@ loqt_gemm_kernel(const __grid_constant__ TensorMaps maps, const GemmParams p) {
           const int s = it % kStages;
           const uint32_t ph = (it / kStages) & 1u;
           if (!(ok = ptx::mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, p.status))) break;
+          // tell the partner that this CTA's slot s may be overwritten
+          if (PAIR) ptx::mbar_arrive_cluster(ptx::map_to_cta(pempty_bar(s), peer));
           const int sidx = kb < sched.kb_seg0 ? 0 : 1;
           const int k0 = (sidx == 0 ? kb : kb - sched.kb_seg0) * kBK;
           const Segment &sg = p.seg[sidx];
@@ -434,7 +463,7 @@ loqt_gemm_kernel(const __grid_constant__ TensorMaps maps, const GemmParams p) {
         for (int kb = kb_lo; kb < kb_hi; ++kb, ++it) {
           const int s = it % kStages;
           const uint32_t ph = (it / kStages) & 1u;
-          if (!(ok = ptx::mbar_wait(full_bar(s), ph, abort_flag, p.status))) break;
+          if (!(ok = ptx::mbar_wait<PAIR>(full_bar(s), ph, abort_flag, p.status))) break;
           ptx::tc_fence_after();
           const Segment &sg = p.seg[kb < sched.kb_seg0 ? 0 : 1];
           const bool a_mn = (sg.a_kind == OP_TMA_MN);
@@ -591,8 +620,9 @@ loqt_gemm_kernel(const __grid_constant__ TensorMaps maps, const GemmParams p) {
   }
   // =========================================================== NF4 dequant
   else {
-    if (p.has_nf4) {
-      const int t = threadIdx.x - kDeqWarp0 * 32;
+    if (p.has_nf4 && (!PAIR || warp < kDeqWarp0 + kDeqWarps / 2)) {
+      // PAIR: this CTA stages blocks [128 rank, 128 rank + 128) of every B tile
+      const int t = threadIdx.x - kDeqWarp0 * 32 + (PAIR ? static_cast<int>(peer ^ 1u) * 128 : 0);
       // Position of the k-block being staged and of the one whose scale is fetched ahead.
       int u = blockIdx.x, kb = 0, kb_hi = 0, m_blk = 0, n_blk = 0, split = 0;
       auto open_unit = [&]() {
@@ -628,11 +658,14 @@ loqt_gemm_kernel(const __grid_constant__ TensorMaps maps, const GemmParams p) {
         // codes landed (requested several stages ago), then the operand slot is free
         if (!(ok = ptx::mbar_wait(cfull_bar(sc), (it / kCS) & 1u, abort_flag, p.status))) break;
         if (!(ok = ptx::mbar_wait(empty_bar(s), ((it / kStages) & 1u) ^ 1u, abort_flag, p.status))) break;
-        deq_store(cur, smem_base + s * L::kStageBytes, code_tile(sc));
-        ptx::fence_proxy_async_smem();
+        if (PAIR && !(ok = ptx::mbar_wait<true>(pempty_bar(s), (it / kStages) & 1u, abort_flag, p.status))) break;
+        deq_store<PAIR>(cur, smem_base + s * L::kStageBytes, code_tile(sc), peer);
+        if (PAIR) ptx::fence_proxy_async_all();
+        else ptx::fence_proxy_async_smem();
         __syncwarp();
         if (lane == 0) {
           ptx::mbar_arrive(full_bar(s));
+          if (PAIR) ptx::mbar_arrive_cluster(ptx::map_to_cta(full_bar(s), peer));
           ptx::mbar_arrive(cempty_bar(sc));  // this warp has read its codes
         }
         ++it;
@@ -647,6 +680,8 @@ loqt_gemm_kernel(const __grid_constant__ TensorMaps maps, const GemmParams p) {
     ptx::tc_fence_after();
     ptx::tmem_dealloc(tmem_base, kTmemCols);
   }
+  // the partner may still be writing into this CTA's shared memory or barriers
+  if (PAIR) ptx::cluster_sync_all();
 }
 
 // Deterministic split-K reduction: out = (accumulate ? out : 0) + sum_s partial[s].
