@@ -19,12 +19,12 @@
 // operand slot frees, so the codes are already in shared memory when the
 // dequant warps get the slot.
 //
-// PAIR mode (NF4 B operand): two CTAs on neighbouring M tiles form a cluster and
-// share the dequantisation of every B tile.  Each dequantises half of the
-// tile's blocks and writes its rows into both CTAs' shared memory (a local
-// store and a distributed-shared-memory store), then arrives on both CTAs'
-// full barriers; each CTA still issues its own MMAs.  This halves the ALU work
-// per flop, which is what bounds the fused products.
+// PAIR mode (NF4 B operand, BN = 256): two CTAs on neighbouring M tiles form a
+// cluster and share the dequantisation of every B tile.  Each dequantises half
+// of the tile's blocks into its own shared memory and ships the finished rows
+// to its partner with an asynchronous shared-to-shared bulk copy that completes
+// on the partner's full barrier; each CTA still issues its own MMAs.  This
+// halves the ALU work per flop, which is what bounds the fused products.
 //
 // Warp roles (480 threads): warp 0 TMA producer of the operand stages, warp 1
 // MMA issuer + TMEM owner, warps 2-5 epilogue (one per TMEM lane quarter),
@@ -177,6 +177,8 @@ struct DeqTask {
   uint32_t src2;
   uint32_t dst;  // byte offset of the 128-byte operand row inside the stage
   uint32_t sw;   // row index & 7 (swizzle key of the operand row)
+  int nf4;       // the stage has an NF4 operand (whether or not this thread's row is inside the matrix)
+  int mn;        // that operand is staged MN-major
 };
 
 template <int BN, int MH>
@@ -187,11 +189,14 @@ __device__ __forceinline__ DeqTask deq_plan(const GemmParams &p, int seg_idx, in
   task.mode = 0;
   task.M = 0.0f;
   task.src = task.src2 = task.dst = task.sw = 0;
+  task.nf4 = task.mn = 0;
   const Segment &sg = p.seg[seg_idx];
   const bool a_nf4 = sg.a_kind >= OP_NF4_K;
   const bool b_nf4 = sg.b_kind >= OP_NF4_K;
   if (!a_nf4 && !b_nf4) return task;
   const int kind = a_nf4 ? sg.a_kind : sg.b_kind;
+  task.nf4 = 1;
+  task.mn = (kind == OP_NF4_MN);
   const Nf4Src &src = a_nf4 ? sg.a_nf4 : sg.b_nf4;
   const int rows_tile = a_nf4 ? L::kBM : BN;
   if (t >= rows_tile) return task;
@@ -252,18 +257,12 @@ __device__ __forceinline__ uint4 ld_shared_v4(uint32_t addr) {
   return v;
 }
 
-// PAIR: every row is also written to the same place in the partner CTA.
-template <bool PAIR>
-__device__ __forceinline__ void deq_store(const DeqTask &task, uint32_t stage_base, uint32_t code_base, uint32_t peer) {
+__device__ __forceinline__ void deq_store(const DeqTask &task, uint32_t stage_base, uint32_t code_base) {
   if (task.mode == 0) return;
   const uint32_t dst = stage_base + task.dst;
-  const uint32_t rdst = PAIR ? ptx::map_to_cta(dst, peer) : 0u;
   if (task.mode == 2) {
 #pragma unroll
-    for (uint32_t c = 0; c < 8; ++c) {
-      st_shared_v4(dst + ((c ^ task.sw) << 4), make_uint4(0, 0, 0, 0));
-      if (PAIR) ptx::st_cluster_v4(rdst + ((c ^ task.sw) << 4), make_uint4(0, 0, 0, 0));
-    }
+    for (uint32_t c = 0; c < 8; ++c) st_shared_v4(dst + ((c ^ task.sw) << 4), make_uint4(0, 0, 0, 0));
     return;
   }
   const uint4 c0 = ld_shared_v4(code_base + task.src);
@@ -272,11 +271,7 @@ __device__ __forceinline__ void deq_store(const DeqTask &task, uint32_t stage_ba
   nf4_block_table(task.M, tab);
   const uint32_t w[8] = {c0.x, c0.y, c0.z, c0.w, c1.x, c1.y, c1.z, c1.w};
 #pragma unroll
-  for (uint32_t c = 0; c < 8; ++c) {
-    const uint4 v = nf4_dequant8(tab, w[c]);
-    st_shared_v4(dst + ((c ^ task.sw) << 4), v);
-    if (PAIR) ptx::st_cluster_v4(rdst + ((c ^ task.sw) << 4), v);
-  }
+  for (uint32_t c = 0; c < 8; ++c) st_shared_v4(dst + ((c ^ task.sw) << 4), nf4_dequant8(tab, w[c]));
 }
 
 __device__ __forceinline__ bool helpers_of(const GemmParams &p, int mh) { return mh == 1 && p.epi == EPI_REQUANT; }
@@ -327,8 +322,9 @@ loqt_gemm_kernel(const __grid_constant__ TensorMaps maps, const GemmParams p) {
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) {
-      // arrivals: the TMA producer, the local dequant warps, and in PAIR mode the partner's
-      ptx::mbar_init(full_bar(s), 1 + (p.has_nf4 ? deq_local * (PAIR ? 2 : 1) : 0));
+      // arrivals: the TMA producer and the local dequant warps (the partner's half of a
+      // dequantised tile is counted in transaction bytes)
+      ptx::mbar_init(full_bar(s), 1 + (p.has_nf4 ? deq_local : 0));
       ptx::mbar_init(empty_bar(s), 1);
       ptx::mbar_init(pempty_bar(s), 1);
     }
@@ -381,6 +377,7 @@ loqt_gemm_kernel(const __grid_constant__ TensorMaps maps, const GemmParams p) {
           uint32_t bytes = 0;
           if (sg.a_kind <= OP_TMA_MN) bytes += L::kABytes;
           if (sg.b_kind <= OP_TMA_MN) bytes += L::kBBytes;
+          else if (PAIR) bytes += L::kBBytes / 2;  // the partner's half of the dequantised tile
           ptx::mbar_arrive_expect_tx(full_bar(s), bytes);
           if (sg.a_kind == OP_TMA_K) {
             ptx::tma_load_2d(a_dst, &maps.a[sidx], full_bar(s), k0, m_blk * kBM);
@@ -659,13 +656,25 @@ loqt_gemm_kernel(const __grid_constant__ TensorMaps maps, const GemmParams p) {
         if (!(ok = ptx::mbar_wait(cfull_bar(sc), (it / kCS) & 1u, abort_flag, p.status))) break;
         if (!(ok = ptx::mbar_wait(empty_bar(s), ((it / kStages) & 1u) ^ 1u, abort_flag, p.status))) break;
         if (PAIR && !(ok = ptx::mbar_wait<true>(pempty_bar(s), (it / kStages) & 1u, abort_flag, p.status))) break;
-        deq_store<PAIR>(cur, smem_base + s * L::kStageBytes, code_tile(sc), peer);
-        if (PAIR) ptx::fence_proxy_async_all();
-        else ptx::fence_proxy_async_smem();
+        const uint32_t stage_base = smem_base + s * L::kStageBytes;
+        deq_store(cur, stage_base, code_tile(sc));
+        ptx::fence_proxy_async_smem();
         __syncwarp();
         if (lane == 0) {
+          if (PAIR && cur.nf4) {
+            // ship this warp's 32 finished rows (4 KiB) to the partner: one run of four
+            // 1 KiB groups (K-major), or one 1 KiB group in each 64-column chunk (MN-major)
+            const uint32_t src = stage_base + cur.dst;
+            const uint32_t rbar = ptx::map_to_cta(full_bar(s), peer);
+            if (!cur.mn) {
+              ptx::bulk_copy_to_cta(ptx::map_to_cta(src, peer), src, 4096, rbar);
+            } else {
+#pragma unroll
+              for (uint32_t j = 0; j < 4; ++j)
+                ptx::bulk_copy_to_cta(ptx::map_to_cta(src + j * 8192, peer), src + j * 8192, 1024, rbar);
+            }
+          }
           ptx::mbar_arrive(full_bar(s));
-          if (PAIR) ptx::mbar_arrive_cluster(ptx::map_to_cta(full_bar(s), peer));
           ptx::mbar_arrive(cempty_bar(sc));  // this warp has read its codes
         }
         ++it;

@@ -190,11 +190,8 @@ static loqt_status launch(GemmCall &c, cudaStream_t stream) {
   const int mt = (c.p.M + t.mh * kHM - 1) / (t.mh * kHM);
   bool b_nf4 = false;
   for (int s = 0; s < c.p.num_segs; ++s) b_nf4 = b_nf4 || c.p.seg[s].b_kind >= OP_NF4_K;
-  const bool pair = b_nf4 && (mt % 2 == 0) && c.p.splits == 1;
-  if (pair) {
-    if (t.bn == 256) return t.mh == 2 ? launch_cfg<256, 2, true>(c, stream) : launch_cfg<256, 1, true>(c, stream);
-    return t.mh == 2 ? launch_cfg<128, 2, true>(c, stream) : launch_cfg<128, 1, true>(c, stream);
-  }
+  const bool pair = b_nf4 && t.bn == 256 && (mt % 2 == 0) && c.p.splits == 1;
+  if (pair) return t.mh == 2 ? launch_cfg<256, 2, true>(c, stream) : launch_cfg<256, 1, true>(c, stream);
   if (t.bn == 256) return t.mh == 2 ? launch_cfg<256, 2, false>(c, stream) : launch_cfg<256, 1, false>(c, stream);
   return t.mh == 2 ? launch_cfg<128, 2, false>(c, stream) : launch_cfg<128, 1, false>(c, stream);
 }
