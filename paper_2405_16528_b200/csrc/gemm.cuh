@@ -13,23 +13,9 @@
 // next; MH = 2 computes two 128-row halves against the same B tile (each
 // dequantised weight is then reused by 256 rows), filling TMEM with one tile.
 //
-// Packed codes travel through a ring of their own (kCodeSlots tiles of 8 KiB,
-// deeper than the operand ring): a code tile is requested as soon as the
-// dequant warps have read the one it replaces, several stages before its
-// operand slot frees, so the codes are already in shared memory when the
-// dequant warps get the slot.
-//
-// PAIR mode (NF4 B operand, BN = 256): two CTAs on neighbouring M tiles form a
-// cluster and share the dequantisation of every B tile.  Each dequantises half
-// of the tile's blocks into its own shared memory and ships the finished rows
-// to its partner with an asynchronous shared-to-shared bulk copy that completes
-// on the partner's full barrier; each CTA still issues its own MMAs.  This
-// halves the ALU work per flop, which is what bounds the fused products.
-//
-// Warp roles (480 threads): warp 0 TMA producer of the operand stages, warp 1
-// MMA issuer + TMEM owner, warps 2-5 epilogue (one per TMEM lane quarter),
-// warps 6-13 NF4 dequantisation, warp 14 TMA producer of the code ring.  One
-// CTA per SM.
+// Warp roles (448 threads): warp 0 TMA producer, warp 1 MMA issuer + TMEM
+// owner, warps 2-5 epilogue (one per TMEM lane quarter), warps 6-13 NF4
+// dequantisation.  One CTA per SM.
 #pragma once
 #include "nf4_dequant.cuh"
 #include "ptx.cuh"
@@ -39,8 +25,7 @@ namespace loqt {
 constexpr int kHM = 128;      // rows of one MMA (M of tcgen05.mma)
 constexpr int kBK = 64;       // K elements per pipeline stage (one 128-byte swizzle row of bf16)
 constexpr int kUmmaK = 16;    // K of one tcgen05.mma for 16-bit inputs
-constexpr int kNumThreads = 480;
-constexpr int kCodeWarp = 14;  // TMA producer of the code ring
+constexpr int kNumThreads = 448;
 constexpr int kEpiWarp0 = 2;  // warps 2..5
 constexpr int kDeqWarp0 = 6;  // warps 6..13
 constexpr int kDeqWarps = 8;
@@ -106,12 +91,10 @@ struct SmemLayout {
   static constexpr int kABytes = kBM * kBK * 2;
   static constexpr int kBBytes = BN * kBK * 2;
   static constexpr int kCodeBytes = 8192;  // 256 blocks x 32 bytes
-  static constexpr int kCodeSlots = 4;
-  static constexpr int kStageBytes = kABytes + kBBytes;
-  static constexpr int kCodeOffset = kStages * kStageBytes;
-  static constexpr int kBarOffset = kCodeOffset + kCodeSlots * kCodeBytes;
-  // full[S], empty[S], cfull[C], cempty[C], tfull[2], tempty[2], drain, pempty[S]
-  static constexpr int kNumBars = 3 * kStages + 2 * kCodeSlots + 5;
+  static constexpr int kStageBytes = kABytes + kBBytes + kCodeBytes;
+  static constexpr int kBarOffset = kStages * kStageBytes;
+  // full[S], empty[S], codes[S], tfull[2], tempty[2], drain
+  static constexpr int kNumBars = 3 * kStages + 5;
   static constexpr int kMiscOffset = kBarOffset + kNumBars * 8;
   static constexpr int kTablesOffset = kMiscOffset + 16;
   static constexpr int kTotal = kTablesOffset + static_cast<int>(sizeof(Nf4Tables));
@@ -177,8 +160,6 @@ struct DeqTask {
   uint32_t src2;
   uint32_t dst;  // byte offset of the 128-byte operand row inside the stage
   uint32_t sw;   // row index & 7 (swizzle key of the operand row)
-  int nf4;       // the stage has an NF4 operand (whether or not this thread's row is inside the matrix)
-  int mn;        // that operand is staged MN-major
 };
 
 template <int BN, int MH>
@@ -189,14 +170,11 @@ __device__ __forceinline__ DeqTask deq_plan(const GemmParams &p, int seg_idx, in
   task.mode = 0;
   task.M = 0.0f;
   task.src = task.src2 = task.dst = task.sw = 0;
-  task.nf4 = task.mn = 0;
   const Segment &sg = p.seg[seg_idx];
   const bool a_nf4 = sg.a_kind >= OP_NF4_K;
   const bool b_nf4 = sg.b_kind >= OP_NF4_K;
   if (!a_nf4 && !b_nf4) return task;
   const int kind = a_nf4 ? sg.a_kind : sg.b_kind;
-  task.nf4 = 1;
-  task.mn = (kind == OP_NF4_MN);
   const Nf4Src &src = a_nf4 ? sg.a_nf4 : sg.b_nf4;
   const int rows_tile = a_nf4 ? L::kBM : BN;
   if (t >= rows_tile) return task;
@@ -274,12 +252,10 @@ __device__ __forceinline__ void deq_store(const DeqTask &task, uint32_t stage_ba
   for (uint32_t c = 0; c < 8; ++c) st_shared_v4(dst + ((c ^ task.sw) << 4), nf4_dequant8(tab, w[c]));
 }
 
-__device__ __forceinline__ bool helpers_of(const GemmParams &p, int mh) { return mh == 1 && p.epi == EPI_REQUANT; }
-
 // ---------------------------------------------------------------------------
 // The kernel
 // ---------------------------------------------------------------------------
-template <int BN, int MH, bool PAIR>
+template <int BN, int MH>
 __global__ void __launch_bounds__(kNumThreads, 1)
 loqt_gemm_kernel(const __grid_constant__ TensorMaps maps, const GemmParams p) {
   using L = SmemLayout<BN, MH>;
@@ -293,18 +269,10 @@ loqt_gemm_kernel(const __grid_constant__ TensorMaps maps, const GemmParams p) {
   const uint32_t bar0 = smem_base + L::kBarOffset;
   auto full_bar = [&](int s) { return bar0 + 8u * s; };
   auto empty_bar = [&](int s) { return bar0 + 8u * (kStages + s); };
-  constexpr int kCS = L::kCodeSlots;
-  auto cfull_bar = [&](int s) { return bar0 + 8u * (2 * kStages + s); };
-  auto cempty_bar = [&](int s) { return bar0 + 8u * (2 * kStages + kCS + s); };
-  auto tfull_bar = [&](int a) { return bar0 + 8u * (2 * kStages + 2 * kCS + a); };
-  auto tempty_bar = [&](int a) { return bar0 + 8u * (2 * kStages + 2 * kCS + 2 + a); };
-  const uint32_t drain_bar = bar0 + 8u * (2 * kStages + 2 * kCS + 4);
-  auto pempty_bar = [&](int s) { return bar0 + 8u * (2 * kStages + 2 * kCS + 5 + s); };  // partner released slot s
-  const uint32_t peer = PAIR ? (ptx::cluster_ctarank() ^ 1u) : 0u;
-  // dequant warps that take part: all eight, four in the merge kernel (the rest
-  // help its epilogue), four per CTA in PAIR mode (each CTA does half the tile)
-  const int deq_local = (helpers_of(p, MH) || PAIR) ? kDeqWarps / 2 : kDeqWarps;
-  auto code_tile = [&](int s) { return smem_base + L::kCodeOffset + s * L::kCodeBytes; };
+  auto codes_bar = [&](int s) { return bar0 + 8u * (2 * kStages + s); };
+  auto tfull_bar = [&](int a) { return bar0 + 8u * (3 * kStages + a); };
+  auto tempty_bar = [&](int a) { return bar0 + 8u * (3 * kStages + 2 + a); };
+  const uint32_t drain_bar = bar0 + 8u * (3 * kStages + 4);
   volatile uint32_t *misc = reinterpret_cast<volatile uint32_t *>(smem_gen + L::kMiscOffset);
   volatile uint32_t *tmem_slot = misc;       // written by tcgen05.alloc
   volatile uint32_t *abort_flag = misc + 1;  // raised by any role whose wait expired
@@ -322,15 +290,9 @@ loqt_gemm_kernel(const __grid_constant__ TensorMaps maps, const GemmParams p) {
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) {
-      // arrivals: the TMA producer and the local dequant warps (the partner's half of a
-      // dequantised tile is counted in transaction bytes)
-      ptx::mbar_init(full_bar(s), 1 + (p.has_nf4 ? deq_local : 0));
+      ptx::mbar_init(full_bar(s), 1 + (p.has_nf4 ? (helpers ? kDeqWarps / 2 : kDeqWarps) : 0));
       ptx::mbar_init(empty_bar(s), 1);
-      ptx::mbar_init(pempty_bar(s), 1);
-    }
-    for (int s = 0; s < kCS; ++s) {
-      ptx::mbar_init(cfull_bar(s), 1);
-      ptx::mbar_init(cempty_bar(s), deq_local);
+      ptx::mbar_init(codes_bar(s), 1);
     }
     for (int a = 0; a < 2; ++a) {
       ptx::mbar_init(tfull_bar(a), 1);
@@ -347,7 +309,6 @@ loqt_gemm_kernel(const __grid_constant__ TensorMaps maps, const GemmParams p) {
   }
   ptx::tc_fence_before();
   __syncthreads();
-  if (PAIR) ptx::cluster_sync_all();  // the partner's barriers exist before anything arrives on them
   ptx::tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
@@ -355,8 +316,8 @@ loqt_gemm_kernel(const __grid_constant__ TensorMaps maps, const GemmParams p) {
   if (warp == 0) {
     if (lane == 0) {
       for (int s = 0; s < p.num_segs; ++s) {
-        if (p.seg[s].a_kind <= OP_TMA_MN) ptx::prefetch_tensormap(&maps.a[s]);
-        if (p.seg[s].b_kind <= OP_TMA_MN) ptx::prefetch_tensormap(&maps.b[s]);
+        ptx::prefetch_tensormap(p.seg[s].a_kind <= OP_TMA_MN ? &maps.a[s] : &maps.ca[s]);
+        ptx::prefetch_tensormap(p.seg[s].b_kind <= OP_TMA_MN ? &maps.b[s] : &maps.cb[s]);
       }
       uint32_t it = 0;
       bool ok = true;
@@ -367,17 +328,30 @@ loqt_gemm_kernel(const __grid_constant__ TensorMaps maps, const GemmParams p) {
           const int s = it % kStages;
           const uint32_t ph = (it / kStages) & 1u;
           if (!(ok = ptx::mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, p.status))) break;
-          // tell the partner that this CTA's slot s may be overwritten
-          if (PAIR) ptx::mbar_arrive_cluster(ptx::map_to_cta(pempty_bar(s), peer));
           const int sidx = kb < sched.kb_seg0 ? 0 : 1;
           const int k0 = (sidx == 0 ? kb : kb - sched.kb_seg0) * kBK;
           const Segment &sg = p.seg[sidx];
           const uint32_t a_dst = smem_base + s * L::kStageBytes;
           const uint32_t b_dst = a_dst + L::kABytes;
+          const uint32_t c_dst = b_dst + L::kBBytes;
+          // packed codes of the stage's NF4 operand (if any) -> code tile
+          if (p.has_nf4) {
+            if (sg.a_kind == OP_NF4_K) {
+              ptx::mbar_arrive_expect_tx(codes_bar(s), kBM * 32);
+              ptx::tma_load_2d(c_dst, &maps.ca[sidx], codes_bar(s), k0 >> 1, m_blk * kBM);
+            } else if (sg.b_kind == OP_NF4_K) {
+              ptx::mbar_arrive_expect_tx(codes_bar(s), BN * 32);
+              ptx::tma_load_2d(c_dst, &maps.cb[sidx], codes_bar(s), k0 >> 1, n_blk * BN);
+            } else if (sg.b_kind == OP_NF4_MN) {
+              ptx::mbar_arrive_expect_tx(codes_bar(s), BN * 32);
+              ptx::tma_load_2d(c_dst, &maps.cb[sidx], codes_bar(s), (n_blk * BN) >> 1, k0);
+            } else {
+              ptx::mbar_arrive(codes_bar(s));  // nothing to dequantise in this stage
+            }
+          }
           uint32_t bytes = 0;
           if (sg.a_kind <= OP_TMA_MN) bytes += L::kABytes;
           if (sg.b_kind <= OP_TMA_MN) bytes += L::kBBytes;
-          else if (PAIR) bytes += L::kBBytes / 2;  // the partner's half of the dequantised tile
           ptx::mbar_arrive_expect_tx(full_bar(s), bytes);
           if (sg.a_kind == OP_TMA_K) {
             ptx::tma_load_2d(a_dst, &maps.a[sidx], full_bar(s), k0, m_blk * kBM);
@@ -404,46 +378,6 @@ loqt_gemm_kernel(const __grid_constant__ TensorMaps maps, const GemmParams p) {
       }
     }
   }
-  // =========================================================== code-ring producer
-  else if (warp == kCodeWarp) {
-    if (lane == 0 && p.has_nf4) {
-      for (int s = 0; s < p.num_segs; ++s) {
-        if (p.seg[s].a_kind >= OP_NF4_K) ptx::prefetch_tensormap(&maps.ca[s]);
-        if (p.seg[s].b_kind >= OP_NF4_K) ptx::prefetch_tensormap(&maps.cb[s]);
-      }
-      uint32_t it = 0;
-      bool ok = true;
-      for (int u = blockIdx.x; ok && u < sched.units; u += gridDim.x) {
-        int m_blk, n_blk, split, kb_lo, kb_hi;
-        sched.unit(u, m_blk, n_blk, split, kb_lo, kb_hi);
-        for (int kb = kb_lo; kb < kb_hi; ++kb, ++it) {
-          const int sc = it % kCS;
-          const uint32_t ph = (it / kCS) & 1u;
-          if (!(ok = ptx::mbar_wait(cempty_bar(sc), ph ^ 1u, abort_flag, p.status))) break;
-          const int sidx = kb < sched.kb_seg0 ? 0 : 1;
-          const int k0 = (sidx == 0 ? kb : kb - sched.kb_seg0) * kBK;
-          const Segment &sg = p.seg[sidx];
-          if (sg.a_kind == OP_NF4_K) {
-            ptx::mbar_arrive_expect_tx(cfull_bar(sc), kBM * 32);
-            ptx::tma_load_2d(code_tile(sc), &maps.ca[sidx], cfull_bar(sc), k0 >> 1, m_blk * kBM);
-          } else if (sg.b_kind == OP_NF4_K) {
-            ptx::mbar_arrive_expect_tx(cfull_bar(sc), BN * 32);
-            ptx::tma_load_2d(code_tile(sc), &maps.cb[sidx], cfull_bar(sc), k0 >> 1, n_blk * BN);
-          } else if (sg.b_kind == OP_NF4_MN) {
-            ptx::mbar_arrive_expect_tx(cfull_bar(sc), BN * 32);
-            ptx::tma_load_2d(code_tile(sc), &maps.cb[sidx], cfull_bar(sc), (n_blk * BN) >> 1, k0);
-          } else {
-            ptx::mbar_arrive(cfull_bar(sc));  // nothing to dequantise in this stage
-          }
-        }
-      }
-      if (!ok) {
-        const uint64_t t0 = ptx::globaltimer_ns();
-        while (ptx::globaltimer_ns() - t0 < 200000ull) {
-        }
-      }
-    }
-  }
   // =========================================================== MMA issuer
   else if (warp == 1) {
     if (lane == 0) {
@@ -460,7 +394,7 @@ loqt_gemm_kernel(const __grid_constant__ TensorMaps maps, const GemmParams p) {
         for (int kb = kb_lo; kb < kb_hi; ++kb, ++it) {
           const int s = it % kStages;
           const uint32_t ph = (it / kStages) & 1u;
-          if (!(ok = ptx::mbar_wait<PAIR>(full_bar(s), ph, abort_flag, p.status))) break;
+          if (!(ok = ptx::mbar_wait(full_bar(s), ph, abort_flag, p.status))) break;
           ptx::tc_fence_after();
           const Segment &sg = p.seg[kb < sched.kb_seg0 ? 0 : 1];
           const bool a_mn = (sg.a_kind == OP_TMA_MN);
@@ -490,7 +424,7 @@ loqt_gemm_kernel(const __grid_constant__ TensorMaps maps, const GemmParams p) {
     }
   }
   // =========================================================== epilogue
-  else if (warp < kDeqWarp0 || (helpers && warp >= kDeqWarp0 + kDeqWarps / 2 && warp < kDeqWarp0 + kDeqWarps)) {
+  else if (warp < kDeqWarp0 || (helpers && warp >= kDeqWarp0 + kDeqWarps / 2)) {
     const int q = warp & 3;  // TMEM lane quarter this warp may access
     const int grp = warp < kDeqWarp0 ? 0 : 1;
     uint32_t tile = 0;
@@ -617,9 +551,8 @@ loqt_gemm_kernel(const __grid_constant__ TensorMaps maps, const GemmParams p) {
   }
   // =========================================================== NF4 dequant
   else {
-    if (p.has_nf4 && (!PAIR || warp < kDeqWarp0 + kDeqWarps / 2)) {
-      // PAIR: this CTA stages blocks [128 rank, 128 rank + 128) of every B tile
-      const int t = threadIdx.x - kDeqWarp0 * 32 + (PAIR ? static_cast<int>(peer ^ 1u) * 128 : 0);
+    if (p.has_nf4) {
+      const int t = threadIdx.x - kDeqWarp0 * 32;
       // Position of the k-block being staged and of the one whose scale is fetched ahead.
       int u = blockIdx.x, kb = 0, kb_hi = 0, m_blk = 0, n_blk = 0, split = 0;
       auto open_unit = [&]() {
@@ -651,32 +584,15 @@ loqt_gemm_kernel(const __grid_constant__ TensorMaps maps, const GemmParams p) {
           have = open_unit();
         }
         if (have) next = plan();
-        const int s = it % kStages, sc = it % kCS;
-        // codes landed (requested several stages ago), then the operand slot is free
-        if (!(ok = ptx::mbar_wait(cfull_bar(sc), (it / kCS) & 1u, abort_flag, p.status))) break;
-        if (!(ok = ptx::mbar_wait(empty_bar(s), ((it / kStages) & 1u) ^ 1u, abort_flag, p.status))) break;
-        if (PAIR && !(ok = ptx::mbar_wait<true>(pempty_bar(s), (it / kStages) & 1u, abort_flag, p.status))) break;
+        const int s = it % kStages;
+        const uint32_t ph = (it / kStages) & 1u;
+        // The code tile landing implies the stage's previous contents were consumed.
+        if (!(ok = ptx::mbar_wait(codes_bar(s), ph, abort_flag, p.status))) break;
         const uint32_t stage_base = smem_base + s * L::kStageBytes;
-        deq_store(cur, stage_base, code_tile(sc));
+        deq_store(cur, stage_base, stage_base + L::kABytes + L::kBBytes);
         ptx::fence_proxy_async_smem();
         __syncwarp();
-        if (lane == 0) {
-          if (PAIR && cur.nf4) {
-            // ship this warp's 32 finished rows (4 KiB) to the partner: one run of four
-            // 1 KiB groups (K-major), or one 1 KiB group in each 64-column chunk (MN-major)
-            const uint32_t src = stage_base + cur.dst;
-            const uint32_t rbar = ptx::map_to_cta(full_bar(s), peer);
-            if (!cur.mn) {
-              ptx::bulk_copy_to_cta(ptx::map_to_cta(src, peer), src, 4096, rbar);
-            } else {
-#pragma unroll
-              for (uint32_t j = 0; j < 4; ++j)
-                ptx::bulk_copy_to_cta(ptx::map_to_cta(src + j * 8192, peer), src + j * 8192, 1024, rbar);
-            }
-          }
-          ptx::mbar_arrive(full_bar(s));
-          ptx::mbar_arrive(cempty_bar(sc));  // this warp has read its codes
-        }
+        if (lane == 0) ptx::mbar_arrive(full_bar(s));
         ++it;
       }
     }
@@ -689,8 +605,6 @@ loqt_gemm_kernel(const __grid_constant__ TensorMaps maps, const GemmParams p) {
     ptx::tc_fence_after();
     ptx::tmem_dealloc(tmem_base, kTmemCols);
   }
-  // the partner may still be writing into this CTA's shared memory or barriers
-  if (PAIR) ptx::cluster_sync_all();
 }
 
 // Deterministic split-K reduction: out = (accumulate ? out : 0) + sum_s partial[s].

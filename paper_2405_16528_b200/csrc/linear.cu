@@ -91,7 +91,7 @@ constexpr double kCyclesDequantRow = 3.3;
 constexpr double kCyclesEpilogueRow = 400.0;
 constexpr double kCyclesFixed = 3000.0;
 
-template <int BN, int MH, bool PAIR>
+template <int BN, int MH>
 static loqt_status launch_cfg(const GemmCall &c, cudaStream_t stream) {
   using L = SmemLayout<BN, MH>;
   TensorMaps maps;
@@ -115,31 +115,15 @@ static loqt_status launch_cfg(const GemmCall &c, cudaStream_t stream) {
         return LOQT_ERR_CUDA;
     }
   }
-  auto kernel = loqt_gemm_kernel<BN, MH, PAIR>;
-  if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kDynamicBytes) != cudaSuccess)
+  if (cudaFuncSetAttribute(loqt_gemm_kernel<BN, MH>, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kDynamicBytes) !=
+      cudaSuccess)
     return LOQT_ERR_CUDA;
   const int mt = (c.p.M + L::kBM - 1) / L::kBM, nt = (c.p.N + BN - 1) / BN;
   const int units = mt * nt * c.p.splits;
-  int grid = units < sm_count() ? units : sm_count();
-  cudaLaunchConfig_t cfg;
-  memset(&cfg, 0, sizeof(cfg));
-  cudaLaunchAttribute attr[1];
-  if (PAIR) {
-    grid &= ~1;  // whole pairs; `units` is even here
-    attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = 2;
-    attr[0].val.clusterDim.y = 1;
-    attr[0].val.clusterDim.z = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
-  }
-  cfg.gridDim = dim3(grid);
-  cfg.blockDim = dim3(kNumThreads);
-  cfg.dynamicSmemBytes = L::kDynamicBytes;
-  cfg.stream = stream;
-  const cudaError_t err = cudaLaunchKernelEx(&cfg, kernel, maps, c.p);
+  const int grid = units < sm_count() ? units : sm_count();
+  loqt_gemm_kernel<BN, MH><<<grid, kNumThreads, L::kDynamicBytes, stream>>>(maps, c.p);
   count_launch();
-  return (err == cudaSuccess && cudaGetLastError() == cudaSuccess) ? LOQT_OK : LOQT_ERR_CUDA;
+  return cudaGetLastError() == cudaSuccess ? LOQT_OK : LOQT_ERR_CUDA;
 }
 
 // Tile selection.  Candidates: BN in {256, 128}, rows per CTA 128 (two TMEM
@@ -184,16 +168,8 @@ static loqt_status launch(GemmCall &c, cudaStream_t stream) {
   for (int s = 0; s < c.p.num_segs; ++s)
     if (c.p.seg[s].a_kind >= OP_NF4_K || c.p.seg[s].b_kind >= OP_NF4_K) c.p.has_nf4 = 1;
   const TileCfg t = pick_tile(c);
-  // Two CTAs on neighbouring M tiles can share the dequantisation of an NF4 B
-  // operand when tiles pair up exactly: an even number of M tiles (so a pair
-  // has the same N tile) and no split-K.
-  const int mt = (c.p.M + t.mh * kHM - 1) / (t.mh * kHM);
-  bool b_nf4 = false;
-  for (int s = 0; s < c.p.num_segs; ++s) b_nf4 = b_nf4 || c.p.seg[s].b_kind >= OP_NF4_K;
-  const bool pair = b_nf4 && t.bn == 256 && (mt % 2 == 0) && c.p.splits == 1;
-  if (pair) return t.mh == 2 ? launch_cfg<256, 2, true>(c, stream) : launch_cfg<256, 1, true>(c, stream);
-  if (t.bn == 256) return t.mh == 2 ? launch_cfg<256, 2, false>(c, stream) : launch_cfg<256, 1, false>(c, stream);
-  return t.mh == 2 ? launch_cfg<128, 2, false>(c, stream) : launch_cfg<128, 1, false>(c, stream);
+  if (t.bn == 256) return t.mh == 2 ? launch_cfg<256, 2>(c, stream) : launch_cfg<256, 1>(c, stream);
+  return t.mh == 2 ? launch_cfg<128, 2>(c, stream) : launch_cfg<128, 1>(c, stream);
 }
 
 // ---------------------------------------------------------------------------
