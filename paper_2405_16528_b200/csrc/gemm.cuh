@@ -13,6 +13,16 @@
 // next; MH = 2 computes two 128-row halves against the same B tile (each
 // dequantised weight is then reused by 256 rows), filling TMEM with one tile.
 //
+// TWO mode (tcgen05 cta_group::2): two CTAs on neighbouring M tiles form a
+// cluster and run every MMA together.  Each keeps its own A tile and its own
+// accumulators but stages only half of the B tile (128 of the 256 N rows), and
+// one thread of the leader CTA issues M = 256 instructions that drive both SMs'
+// tensor cores.  Per SM this halves the dequantisation work, the B bytes written
+// to shared memory and the B bytes the tensor core reads from it.  Barriers the
+// MMA thread waits on live in the leader; the follower arrives on them through
+// the cluster's shared-memory window, and the leader forwards "slot free" and
+// "accumulator ready" to the follower the same way.
+//
 // Warp roles (448 threads): warp 0 TMA producer, warp 1 MMA issuer + TMEM
 // owner, warps 2-5 epilogue (one per TMEM lane quarter), warps 6-13 NF4
 // dequantisation.  One CTA per SM.
@@ -84,14 +94,15 @@ struct TensorMaps {
   CUtensorMap cb[2];
 };
 
-template <int BN, int MH>
+template <int BN, int MH, bool TWO>
 struct SmemLayout {
-  static constexpr int kStages = (MH == 1) ? 4 : 3;
   static constexpr int kBM = MH * kHM;
+  static constexpr int kBNL = TWO ? BN / 2 : BN;  // B rows staged by this CTA
   static constexpr int kABytes = kBM * kBK * 2;
-  static constexpr int kBBytes = BN * kBK * 2;
-  static constexpr int kCodeBytes = 8192;  // 256 blocks x 32 bytes
+  static constexpr int kBBytes = kBNL * kBK * 2;
+  static constexpr int kCodeBytes = 8192;  // up to 256 blocks x 32 bytes
   static constexpr int kStageBytes = kABytes + kBBytes + kCodeBytes;
+  static constexpr int kStages = (225 * 1024 / kStageBytes) < 6 ? (225 * 1024 / kStageBytes) : 6;
   static constexpr int kBarOffset = kStages * kStageBytes;
   // full[S], empty[S], codes[S], tfull[2], tempty[2], drain
   static constexpr int kNumBars = 3 * kStages + 5;
@@ -99,8 +110,10 @@ struct SmemLayout {
   static constexpr int kTablesOffset = kMiscOffset + 16;
   static constexpr int kTotal = kTablesOffset + static_cast<int>(sizeof(Nf4Tables));
   static constexpr int kDynamicBytes = kTotal + 1024;  // slack for 1024-byte alignment
+  static_assert(kStages >= 3, "pipeline too shallow");
   static_assert(kDynamicBytes <= 232448, "exceeds the 227 KiB shared memory of one CTA");
-  static_assert(kBM * 32 <= kCodeBytes && BN * 32 <= kCodeBytes, "code tile too large");
+  static_assert(kBM * 32 <= kCodeBytes && kBNL * 32 <= kCodeBytes, "code tile too large");
+  static_assert(!TWO || BN == 256, "pairs run 256-wide tiles");
 };
 
 // Shared-memory matrix descriptor (tcgen05), 128-byte swizzle.
@@ -114,12 +127,12 @@ __device__ __forceinline__ uint64_t make_smem_desc(uint32_t saddr, bool mn_major
   return start | (lbo << 16) | (sbo << 32) | (1ull << 46) | (2ull << 61);
 }
 
-__device__ __forceinline__ uint32_t make_idesc(int bn, bool a_mn, bool b_mn) {
+__device__ __forceinline__ uint32_t make_idesc(int m, int bn, bool a_mn, bool b_mn) {
   return (1u << 4)                                  // D format fp32
          | (1u << 7) | (1u << 10)                   // A, B format bf16
          | (a_mn ? (1u << 15) : 0u) | (b_mn ? (1u << 16) : 0u)
          | (static_cast<uint32_t>(bn >> 3) << 17)   // N
-         | (static_cast<uint32_t>(kHM >> 4) << 24); // M
+         | (static_cast<uint32_t>(m >> 4) << 24);   // M (128, or 256 for a CTA pair)
 }
 
 // Work decomposition shared by all roles.
@@ -162,10 +175,12 @@ struct DeqTask {
   uint32_t sw;   // row index & 7 (swizzle key of the operand row)
 };
 
-template <int BN, int MH>
+// BN here is the number of B rows this CTA stages (half a tile in TWO mode) and
+// n_blk counts in units of it.
+template <int BN, int kBM, int kABytes>
 __device__ __forceinline__ DeqTask deq_plan(const GemmParams &p, int seg_idx, int kb_in_seg, int m_blk, int n_blk,
                                             int t) {
-  using L = SmemLayout<BN, MH>;
+
   DeqTask task;
   task.mode = 0;
   task.M = 0.0f;
@@ -176,10 +191,10 @@ __device__ __forceinline__ DeqTask deq_plan(const GemmParams &p, int seg_idx, in
   if (!a_nf4 && !b_nf4) return task;
   const int kind = a_nf4 ? sg.a_kind : sg.b_kind;
   const Nf4Src &src = a_nf4 ? sg.a_nf4 : sg.b_nf4;
-  const int rows_tile = a_nf4 ? L::kBM : BN;
+  const int rows_tile = a_nf4 ? kBM : BN;
   if (t >= rows_tile) return task;
-  const uint32_t base = a_nf4 ? 0u : static_cast<uint32_t>(L::kABytes);
-  const int mn0 = a_nf4 ? m_blk * L::kBM : n_blk * BN;
+  const uint32_t base = a_nf4 ? 0u : static_cast<uint32_t>(kABytes);
+  const int mn0 = a_nf4 ? m_blk * kBM : n_blk * BN;
   const int k0 = kb_in_seg * kBK;
   int row, col0, r8;
   if (kind == OP_NF4_K) {
@@ -255,12 +270,13 @@ __device__ __forceinline__ void deq_store(const DeqTask &task, uint32_t stage_ba
 // ---------------------------------------------------------------------------
 // The kernel
 // ---------------------------------------------------------------------------
-template <int BN, int MH>
+template <int BN, int MH, bool TWO>
 __global__ void __launch_bounds__(kNumThreads, 1)
 loqt_gemm_kernel(const __grid_constant__ TensorMaps maps, const GemmParams p) {
-  using L = SmemLayout<BN, MH>;
+  using L = SmemLayout<BN, MH, TWO>;
   constexpr int kStages = L::kStages;
   constexpr int kBM = L::kBM;
+  constexpr int kBNL = L::kBNL;
   constexpr int kAccBufs = (MH == 1) ? 2 : 1;  // TMEM accumulator buffers (each MH * BN columns)
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -281,22 +297,31 @@ loqt_gemm_kernel(const __grid_constant__ TensorMaps maps, const GemmParams p) {
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
   const Sched sched(p, kBM, BN);
+  // TWO: rank 0 of the pair is the leader (issues the MMAs, owns the barriers the
+  // MMA thread waits on); `peer` is the other CTA's rank.
+  const uint32_t rank = TWO ? ptx::cluster_ctarank() : 0u;
+  const uint32_t peer = rank ^ 1u;
+  const bool leader = (rank == 0);
   // In the merge kernel (128-row tiles) only four dequant warps have rows to
   // stage; the other four (warps 10-13, TMEM lane quarters 2,3,0,1) join the
   // requantising epilogue and take every second 64-column block.
-  const bool helpers = (MH == 1) && (p.epi == EPI_REQUANT);
+  const bool helpers = !TWO && (MH == 1) && (p.epi == EPI_REQUANT);
   const int epi_groups = helpers ? 2 : 1;
+  // dequant warps with rows to stage: eight for a 256-row B tile, four for 128 rows
+  const int deq_warps = (helpers || kBNL == 128) ? kDeqWarps / 2 : kDeqWarps;
   constexpr uint32_t kTmemCols = 2 * BN;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) {
-      ptx::mbar_init(full_bar(s), 1 + (p.has_nf4 ? (helpers ? kDeqWarps / 2 : kDeqWarps) : 0));
+      // arrivals: the leader's TMA producer (which also posts the follower's bytes) and
+      // the dequant warps of every CTA of the pair
+      ptx::mbar_init(full_bar(s), 1 + (p.has_nf4 ? deq_warps * (TWO ? 2 : 1) : 0));
       ptx::mbar_init(empty_bar(s), 1);
       ptx::mbar_init(codes_bar(s), 1);
     }
     for (int a = 0; a < 2; ++a) {
       ptx::mbar_init(tfull_bar(a), 1);
-      ptx::mbar_init(tempty_bar(a), 4 * epi_groups);
+      ptx::mbar_init(tempty_bar(a), 4 * epi_groups * (TWO ? 2 : 1));
     }
     ptx::mbar_init(drain_bar, 1);
     *abort_flag = 0;
@@ -304,11 +329,17 @@ loqt_gemm_kernel(const __grid_constant__ TensorMaps maps, const GemmParams p) {
   }
   if (p.epi == EPI_REQUANT) nf4_tables_init(tables, threadIdx.x);
   if (warp == 1) {
-    ptx::tmem_alloc(smem_u32(const_cast<uint32_t *>(tmem_slot)), kTmemCols);
-    ptx::tmem_relinquish();
+    if (TWO) {
+      ptx::tmem_alloc_pair(smem_u32(const_cast<uint32_t *>(tmem_slot)), kTmemCols);
+      ptx::tmem_relinquish_pair();
+    } else {
+      ptx::tmem_alloc(smem_u32(const_cast<uint32_t *>(tmem_slot)), kTmemCols);
+      ptx::tmem_relinquish();
+    }
   }
   ptx::tc_fence_before();
   __syncthreads();
+  if (TWO) ptx::cluster_sync_all();  // both CTAs' barriers exist before anything arrives on them
   ptx::tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
@@ -324,27 +355,32 @@ loqt_gemm_kernel(const __grid_constant__ TensorMaps maps, const GemmParams p) {
       for (int u = blockIdx.x; ok && u < sched.units; u += gridDim.x) {
         int m_blk, n_blk, split, kb_lo, kb_hi;
         sched.unit(u, m_blk, n_blk, split, kb_lo, kb_hi);
+        // first B row staged by this CTA (the follower of a pair takes the upper half of the tile)
+        const int n_row0 = n_blk * BN + (TWO ? static_cast<int>(rank) * kBNL : 0);
         for (int kb = kb_lo; kb < kb_hi; ++kb, ++it) {
           const int s = it % kStages;
           const uint32_t ph = (it / kStages) & 1u;
-          if (!(ok = ptx::mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, p.status))) break;
+          if (!(ok = ptx::mbar_wait<TWO>(empty_bar(s), ph ^ 1u, abort_flag, p.status))) break;
+          // the MMA thread frees a slot on the leader's barrier; pass it on
+          // (only real releases: the first pass over the ring waits for nothing)
+          if (TWO && leader && it >= static_cast<uint32_t>(kStages)) ptx::mbar_arrive_cluster(ptx::map_to_cta(empty_bar(s), peer));
           const int sidx = kb < sched.kb_seg0 ? 0 : 1;
           const int k0 = (sidx == 0 ? kb : kb - sched.kb_seg0) * kBK;
           const Segment &sg = p.seg[sidx];
           const uint32_t a_dst = smem_base + s * L::kStageBytes;
           const uint32_t b_dst = a_dst + L::kABytes;
           const uint32_t c_dst = b_dst + L::kBBytes;
-          // packed codes of the stage's NF4 operand (if any) -> code tile
+          // packed codes of the stage's NF4 operand (if any) -> this CTA's code tile
           if (p.has_nf4) {
             if (sg.a_kind == OP_NF4_K) {
               ptx::mbar_arrive_expect_tx(codes_bar(s), kBM * 32);
               ptx::tma_load_2d(c_dst, &maps.ca[sidx], codes_bar(s), k0 >> 1, m_blk * kBM);
             } else if (sg.b_kind == OP_NF4_K) {
-              ptx::mbar_arrive_expect_tx(codes_bar(s), BN * 32);
-              ptx::tma_load_2d(c_dst, &maps.cb[sidx], codes_bar(s), k0 >> 1, n_blk * BN);
+              ptx::mbar_arrive_expect_tx(codes_bar(s), kBNL * 32);
+              ptx::tma_load_2d(c_dst, &maps.cb[sidx], codes_bar(s), k0 >> 1, n_row0);
             } else if (sg.b_kind == OP_NF4_MN) {
-              ptx::mbar_arrive_expect_tx(codes_bar(s), BN * 32);
-              ptx::tma_load_2d(c_dst, &maps.cb[sidx], codes_bar(s), (n_blk * BN) >> 1, k0);
+              ptx::mbar_arrive_expect_tx(codes_bar(s), kBNL * 32);
+              ptx::tma_load_2d(c_dst, &maps.cb[sidx], codes_bar(s), n_row0 >> 1, k0);
             } else {
               ptx::mbar_arrive(codes_bar(s));  // nothing to dequantise in this stage
             }
@@ -352,20 +388,25 @@ loqt_gemm_kernel(const __grid_constant__ TensorMaps maps, const GemmParams p) {
           uint32_t bytes = 0;
           if (sg.a_kind <= OP_TMA_MN) bytes += L::kABytes;
           if (sg.b_kind <= OP_TMA_MN) bytes += L::kBBytes;
-          ptx::mbar_arrive_expect_tx(full_bar(s), bytes);
+          // the pair's full barrier lives in the leader, which expects both CTAs' bytes
+          const uint32_t fbar = TWO ? ptx::map_to_cta(full_bar(s), 0) : full_bar(s);
+          if (!TWO) ptx::mbar_arrive_expect_tx(fbar, bytes);
+          else if (leader) ptx::mbar_arrive_expect_tx(full_bar(s), 2 * bytes);
+          auto load = [&](uint32_t dst, const CUtensorMap *m, int c0, int c1) {
+            if (TWO) ptx::tma_load_2d_pair(dst, m, fbar, c0, c1);
+            else ptx::tma_load_2d(dst, m, fbar, c0, c1);
+          };
           if (sg.a_kind == OP_TMA_K) {
-            ptx::tma_load_2d(a_dst, &maps.a[sidx], full_bar(s), k0, m_blk * kBM);
+            load(a_dst, &maps.a[sidx], k0, m_blk * kBM);
           } else if (sg.a_kind == OP_TMA_MN) {
 #pragma unroll
-            for (int j = 0; j < kBM / 64; ++j)
-              ptx::tma_load_2d(a_dst + j * 8192, &maps.a[sidx], full_bar(s), m_blk * kBM + 64 * j, k0);
+            for (int j = 0; j < kBM / 64; ++j) load(a_dst + j * 8192, &maps.a[sidx], m_blk * kBM + 64 * j, k0);
           }
           if (sg.b_kind == OP_TMA_K) {
-            ptx::tma_load_2d(b_dst, &maps.b[sidx], full_bar(s), k0, n_blk * BN);
+            load(b_dst, &maps.b[sidx], k0, n_row0);
           } else if (sg.b_kind == OP_TMA_MN) {
 #pragma unroll
-            for (int j = 0; j < BN / 64; ++j)
-              ptx::tma_load_2d(b_dst + j * 8192, &maps.b[sidx], full_bar(s), n_blk * BN + 64 * j, k0);
+            for (int j = 0; j < kBNL / 64; ++j) load(b_dst + j * 8192, &maps.b[sidx], n_row0 + 64 * j, k0);
           }
         }
       }
@@ -380,7 +421,7 @@ loqt_gemm_kernel(const __grid_constant__ TensorMaps maps, const GemmParams p) {
   }
   // =========================================================== MMA issuer
   else if (warp == 1) {
-    if (lane == 0) {
+    if (lane == 0 && leader) {
       uint32_t it = 0, tile = 0;
       bool ok = true;
       for (int u = blockIdx.x; ok && u < sched.units; u += gridDim.x, ++tile) {
@@ -388,18 +429,18 @@ loqt_gemm_kernel(const __grid_constant__ TensorMaps maps, const GemmParams p) {
         sched.unit(u, m_blk, n_blk, split, kb_lo, kb_hi);
         const uint32_t acc = tile % kAccBufs;
         const uint32_t acc_ph = (tile / kAccBufs) & 1u;
-        if (!(ok = ptx::mbar_wait(tempty_bar(acc), acc_ph ^ 1u, abort_flag, p.status))) break;
+        if (!(ok = ptx::mbar_wait<TWO>(tempty_bar(acc), acc_ph ^ 1u, abort_flag, p.status))) break;
         ptx::tc_fence_after();
         const uint32_t d_tmem = tmem_base + acc * (MH * BN);
         for (int kb = kb_lo; kb < kb_hi; ++kb, ++it) {
           const int s = it % kStages;
           const uint32_t ph = (it / kStages) & 1u;
-          if (!(ok = ptx::mbar_wait(full_bar(s), ph, abort_flag, p.status))) break;
+          if (!(ok = ptx::mbar_wait<TWO>(full_bar(s), ph, abort_flag, p.status))) break;
           ptx::tc_fence_after();
           const Segment &sg = p.seg[kb < sched.kb_seg0 ? 0 : 1];
           const bool a_mn = (sg.a_kind == OP_TMA_MN);
           const bool b_mn = (sg.b_kind == OP_TMA_MN) || (sg.b_kind == OP_NF4_MN);
-          const uint32_t idesc = make_idesc(BN, a_mn, b_mn);
+          const uint32_t idesc = make_idesc(TWO ? 2 * kHM : kHM, BN, a_mn, b_mn);
           const uint32_t a_addr = smem_base + s * L::kStageBytes;
           const uint32_t b_addr = a_addr + L::kABytes;
           const uint64_t b_desc = make_smem_desc(b_addr, b_mn);
@@ -410,17 +451,25 @@ loqt_gemm_kernel(const __grid_constant__ TensorMaps maps, const GemmParams p) {
             // half h: rows 128 h .. 128 h + 127 of the A tile (16 KiB further in either layout)
             const uint64_t a_desc = make_smem_desc(a_addr + h * (kHM * kBK * 2), a_mn);
 #pragma unroll
-            for (uint32_t k = 0; k < kBK / kUmmaK; ++k)
-              ptx::mma_bf16_ss(d_tmem + h * BN, a_desc + k * a_step, b_desc + k * b_step, idesc,
-                               (kb > kb_lo || k > 0) ? 1u : 0u);
+            for (uint32_t k = 0; k < kBK / kUmmaK; ++k) {
+              const uint32_t accum = (kb > kb_lo || k > 0) ? 1u : 0u;
+              if (TWO) ptx::mma_bf16_ss_pair(d_tmem + h * BN, a_desc + k * a_step, b_desc + k * b_step, idesc, accum);
+              else ptx::mma_bf16_ss(d_tmem + h * BN, a_desc + k * a_step, b_desc + k * b_step, idesc, accum);
+            }
           }
-          ptx::mma_commit(empty_bar(s));  // stage reusable once these MMAs have read it
+          // stage reusable (in both CTAs) once these MMAs have read it
+          if (TWO) ptx::mma_commit_pair(empty_bar(s));
+          else ptx::mma_commit(empty_bar(s));
         }
-        if (ok) ptx::mma_commit(tfull_bar(acc));
+        if (ok) {
+          if (TWO) ptx::mma_commit_pair(tfull_bar(acc));
+          else ptx::mma_commit(tfull_bar(acc));
+        }
       }
       // Every MMA issued above must have finished before TMEM is freed.
-      ptx::mma_commit(drain_bar);
-      ptx::mbar_wait(drain_bar, 0, abort_flag, p.status);
+      if (TWO) ptx::mma_commit_pair(drain_bar);
+      else ptx::mma_commit(drain_bar);
+      ptx::mbar_wait<TWO>(drain_bar, 0, abort_flag, p.status);
     }
   }
   // =========================================================== epilogue
@@ -434,7 +483,9 @@ loqt_gemm_kernel(const __grid_constant__ TensorMaps maps, const GemmParams p) {
       sched.unit(u, m_blk, n_blk, split, kb_lo, kb_hi);
       const uint32_t acc = tile % kAccBufs;
       const uint32_t acc_ph = (tile / kAccBufs) & 1u;
-      if (!(ok = ptx::mbar_wait(tfull_bar(acc), acc_ph, abort_flag, p.status))) break;
+      if (!(ok = ptx::mbar_wait<TWO>(tfull_bar(acc), acc_ph, abort_flag, p.status))) break;
+      // the MMA thread signals the leader's barrier; one leader warp passes it on
+      if (TWO && leader && warp == kEpiWarp0 && lane == 0) ptx::mbar_arrive_cluster(ptx::map_to_cta(tfull_bar(acc), peer));
       ptx::tc_fence_after();
       const int n_base = n_blk * BN;
 #pragma unroll 1
@@ -546,12 +597,15 @@ loqt_gemm_kernel(const __grid_constant__ TensorMaps maps, const GemmParams p) {
       // Accumulator fully read: hand the TMEM buffer back to the MMA warp.
       ptx::tc_fence_before();
       __syncwarp();
-      if (lane == 0) ptx::mbar_arrive(tempty_bar(acc));
+      if (lane == 0) {
+        if (TWO && !leader) ptx::mbar_arrive_cluster(ptx::map_to_cta(tempty_bar(acc), 0));
+        else ptx::mbar_arrive(tempty_bar(acc));
+      }
     }
   }
   // =========================================================== NF4 dequant
   else {
-    if (p.has_nf4) {
+    if (p.has_nf4 && warp < kDeqWarp0 + deq_warps) {
       const int t = threadIdx.x - kDeqWarp0 * 32;
       // Position of the k-block being staged and of the one whose scale is fetched ahead.
       int u = blockIdx.x, kb = 0, kb_hi = 0, m_blk = 0, n_blk = 0, split = 0;
@@ -568,7 +622,8 @@ loqt_gemm_kernel(const __grid_constant__ TensorMaps maps, const GemmParams p) {
       auto plan = [&]() {
         const int sidx = kb < sched.kb_seg0 ? 0 : 1;
         const int kb_in = sidx == 0 ? kb : kb - sched.kb_seg0;
-        return deq_plan<BN, MH>(p, sidx, kb_in, m_blk, n_blk, t);
+        // this CTA's B rows start at local block (TWO: 2 n_blk + rank) of kBNL rows
+        return deq_plan<kBNL, kBM, L::kABytes>(p, sidx, kb_in, m_blk, TWO ? 2 * n_blk + static_cast<int>(rank) : n_blk, t);
       };
       uint32_t it = 0;
       DeqTask next;
@@ -590,9 +645,13 @@ loqt_gemm_kernel(const __grid_constant__ TensorMaps maps, const GemmParams p) {
         if (!(ok = ptx::mbar_wait(codes_bar(s), ph, abort_flag, p.status))) break;
         const uint32_t stage_base = smem_base + s * L::kStageBytes;
         deq_store(cur, stage_base, stage_base + L::kABytes + L::kBBytes);
-        ptx::fence_proxy_async_smem();
+        if (TWO) ptx::fence_proxy_async_all();
+        else ptx::fence_proxy_async_smem();
         __syncwarp();
-        if (lane == 0) ptx::mbar_arrive(full_bar(s));
+        if (lane == 0) {
+          if (TWO && !leader) ptx::mbar_arrive_cluster(ptx::map_to_cta(full_bar(s), 0));
+          else ptx::mbar_arrive(full_bar(s));
+        }
         ++it;
       }
     }
@@ -601,9 +660,13 @@ loqt_gemm_kernel(const __grid_constant__ TensorMaps maps, const GemmParams p) {
   // =========================================================== teardown
   ptx::tc_fence_before();
   __syncthreads();
+  // neither CTA of a pair may free TMEM or leave while the other still uses the
+  // pair's barriers, its shared memory (MMA operands) or its accumulators
+  if (TWO) ptx::cluster_sync_all();
   if (warp == 1) {
     ptx::tc_fence_after();
-    ptx::tmem_dealloc(tmem_base, kTmemCols);
+    if (TWO) ptx::tmem_dealloc_pair(tmem_base, kTmemCols);
+    else ptx::tmem_dealloc(tmem_base, kTmemCols);
   }
 }
 

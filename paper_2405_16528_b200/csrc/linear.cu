@@ -91,9 +91,10 @@ constexpr double kCyclesDequantRow = 3.3;
 constexpr double kCyclesEpilogueRow = 400.0;
 constexpr double kCyclesFixed = 3000.0;
 
-template <int BN, int MH>
+template <int BN, int MH, bool TWO>
 static loqt_status launch_cfg(const GemmCall &c, cudaStream_t stream) {
-  using L = SmemLayout<BN, MH>;
+  using L = SmemLayout<BN, MH, TWO>;
+  constexpr int BNL = L::kBNL;  // B rows one CTA stages
   TensorMaps maps;
   memset(&maps, 0, sizeof(maps));
   for (int s = 0; s < c.p.num_segs; ++s) {
@@ -106,24 +107,40 @@ static loqt_status launch_cfg(const GemmCall &c, cudaStream_t stream) {
       return LOQT_ERR_UNSUPPORTED;
     }
     if (sg.b_kind <= OP_TMA_MN) {
-      if (!map_operand(&maps.b[s], sg.b_kind, c.b[s], c.p.N, sg.K, BN)) return LOQT_ERR_CUDA;
+      if (!map_operand(&maps.b[s], sg.b_kind, c.b[s], c.p.N, sg.K, BNL)) return LOQT_ERR_CUDA;
     } else if (sg.b_kind == OP_NF4_K) {
-      if (!make_code_map(&maps.cb[s], sg.b_nf4, 32, BN, CU_TENSOR_MAP_SWIZZLE_NONE)) return LOQT_ERR_CUDA;
+      if (!make_code_map(&maps.cb[s], sg.b_nf4, 32, BNL, CU_TENSOR_MAP_SWIZZLE_NONE)) return LOQT_ERR_CUDA;
     } else {
-      if (!make_code_map(&maps.cb[s], sg.b_nf4, BN / 2, kBK,
-                         BN == 256 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B))
+      if (!make_code_map(&maps.cb[s], sg.b_nf4, BNL / 2, kBK,
+                         BNL == 256 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B))
         return LOQT_ERR_CUDA;
     }
   }
-  if (cudaFuncSetAttribute(loqt_gemm_kernel<BN, MH>, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kDynamicBytes) !=
-      cudaSuccess)
+  auto kernel = loqt_gemm_kernel<BN, MH, TWO>;
+  if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kDynamicBytes) != cudaSuccess)
     return LOQT_ERR_CUDA;
   const int mt = (c.p.M + L::kBM - 1) / L::kBM, nt = (c.p.N + BN - 1) / BN;
   const int units = mt * nt * c.p.splits;
-  const int grid = units < sm_count() ? units : sm_count();
-  loqt_gemm_kernel<BN, MH><<<grid, kNumThreads, L::kDynamicBytes, stream>>>(maps, c.p);
+  int grid = units < sm_count() ? units : sm_count();
+  cudaLaunchConfig_t cfg;
+  memset(&cfg, 0, sizeof(cfg));
+  cudaLaunchAttribute attr[1];
+  if (TWO) {
+    grid &= ~1;  // whole pairs (`units` is even in this mode)
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+  }
+  cfg.gridDim = dim3(grid);
+  cfg.blockDim = dim3(kNumThreads);
+  cfg.dynamicSmemBytes = L::kDynamicBytes;
+  cfg.stream = stream;
+  const cudaError_t err = cudaLaunchKernelEx(&cfg, kernel, maps, c.p);
   count_launch();
-  return cudaGetLastError() == cudaSuccess ? LOQT_OK : LOQT_ERR_CUDA;
+  return (err == cudaSuccess && cudaGetLastError() == cudaSuccess) ? LOQT_OK : LOQT_ERR_CUDA;
 }
 
 // Tile selection.  Candidates: BN in {256, 128}, rows per CTA 128 (two TMEM
@@ -168,8 +185,15 @@ static loqt_status launch(GemmCall &c, cudaStream_t stream) {
   for (int s = 0; s < c.p.num_segs; ++s)
     if (c.p.seg[s].a_kind >= OP_NF4_K || c.p.seg[s].b_kind >= OP_NF4_K) c.p.has_nf4 = 1;
   const TileCfg t = pick_tile(c);
-  if (t.bn == 256) return t.mh == 2 ? launch_cfg<256, 2>(c, stream) : launch_cfg<256, 1>(c, stream);
-  return t.mh == 2 ? launch_cfg<128, 2>(c, stream) : launch_cfg<128, 1>(c, stream);
+  // Two CTAs on neighbouring M tiles can run as a tcgen05 pair when tiles pair up
+  // exactly: 256-wide tiles, an even number of M tiles (so both CTAs of a pair
+  // have the same N tile), no split-K, and not the merge (its epilogue wants all
+  // twelve worker warps of a CTA).
+  const int mt = (c.p.M + t.mh * kHM - 1) / (t.mh * kHM);
+  const bool two = t.bn == 256 && (mt % 2 == 0) && c.p.splits == 1 && c.p.epi != EPI_REQUANT;
+  if (two) return t.mh == 2 ? launch_cfg<256, 2, true>(c, stream) : launch_cfg<256, 1, true>(c, stream);
+  if (t.bn == 256) return t.mh == 2 ? launch_cfg<256, 2, false>(c, stream) : launch_cfg<256, 1, false>(c, stream);
+  return t.mh == 2 ? launch_cfg<128, 2, false>(c, stream) : launch_cfg<128, 1, false>(c, stream);
 }
 
 // ---------------------------------------------------------------------------
