@@ -163,79 +163,91 @@ struct Sched {
   }
 };
 
-// What one dequant thread does for one stage: where its 32 bytes of codes sit in
-// the stage's code tile, where its 128-byte operand row goes, and the block
-// scale (fetched from global memory one stage ahead).
+// What one dequant thread does, fixed for as long as it stays in the same tile
+// and K segment: where its 32 bytes of codes sit in a code tile, where its
+// 128-byte operand row goes, and where its block scales come from.
+struct DeqGeom {
+  uint32_t src, src2;  // byte offsets of the two 16-byte code chunks inside the code tile
+  uint32_t dst;        // byte offset of the 128-byte operand row inside the stage
+  uint32_t sw;         // row index & 7 (swizzle key of the operand row)
+  int active;          // 0: this thread has no row inside the matrix (outputs it would feed are discarded)
+  const float *mptr;   // block scale of k-block 0 of the segment
+  int mstride;         // floats between consecutive k-blocks
+  int kb_valid;        // k-blocks of the segment for which the row exists; later ones are the K tail (zeros)
+};
+
+// The per-stage part: the scale, fetched from global memory one stage ahead.
 struct DeqTask {
   float M;
-  int mode;      // 0: nothing to do, 1: dequantise, 2: write zeros
-  uint32_t src;  // byte offsets of the two 16-byte code chunks inside the code tile
-  uint32_t src2;
-  uint32_t dst;  // byte offset of the 128-byte operand row inside the stage
-  uint32_t sw;   // row index & 7 (swizzle key of the operand row)
+  int mode;  // 0: nothing to do, 1: dequantise, 2: write zeros
 };
 
 // BN here is the number of B rows this CTA stages (half a tile in TWO mode) and
 // n_blk counts in units of it.
 template <int BN, int kBM, int kABytes>
-__device__ __forceinline__ DeqTask deq_plan(const GemmParams &p, int seg_idx, int kb_in_seg, int m_blk, int n_blk,
-                                            int t) {
-
-  DeqTask task;
-  task.mode = 0;
-  task.M = 0.0f;
-  task.src = task.src2 = task.dst = task.sw = 0;
+__device__ __forceinline__ DeqGeom deq_geom(const GemmParams &p, int seg_idx, int m_blk, int n_blk, int t) {
+  DeqGeom g;
+  g.src = g.src2 = g.dst = g.sw = 0;
+  g.active = 0;
+  g.mptr = nullptr;
+  g.mstride = 0;
+  g.kb_valid = 0;
   const Segment &sg = p.seg[seg_idx];
   const bool a_nf4 = sg.a_kind >= OP_NF4_K;
   const bool b_nf4 = sg.b_kind >= OP_NF4_K;
-  if (!a_nf4 && !b_nf4) return task;
+  if (!a_nf4 && !b_nf4) return g;
   const int kind = a_nf4 ? sg.a_kind : sg.b_kind;
   const Nf4Src &src = a_nf4 ? sg.a_nf4 : sg.b_nf4;
   const int rows_tile = a_nf4 ? kBM : BN;
-  if (t >= rows_tile) return task;
+  if (t >= rows_tile) return g;
   const uint32_t base = a_nf4 ? 0u : static_cast<uint32_t>(kABytes);
   const int mn0 = a_nf4 ? m_blk * kBM : n_blk * BN;
-  const int k0 = kb_in_seg * kBK;
-  int row, col0, r8;
+  const int nb = src.ld >> 6;
   if (kind == OP_NF4_K) {
-    // tile row t <- matrix row mn0 + t, codes k0 .. k0+63; code tile is [rows][32 B]
-    row = mn0 + t;
-    col0 = k0;
-    r8 = t & 7;
-    task.dst = base + static_cast<uint32_t>((t >> 3) * 1024 + r8 * 128);
-    task.src = static_cast<uint32_t>(t * 32);
-    task.src2 = task.src + 16;
-    if (row >= src.rows) return task;  // feeds only discarded outputs
+    // tile row t <- matrix row mn0 + t, codes of one k-block; code tile is [rows][32 B]
+    const int row = mn0 + t;
+    g.sw = static_cast<uint32_t>(t & 7);
+    g.dst = base + static_cast<uint32_t>((t >> 3) * 1024 + (t & 7) * 128);
+    g.src = static_cast<uint32_t>(t * 32);
+    g.src2 = g.src + 16;
+    if (row >= src.rows) return g;
+    g.active = 1;
+    g.mptr = src.absmax + static_cast<int64_t>(row) * nb;
+    g.mstride = 1;
+    g.kb_valid = 0x7fffffff;  // padded columns hold the zero level
   } else {
-    // 64-column chunk j, K-row kk <- matrix row k0 + kk, codes of columns mn0 + 64 j ..
+    // 64-column chunk j, K-row kk <- matrix row 64 kb + kk, codes of columns mn0 + 64 j ..
     // A warp takes 8 consecutive K-rows of every chunk, so that its operand-row
     // stores and its code-tile loads each touch 8 different swizzle positions.
     constexpr int JB = BN / 64;
     constexpr int jbits = (JB == 4) ? 2 : 1;
     const int j = (t >> 3) & (JB - 1);
     const int kk = (t & 7) | ((t >> (3 + jbits)) << 3);
-    row = k0 + kk;
-    col0 = mn0 + 64 * j;
-    r8 = kk & 7;
-    task.dst = base + static_cast<uint32_t>(j * 8192 + (kk >> 3) * 1024 + r8 * 128);
+    const int col0 = mn0 + 64 * j;
+    g.sw = static_cast<uint32_t>(kk & 7);
+    g.dst = base + static_cast<uint32_t>(j * 8192 + (kk >> 3) * 1024 + (kk & 7) * 128);
     // code tile is [64 K-rows][BN/2 bytes], TMA-swizzled (128 B rows: 128-byte
     // swizzle, 64 B rows: 64-byte swizzle): chunk ^= (offset >> 7) & mask
     constexpr uint32_t RB = BN / 2;
     constexpr uint32_t mask = (RB == 128) ? 7u : 3u;
     const uint32_t o0 = static_cast<uint32_t>(kk) * RB + static_cast<uint32_t>(j) * 32u;
     const uint32_t o1 = o0 + 16u;
-    task.src = o0 ^ (((o0 >> 7) & mask) << 4);
-    task.src2 = o1 ^ (((o1 >> 7) & mask) << 4);
-    if (col0 >= src.ld) return task;  // beyond the matrix: discarded outputs
-    if (row >= src.rows) {            // K tail: must contribute zero
-      task.mode = 2;
-      task.sw = static_cast<uint32_t>(r8);
-      return task;
-    }
+    g.src = o0 ^ (((o0 >> 7) & mask) << 4);
+    g.src2 = o1 ^ (((o1 >> 7) & mask) << 4);
+    if (col0 >= src.ld) return g;
+    g.active = 1;
+    g.mptr = src.absmax + static_cast<int64_t>(kk) * nb + (col0 >> 6);
+    g.mstride = 64 * nb;
+    g.kb_valid = src.rows > kk ? (src.rows - kk + 63) >> 6 : 0;  // beyond: the K tail must contribute zero
   }
-  task.sw = static_cast<uint32_t>(r8);
-  task.mode = 1;
-  task.M = __ldg(src.absmax + static_cast<int64_t>(row) * (src.ld >> 6) + (col0 >> 6));
+  return g;
+}
+
+__device__ __forceinline__ DeqTask deq_fetch(const DeqGeom &g, int kb_in_seg) {
+  DeqTask task;
+  task.M = 0.0f;
+  task.mode = !g.active ? 0 : (kb_in_seg < g.kb_valid ? 1 : 2);
+  if (task.mode == 1) task.M = __ldg(g.mptr + static_cast<int64_t>(kb_in_seg) * g.mstride);
   return task;
 }
 
@@ -250,21 +262,22 @@ __device__ __forceinline__ uint4 ld_shared_v4(uint32_t addr) {
   return v;
 }
 
-__device__ __forceinline__ void deq_store(const DeqTask &task, uint32_t stage_base, uint32_t code_base) {
+__device__ __forceinline__ void deq_store(const DeqGeom &g, const DeqTask &task, uint32_t stage_base,
+                                          uint32_t code_base) {
   if (task.mode == 0) return;
-  const uint32_t dst = stage_base + task.dst;
+  const uint32_t dst = stage_base + g.dst;
   if (task.mode == 2) {
 #pragma unroll
-    for (uint32_t c = 0; c < 8; ++c) st_shared_v4(dst + ((c ^ task.sw) << 4), make_uint4(0, 0, 0, 0));
+    for (uint32_t c = 0; c < 8; ++c) st_shared_v4(dst + ((c ^ g.sw) << 4), make_uint4(0, 0, 0, 0));
     return;
   }
-  const uint4 c0 = ld_shared_v4(code_base + task.src);
-  const uint4 c1 = ld_shared_v4(code_base + task.src2);
+  const uint4 c0 = ld_shared_v4(code_base + g.src);
+  const uint4 c1 = ld_shared_v4(code_base + g.src2);
   Nf4BlockTable tab;
   nf4_block_table(task.M, tab);
   const uint32_t w[8] = {c0.x, c0.y, c0.z, c0.w, c1.x, c1.y, c1.z, c1.w};
 #pragma unroll
-  for (uint32_t c = 0; c < 8; ++c) st_shared_v4(dst + ((c ^ task.sw) << 4), nf4_dequant8(tab, w[c]));
+  for (uint32_t c = 0; c < 8; ++c) st_shared_v4(dst + ((c ^ g.sw) << 4), nf4_dequant8(tab, w[c]));
 }
 
 // ---------------------------------------------------------------------------
@@ -607,44 +620,63 @@ loqt_gemm_kernel(const __grid_constant__ TensorMaps maps, const GemmParams p) {
   else {
     if (p.has_nf4 && warp < kDeqWarp0 + deq_warps) {
       const int t = threadIdx.x - kDeqWarp0 * 32;
-      // Position of the k-block being staged and of the one whose scale is fetched ahead.
-      int u = blockIdx.x, kb = 0, kb_hi = 0, m_blk = 0, n_blk = 0, split = 0;
-      auto open_unit = [&]() {
-        while (u < sched.units) {
-          int lo;
-          sched.unit(u, m_blk, n_blk, split, lo, kb_hi);
-          kb = lo;
-          if (kb < kb_hi) return true;
-          u += gridDim.x;
+      // Two cursors over this CTA's k-blocks: the one being staged and, one step
+      // ahead, the one whose scale is being fetched.  A cursor recomputes its
+      // geometry only when it enters a new tile or K segment.
+      struct Cursor {
+        int u, kb, kb_hi, m_blk, n_blk, seg;
+        DeqGeom g;
+      };
+      auto enter = [&](Cursor &c) {  // c.kb valid: (re)compute segment and geometry
+        c.seg = c.kb < sched.kb_seg0 ? 0 : 1;
+        // this CTA's B rows start at local block (TWO: 2 n_blk + rank) of kBNL rows
+        c.g = deq_geom<kBNL, kBM, L::kABytes>(p, c.seg, c.m_blk, TWO ? 2 * c.n_blk + static_cast<int>(rank) : c.n_blk, t);
+      };
+      auto open = [&](Cursor &c) {
+        while (c.u < sched.units) {
+          int split, lo;
+          sched.unit(c.u, c.m_blk, c.n_blk, split, lo, c.kb_hi);
+          c.kb = lo;
+          if (c.kb < c.kb_hi) {
+            enter(c);
+            return true;
+          }
+          c.u += gridDim.x;
         }
         return false;
       };
-      auto plan = [&]() {
-        const int sidx = kb < sched.kb_seg0 ? 0 : 1;
-        const int kb_in = sidx == 0 ? kb : kb - sched.kb_seg0;
-        // this CTA's B rows start at local block (TWO: 2 n_blk + rank) of kBNL rows
-        return deq_plan<kBNL, kBM, L::kABytes>(p, sidx, kb_in, m_blk, TWO ? 2 * n_blk + static_cast<int>(rank) : n_blk, t);
+      auto advance = [&](Cursor &c) {
+        if (++c.kb < c.kb_hi) {
+          if (c.kb == sched.kb_seg0) enter(c);  // crossed into the second segment
+          return true;
+        }
+        c.u += gridDim.x;
+        return open(c);
       };
+      auto fetch = [&](const Cursor &c) { return deq_fetch(c.g, c.seg == 0 ? c.kb : c.kb - sched.kb_seg0); };
+
+      Cursor cur, nxt;
+      cur.u = blockIdx.x;
+      bool have = open(cur);
+      DeqTask task;
+      task.mode = 0;
+      task.M = 0.0f;
+      if (have) task = fetch(cur);
+      nxt = cur;
+      bool have_next = have && advance(nxt);
       uint32_t it = 0;
-      DeqTask next;
-      next.mode = 0;
-      bool have = open_unit();
-      if (have) next = plan();
       bool ok = true;
       while (have && ok) {
-        const DeqTask cur = next;
-        ++kb;
-        if (kb >= kb_hi) {
-          u += gridDim.x;
-          have = open_unit();
-        }
-        if (have) next = plan();
+        DeqTask task_next;
+        task_next.mode = 0;
+        task_next.M = 0.0f;
+        if (have_next) task_next = fetch(nxt);  // in flight while this stage is dequantised
         const int s = it % kStages;
         const uint32_t ph = (it / kStages) & 1u;
         // The code tile landing implies the stage's previous contents were consumed.
         if (!(ok = ptx::mbar_wait(codes_bar(s), ph, abort_flag, p.status))) break;
         const uint32_t stage_base = smem_base + s * L::kStageBytes;
-        deq_store(cur, stage_base, stage_base + L::kABytes + L::kBBytes);
+        deq_store(cur.g, task, stage_base, stage_base + L::kABytes + L::kBBytes);
         if (TWO) ptx::fence_proxy_async_all();
         else ptx::fence_proxy_async_smem();
         __syncwarp();
@@ -653,6 +685,10 @@ loqt_gemm_kernel(const __grid_constant__ TensorMaps maps, const GemmParams p) {
           else ptx::mbar_arrive(full_bar(s));
         }
         ++it;
+        cur = nxt;
+        have = have_next;
+        task = task_next;
+        if (have_next) have_next = advance(nxt);
       }
     }
   }

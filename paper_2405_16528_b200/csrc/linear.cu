@@ -91,6 +91,12 @@ constexpr double kCyclesDequantRow = 3.3;
 constexpr double kCyclesEpilogueRow = 400.0;
 constexpr double kCyclesFixed = 3000.0;
 
+// Run eligible products as tcgen05 CTA pairs (cta_group::2).
+#ifndef LOQT_USE_PAIRS
+#define LOQT_USE_PAIRS 0
+#endif
+constexpr bool kUsePairs = LOQT_USE_PAIRS != 0;
+
 template <int BN, int MH, bool TWO>
 static loqt_status launch_cfg(const GemmCall &c, cudaStream_t stream) {
   using L = SmemLayout<BN, MH, TWO>;
@@ -190,7 +196,7 @@ static loqt_status launch(GemmCall &c, cudaStream_t stream) {
   // have the same N tile), no split-K, and not the merge (its epilogue wants all
   // twelve worker warps of a CTA).
   const int mt = (c.p.M + t.mh * kHM - 1) / (t.mh * kHM);
-  const bool two = t.bn == 256 && (mt % 2 == 0) && c.p.splits == 1 && c.p.epi != EPI_REQUANT;
+  const bool two = kUsePairs && t.bn == 256 && (mt % 2 == 0) && c.p.splits == 1 && c.p.epi != EPI_REQUANT;
   if (two) return t.mh == 2 ? launch_cfg<256, 2, true>(c, stream) : launch_cfg<256, 1, true>(c, stream);
   if (t.bn == 256) return t.mh == 2 ? launch_cfg<256, 2, false>(c, stream) : launch_cfg<256, 1, false>(c, stream);
   return t.mh == 2 ? launch_cfg<128, 2, false>(c, stream) : launch_cfg<128, 1, false>(c, stream);
