@@ -276,8 +276,10 @@ __device__ __forceinline__ void deq_store(const DeqGeom &g, const DeqTask &task,
   Nf4BlockTable tab;
   nf4_block_table(task.M, tab);
   const uint32_t w[8] = {c0.x, c0.y, c0.z, c0.w, c1.x, c1.y, c1.z, c1.w};
+  // the row is 128-byte aligned, so the swizzled chunk address is a pure XOR
+  const uint32_t dst_x = dst ^ (g.sw << 4);
 #pragma unroll
-  for (uint32_t c = 0; c < 8; ++c) st_shared_v4(dst + ((c ^ g.sw) << 4), nf4_dequant8(tab, w[c]));
+  for (uint32_t c = 0; c < 8; ++c) st_shared_v4(dst_x ^ (c << 4), nf4_dequant8(tab, w[c]));
 }
 
 // ---------------------------------------------------------------------------

@@ -69,24 +69,30 @@ LOQT_HD void nf4_block_table(float M, Nf4BlockTable &t) {
   }
 }
 
-// Four codes (nibbles 0..3 of `c`, higher bits ignored except as noted) ->
-// two registers of packed bf16: out01 = elements 0,1; out23 = elements 2,3.
-// `c4` must equal c << 4 in its low 16 bits (it supplies bit 3 of the even
-// codes as byte sign bits).
-LOQT_HD void nf4_lookup4(const Nf4BlockTable &t, uint32_t c, uint32_t c4, uint32_t &out01, uint32_t &out23) {
-  const uint32_t idx = c & 0x7777u;
-  const uint32_t upper = hd_prmt(c4, c, 0xD9C8u);  // byte e = 0xFF iff code e >= 8
-  const uint32_t lo = (hd_prmt(t.lo[0], t.lo[1], idx) & ~upper) | (hd_prmt(t.lo[2], t.lo[3], idx) & upper);
-  const uint32_t hi = (hd_prmt(t.hi[0], t.hi[1], idx) & ~upper) | (hd_prmt(t.hi[2], t.hi[3], idx) & upper);
-  out01 = hd_prmt(lo, hi, 0x5140u);
-  out23 = hd_prmt(lo, hi, 0x7362u);
-}
-
 // One code word (8 codes, element j in nibble j) -> 8 bf16 (16 bytes).
+// Codes 0..3 use the selector's low half directly; codes 4..7 the same word
+// shifted down.  Bit 3 of every code is turned into a byte mask by a permute in
+// sign-replication mode: the sign bits of bytes 0..3 of w hold bit 3 of the odd
+// codes, those of w << 4 bit 3 of the even codes.
 LOQT_HD uint4 nf4_dequant8(const Nf4BlockTable &t, uint32_t w) {
+  const uint32_t w4 = w << 4;
+  const uint32_t idx = w & 0x77777777u;  // 3-bit table indices; a permute reads the low 16 bits of its selector
+  const uint32_t idxh = idx >> 16;
+  const uint32_t up_l = hd_prmt(w4, w, 0xD9C8u);  // byte e = 0xFF iff code e >= 8       (e = 0..3)
+  const uint32_t up_h = hd_prmt(w4, w, 0xFBEAu);  // byte e = 0xFF iff code 4 + e >= 8
   uint4 o;
-  nf4_lookup4(t, w, w << 4, o.x, o.y);
-  nf4_lookup4(t, w >> 16, w >> 12, o.z, o.w);
+  {
+    const uint32_t lo = (hd_prmt(t.lo[0], t.lo[1], idx) & ~up_l) | (hd_prmt(t.lo[2], t.lo[3], idx) & up_l);
+    const uint32_t hi = (hd_prmt(t.hi[0], t.hi[1], idx) & ~up_l) | (hd_prmt(t.hi[2], t.hi[3], idx) & up_l);
+    o.x = hd_prmt(lo, hi, 0x5140u);
+    o.y = hd_prmt(lo, hi, 0x7362u);
+  }
+  {
+    const uint32_t lo = (hd_prmt(t.lo[0], t.lo[1], idxh) & ~up_h) | (hd_prmt(t.lo[2], t.lo[3], idxh) & up_h);
+    const uint32_t hi = (hd_prmt(t.hi[0], t.hi[1], idxh) & ~up_h) | (hd_prmt(t.hi[2], t.hi[3], idxh) & up_h);
+    o.z = hd_prmt(lo, hi, 0x5140u);
+    o.w = hd_prmt(lo, hi, 0x7362u);
+  }
   return o;
 }
 
