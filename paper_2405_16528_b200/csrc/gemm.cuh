@@ -174,6 +174,11 @@ struct DeqGeom {
   const float *mptr;   // block scale of k-block 0 of the segment
   int mstride;         // floats between consecutive k-blocks
   int kb_valid;        // k-blocks of the segment for which the row exists; later ones are the K tail (zeros)
+  // A thread of a 256-row tile owns a second block, 128 tasks further on: the same
+  // geometry shifted by constant offsets.
+  int active2, kb_valid2;
+  uint32_t d2, s2;     // byte offsets added to dst / src, src2
+  int m2;              // floats added to mptr
 };
 
 // The per-stage part: the scale, fetched from global memory one stage ahead.
@@ -192,6 +197,9 @@ __device__ __forceinline__ DeqGeom deq_geom(const GemmParams &p, int seg_idx, in
   g.mptr = nullptr;
   g.mstride = 0;
   g.kb_valid = 0;
+  g.active2 = g.kb_valid2 = 0;
+  g.d2 = g.s2 = 0;
+  g.m2 = 0;
   const Segment &sg = p.seg[seg_idx];
   const bool a_nf4 = sg.a_kind >= OP_NF4_K;
   const bool b_nf4 = sg.b_kind >= OP_NF4_K;
@@ -215,6 +223,12 @@ __device__ __forceinline__ DeqGeom deq_geom(const GemmParams &p, int seg_idx, in
     g.mptr = src.absmax + static_cast<int64_t>(row) * nb;
     g.mstride = 1;
     g.kb_valid = 0x7fffffff;  // padded columns hold the zero level
+    // second block: tile row t + 128
+    g.active2 = (t + 128 < rows_tile) && (row + 128 < src.rows);
+    g.kb_valid2 = g.kb_valid;
+    g.d2 = 128u * 128u;
+    g.s2 = 128u * 32u;
+    g.m2 = 128 * nb;
   } else {
     // 64-column chunk j, K-row kk <- matrix row 64 kb + kk, codes of columns mn0 + 64 j ..
     // A warp takes 8 consecutive K-rows of every chunk, so that its operand-row
@@ -239,15 +253,24 @@ __device__ __forceinline__ DeqGeom deq_geom(const GemmParams &p, int seg_idx, in
     g.mptr = src.absmax + static_cast<int64_t>(kk) * nb + (col0 >> 6);
     g.mstride = 64 * nb;
     g.kb_valid = src.rows > kk ? (src.rows - kk + 63) >> 6 : 0;  // beyond: the K tail must contribute zero
+    // second block (256-row tiles only): same chunk, K-row kk + 32
+    g.active2 = (BN == 256);
+    g.kb_valid2 = src.rows > kk + 32 ? (src.rows - kk - 32 + 63) >> 6 : 0;
+    g.d2 = 4u * 1024u;
+    g.s2 = 32u * RB;
+    g.m2 = 32 * nb;
   }
   return g;
 }
 
+template <int kSecond>
 __device__ __forceinline__ DeqTask deq_fetch(const DeqGeom &g, int kb_in_seg) {
   DeqTask task;
   task.M = 0.0f;
-  task.mode = !g.active ? 0 : (kb_in_seg < g.kb_valid ? 1 : 2);
-  if (task.mode == 1) task.M = __ldg(g.mptr + static_cast<int64_t>(kb_in_seg) * g.mstride);
+  const int active = kSecond ? g.active2 : g.active;
+  const int valid = kSecond ? g.kb_valid2 : g.kb_valid;
+  task.mode = !active ? 0 : (kb_in_seg < valid ? 1 : 2);
+  if (task.mode == 1) task.M = __ldg(g.mptr + static_cast<int64_t>(kb_in_seg) * g.mstride + (kSecond ? g.m2 : 0));
   return task;
 }
 
@@ -262,17 +285,18 @@ __device__ __forceinline__ uint4 ld_shared_v4(uint32_t addr) {
   return v;
 }
 
+template <int kSecond>
 __device__ __forceinline__ void deq_store(const DeqGeom &g, const DeqTask &task, uint32_t stage_base,
                                           uint32_t code_base) {
   if (task.mode == 0) return;
-  const uint32_t dst = stage_base + g.dst;
+  const uint32_t dst = stage_base + g.dst + (kSecond ? g.d2 : 0u);
   if (task.mode == 2) {
 #pragma unroll
     for (uint32_t c = 0; c < 8; ++c) st_shared_v4(dst + ((c ^ g.sw) << 4), make_uint4(0, 0, 0, 0));
     return;
   }
-  const uint4 c0 = ld_shared_v4(code_base + g.src);
-  const uint4 c1 = ld_shared_v4(code_base + g.src2);
+  const uint4 c0 = ld_shared_v4(code_base + g.src + (kSecond ? g.s2 : 0u));
+  const uint4 c1 = ld_shared_v4(code_base + g.src2 + (kSecond ? g.s2 : 0u));
   Nf4BlockTable tab;
   nf4_block_table(task.M, tab);
   const uint32_t w[8] = {c0.x, c0.y, c0.z, c0.w, c1.x, c1.y, c1.z, c1.w};
@@ -322,15 +346,20 @@ loqt_gemm_kernel(const __grid_constant__ TensorMaps maps, const GemmParams p) {
   // requantising epilogue and take every second 64-column block.
   const bool helpers = !TWO && (MH == 1) && (p.epi == EPI_REQUANT);
   const int epi_groups = helpers ? 2 : 1;
-  // dequant warps with rows to stage: eight for a 256-row B tile, four for 128 rows
-  const int deq_warps = (helpers || kBNL == 128) ? kDeqWarps / 2 : kDeqWarps;
+  // The eight dequant warps work as two groups of four that take alternate stages,
+  // so that one group's barrier, fence and bookkeeping time is covered by the
+  // other's table lookups (the ALU pipe is what bounds the fused products).  A
+  // group stages a whole tile: one block per thread for 128 rows, two for 256.
+  // In the merge kernel only one group stages (the other helps the epilogue).
+  const int deq_groups = helpers ? 1 : 2;
+  constexpr int kGroupWarps = kDeqWarps / 2;
   constexpr uint32_t kTmemCols = 2 * BN;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) {
       // arrivals: the leader's TMA producer (which also posts the follower's bytes) and
       // the dequant warps of every CTA of the pair
-      ptx::mbar_init(full_bar(s), 1 + (p.has_nf4 ? deq_warps * (TWO ? 2 : 1) : 0));
+      ptx::mbar_init(full_bar(s), 1 + (p.has_nf4 ? kGroupWarps * (TWO ? 2 : 1) : 0));
       ptx::mbar_init(empty_bar(s), 1);
       ptx::mbar_init(codes_bar(s), 1);
     }
@@ -620,8 +649,10 @@ loqt_gemm_kernel(const __grid_constant__ TensorMaps maps, const GemmParams p) {
   }
   // =========================================================== NF4 dequant
   else {
-    if (p.has_nf4 && warp < kDeqWarp0 + deq_warps) {
-      const int t = threadIdx.x - kDeqWarp0 * 32;
+    if (p.has_nf4 && warp < kDeqWarp0 + kGroupWarps * deq_groups) {
+      const int grp = (warp - kDeqWarp0) / kGroupWarps;  // this group's stages: it = grp (mod deq_groups)
+      const int t = (threadIdx.x - kDeqWarp0 * 32) & (kGroupWarps * 32 - 1);
+      constexpr bool kTwoRows = (kBNL == 256);  // (an NF4 A tile is 128 rows: one block per thread)
       // Two cursors over this CTA's k-blocks: the one being staged and, one step
       // ahead, the one whose scale is being fetched.  A cursor recomputes its
       // geometry only when it enters a new tile or K segment.
@@ -655,30 +686,47 @@ loqt_gemm_kernel(const __grid_constant__ TensorMaps maps, const GemmParams p) {
         c.u += gridDim.x;
         return open(c);
       };
-      auto fetch = [&](const Cursor &c) { return deq_fetch(c.g, c.seg == 0 ? c.kb : c.kb - sched.kb_seg0); };
+      auto kb_in = [&](const Cursor &c) { return c.seg == 0 ? c.kb : c.kb - sched.kb_seg0; };
+      auto advance_group = [&](Cursor &c) {  // to this group's next stage
+        for (int i = 0; i < deq_groups; ++i)
+          if (!advance(c)) return false;
+        return true;
+      };
 
       Cursor cur, nxt;
       cur.u = blockIdx.x;
       bool have = open(cur);
-      DeqTask task;
-      task.mode = 0;
-      task.M = 0.0f;
-      if (have) task = fetch(cur);
-      nxt = cur;
-      bool have_next = have && advance(nxt);
       uint32_t it = 0;
+      if (have && grp == 1) {
+        have = advance(cur);
+        it = 1;
+      }
+      DeqTask task0, task1;
+      task0.mode = task1.mode = 0;
+      task0.M = task1.M = 0.0f;
+      if (have) {
+        task0 = deq_fetch<0>(cur.g, kb_in(cur));
+        if (kTwoRows) task1 = deq_fetch<1>(cur.g, kb_in(cur));
+      }
+      nxt = cur;
+      bool have_next = have && advance_group(nxt);
       bool ok = true;
       while (have && ok) {
-        DeqTask task_next;
-        task_next.mode = 0;
-        task_next.M = 0.0f;
-        if (have_next) task_next = fetch(nxt);  // in flight while this stage is dequantised
+        DeqTask next0, next1;
+        next0.mode = next1.mode = 0;
+        next0.M = next1.M = 0.0f;
+        if (have_next) {  // in flight while this stage is dequantised
+          next0 = deq_fetch<0>(nxt.g, kb_in(nxt));
+          if (kTwoRows) next1 = deq_fetch<1>(nxt.g, kb_in(nxt));
+        }
         const int s = it % kStages;
         const uint32_t ph = (it / kStages) & 1u;
         // The code tile landing implies the stage's previous contents were consumed.
         if (!(ok = ptx::mbar_wait(codes_bar(s), ph, abort_flag, p.status))) break;
         const uint32_t stage_base = smem_base + s * L::kStageBytes;
-        deq_store(cur.g, task, stage_base, stage_base + L::kABytes + L::kBBytes);
+        const uint32_t code_base = stage_base + L::kABytes + L::kBBytes;
+        deq_store<0>(cur.g, task0, stage_base, code_base);
+        if (kTwoRows) deq_store<1>(cur.g, task1, stage_base, code_base);
         if (TWO) ptx::fence_proxy_async_all();
         else ptx::fence_proxy_async_smem();
         __syncwarp();
@@ -686,11 +734,12 @@ loqt_gemm_kernel(const __grid_constant__ TensorMaps maps, const GemmParams p) {
           if (TWO && !leader) ptx::mbar_arrive_cluster(ptx::map_to_cta(full_bar(s), 0));
           else ptx::mbar_arrive(full_bar(s));
         }
-        ++it;
+        it += deq_groups;
         cur = nxt;
         have = have_next;
-        task = task_next;
-        if (have_next) have_next = advance(nxt);
+        task0 = next0;
+        task1 = next1;
+        if (have_next) have_next = advance_group(nxt);
       }
     }
   }
