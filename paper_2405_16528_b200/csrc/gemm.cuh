@@ -721,7 +721,11 @@ loqt_gemm_kernel(const __grid_constant__ TensorMaps maps, const GemmParams p) {
         }
         const int s = it % kStages;
         const uint32_t ph = (it / kStages) & 1u;
-        // The code tile landing implies the stage's previous contents were consumed.
+        // First the slot's release (the same event the producer waits for): with an odd
+        // number of stages the two groups share slots, and a group that ran a whole ring
+        // ahead of the other would otherwise test the code barrier two phases early and
+        // read "already complete".  Then the code tile of this stage.
+        if (!(ok = ptx::mbar_wait<TWO>(empty_bar(s), ph ^ 1u, abort_flag, p.status))) break;
         if (!(ok = ptx::mbar_wait(codes_bar(s), ph, abort_flag, p.status))) break;
         const uint32_t stage_base = smem_base + s * L::kStageBytes;
         const uint32_t code_base = stage_base + L::kABytes + L::kBBytes;
