@@ -17,7 +17,9 @@ __global__ void __launch_bounds__(kQThreads)
 nf4_quantize_kernel(const float *__restrict__ src, int64_t ld_src, uint8_t *__restrict__ codes,
                     float *__restrict__ absmax, int rows, int cols, int ld) {
   __shared__ Nf4Tables tab;
+  __shared__ __align__(16) uint8_t bins[kNf4Bins];
   nf4_tables_init(tab, threadIdx.x);
+  nf4_bins_load(bins, threadIdx.x, kQThreads);
   __syncthreads();
 
   const int nb = ld / kBlock;
@@ -59,7 +61,7 @@ nf4_quantize_kernel(const float *__restrict__ src, int64_t ld_src, uint8_t *__re
     if (!live) continue;
 
     uint32_t w = kZeroWord;
-    if (m > 0.0f) w = nf4_quantize8(tab, v, nf4_divisor(m));
+    if (m > 0.0f) w = nf4_quantize8(tab, bins, v, nf4_divisor(m));
     uint8_t *crow = codes + static_cast<int64_t>(row) * (ld / 2) + c0 / 2;
     *reinterpret_cast<uint16_t *>(crow + 2 * l) = static_cast<uint16_t>(w & 0xffffu);
     *reinterpret_cast<uint16_t *>(crow + 16 + 2 * l) = static_cast<uint16_t>(w >> 16);
