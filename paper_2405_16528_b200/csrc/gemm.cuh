@@ -392,6 +392,11 @@ loqt_gemm_kernel(const __grid_constant__ TensorMaps maps, const GemmParams p) {
   if (TWO) ptx::cluster_sync_all();  // both CTAs' barriers exist before anything arrives on them
   ptx::tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  // Everything above (barriers, TMEM, tables) touched no global data, so it may
+  // overlap the tail of the previous kernel of the stream; from here on global
+  // memory is read and written.
+  ptx::grid_launch_dependents();
+  ptx::grid_dependency_wait();
 
   // =========================================================== TMA producer
   if (warp == 0) {

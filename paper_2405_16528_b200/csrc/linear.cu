@@ -130,16 +130,23 @@ static loqt_status launch_cfg(const GemmCall &c, cudaStream_t stream) {
   int grid = units < sm_count() ? units : sm_count();
   cudaLaunchConfig_t cfg;
   memset(&cfg, 0, sizeof(cfg));
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
+  int nattr = 0;
+  // programmatic dependent launch: this kernel's prologue may overlap the previous
+  // kernel's tail (the kernel itself waits before it touches global memory)
+  attr[nattr].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[nattr].val.programmaticStreamSerializationAllowed = 1;
+  ++nattr;
   if (TWO) {
     grid &= ~1;  // whole pairs (`units` is even in this mode)
-    attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = 2;
-    attr[0].val.clusterDim.y = 1;
-    attr[0].val.clusterDim.z = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    attr[nattr].id = cudaLaunchAttributeClusterDimension;
+    attr[nattr].val.clusterDim.x = 2;
+    attr[nattr].val.clusterDim.y = 1;
+    attr[nattr].val.clusterDim.z = 1;
+    ++nattr;
   }
+  cfg.attrs = attr;
+  cfg.numAttrs = nattr;
   cfg.gridDim = dim3(grid);
   cfg.blockDim = dim3(kNumThreads);
   cfg.dynamicSmemBytes = L::kDynamicBytes;

@@ -93,6 +93,14 @@ __device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t par
   return ok != 0;
 }
 
+// ---------------------------------------------------------------- programmatic dependent launch
+// wait: blocks until the kernel this one was ordered after has completed and its
+// memory is visible (returns at once when launched without the attribute).
+// launch_dependents: lets the next kernel of the stream start its own prologue
+// on SMs this grid no longer occupies.
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 // ---------------------------------------------------------------- fences
 __device__ __forceinline__ void fence_barrier_init() {
   asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
