@@ -371,13 +371,7 @@ loqt_gemm_kernel(const __grid_constant__ TensorMaps maps, const GemmParams p) {
     *abort_flag = 0;
     ptx::fence_barrier_init();
   }
-  // The merge's bin table sits in the unused upper half of stage 0's code tile (an
-  // NF4 A tile of 128 rows needs only 4 KiB of the 8 KiB slot).
-  const uint8_t *bins = smem_gen + L::kABytes + L::kBBytes + 4096;
-  if (p.epi == EPI_REQUANT) {
-    nf4_tables_init(tables, threadIdx.x);
-    nf4_bins_load(smem_gen + L::kABytes + L::kBBytes + 4096, threadIdx.x, kNumThreads);
-  }
+  if (p.epi == EPI_REQUANT) nf4_tables_init(tables, threadIdx.x);
   if (warp == 1) {
     if (TWO) {
       ptx::tmem_alloc_pair(smem_u32(const_cast<uint32_t *>(tmem_slot)), kTmemCols);
