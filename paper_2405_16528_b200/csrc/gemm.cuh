@@ -544,53 +544,46 @@ loqt_gemm_kernel(const __grid_constant__ TensorMaps maps, const GemmParams p) {
         const uint32_t t_row = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + acc * (MH * BN) + h * BN;
 
         if (p.epi == EPI_REQUANT) {
-          // One NF4 block of W_q per 64 accumulator columns of this thread's row, in two
-          // passes over the accumulator (TMEM reads are cheap, and not keeping 64 merged
-          // values in registers keeps the code and the register footprint small):
-          // pass 1 finds the block's new scale, pass 2 forms each merged value again,
-          // normalises it and writes its code.
+          // One NF4 block of W_q per 64 accumulator columns of this thread's row.
 #pragma unroll 1
           for (int jb = grp; jb < BN / 64; jb += epi_groups) {
+            uint32_t d0[32], d1[32];
+            ptx::tmem_ld32(t_row + jb * 64, d0);
+            ptx::tmem_ld32(t_row + jb * 64 + 32, d1);
+            ptx::tmem_ld_wait();
             const int c0 = n_base + jb * 64;
-            const bool valid = row_ok && c0 < p.wq_ld;
-            uint32_t *cw = reinterpret_cast<uint32_t *>(p.wq_codes + static_cast<int64_t>(valid ? row : 0) * (p.wq_ld >> 1) +
-                                                        ((valid ? c0 : 0) >> 1));
-            float *mp = p.wq_absmax + static_cast<int64_t>(valid ? row : 0) * (p.wq_ld >> 6) + ((valid ? c0 : 0) >> 6);
-            const float Mold = valid ? *mp : 0.0f;
-            const uint32_t tcol = t_row + jb * 64;
-            auto merged8 = [&](const uint32_t (&d)[8], uint32_t w, float (&v)[8]) {
+            if (row_ok && c0 < p.wq_ld) {
+              uint4 *cp = reinterpret_cast<uint4 *>(p.wq_codes + static_cast<int64_t>(row) * (p.wq_ld >> 1) + (c0 >> 1));
+              float *mp = p.wq_absmax + static_cast<int64_t>(row) * (p.wq_ld >> 6) + (c0 >> 6);
+              const uint4 ca = *cp, cb = *(cp + 1);
+              const float Mold = *mp;
+              const uint32_t w[8] = {ca.x, ca.y, ca.z, ca.w, cb.x, cb.y, cb.z, cb.w};
+              float v[64];
+              float Mnew = 0.0f;
 #pragma unroll
-              for (int e = 0; e < 8; ++e)
-                v[e] = fmaf(p.alpha, __uint_as_float(d[e]), Mold * tables.level[(w >> (4 * e)) & 15u]);
-            };
-            float Mnew = 0.0f;
-#pragma unroll 1
-            for (int g = 0; g < 8; ++g) {
-              uint32_t d[8];
-              ptx::tmem_ld8(tcol + 8 * g, d);
-              ptx::tmem_ld_wait();
-              if (valid) {
-                float v[8];
-                merged8(d, cw[g], v);
+              for (int e = 0; e < 64; ++e) {
+                const float deq = Mold * tables.level[(w[e >> 3] >> (4 * (e & 7))) & 15u];
+                const float delta = __uint_as_float(e < 32 ? d0[e] : d1[e - 32]);
+                v[e] = fmaf(p.alpha, delta, deq);
+                Mnew = fmaxf(Mnew, fabsf(v[e]));
+              }
+              uint32_t o[8];
+              const Nf4Divisor dv = nf4_divisor(Mnew);
 #pragma unroll
-                for (int e = 0; e < 8; ++e) Mnew = fmaxf(Mnew, fabsf(v[e]));
+              for (int g = 0; g < 8; ++g) {
+                if (Mnew > 0.0f) {
+                  const float vv[8] = {v[8 * g], v[8 * g + 1], v[8 * g + 2], v[8 * g + 3],
+                                       v[8 * g + 4], v[8 * g + 5], v[8 * g + 6], v[8 * g + 7]};
+                  o[g] = nf4_quantize8_tree(vv, dv);
+                } else {
+                  o[g] = kZeroWord;
+                }
               }
-              __syncwarp();
+              *cp = make_uint4(o[0], o[1], o[2], o[3]);
+              *(cp + 1) = make_uint4(o[4], o[5], o[6], o[7]);
+              *mp = Mnew;
             }
-            const Nf4Divisor dv = nf4_divisor(Mnew);
-#pragma unroll 1
-            for (int g = 0; g < 8; ++g) {
-              uint32_t d[8];
-              ptx::tmem_ld8(tcol + 8 * g, d);
-              ptx::tmem_ld_wait();
-              if (valid) {
-                float v[8];
-                merged8(d, cw[g], v);
-                cw[g] = (Mnew > 0.0f) ? nf4_quantize8(tables, bins, v, dv) : kZeroWord;
-              }
-              __syncwarp();
-            }
-            if (valid) *mp = Mnew;
+            __syncwarp();
           }
         } else {
 #pragma unroll 1
