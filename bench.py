@@ -142,7 +142,8 @@ def alloc_outputs(cfg, mats, device):
                 "dB": torch.empty((cfg.r, m["in"]), dtype=torch.float32, device=device),
             }
         ws_bytes = max(ws_bytes, L.loqt_workspace_bytes(L.LOQT_OP_FWD, m["out"], m["in"], cfg.r, cfg.T),
-                       L.loqt_workspace_bytes(L.LOQT_OP_BWD, m["out"], m["in"], cfg.r, cfg.T))
+                       L.loqt_workspace_bytes(L.LOQT_OP_BWD, m["out"], m["in"], cfg.r, cfg.T),
+                       256 + min(8, len(mats)) * (L.loqt_workspace_bytes(L.LOQT_OP_MERGE, m["out"], m["in"], cfg.r, 0) - 256))
     return bufs, L.new_workspace(ws_bytes, device)
 
 
@@ -229,7 +230,8 @@ def run_per_shape(args):
         y = torch.empty((T, pad8(out)), dtype=torch.bfloat16, device="cuda")[:, :out]
         dx = torch.empty((T, pad8(inn)), dtype=torch.bfloat16, device="cuda")[:, :inn]
         dB = torch.empty((r, inn), dtype=torch.float32, device="cuda")
-        ws = L.new_workspace(L.loqt_workspace_bytes(L.LOQT_OP_BWD, out, inn, r, T))
+        ws = L.new_workspace(max(L.loqt_workspace_bytes(L.LOQT_OP_BWD, out, inn, r, T),
+                                 L.loqt_workspace_bytes(L.LOQT_OP_MERGE, out, inn, r, 0)))
         tf = timeit(lambda: L.loqt_linear_fwd(Wq, Pq, B, 1.0, x, y=y, ws=ws))
         tb = timeit(lambda: L.loqt_linear_bwd(Wq, Pq, B, 1.0, x, dy, dx=dx, dB=dB, ws=ws))
         Wc = Wq.clone()

@@ -40,7 +40,7 @@ typedef enum {
   LOQT_OK = 0,
   LOQT_ERR_INVALID_ARG = 1, /* null pointer, non-positive size, ld too small      */
   LOQT_ERR_ALIGNMENT = 2,   /* pointer or leading dimension violates alignment    */
-  LOQT_ERR_UNSUPPORTED = 3, /* block size other than 64                            */
+  LOQT_ERR_UNSUPPORTED = 3, /* block size other than 64, or a size beyond the stated limit */
   LOQT_ERR_WORKSPACE = 4,   /* workspace missing or smaller than required          */
   LOQT_ERR_CUDA = 5,        /* a CUDA runtime / driver call failed                 */
   LOQT_ERR_TIMEOUT = 6,     /* a bounded device-side wait expired                  */
@@ -77,6 +77,7 @@ enum { LOQT_OP_FWD = 0, LOQT_OP_BWD = 1, LOQT_OP_MERGE = 2 };
  * tie; an all-zero block gets M = 0 and code 7).
  *   src : fp32 [dst.rows][ld_src] on the device, ld_src >= dst.cols.
  *   dst : receives codes and absmax, padding included.
+ * rows * (ld / 64) must stay below 2^30 (LOQT_ERR_UNSUPPORTED otherwise).
  */
 loqt_status loqt_nf4_quantize(const float *src, int64_t ld_src, loqt_nf4_mat dst, void *stream);
 
@@ -84,7 +85,8 @@ loqt_status loqt_nf4_quantize(const float *src, int64_t ld_src, loqt_nf4_mat dst
  * q_NF4^{-1} (Section 5.1, last two displayed equations): w = M * q[code],
  * one fp32 multiply.  Writes src.rows x src.cols elements to `dst` (row-major,
  * ld_dst elements per row), as fp32 when dst_is_bf16 == 0, else rounded once
- * to bf16 (nearest even).
+ * to bf16 (nearest even).  rows * (ld / 8) must stay below 2^31
+ * (LOQT_ERR_UNSUPPORTED otherwise).
  */
 loqt_status loqt_nf4_dequantize(loqt_nf4_mat src, void *dst, int64_t ld_dst, int dst_is_bf16,
                                 void *stream);
@@ -124,6 +126,9 @@ loqt_status loqt_linear_bwd(loqt_nf4_mat Wq, loqt_nf4_mat Pq, const void *B, int
  * deq(W_q) enters as the unrounded fp32 product M*q, deq(P_q) as the bf16
  * operand of the tensor-core product, the sum is formed in fp32.  Each block of
  * W_q depends only on its own previous contents, so the update is in place.
+ * Two launches: deq(P_q) is written once, as bf16, into the workspace
+ * (loqt_workspace_bytes(LOQT_OP_MERGE, ...) bytes), then one product kernel
+ * requantises W_q in its epilogue.
  */
 loqt_status loqt_merge_requant(loqt_nf4_mat Wq, loqt_nf4_mat Pq, const void *B, int64_t ldb,
                                float s, void *ws, size_t ws_bytes, void *stream);
@@ -131,7 +136,9 @@ loqt_status loqt_merge_requant(loqt_nf4_mat Wq, loqt_nf4_mat Pq, const void *B, 
 /*
  * The same merge for n independent matrices in one call (a whole model at a
  * merge step).  Wq, Pq, B, ldb are HOST arrays of length n; the workspace is
- * shared and must satisfy the largest matrix.
+ * shared and must satisfy the largest matrix.  A workspace of 256 + k times the
+ * largest matrix's scratch (k up to 8) lets the call stage k matrices ahead,
+ * which keeps the GPU from draining between products.
  */
 loqt_status loqt_merge_requant_many(int32_t n, const loqt_nf4_mat *Wq, const loqt_nf4_mat *Pq,
                                     const void *const *B, const int64_t *ldb, float s, void *ws,

@@ -204,11 +204,19 @@ def loqt_merge_requant(Wq: NF4Tensor, Pq: NF4Tensor, B: torch.Tensor, s: float, 
     return Wq
 
 
+def merge_many_workspace_bytes(Wqs, Pqs, group: int = 8) -> int:
+    """Workspace that lets loqt_merge_requant_many stage `group` matrices ahead
+    (the status block plus `group` scratch slots of the largest matrix)."""
+    if not Wqs:
+        return 256
+    need = max(loqt_workspace_bytes(LOQT_OP_MERGE, w.rows, w.cols, p.cols, 0) for w, p in zip(Wqs, Pqs))
+    return 256 + max(1, min(group, len(Wqs))) * (need - 256)
+
+
 def loqt_merge_requant_many(Wqs, Pqs, Bs, s: float, ws: torch.Tensor | None = None):
     n = len(Wqs)
     if ws is None:
-        need = max(loqt_workspace_bytes(LOQT_OP_MERGE, w.rows, w.cols, p.cols, 0) for w, p in zip(Wqs, Pqs))
-        ws = new_workspace(need, Bs[0].device)
+        ws = new_workspace(merge_many_workspace_bytes(Wqs, Pqs), Bs[0].device)
     aW = (loqt_nf4_mat * n)(*[w.view() for w in Wqs])
     aP = (loqt_nf4_mat * n)(*[p.view() for p in Pqs])
     aB = (ctypes.c_void_p * n)(*[_dev(b, torch.bfloat16) for b in Bs])

@@ -341,17 +341,19 @@ loqt_gemm_kernel(const __grid_constant__ TensorMaps maps, const GemmParams p) {
   const uint32_t rank = TWO ? ptx::cluster_ctarank() : 0u;
   const uint32_t peer = rank ^ 1u;
   const bool leader = (rank == 0);
-  // In the merge kernel (128-row tiles) only four dequant warps have rows to
-  // stage; the other four (warps 10-13, TMEM lane quarters 2,3,0,1) join the
-  // requantising epilogue and take every second 64-column block.
-  const bool helpers = !TWO && (MH == 1) && (p.epi == EPI_REQUANT);
-  const int epi_groups = helpers ? 2 : 1;
-  // The eight dequant warps work as two groups of four that take alternate stages,
+  // The requantising epilogue of the merge is the heaviest one, so dequant warps
+  // that have nothing to stage join it in groups of four (one warp per TMEM lane
+  // quarter: warps 6-9 and 10-13 cover quarters 2,3,0,1).  With both operands
+  // arriving by TMA both groups help; with an NF4 A operand (128-row tiles) one
+  // group stages and the other helps.  The 64-column blocks of a tile are dealt
+  // to the epilogue groups round-robin, continuing across tiles.
+  const bool requant_helpers = !TWO && (MH == 1) && (p.epi == EPI_REQUANT);
+  const int epi_groups = requant_helpers ? (p.has_nf4 ? 2 : 3) : 1;
+  // The dequant warps work as two groups of four that take alternate stages,
   // so that one group's barrier, fence and bookkeeping time is covered by the
   // other's table lookups (the ALU pipe is what bounds the fused products).  A
   // group stages a whole tile: one block per thread for 128 rows, two for 256.
-  // In the merge kernel only one group stages (the other helps the epilogue).
-  const int deq_groups = helpers ? 1 : 2;
+  const int deq_groups = !p.has_nf4 ? 0 : (requant_helpers ? 1 : 2);
   constexpr int kGroupWarps = kDeqWarps / 2;
   constexpr uint32_t kTmemCols = 2 * BN;
 
@@ -522,9 +524,9 @@ loqt_gemm_kernel(const __grid_constant__ TensorMaps maps, const GemmParams p) {
     }
   }
   // =========================================================== epilogue
-  else if (warp < kDeqWarp0 || (helpers && warp >= kDeqWarp0 + kDeqWarps / 2)) {
+  else if (warp < kDeqWarp0 || warp >= kDeqWarp0 + kGroupWarps * (3 - epi_groups)) {
     const int q = warp & 3;  // TMEM lane quarter this warp may access
-    const int grp = warp < kDeqWarp0 ? 0 : 1;
+    const int grp = warp < kDeqWarp0 ? 0 : epi_groups - 1 - (kDeqWarp0 + kDeqWarps - 1 - warp) / kGroupWarps;
     uint32_t tile = 0;
     bool ok = true;
     for (int u = blockIdx.x; ok && u < sched.units; u += gridDim.x, ++tile) {
@@ -546,7 +548,8 @@ loqt_gemm_kernel(const __grid_constant__ TensorMaps maps, const GemmParams p) {
         if (p.epi == EPI_REQUANT) {
           // One NF4 block of W_q per 64 accumulator columns of this thread's row.
 #pragma unroll 1
-          for (int jb = grp; jb < BN / 64; jb += epi_groups) {
+          for (int jb = 0; jb < BN / 64; ++jb) {
+            if (static_cast<int>((tile * (BN / 64) + jb) % epi_groups) != grp) continue;
             uint32_t d0[32], d1[32];
             ptx::tmem_ld32(t_row + jb * 64, d0);
             ptx::tmem_ld32(t_row + jb * 64 + 32, d1);
@@ -574,7 +577,7 @@ loqt_gemm_kernel(const __grid_constant__ TensorMaps maps, const GemmParams p) {
                 if (Mnew > 0.0f) {
                   const float vv[8] = {v[8 * g], v[8 * g + 1], v[8 * g + 2], v[8 * g + 3],
                                        v[8 * g + 4], v[8 * g + 5], v[8 * g + 6], v[8 * g + 7]};
-                  o[g] = nf4_quantize8_tree(vv, dv);
+                  o[g] = nf4_quantize8(tables, vv, dv);
                 } else {
                   o[g] = kZeroWord;
                 }

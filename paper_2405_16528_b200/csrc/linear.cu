@@ -240,7 +240,8 @@ extern "C" size_t loqt_workspace_bytes(int op, int32_t out, int32_t in, int32_t 
     db_splits(r, in, T > 0 ? T : 1, splits, kbps);
     if (splits > 1) total += align256(static_cast<size_t>(splits) * r * ((static_cast<size_t>(in) + 3) / 4 * 4) * 4);
   }
-  (void)out;
+  // merge: deq(P_q) as bf16, out x roundup(r, 64)
+  if (op == LOQT_OP_MERGE) total += align256(static_cast<size_t>(out > 0 ? out : 0) * ld_lowrank(r) * 2);
   return total;
 }
 
@@ -363,13 +364,23 @@ extern "C" loqt_status loqt_linear_bwd(loqt_nf4_mat Wq, loqt_nf4_mat Pq, const v
   return LOQT_OK;
 }
 
-static loqt_status merge_one(const loqt_nf4_mat &Wq, const loqt_nf4_mat &Pq, const void *B, int64_t ldb, float s,
-                             uint32_t *status, cudaStream_t stm) {
-  // Delta = deq(P_q) B  (out x in; K = r; P_q blocks along K), requantised in the epilogue.
+// The merge of one matrix, in two launches.  `phat` is scratch for deq(P_q).
+static size_t merge_scratch_bytes(const loqt_nf4_mat &Pq) {
+  return align256(static_cast<size_t>(Pq.rows) * ld_lowrank(Pq.cols) * 2);
+}
+
+// P-hat = bf16(deq(P_q)), once, instead of once per column tile inside the product.
+static loqt_status merge_stage(const loqt_nf4_mat &Pq, void *phat, cudaStream_t stm) {
+  return loqt_nf4_dequantize(Pq, phat, ld_lowrank(Pq.cols), 1, stm);
+}
+
+// Delta = P-hat B  (out x in; K = r, both operands by TMA), requantised in the epilogue.
+static loqt_status merge_product(const loqt_nf4_mat &Wq, const loqt_nf4_mat &Pq, const void *phat, const void *B,
+                                 int64_t ldb, float s, uint32_t *status, cudaStream_t stm) {
   GemmCall c{};
   c.p.M = Wq.rows; c.p.N = Wq.cols; c.p.num_segs = 1;
-  c.p.seg[0].K = Pq.cols; c.p.seg[0].a_kind = OP_NF4_K; c.p.seg[0].a_nf4 = nf4_src(Pq); c.p.seg[0].b_kind = OP_TMA_MN;
-  c.b[0] = {B, ldb};
+  c.p.seg[0].K = Pq.cols; c.p.seg[0].a_kind = OP_TMA_K; c.p.seg[0].b_kind = OP_TMA_MN;
+  c.a[0] = {phat, ld_lowrank(Pq.cols)}; c.b[0] = {B, ldb};
   c.p.splits = 1;
   c.p.epi = EPI_REQUANT; c.p.alpha = s; c.p.status = status;
   c.p.wq_codes = Wq.codes; c.p.wq_absmax = Wq.absmax; c.p.wq_ld = Wq.ld;
@@ -380,9 +391,12 @@ extern "C" loqt_status loqt_merge_requant(loqt_nf4_mat Wq, loqt_nf4_mat Pq, cons
                                           void *ws, size_t ws_bytes, void *stream) {
   loqt_status st;
   if ((st = check_layer(Wq, Pq, B, ldb)) != LOQT_OK) return st;
-  if ((st = check_ws(ws, ws_bytes, 256)) != LOQT_OK) return st;
+  if ((st = check_ws(ws, ws_bytes, 256 + merge_scratch_bytes(Pq))) != LOQT_OK) return st;
   if ((st = check_arch()) != LOQT_OK) return st;
-  return merge_one(Wq, Pq, B, ldb, s, static_cast<uint32_t *>(ws), static_cast<cudaStream_t>(stream));
+  cudaStream_t stm = static_cast<cudaStream_t>(stream);
+  void *phat = static_cast<uint8_t *>(ws) + 256;
+  if ((st = merge_stage(Pq, phat, stm)) != LOQT_OK) return st;
+  return merge_product(Wq, Pq, phat, B, ldb, s, static_cast<uint32_t *>(ws), stm);
 }
 
 extern "C" loqt_status loqt_merge_requant_many(int32_t n, const loqt_nf4_mat *Wq, const loqt_nf4_mat *Pq,
@@ -390,13 +404,32 @@ extern "C" loqt_status loqt_merge_requant_many(int32_t n, const loqt_nf4_mat *Wq
                                                size_t ws_bytes, void *stream) {
   if (n < 0 || (n > 0 && (Wq == nullptr || Pq == nullptr || B == nullptr || ldb == nullptr))) return LOQT_ERR_INVALID_ARG;
   loqt_status st;
-  for (int i = 0; i < n; ++i)
+  size_t slot = 0;
+  for (int i = 0; i < n; ++i) {
     if ((st = check_layer(Wq[i], Pq[i], B[i], ldb[i])) != LOQT_OK) return st;
-  if ((st = check_ws(ws, ws_bytes, 256)) != LOQT_OK) return st;
+    const size_t need = merge_scratch_bytes(Pq[i]);
+    if (need > slot) slot = need;
+  }
+  if ((st = check_ws(ws, ws_bytes, 256 + slot)) != LOQT_OK) return st;
   if ((st = check_arch()) != LOQT_OK) return st;
-  for (int i = 0; i < n; ++i)
-    if ((st = merge_one(Wq[i], Pq[i], B[i], ldb[i], s, static_cast<uint32_t *>(ws), static_cast<cudaStream_t>(stream))) != LOQT_OK)
-      return st;
+  if (n == 0) return LOQT_OK;
+  cudaStream_t stm = static_cast<cudaStream_t>(stream);
+  // The workspace holds as many P-hat slots as fit (at most kMergeGroup): a group's
+  // P-hats are staged back to back, then its products run back to back, so that
+  // the short staging kernels do not drain the GPU between every two products.
+  constexpr int kMergeGroup = 8;
+  int slots = static_cast<int>((ws_bytes - 256) / slot);
+  if (slots > kMergeGroup) slots = kMergeGroup;
+  uint8_t *base = static_cast<uint8_t *>(ws) + 256;
+  for (int g0 = 0; g0 < n; g0 += slots) {
+    const int g1 = g0 + slots < n ? g0 + slots : n;
+    for (int i = g0; i < g1; ++i)
+      if ((st = merge_stage(Pq[i], base + static_cast<size_t>(i - g0) * slot, stm)) != LOQT_OK) return st;
+    for (int i = g0; i < g1; ++i)
+      if ((st = merge_product(Wq[i], Pq[i], base + static_cast<size_t>(i - g0) * slot, B[i], ldb[i], s,
+                              static_cast<uint32_t *>(ws), stm)) != LOQT_OK)
+        return st;
+  }
   return LOQT_OK;
 }
 

@@ -11,67 +11,71 @@ constexpr int kQThreads = 256;
 
 // ---------------------------------------------------------------------------
 // quantise: fp32 [rows][ld_src] -> codes [rows][ld/2], absmax [rows][ld/64]
+// Four threads share one block of 64 weights; each owns 16 consecutive elements
+// (four 128-bit loads in flight, one 64-bit store of 16 codes).
 // ---------------------------------------------------------------------------
 template <bool kVec>
 __global__ void __launch_bounds__(kQThreads)
 nf4_quantize_kernel(const float *__restrict__ src, int64_t ld_src, uint8_t *__restrict__ codes,
                     float *__restrict__ absmax, int rows, int cols, int ld) {
   __shared__ Nf4Tables tab;
-  __shared__ __align__(16) uint8_t bins[kNf4Bins];
   nf4_tables_init(tab, threadIdx.x);
-  nf4_bins_load(bins, threadIdx.x, kQThreads);
   __syncthreads();
 
-  const int nb = ld / kBlock;
-  const int64_t n_items = static_cast<int64_t>(rows) * nb;  // one item = one NF4 block
-  const int l = threadIdx.x & 7;                            // lane within the 8-thread group
-  const int64_t group0 = (static_cast<int64_t>(blockIdx.x) * kQThreads + threadIdx.x) >> 3;
-  const int64_t stride = (static_cast<int64_t>(gridDim.x) * kQThreads) >> 3;
-  // All 8 threads of a group run the same trip count, and a warp holds 4 whole
-  // groups; inactive groups still take part in the shuffles.
-  const int64_t trips = (n_items + stride - 1) / stride;
+  const uint32_t nb = static_cast<uint32_t>(ld / kBlock);
+  const uint32_t n_items = static_cast<uint32_t>(rows) * nb;  // one item = one NF4 block (host checks < 2^30)
+  const uint32_t l = threadIdx.x & 3;                         // lane within the 4-thread group
+  const uint32_t group0 = (blockIdx.x * kQThreads + threadIdx.x) >> 2;
+  const uint32_t stride = (gridDim.x * kQThreads) >> 2;
+  // All threads of a warp run the same trip count: idle groups still take part in the shuffles.
+  const uint32_t trips = (n_items + stride - 1) / stride;
 
-  for (int64_t it = 0; it < trips; ++it) {
-    const int64_t item = group0 + it * stride;
+  for (uint32_t it = 0; it < trips; ++it) {
+    const uint32_t item = group0 + it * stride;
     const bool live = item < n_items;
-    const int row = live ? static_cast<int>(item / nb) : 0;
-    const int b = live ? static_cast<int>(item - static_cast<int64_t>(row) * nb) : 0;
-    const int c0 = b * kBlock;
+    const uint32_t row = live ? item / nb : 0;
+    const uint32_t b = live ? item - row * nb : 0;
+    const int c0 = static_cast<int>(b) * kBlock + 16 * static_cast<int>(l);
     const float *p = src + static_cast<int64_t>(row) * ld_src + c0;
-    // thread l owns elements [4l, 4l+4) and [32+4l, 32+4l+4) of the block
-    float v[8];
-    if (kVec && live && c0 + kBlock <= cols) {
-      const float4 a = __ldg(reinterpret_cast<const float4 *>(p) + l);
-      const float4 c = __ldg(reinterpret_cast<const float4 *>(p) + 8 + l);
-      v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w;
-      v[4] = c.x; v[5] = c.y; v[6] = c.z; v[7] = c.w;
+    float v[16];
+    if (kVec && live && c0 + 16 <= cols) {
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        const float4 a = __ldg(reinterpret_cast<const float4 *>(p) + k);
+        v[4 * k] = a.x; v[4 * k + 1] = a.y; v[4 * k + 2] = a.z; v[4 * k + 3] = a.w;
+      }
     } else {
 #pragma unroll
-      for (int j = 0; j < 8; ++j) {
-        const int e = (j < 4) ? (4 * l + j) : (32 + 4 * l + j - 4);
-        v[j] = (live && c0 + e < cols) ? __ldg(p + e) : 0.0f;
-      }
+      for (int j = 0; j < 16; ++j) v[j] = (live && c0 + j < cols) ? __ldg(p + j) : 0.0f;
     }
     float m = 0.0f;
 #pragma unroll
-    for (int j = 0; j < 8; ++j) m = fmaxf(m, fabsf(v[j]));
+    for (int j = 0; j < 16; ++j) m = fmaxf(m, fabsf(v[j]));
     m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 1));
     m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 2));
-    m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 4));
     if (!live) continue;
 
-    uint32_t w = kZeroWord;
-    if (m > 0.0f) w = nf4_quantize8(tab, bins, v, nf4_divisor(m));
-    uint8_t *crow = codes + static_cast<int64_t>(row) * (ld / 2) + c0 / 2;
-    *reinterpret_cast<uint16_t *>(crow + 2 * l) = static_cast<uint16_t>(w & 0xffffu);
-    *reinterpret_cast<uint16_t *>(crow + 16 + 2 * l) = static_cast<uint16_t>(w >> 16);
+    uint2 w = make_uint2(kZeroWord, kZeroWord);
+    if (m > 0.0f) {
+      const Nf4Divisor d = nf4_divisor(m);
+      const float lo[8] = {v[0], v[1], v[2], v[3], v[4], v[5], v[6], v[7]};
+      const float hi[8] = {v[8], v[9], v[10], v[11], v[12], v[13], v[14], v[15]};
+      w.x = nf4_quantize8(tab, lo, d);
+      w.y = nf4_quantize8(tab, hi, d);
+    }
+    uint8_t *crow = codes + static_cast<int64_t>(row) * (ld / 2) + (c0 >> 1);
+    *reinterpret_cast<uint2 *>(crow) = w;
     if (l == 0) absmax[static_cast<int64_t>(row) * nb + b] = m;
   }
 }
 
 // ---------------------------------------------------------------------------
-// dequantise: one thread per 8 consecutive elements (one 32-bit code word)
+// dequantise: one thread per 8 consecutive elements (one 32-bit word of codes,
+// one 16- or 32-byte store, so that a warp's stores are contiguous), four
+// independent words per trip so that enough loads are in flight.
 // ---------------------------------------------------------------------------
+constexpr int kDqUnroll = 4;
+
 template <bool kBf16, bool kVec>
 __global__ void __launch_bounds__(kQThreads)
 nf4_dequantize_kernel(const uint8_t *__restrict__ codes, const float *__restrict__ absmax,
@@ -80,45 +84,61 @@ nf4_dequantize_kernel(const uint8_t *__restrict__ codes, const float *__restrict
   nf4_tables_init(tab, threadIdx.x);
   __syncthreads();
 
-  const int wpr = ld / 8;  // code words per row
-  const int nb = ld / kBlock;
-  const int64_t n_items = static_cast<int64_t>(rows) * wpr;
-  const int64_t stride = static_cast<int64_t>(gridDim.x) * kQThreads;
-  for (int64_t item = static_cast<int64_t>(blockIdx.x) * kQThreads + threadIdx.x; item < n_items;
-       item += stride) {
-    const int row = static_cast<int>(item / wpr);
-    const int wi = static_cast<int>(item - static_cast<int64_t>(row) * wpr);
-    const int c0 = wi * 8;
-    if (c0 >= cols) continue;
-    const uint32_t w = __ldg(reinterpret_cast<const uint32_t *>(codes + static_cast<int64_t>(row) * (ld / 2)) + wi);
-    const float M = __ldg(absmax + static_cast<int64_t>(row) * nb + (c0 >> 6));
-    float v[8];
+  const uint32_t wpr = static_cast<uint32_t>(ld / 8);  // code words per row
+  const uint32_t nb = static_cast<uint32_t>(ld / kBlock);
+  const uint32_t n_items = static_cast<uint32_t>(rows) * wpr;  // (host checks < 2^31)
+  const uint32_t stride = gridDim.x * kQThreads;
+  for (uint32_t base = blockIdx.x * kQThreads + threadIdx.x; base < n_items; base += kDqUnroll * stride) {
+    uint32_t w[kDqUnroll], row[kDqUnroll];
+    int c0[kDqUnroll];
+    float M[kDqUnroll];
+    bool live[kDqUnroll];
 #pragma unroll
-    for (int j = 0; j < 8; ++j) v[j] = M * tab.level[(w >> (4 * j)) & 15u];
-    const bool full = kVec && (c0 + 8 <= cols);
-    if (kBf16) {
-      __nv_bfloat16 *o = reinterpret_cast<__nv_bfloat16 *>(dst) + static_cast<int64_t>(row) * ld_dst + c0;
-      if (full) {
-        uint4 q;
-        q.x = pack_bf16x2(v[0], v[1]);
-        q.y = pack_bf16x2(v[2], v[3]);
-        q.z = pack_bf16x2(v[4], v[5]);
-        q.w = pack_bf16x2(v[6], v[7]);
-        *reinterpret_cast<uint4 *>(o) = q;
-      } else {
-#pragma unroll
-        for (int j = 0; j < 8; ++j)
-          if (c0 + j < cols) o[j] = __float2bfloat16_rn(v[j]);
+    for (int u = 0; u < kDqUnroll; ++u) {
+      const uint32_t item = base + u * stride;
+      live[u] = item < n_items;
+      row[u] = live[u] ? item / wpr : 0;
+      const uint32_t h = live[u] ? item - row[u] * wpr : 0;
+      c0[u] = static_cast<int>(h) * 8;
+      live[u] = live[u] && c0[u] < cols;
+      w[u] = kZeroWord;
+      M[u] = 0.0f;
+      if (live[u]) {
+        w[u] = __ldg(reinterpret_cast<const uint32_t *>(codes + static_cast<int64_t>(row[u]) * (ld / 2)) + h);
+        M[u] = __ldg(absmax + static_cast<int64_t>(row[u]) * nb + (h >> 3));
       }
-    } else {
-      float *o = reinterpret_cast<float *>(dst) + static_cast<int64_t>(row) * ld_dst + c0;
-      if (full) {
-        reinterpret_cast<float4 *>(o)[0] = make_float4(v[0], v[1], v[2], v[3]);
-        reinterpret_cast<float4 *>(o)[1] = make_float4(v[4], v[5], v[6], v[7]);
-      } else {
+    }
 #pragma unroll
-        for (int j = 0; j < 8; ++j)
-          if (c0 + j < cols) o[j] = v[j];
+    for (int u = 0; u < kDqUnroll; ++u) {
+      if (!live[u]) continue;
+      float v[8];
+#pragma unroll
+      for (int j = 0; j < 8; ++j) v[j] = M[u] * tab.level[(w[u] >> (4 * j)) & 15u];
+      const bool full = kVec && (c0[u] + 8 <= cols);
+      if (kBf16) {
+        __nv_bfloat16 *o = reinterpret_cast<__nv_bfloat16 *>(dst) + static_cast<int64_t>(row[u]) * ld_dst + c0[u];
+        if (full) {
+          uint4 pk;
+          pk.x = pack_bf16x2(v[0], v[1]);
+          pk.y = pack_bf16x2(v[2], v[3]);
+          pk.z = pack_bf16x2(v[4], v[5]);
+          pk.w = pack_bf16x2(v[6], v[7]);
+          *reinterpret_cast<uint4 *>(o) = pk;
+        } else {
+#pragma unroll
+          for (int j = 0; j < 8; ++j)
+            if (c0[u] + j < cols) o[j] = __float2bfloat16_rn(v[j]);
+        }
+      } else {
+        float *o = reinterpret_cast<float *>(dst) + static_cast<int64_t>(row[u]) * ld_dst + c0[u];
+        if (full) {
+          reinterpret_cast<float4 *>(o)[0] = make_float4(v[0], v[1], v[2], v[3]);
+          reinterpret_cast<float4 *>(o)[1] = make_float4(v[4], v[5], v[6], v[7]);
+        } else {
+#pragma unroll
+          for (int j = 0; j < 8; ++j)
+            if (c0[u] + j < cols) o[j] = v[j];
+        }
       }
     }
   }
@@ -143,7 +163,8 @@ extern "C" loqt_status loqt_nf4_quantize(const float *src, int64_t ld_src, loqt_
   if ((reinterpret_cast<uintptr_t>(src) & 3u) != 0) return LOQT_ERR_ALIGNMENT;
   if ((st = check_arch()) != LOQT_OK) return st;
   const int64_t items = static_cast<int64_t>(dst.rows) * (dst.ld / kBlock);
-  const int grid = grid_for(items * 8);
+  if (items >= (1ll << 30)) return LOQT_ERR_UNSUPPORTED;  // 32-bit block indices in the kernel
+  const int grid = grid_for(items * 4);
   const bool vec = (reinterpret_cast<uintptr_t>(src) & 15u) == 0 && (ld_src % 4) == 0;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   if (vec)
@@ -163,7 +184,8 @@ extern "C" loqt_status loqt_nf4_dequantize(loqt_nf4_mat src, void *dst, int64_t 
   if ((a & (dst_is_bf16 ? 1u : 3u)) != 0) return LOQT_ERR_ALIGNMENT;
   if ((st = check_arch()) != LOQT_OK) return st;
   const int64_t items = static_cast<int64_t>(src.rows) * (src.ld / 8);
-  const int grid = grid_for(items);
+  if (items >= (1ll << 31)) return LOQT_ERR_UNSUPPORTED;  // 32-bit word indices in the kernel
+  const int grid = grid_for((items + kDqUnroll - 1) / kDqUnroll);
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   const bool vec = (a & 15u) == 0 && (ld_dst % (dst_is_bf16 ? 8 : 4)) == 0;
   if (dst_is_bf16) {

@@ -47,7 +47,7 @@ const char *loqt_status_string(loqt_status st) {
     case LOQT_OK: return "ok";
     case LOQT_ERR_INVALID_ARG: return "invalid argument";
     case LOQT_ERR_ALIGNMENT: return "misaligned pointer or leading dimension";
-    case LOQT_ERR_UNSUPPORTED: return "unsupported NF4 block size (must be 64)";
+    case LOQT_ERR_UNSUPPORTED: return "unsupported NF4 block size (must be 64) or size beyond the limit";
     case LOQT_ERR_WORKSPACE: return "workspace missing or too small";
     case LOQT_ERR_CUDA: return "CUDA call failed";
     case LOQT_ERR_TIMEOUT: return "device-side wait timed out";

@@ -34,7 +34,7 @@ def test_status_strings(lib):
 
 
 def test_workspace_sizes(lib):
-    assert L.loqt_workspace_bytes(L.LOQT_OP_MERGE, 4096, 4096, 1024, 0) == 256
+    assert L.loqt_workspace_bytes(L.LOQT_OP_MERGE, 4096, 4096, 1024, 0) == 256 + 4096 * 1024 * 2
     fwd = L.loqt_workspace_bytes(L.LOQT_OP_FWD, 4096, 4096, 1024, 4096)
     assert fwd == 256 + 4096 * 1024 * 2
     assert L.loqt_workspace_bytes(L.LOQT_OP_BWD, 4096, 4096, 1024, 4096) >= fwd
