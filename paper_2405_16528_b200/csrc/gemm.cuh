@@ -27,6 +27,7 @@
 // owner, warps 2-5 epilogue (one per TMEM lane quarter), warps 6-13 NF4
 // dequantisation.  One CTA per SM.
 #pragma once
+#include <type_traits>
 #include "nf4_dequant.cuh"
 #include "ptx.cuh"
 
@@ -572,15 +573,21 @@ loqt_gemm_kernel(const __grid_constant__ TensorMaps maps, const GemmParams p) {
               }
               uint32_t o[8];
               const Nf4Divisor dv = nf4_divisor(Mnew);
+              auto quantise_block = [&](auto exact) {
 #pragma unroll
-              for (int g = 0; g < 8; ++g) {
-                if (Mnew > 0.0f) {
+                for (int g = 0; g < 8; ++g) {
                   const float vv[8] = {v[8 * g], v[8 * g + 1], v[8 * g + 2], v[8 * g + 3],
                                        v[8 * g + 4], v[8 * g + 5], v[8 * g + 6], v[8 * g + 7]};
-                  o[g] = nf4_quantize8(tables, vv, dv);
-                } else {
-                  o[g] = kZeroWord;
+                  o[g] = nf4_quantize8<decltype(exact)::value>(tables, vv, dv);
                 }
+              };
+              if (!(Mnew > 0.0f)) {
+#pragma unroll
+                for (int g = 0; g < 8; ++g) o[g] = kZeroWord;
+              } else if (dv.exact) {
+                quantise_block(std::true_type{});
+              } else {
+                quantise_block(std::false_type{});
               }
               *cp = make_uint4(o[0], o[1], o[2], o[3]);
               *(cp + 1) = make_uint4(o[4], o[5], o[6], o[7]);

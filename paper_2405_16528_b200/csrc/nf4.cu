@@ -60,8 +60,13 @@ nf4_quantize_kernel(const float *__restrict__ src, int64_t ld_src, uint8_t *__re
       const Nf4Divisor d = nf4_divisor(m);
       const float lo[8] = {v[0], v[1], v[2], v[3], v[4], v[5], v[6], v[7]};
       const float hi[8] = {v[8], v[9], v[10], v[11], v[12], v[13], v[14], v[15]};
-      w.x = nf4_quantize8(tab, lo, d);
-      w.y = nf4_quantize8(tab, hi, d);
+      if (d.exact) {
+        w.x = nf4_quantize8<true>(tab, lo, d);
+        w.y = nf4_quantize8<true>(tab, hi, d);
+      } else {
+        w.x = nf4_quantize8<false>(tab, lo, d);
+        w.y = nf4_quantize8<false>(tab, hi, d);
+      }
     }
     uint8_t *crow = codes + static_cast<int64_t>(row) * (ld / 2) + (c0 >> 1);
     *reinterpret_cast<uint2 *>(crow) = w;
