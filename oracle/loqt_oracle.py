@@ -204,3 +204,14 @@ def loqt_merge_values(wq, pq, B, s, shape) -> np.ndarray:
 def loqt_merge_requant(wq, pq, B, s, shape):
     """W_q <- q_NF4( deq(W_q) + s deq(P_q) B ).  Returns (codes, absmax)."""
     return nf4_quantize(loqt_merge_values(wq, pq, B, s, shape))
+
+
+def nf4_requantize(wq, delta, s, cols):
+    """The requantising half of the merge with the product already formed
+    (Section 2.4; Algorithm 1, merge line; quantiser of Section 5.1):
+    W_q <- q_NF4( fl32( deq32(W_q) + s * delta ) ) for an fp32 matrix `delta`
+    ([rows, cols]); the sum is formed in float64 and rounded once.  Returns
+    (codes, absmax)."""
+    W32 = nf4_dequantize(wq[0], wq[1], cols).astype(np.float64)
+    d = np.asarray(delta, dtype=np.float32).astype(np.float64)
+    return nf4_quantize((W32 + float(s) * d).astype(np.float32))

@@ -179,3 +179,35 @@ def test_merged_weight_reproduces_adapter_output():
     y_merged = O.loqt_forward((c, m), pq, np.zeros_like(B), s, x, shape)
     bound = np.abs(x.astype(np.float64)) @ (np.repeat(m.astype(np.float64), 64, axis=1)[:, :inn] * (half_gap + 2 ** -8)).T
     assert np.all(np.abs(y_adapt - y_merged) <= bound + 1e-9)
+
+
+def test_requantize_zero_delta_is_identity():
+    out, inn, r, T = 48, 200, 8, 2
+    wq, pq, B, x, dy = _layer(21, out, inn, r, T)
+    c, m = O.nf4_requantize(wq, np.zeros((out, inn), np.float32), 1.0, inn)
+    assert np.array_equal(c, wq[0]) and np.array_equal(m, wq[1])
+
+
+def test_requantize_cancelling_delta_gives_zero_weights():
+    # s * delta = -deq32(W) exactly (halving and doubling are exact): every block
+    # becomes all-zero, i.e. code 7 and scale 0.  A wrong sign or a dropped s fails.
+    out, inn, r, T = 32, 128, 8, 2
+    wq, pq, B, x, dy = _layer(22, out, inn, r, T)
+    W32 = O.nf4_dequantize(wq[0], wq[1], inn)
+    c, m = O.nf4_requantize(wq, -0.5 * W32, 2.0, inn)
+    assert np.all(c == 7) and np.all(m == 0)
+
+
+@pytest.mark.parametrize("s", [1.0, 0.25])
+def test_requantize_equals_merge_for_rank_one(s):
+    # With r = 1 every element of P_BF16 @ B is one product of two bf16 numbers,
+    # exact in fp32, so handing that product to the requantiser must reproduce the
+    # merge bit for bit.
+    out, inn, r, T = 40, 192, 1, 2
+    wq, pq, B, x, dy = _layer(23, out, inn, r, T)
+    P = O.nf4_dequantize_bf16(pq[0], pq[1], r).astype(np.float64)
+    delta = (P @ B.astype(np.float64)).astype(np.float32)
+    assert np.array_equal(delta.astype(np.float64), P @ B.astype(np.float64))
+    c, m = O.nf4_requantize(wq, delta, s, inn)
+    rc, rm = O.loqt_merge_requant(wq, pq, B, s, (out, inn, r))
+    assert np.array_equal(c, rc) and np.array_equal(m, rm)
