@@ -231,16 +231,22 @@ def run_per_shape(args):
         dx = torch.empty((T, pad8(inn)), dtype=torch.bfloat16, device="cuda")[:, :inn]
         dB = torch.empty((r, inn), dtype=torch.float32, device="cuda")
         ws = L.new_workspace(max(L.loqt_workspace_bytes(L.LOQT_OP_BWD, out, inn, r, T),
-                                 L.loqt_workspace_bytes(L.LOQT_OP_MERGE, out, inn, r, 0)))
+                                 L.loqt_workspace_bytes(L.LOQT_OP_MERGE_SPLIT, out, inn, r, 0)))
         tf = timeit(lambda: L.loqt_linear_fwd(Wq, Pq, B, 1.0, x, y=y, ws=ws))
         tb = timeit(lambda: L.loqt_linear_bwd(Wq, Pq, B, 1.0, x, dy, dx=dx, dB=dB, ws=ws))
         Wc = Wq.clone()
         tm = timeit(lambda: L.loqt_merge_requant(Wc, Pq, B, 1.0, ws=ws))
+        ts = timeit(lambda: L.loqt_merge_requant_split(Wc, Pq, B, 1.0, ws=ws))
+        # the streaming half alone: read delta (fp32) + codes + scales, write codes + scales
+        delta = torch.randn((out, Wq.ld), dtype=torch.float32, device="cuda")[:, :inn] * 1e-3
+        tr = timeit(lambda: L.loqt_nf4_requantize(delta, 1.0, Wc))
+        requant_bytes = out * inn * 4 + 2 * synth.nf4_bytes(out, inn)
         L.loqt_device_status(ws)
         res[f"{out}x{inn}"] = {
-            "fwd_ms": round(tf, 4), "bwd_ms": round(tb, 4), "merge_ms": round(tm, 4),
+            "fwd_ms": round(tf, 4), "bwd_ms": round(tb, 4), "merge_ms": round(tm, 4), "merge_split_ms": round(ts, 4),
             "fwdbwd_tflops": round(synth.fwd_bwd_flops(out, inn, r, T) / (tf + tb) / 1e9, 1),
             "merge_gb_s": round(synth.merge_bytes(out, inn, r) / tm / 1e6, 1),
+            "requant_stage_ms": round(tr, 4), "requant_stage_gb_s": round(requant_bytes / tr / 1e6, 1),
         }
     print(json.dumps({"per_shape": res, "config": cfg.name}), flush=True)
 

@@ -69,7 +69,7 @@ typedef struct {
 } loqt_nf4_mat;
 
 /* Operation selector for loqt_workspace_bytes(). */
-enum { LOQT_OP_FWD = 0, LOQT_OP_BWD = 1, LOQT_OP_MERGE = 2 };
+enum { LOQT_OP_FWD = 0, LOQT_OP_BWD = 1, LOQT_OP_MERGE = 2, LOQT_OP_MERGE_SPLIT = 3 };
 
 /*
  * q_NF4 (Section 5.1, first two displayed equations): per block M = max|w|,
@@ -132,6 +132,29 @@ loqt_status loqt_linear_bwd(loqt_nf4_mat Wq, loqt_nf4_mat Pq, const void *B, int
  */
 loqt_status loqt_merge_requant(loqt_nf4_mat Wq, loqt_nf4_mat Pq, const void *B, int64_t ldb,
                                float s, void *ws, size_t ws_bytes, void *stream);
+
+/*
+ * The requantising half of the merge on its own (Section 2.4; Algorithm 1 merge
+ * line; quantiser of Section 5.1):
+ *     W_q <- q_NF4( deq(W_q) + s * delta )            in place
+ *   delta : fp32 [Wq.rows][ld_delta] on the device, ld_delta >= Wq.cols.
+ * deq(W_q) is the unrounded fp32 product M*q; the sum is one fused multiply-add.
+ * Padding elements of a short last block keep code 7.  rows * (ld / 64) must
+ * stay below 2^30 (LOQT_ERR_UNSUPPORTED otherwise).
+ */
+loqt_status loqt_nf4_requantize(const float *delta, int64_t ld_delta, float s, loqt_nf4_mat Wq,
+                                void *stream);
+
+/*
+ * The merge of loqt_merge_requant in two passes, with the same result bit for
+ * bit: deq(P_q) B is written to the workspace as fp32 (out x roundup(in, 64)),
+ * then loqt_nf4_requantize streams over it.  Workspace:
+ * loqt_workspace_bytes(LOQT_OP_MERGE_SPLIT, ...).  The fused form is the faster
+ * one at large shapes; this one exposes the streaming stage for measurement
+ * and serves callers that already hold the product.
+ */
+loqt_status loqt_merge_requant_split(loqt_nf4_mat Wq, loqt_nf4_mat Pq, const void *B, int64_t ldb,
+                                     float s, void *ws, size_t ws_bytes, void *stream);
 
 /*
  * The same merge for n independent matrices in one call (a whole model at a

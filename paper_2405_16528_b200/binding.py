@@ -16,12 +16,13 @@ import torch
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libloqt.so")
 
-LOQT_OP_FWD, LOQT_OP_BWD, LOQT_OP_MERGE = 0, 1, 2
+LOQT_OP_FWD, LOQT_OP_BWD, LOQT_OP_MERGE, LOQT_OP_MERGE_SPLIT = 0, 1, 2, 3
 BLOCK = 64
 
 EXPORTS = (
     "loqt_nf4_quantize", "loqt_nf4_dequantize", "loqt_linear_fwd", "loqt_linear_bwd",
-    "loqt_merge_requant", "loqt_merge_requant_many", "loqt_linear_fwd_static", "loqt_workspace_bytes",
+    "loqt_merge_requant", "loqt_merge_requant_many", "loqt_merge_requant_split", "loqt_nf4_requantize",
+    "loqt_linear_fwd_static", "loqt_workspace_bytes",
     "loqt_device_status", "loqt_launch_count", "loqt_status_string",
 )
 
@@ -64,6 +65,8 @@ def lib():
     L.loqt_linear_fwd_static.argtypes = [M, M, vp, i64, f32, vp, i64, i32, vp, i64, ctypes.c_int, vp]
     L.loqt_linear_fwd_static.restype = ctypes.c_int
     L.loqt_merge_requant.argtypes = [M, M, vp, i64, f32, vp, sz, vp]
+    L.loqt_merge_requant_split.argtypes = [M, M, vp, i64, f32, vp, sz, vp]
+    L.loqt_nf4_requantize.argtypes = [vp, i64, f32, M, vp]
     L.loqt_merge_requant_many.argtypes = [i32, ctypes.POINTER(M), ctypes.POINTER(M), ctypes.POINTER(vp), ctypes.POINTER(i64), f32, vp, sz, vp]
     L.loqt_workspace_bytes.argtypes = [ctypes.c_int, i32, i32, i32, i32]
     L.loqt_workspace_bytes.restype = sz
@@ -73,7 +76,8 @@ def lib():
     L.loqt_status_string.argtypes = [ctypes.c_int]
     L.loqt_status_string.restype = ctypes.c_char_p
     for name in ("loqt_nf4_quantize", "loqt_nf4_dequantize", "loqt_linear_fwd", "loqt_linear_bwd",
-                 "loqt_merge_requant", "loqt_merge_requant_many", "loqt_device_status"):
+                 "loqt_merge_requant", "loqt_merge_requant_many", "loqt_merge_requant_split", "loqt_nf4_requantize",
+                 "loqt_device_status"):
         getattr(L, name).restype = ctypes.c_int
     _lib = L
     return L
@@ -201,6 +205,21 @@ def loqt_merge_requant(Wq: NF4Tensor, Pq: NF4Tensor, B: torch.Tensor, s: float, 
         ws = new_workspace(loqt_workspace_bytes(LOQT_OP_MERGE, Wq.rows, Wq.cols, Pq.cols, 0), B.device)
     _check(lib().loqt_merge_requant(Wq.view(), Pq.view(), _dev(B, torch.bfloat16), B.stride(0), float(s),
                                     ws.data_ptr(), ws.numel(), _stream()), "loqt_merge_requant")
+    return Wq
+
+
+def loqt_merge_requant_split(Wq: NF4Tensor, Pq: NF4Tensor, B: torch.Tensor, s: float,
+                             ws: torch.Tensor | None = None) -> NF4Tensor:
+    if ws is None:
+        ws = new_workspace(loqt_workspace_bytes(LOQT_OP_MERGE_SPLIT, Wq.rows, Wq.cols, Pq.cols, 0), B.device)
+    _check(lib().loqt_merge_requant_split(Wq.view(), Pq.view(), _dev(B, torch.bfloat16), B.stride(0), float(s),
+                                          ws.data_ptr(), ws.numel(), _stream()), "loqt_merge_requant_split")
+    return Wq
+
+
+def loqt_nf4_requantize(delta: torch.Tensor, s: float, Wq: NF4Tensor) -> NF4Tensor:
+    _check(lib().loqt_nf4_requantize(_dev(delta, torch.float32), delta.stride(0), float(s), Wq.view(), _stream()),
+           "loqt_nf4_requantize")
     return Wq
 
 

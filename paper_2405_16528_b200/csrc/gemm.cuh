@@ -350,12 +350,17 @@ loqt_gemm_kernel(const __grid_constant__ TensorMaps maps, const GemmParams p) {
   // to the epilogue groups round-robin, continuing across tiles.
   const bool requant_helpers = !TWO && (MH == 1) && (p.epi == EPI_REQUANT);
   const int epi_groups = requant_helpers ? (p.has_nf4 ? 2 : 3) : 1;
-  // The dequant warps work as two groups of four that take alternate stages,
-  // so that one group's barrier, fence and bookkeeping time is covered by the
-  // other's table lookups (the ALU pipe is what bounds the fused products).  A
-  // group stages a whole tile: one block per thread for 128 rows, two for 256.
-  const int deq_groups = !p.has_nf4 ? 0 : (requant_helpers ? 1 : 2);
+  // The dequant warps work as two groups of four that take the K stages of a
+  // tile in turn, so that one group's barrier, fence and bookkeeping time is
+  // covered by the other's table lookups (the dequantisation is bound by the
+  // latency of its dependent chains, not by ALU throughput: more warps, more
+  // overlap).  A group stages a whole tile: one block per thread for 128 rows,
+  // two for 256.  (A third group made of the epilogue warps, idle during the main
+  // loop of single-accumulator kernels, was measured 5 % slower: with three stages
+  // in the ring a third group only waits for a slot.)
   constexpr int kGroupWarps = kDeqWarps / 2;
+  const int deq_groups = !p.has_nf4 ? 0 : (requant_helpers ? 1 : 2);
+  const int deq_grp = (warp - kDeqWarp0) / kGroupWarps;
   constexpr uint32_t kTmemCols = 2 * BN;
 
   if (threadIdx.x == 0) {
@@ -394,6 +399,108 @@ loqt_gemm_kernel(const __grid_constant__ TensorMaps maps, const GemmParams p) {
   // memory is read and written.
   ptx::grid_launch_dependents();
   ptx::grid_dependency_wait();
+
+  // ---------------------------------------------------------- NF4 staging worker
+  // State and one-stage step of a staging group.  Group g takes the stages of a
+  // tile whose index within the tile is g modulo the number of groups.
+  constexpr bool kTwoRows = (kBNL == 256);  // (an NF4 A tile is 128 rows: one block per thread)
+  const int deq_t = (threadIdx.x - kDeqWarp0 * 32) & (kGroupWarps * 32 - 1);
+  // Two cursors over this CTA's k-blocks: the one being staged and, one step
+  // ahead, the one whose scale is being fetched.  A cursor recomputes its
+  // geometry only when it enters a new tile or K segment.
+  struct Cursor {
+    int u, kb, kb_lo, kb_hi, m_blk, n_blk, seg;
+    uint32_t it;  // position in the CTA's sequence of stages (all groups count alike)
+    DeqGeom g;
+  };
+  auto cur_enter = [&](Cursor &c) {  // c.kb valid: (re)compute segment and geometry
+    c.seg = c.kb < sched.kb_seg0 ? 0 : 1;
+    // this CTA's B rows start at local block (TWO: 2 n_blk + rank) of kBNL rows
+    c.g = deq_geom<kBNL, kBM, L::kABytes>(p, c.seg, c.m_blk, TWO ? 2 * c.n_blk + static_cast<int>(rank) : c.n_blk, deq_t);
+  };
+  auto cur_open = [&](Cursor &c) {
+    while (c.u < sched.units) {
+      int split;
+      sched.unit(c.u, c.m_blk, c.n_blk, split, c.kb_lo, c.kb_hi);
+      c.kb = c.kb_lo;
+      if (c.kb < c.kb_hi) {
+        cur_enter(c);
+        return true;
+      }
+      c.u += gridDim.x;
+    }
+    return false;
+  };
+  auto cur_advance = [&](Cursor &c) {
+    ++c.it;
+    if (++c.kb < c.kb_hi) {
+      if (c.kb == sched.kb_seg0) cur_enter(c);  // crossed into the second segment
+      return true;
+    }
+    c.u += gridDim.x;
+    return cur_open(c);
+  };
+  auto cur_mine = [&](const Cursor &c) { return (c.kb - c.kb_lo) % deq_groups == deq_grp; };
+  auto cur_next_mine = [&](Cursor &c) {  // to this group's next stage
+    do {
+      if (!cur_advance(c)) return false;
+    } while (!cur_mine(c));
+    return true;
+  };
+  auto cur_kb_in = [&](const Cursor &c) { return c.seg == 0 ? c.kb : c.kb - sched.kb_seg0; };
+
+  Cursor cur, nxt;
+  DeqTask task0, task1;
+  bool deq_have = false, deq_have_next = false;
+  auto deq_begin = [&]() {
+    cur.u = blockIdx.x;
+    cur.it = 0;
+    deq_have = cur_open(cur);
+    if (deq_have && !cur_mine(cur)) deq_have = cur_next_mine(cur);
+    task0.mode = task1.mode = 0;
+    task0.M = task1.M = 0.0f;
+    if (deq_have) {
+      task0 = deq_fetch<0>(cur.g, cur_kb_in(cur));
+      if (kTwoRows) task1 = deq_fetch<1>(cur.g, cur_kb_in(cur));
+    }
+    nxt = cur;
+    deq_have_next = deq_have && cur_next_mine(nxt);
+  };
+  // Stages the block(s) of this thread for the stage under `cur`; false when a wait expired.
+  auto deq_step = [&]() -> bool {
+    DeqTask next0, next1;
+    next0.mode = next1.mode = 0;
+    next0.M = next1.M = 0.0f;
+    if (deq_have_next) {  // in flight while this stage is dequantised
+      next0 = deq_fetch<0>(nxt.g, cur_kb_in(nxt));
+      if (kTwoRows) next1 = deq_fetch<1>(nxt.g, cur_kb_in(nxt));
+    }
+    const int s = cur.it % kStages;
+    const uint32_t ph = (cur.it / kStages) & 1u;
+    // First the slot's release (the same event the producer waits for): groups share
+    // slots, and a group that ran a whole ring ahead of the others would otherwise
+    // test the code barrier two phases early and read "already complete".  Then the
+    // code tile of this stage.
+    if (!ptx::mbar_wait<TWO>(empty_bar(s), ph ^ 1u, abort_flag, p.status)) return false;
+    if (!ptx::mbar_wait(codes_bar(s), ph, abort_flag, p.status)) return false;
+    const uint32_t stage_base = smem_base + s * L::kStageBytes;
+    const uint32_t code_base = stage_base + L::kABytes + L::kBBytes;
+    deq_store<0>(cur.g, task0, stage_base, code_base);
+    if (kTwoRows) deq_store<1>(cur.g, task1, stage_base, code_base);
+    if (TWO) ptx::fence_proxy_async_all();
+    else ptx::fence_proxy_async_smem();
+    __syncwarp();
+    if (lane == 0) {
+      if (TWO && !leader) ptx::mbar_arrive_cluster(ptx::map_to_cta(full_bar(s), 0));
+      else ptx::mbar_arrive(full_bar(s));
+    }
+    cur = nxt;
+    deq_have = deq_have_next;
+    task0 = next0;
+    task1 = next1;
+    if (deq_have_next) deq_have_next = cur_next_mine(nxt);
+    return true;
+  };
 
   // =========================================================== TMA producer
   if (warp == 0) {
@@ -665,100 +772,8 @@ loqt_gemm_kernel(const __grid_constant__ TensorMaps maps, const GemmParams p) {
   // =========================================================== NF4 dequant
   else {
     if (p.has_nf4 && warp < kDeqWarp0 + kGroupWarps * deq_groups) {
-      const int grp = (warp - kDeqWarp0) / kGroupWarps;  // this group's stages: it = grp (mod deq_groups)
-      const int t = (threadIdx.x - kDeqWarp0 * 32) & (kGroupWarps * 32 - 1);
-      constexpr bool kTwoRows = (kBNL == 256);  // (an NF4 A tile is 128 rows: one block per thread)
-      // Two cursors over this CTA's k-blocks: the one being staged and, one step
-      // ahead, the one whose scale is being fetched.  A cursor recomputes its
-      // geometry only when it enters a new tile or K segment.
-      struct Cursor {
-        int u, kb, kb_hi, m_blk, n_blk, seg;
-        DeqGeom g;
-      };
-      auto enter = [&](Cursor &c) {  // c.kb valid: (re)compute segment and geometry
-        c.seg = c.kb < sched.kb_seg0 ? 0 : 1;
-        // this CTA's B rows start at local block (TWO: 2 n_blk + rank) of kBNL rows
-        c.g = deq_geom<kBNL, kBM, L::kABytes>(p, c.seg, c.m_blk, TWO ? 2 * c.n_blk + static_cast<int>(rank) : c.n_blk, t);
-      };
-      auto open = [&](Cursor &c) {
-        while (c.u < sched.units) {
-          int split, lo;
-          sched.unit(c.u, c.m_blk, c.n_blk, split, lo, c.kb_hi);
-          c.kb = lo;
-          if (c.kb < c.kb_hi) {
-            enter(c);
-            return true;
-          }
-          c.u += gridDim.x;
-        }
-        return false;
-      };
-      auto advance = [&](Cursor &c) {
-        if (++c.kb < c.kb_hi) {
-          if (c.kb == sched.kb_seg0) enter(c);  // crossed into the second segment
-          return true;
-        }
-        c.u += gridDim.x;
-        return open(c);
-      };
-      auto kb_in = [&](const Cursor &c) { return c.seg == 0 ? c.kb : c.kb - sched.kb_seg0; };
-      auto advance_group = [&](Cursor &c) {  // to this group's next stage
-        for (int i = 0; i < deq_groups; ++i)
-          if (!advance(c)) return false;
-        return true;
-      };
-
-      Cursor cur, nxt;
-      cur.u = blockIdx.x;
-      bool have = open(cur);
-      uint32_t it = 0;
-      if (have && grp == 1) {
-        have = advance(cur);
-        it = 1;
-      }
-      DeqTask task0, task1;
-      task0.mode = task1.mode = 0;
-      task0.M = task1.M = 0.0f;
-      if (have) {
-        task0 = deq_fetch<0>(cur.g, kb_in(cur));
-        if (kTwoRows) task1 = deq_fetch<1>(cur.g, kb_in(cur));
-      }
-      nxt = cur;
-      bool have_next = have && advance_group(nxt);
-      bool ok = true;
-      while (have && ok) {
-        DeqTask next0, next1;
-        next0.mode = next1.mode = 0;
-        next0.M = next1.M = 0.0f;
-        if (have_next) {  // in flight while this stage is dequantised
-          next0 = deq_fetch<0>(nxt.g, kb_in(nxt));
-          if (kTwoRows) next1 = deq_fetch<1>(nxt.g, kb_in(nxt));
-        }
-        const int s = it % kStages;
-        const uint32_t ph = (it / kStages) & 1u;
-        // First the slot's release (the same event the producer waits for): with an odd
-        // number of stages the two groups share slots, and a group that ran a whole ring
-        // ahead of the other would otherwise test the code barrier two phases early and
-        // read "already complete".  Then the code tile of this stage.
-        if (!(ok = ptx::mbar_wait<TWO>(empty_bar(s), ph ^ 1u, abort_flag, p.status))) break;
-        if (!(ok = ptx::mbar_wait(codes_bar(s), ph, abort_flag, p.status))) break;
-        const uint32_t stage_base = smem_base + s * L::kStageBytes;
-        const uint32_t code_base = stage_base + L::kABytes + L::kBBytes;
-        deq_store<0>(cur.g, task0, stage_base, code_base);
-        if (kTwoRows) deq_store<1>(cur.g, task1, stage_base, code_base);
-        if (TWO) ptx::fence_proxy_async_all();
-        else ptx::fence_proxy_async_smem();
-        __syncwarp();
-        if (lane == 0) {
-          if (TWO && !leader) ptx::mbar_arrive_cluster(ptx::map_to_cta(full_bar(s), 0));
-          else ptx::mbar_arrive(full_bar(s));
-        }
-        it += deq_groups;
-        cur = nxt;
-        have = have_next;
-        task0 = next0;
-        task1 = next1;
-        if (have_next) have_next = advance_group(nxt);
+      deq_begin();
+      while (deq_have && deq_step()) {
       }
     }
   }

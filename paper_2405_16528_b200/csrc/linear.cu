@@ -241,7 +241,11 @@ extern "C" size_t loqt_workspace_bytes(int op, int32_t out, int32_t in, int32_t 
     if (splits > 1) total += align256(static_cast<size_t>(splits) * r * ((static_cast<size_t>(in) + 3) / 4 * 4) * 4);
   }
   // merge: deq(P_q) as bf16, out x roundup(r, 64)
-  if (op == LOQT_OP_MERGE) total += align256(static_cast<size_t>(out > 0 ? out : 0) * ld_lowrank(r) * 2);
+  if (op == LOQT_OP_MERGE || op == LOQT_OP_MERGE_SPLIT)
+    total += align256(static_cast<size_t>(out > 0 ? out : 0) * ld_lowrank(r) * 2);
+  // two-pass merge: the fp32 product P-hat B, out x roundup(in, 64)
+  if (op == LOQT_OP_MERGE_SPLIT)
+    total += align256(static_cast<size_t>(out > 0 ? out : 0) * ((static_cast<size_t>(in > 0 ? in : 0) + 63) / 64 * 64) * 4);
   return total;
 }
 
@@ -397,6 +401,31 @@ extern "C" loqt_status loqt_merge_requant(loqt_nf4_mat Wq, loqt_nf4_mat Pq, cons
   void *phat = static_cast<uint8_t *>(ws) + 256;
   if ((st = merge_stage(Pq, phat, stm)) != LOQT_OK) return st;
   return merge_product(Wq, Pq, phat, B, ldb, s, static_cast<uint32_t *>(ws), stm);
+}
+
+// The same merge in two passes: Delta = P-hat B written as fp32, then the
+// streaming requantiser.  Same arithmetic per element as the fused epilogue.
+extern "C" loqt_status loqt_merge_requant_split(loqt_nf4_mat Wq, loqt_nf4_mat Pq, const void *B, int64_t ldb, float s,
+                                                void *ws, size_t ws_bytes, void *stream) {
+  loqt_status st;
+  if ((st = check_layer(Wq, Pq, B, ldb)) != LOQT_OK) return st;
+  const size_t phat_bytes = merge_scratch_bytes(Pq);
+  const size_t delta_bytes = align256(static_cast<size_t>(Wq.rows) * Wq.ld * 4);
+  if ((st = check_ws(ws, ws_bytes, 256 + phat_bytes + delta_bytes)) != LOQT_OK) return st;
+  if ((st = check_arch()) != LOQT_OK) return st;
+  cudaStream_t stm = static_cast<cudaStream_t>(stream);
+  void *phat = static_cast<uint8_t *>(ws) + 256;
+  float *delta = reinterpret_cast<float *>(static_cast<uint8_t *>(phat) + phat_bytes);
+  if ((st = merge_stage(Pq, phat, stm)) != LOQT_OK) return st;
+  GemmCall c{};
+  c.p.M = Wq.rows; c.p.N = Wq.cols; c.p.num_segs = 1;
+  c.p.seg[0].K = Pq.cols; c.p.seg[0].a_kind = OP_TMA_K; c.p.seg[0].b_kind = OP_TMA_MN;
+  c.a[0] = {phat, ld_lowrank(Pq.cols)}; c.b[0] = {B, ldb};
+  c.p.splits = 1;
+  c.p.epi = EPI_F32; c.p.out = delta; c.p.ld_out = Wq.ld; c.p.alpha = 1.0f; c.p.accumulate = 0;
+  c.p.status = static_cast<uint32_t *>(ws);
+  if ((st = launch(c, stm)) != LOQT_OK) return st;
+  return loqt_nf4_requantize(delta, Wq.ld, s, Wq, stream);
 }
 
 extern "C" loqt_status loqt_merge_requant_many(int32_t n, const loqt_nf4_mat *Wq, const loqt_nf4_mat *Pq,

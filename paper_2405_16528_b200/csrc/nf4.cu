@@ -75,6 +75,83 @@ nf4_quantize_kernel(const float *__restrict__ src, int64_t ld_src, uint8_t *__re
 }
 
 // ---------------------------------------------------------------------------
+// requantise: W_q <- q_NF4(deq32(W_q) + s * delta), in place (the streaming half
+// of the two-pass merge).  Same thread layout as the quantiser: four threads per
+// block, 16 elements each (four 128-bit loads of delta, one 64-bit load and one
+// 64-bit store of codes).
+// ---------------------------------------------------------------------------
+template <bool kVec>
+__global__ void __launch_bounds__(kQThreads)
+nf4_requantize_kernel(const float *__restrict__ delta, int64_t ld_delta, float s, uint8_t *__restrict__ codes,
+                      float *__restrict__ absmax, int rows, int cols, int ld) {
+  __shared__ Nf4Tables tab;
+  nf4_tables_init(tab, threadIdx.x);
+  __syncthreads();
+
+  const uint32_t nb = static_cast<uint32_t>(ld / kBlock);
+  const uint32_t n_items = static_cast<uint32_t>(rows) * nb;
+  const uint32_t l = threadIdx.x & 3;
+  const uint32_t group0 = (blockIdx.x * kQThreads + threadIdx.x) >> 2;
+  const uint32_t stride = (gridDim.x * kQThreads) >> 2;
+  const uint32_t trips = (n_items + stride - 1) / stride;  // uniform: idle groups still shuffle
+
+  for (uint32_t it = 0; it < trips; ++it) {
+    const uint32_t item = group0 + it * stride;
+    const bool live = item < n_items;
+    const uint32_t row = live ? item / nb : 0;
+    const uint32_t b = live ? item - row * nb : 0;
+    const int c0 = static_cast<int>(b) * kBlock + 16 * static_cast<int>(l);
+    const float *p = delta + static_cast<int64_t>(row) * ld_delta + c0;
+    uint8_t *crow = codes + static_cast<int64_t>(row) * (ld / 2) + (c0 >> 1);
+    float *mp = absmax + static_cast<int64_t>(row) * nb + b;
+    float v[16];
+    uint2 old = make_uint2(kZeroWord, kZeroWord);
+    float Mold = 0.0f;
+    if (live) {
+      old = *reinterpret_cast<const uint2 *>(crow);
+      Mold = *mp;
+    }
+    if (kVec && live && c0 + 16 <= cols) {
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        const float4 a = __ldg(reinterpret_cast<const float4 *>(p) + k);
+        v[4 * k] = a.x; v[4 * k + 1] = a.y; v[4 * k + 2] = a.z; v[4 * k + 3] = a.w;
+      }
+    } else {
+#pragma unroll
+      for (int j = 0; j < 16; ++j) v[j] = (live && c0 + j < cols) ? __ldg(p + j) : 0.0f;  // padding: no update
+    }
+    float m = 0.0f;
+#pragma unroll
+    for (int j = 0; j < 16; ++j) {
+      const uint32_t code = ((j < 8 ? old.x : old.y) >> (4 * (j & 7))) & 15u;
+      v[j] = fmaf(s, v[j], Mold * tab.level[code]);
+      m = fmaxf(m, fabsf(v[j]));
+    }
+    // every thread of the block has read the old scale before lane 0 replaces it
+    m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 1));
+    m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 2));
+    if (!live) continue;
+
+    uint2 w = make_uint2(kZeroWord, kZeroWord);
+    if (m > 0.0f) {
+      const Nf4Divisor d = nf4_divisor(m);
+      const float lo[8] = {v[0], v[1], v[2], v[3], v[4], v[5], v[6], v[7]};
+      const float hi[8] = {v[8], v[9], v[10], v[11], v[12], v[13], v[14], v[15]};
+      if (d.exact) {
+        w.x = nf4_quantize8<true>(tab, lo, d);
+        w.y = nf4_quantize8<true>(tab, hi, d);
+      } else {
+        w.x = nf4_quantize8<false>(tab, lo, d);
+        w.y = nf4_quantize8<false>(tab, hi, d);
+      }
+    }
+    *reinterpret_cast<uint2 *>(crow) = w;
+    if (l == 0) *mp = m;
+  }
+}
+
+// ---------------------------------------------------------------------------
 // dequantise: one thread per 8 consecutive elements (one 32-bit word of codes,
 // one 16- or 32-byte store, so that a warp's stores are contiguous), four
 // independent words per trip so that enough loads are in flight.
@@ -149,9 +226,14 @@ nf4_dequantize_kernel(const uint8_t *__restrict__ codes, const float *__restrict
   }
 }
 
-static int grid_for(int64_t threads_needed) {
+// Grid of a streaming kernel: enough blocks for the work, at most as many as
+// are resident at once (the kernels loop with a grid stride).
+template <typename Kernel>
+static int grid_for(Kernel kernel, int64_t threads_needed) {
+  int per_sm = 0;
+  if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, kQThreads, 0) != cudaSuccess || per_sm < 1) per_sm = 1;
   int64_t blocks = (threads_needed + kQThreads - 1) / kQThreads;
-  const int64_t cap = static_cast<int64_t>(sm_count()) * 8;  // 8 resident CTAs of 256 threads per SM
+  const int64_t cap = static_cast<int64_t>(sm_count()) * per_sm;
   if (blocks > cap) blocks = cap;
   if (blocks < 1) blocks = 1;
   return static_cast<int>(blocks);
@@ -169,13 +251,10 @@ extern "C" loqt_status loqt_nf4_quantize(const float *src, int64_t ld_src, loqt_
   if ((st = check_arch()) != LOQT_OK) return st;
   const int64_t items = static_cast<int64_t>(dst.rows) * (dst.ld / kBlock);
   if (items >= (1ll << 30)) return LOQT_ERR_UNSUPPORTED;  // 32-bit block indices in the kernel
-  const int grid = grid_for(items * 4);
   const bool vec = (reinterpret_cast<uintptr_t>(src) & 15u) == 0 && (ld_src % 4) == 0;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
-  if (vec)
-    nf4_quantize_kernel<true><<<grid, kQThreads, 0, s>>>(src, ld_src, dst.codes, dst.absmax, dst.rows, dst.cols, dst.ld);
-  else
-    nf4_quantize_kernel<false><<<grid, kQThreads, 0, s>>>(src, ld_src, dst.codes, dst.absmax, dst.rows, dst.cols, dst.ld);
+  auto kernel = vec ? nf4_quantize_kernel<true> : nf4_quantize_kernel<false>;
+  kernel<<<grid_for(kernel, items * 4), kQThreads, 0, s>>>(src, ld_src, dst.codes, dst.absmax, dst.rows, dst.cols, dst.ld);
   count_launch();
   return cudaGetLastError() == cudaSuccess ? LOQT_OK : LOQT_ERR_CUDA;
 }
@@ -190,16 +269,28 @@ extern "C" loqt_status loqt_nf4_dequantize(loqt_nf4_mat src, void *dst, int64_t 
   if ((st = check_arch()) != LOQT_OK) return st;
   const int64_t items = static_cast<int64_t>(src.rows) * (src.ld / 8);
   if (items >= (1ll << 31)) return LOQT_ERR_UNSUPPORTED;  // 32-bit word indices in the kernel
-  const int grid = grid_for((items + kDqUnroll - 1) / kDqUnroll);
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   const bool vec = (a & 15u) == 0 && (ld_dst % (dst_is_bf16 ? 8 : 4)) == 0;
-  if (dst_is_bf16) {
-    if (vec) nf4_dequantize_kernel<true, true><<<grid, kQThreads, 0, s>>>(src.codes, src.absmax, dst, ld_dst, src.rows, src.cols, src.ld);
-    else nf4_dequantize_kernel<true, false><<<grid, kQThreads, 0, s>>>(src.codes, src.absmax, dst, ld_dst, src.rows, src.cols, src.ld);
-  } else {
-    if (vec) nf4_dequantize_kernel<false, true><<<grid, kQThreads, 0, s>>>(src.codes, src.absmax, dst, ld_dst, src.rows, src.cols, src.ld);
-    else nf4_dequantize_kernel<false, false><<<grid, kQThreads, 0, s>>>(src.codes, src.absmax, dst, ld_dst, src.rows, src.cols, src.ld);
-  }
+  auto kernel = dst_is_bf16 ? (vec ? nf4_dequantize_kernel<true, true> : nf4_dequantize_kernel<true, false>)
+                            : (vec ? nf4_dequantize_kernel<false, true> : nf4_dequantize_kernel<false, false>);
+  kernel<<<grid_for(kernel, (items + kDqUnroll - 1) / kDqUnroll), kQThreads, 0, s>>>(src.codes, src.absmax, dst, ld_dst, src.rows,
+                                                                                     src.cols, src.ld);
+  count_launch();
+  return cudaGetLastError() == cudaSuccess ? LOQT_OK : LOQT_ERR_CUDA;
+}
+
+extern "C" loqt_status loqt_nf4_requantize(const float *delta, int64_t ld_delta, float s, loqt_nf4_mat Wq, void *stream) {
+  loqt_status st = validate_nf4(Wq);
+  if (st != LOQT_OK) return st;
+  if (delta == nullptr || ld_delta < Wq.cols) return LOQT_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(delta) & 3u) != 0) return LOQT_ERR_ALIGNMENT;
+  if ((st = check_arch()) != LOQT_OK) return st;
+  const int64_t items = static_cast<int64_t>(Wq.rows) * (Wq.ld / kBlock);
+  if (items >= (1ll << 30)) return LOQT_ERR_UNSUPPORTED;  // 32-bit block indices in the kernel
+  const bool vec = (reinterpret_cast<uintptr_t>(delta) & 15u) == 0 && (ld_delta % 4) == 0;
+  cudaStream_t stm = static_cast<cudaStream_t>(stream);
+  auto kernel = vec ? nf4_requantize_kernel<true> : nf4_requantize_kernel<false>;
+  kernel<<<grid_for(kernel, items * 4), kQThreads, 0, stm>>>(delta, ld_delta, s, Wq.codes, Wq.absmax, Wq.rows, Wq.cols, Wq.ld);
   count_launch();
   return cudaGetLastError() == cudaSuccess ? LOQT_OK : LOQT_ERR_CUDA;
 }

@@ -91,6 +91,34 @@ def test_merge(shape, sigma_B):
     assert np.all(got_c[:, inn:] == 7)
 
 
+@pytest.mark.parametrize("shape", SHAPES)
+def test_merge_split_matches_fused(shape):
+    # the two-pass merge takes the same accumulators through the same arithmetic
+    out, inn, r, _ = shape
+    h, d = _setup(16, out, inn, r, 8, 1e-2)
+    fused = L.loqt_merge_requant(d["Wq"].clone(), d["Pq"], d["B"], 0.5)
+    split = L.loqt_merge_requant_split(d["Wq"].clone(), d["Pq"], d["B"], 0.5)
+    assert torch.equal(fused.codes, split.codes) and torch.equal(fused.absmax, split.absmax)
+
+
+@pytest.mark.parametrize("shape", [(256, 256), (200, 136), (96, 5461), (1376, 512)])
+@pytest.mark.parametrize("s", [1.0, 0.5])
+def test_requantize_bit_exact(shape, s):
+    # s is a power of two, so s * delta is exact and the oracle's single rounding of
+    # the float64 sum equals the kernel's fused multiply-add.
+    out, inn = shape
+    h, d = _setup(17, out, inn, 8, 8)
+    delta = synth.normal(17, ("delta", out, inn), (out, inn), 5e-3, torch.float32)
+    delta[::7, ::5] = 0.0
+    ref_c, ref_m = O.nf4_requantize(h["wq"], delta.numpy(), s, inn)
+    ld = (inn + 3) // 4 * 4
+    dev_delta = torch.zeros((out, ld), dtype=torch.float32, device="cuda")[:, :inn]
+    dev_delta.copy_(delta)
+    L.loqt_nf4_requantize(dev_delta, s, d["Wq"])
+    got_c, got_m = from_dev_nf4(d["Wq"])
+    assert np.array_equal(got_c, ref_c) and np.array_equal(got_m, ref_m)
+
+
 def test_merge_zero_B_leaves_weights_untouched():
     out, inn, r = 256, 320, 32
     h, d = _setup(13, out, inn, r, 8)
