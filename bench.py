@@ -159,10 +159,13 @@ def pad_rows(t):
     return buf[:, :cols]
 
 
-def time_nf4_kernels(device, peaks, rows=8192, cols=8192, iters=10):
-    """The two streaming kernels on a matrix larger than L2 (fp32 source 268 MB):
+def time_nf4_kernels(device, peaks, rows=16384, cols=8192, iters=10):
+    """The streaming kernels on a matrix whose every stream exceeds twice the L2
+    (fp32 source 537 MB, bf16 output 268 MB; an output of about the L2 size runs
+    at half speed even for a plain fill):
     achieved GB/s on their algorithmic bytes (quantise 4 + 0.5625 B/element,
-    dequantise to bf16 0.5625 + 2 B/element) against the measured HBM copy rate."""
+    dequantise to bf16 0.5625 + 2 B/element, requantise 4 + 1.125 B/element) against
+    the measured HBM copy rate."""
     import torch
 
     from paper_2405_16528_b200 import binding as L
@@ -185,12 +188,17 @@ def time_nf4_kernels(device, peaks, rows=8192, cols=8192, iters=10):
     n = rows * cols
     ms_q = timed(lambda: L.loqt_nf4_quantize(w, q))
     ms_d = timed(lambda: L.loqt_nf4_dequantize(q, dst=out))
+    # the streaming half of the two-pass merge: W_q <- q(deq(W_q) + delta), 4 + 2 * 0.5625 B/element
+    w.mul_(0.05)
+    ms_r = timed(lambda: L.loqt_nf4_requantize(w, 1.0, q))
     gq = n * 4.5625 / (ms_q * 1e-3) / 1e9
     gd = n * 2.5625 / (ms_d * 1e-3) / 1e9
+    gr = n * 5.125 / (ms_r * 1e-3) / 1e9
     return {
         "shape": [rows, cols],
         "quantize_gb_s": round(gq, 1), "quantize_pct_hbm": round(100 * gq / peaks["hbm_gbs"], 1),
         "dequantize_bf16_gb_s": round(gd, 1), "dequantize_pct_hbm": round(100 * gd / peaks["hbm_gbs"], 1),
+        "requantize_gb_s": round(gr, 1), "requantize_pct_hbm": round(100 * gr / peaks["hbm_gbs"], 1),
         "of": peaks["source"],
     }
 

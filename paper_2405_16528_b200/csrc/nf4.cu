@@ -1,8 +1,9 @@
-// NF4 block quantise / dequantise streaming kernels (paper Section 5.1).
+// NF4 block quantise / requantise / dequantise streaming kernels (paper Section 5.1).
 //
-// Both kernels are HBM-bound: quantise moves 4 + 0.5625 bytes per element,
-// dequantise 0.5625 + 2 (bf16) or + 4 (fp32).  Eight threads share one block of
-// 64 weights; loads and stores are 128-bit where alignment allows.
+// All are HBM-bound: quantise moves 4 + 0.5625 bytes per element, requantise
+// 4 + 2 * 0.5625, dequantise 0.5625 + 2 (bf16) or + 4 (fp32).  Loads and stores
+// are 128-bit where alignment allows, and every thread keeps the next trip's
+// loads in flight while it works on the current one.
 #include "common.cuh"
 
 namespace loqt {
@@ -10,13 +11,22 @@ namespace loqt {
 constexpr int kQThreads = 256;
 
 // ---------------------------------------------------------------------------
-// quantise: fp32 [rows][ld_src] -> codes [rows][ld/2], absmax [rows][ld/64]
+// quantise:   fp32 [rows][ld_src] -> codes [rows][ld/2], absmax [rows][ld/64]
+// requantise: W_q <- q_NF4(deq32(W_q) + s * src), in place (the streaming half of
+//             the two-pass merge)
 // Four threads share one block of 64 weights; each owns 16 consecutive elements
-// (four 128-bit loads in flight, one 64-bit store of 16 codes).
+// (four 128-bit loads, one 64-bit store of 16 codes; the requantiser also loads
+// its 16 old codes and the block's old scale).
 // ---------------------------------------------------------------------------
-template <bool kVec>
+struct QuantItem {
+  uint32_t row, b;
+  int c0;
+  bool live;
+};
+
+template <bool kVec, bool kRequant>
 __global__ void __launch_bounds__(kQThreads)
-nf4_quantize_kernel(const float *__restrict__ src, int64_t ld_src, uint8_t *__restrict__ codes,
+nf4_quantize_kernel(const float *__restrict__ src, int64_t ld_src, float s, uint8_t *__restrict__ codes,
                     float *__restrict__ absmax, int rows, int cols, int ld) {
   __shared__ Nf4Tables tab;
   nf4_tables_init(tab, threadIdx.x);
@@ -30,15 +40,26 @@ nf4_quantize_kernel(const float *__restrict__ src, int64_t ld_src, uint8_t *__re
   // All threads of a warp run the same trip count: idle groups still take part in the shuffles.
   const uint32_t trips = (n_items + stride - 1) / stride;
 
-  for (uint32_t it = 0; it < trips; ++it) {
+  auto item_of = [&](uint32_t it) {
+    QuantItem q;
     const uint32_t item = group0 + it * stride;
-    const bool live = item < n_items;
-    const uint32_t row = live ? item / nb : 0;
-    const uint32_t b = live ? item - row * nb : 0;
-    const int c0 = static_cast<int>(b) * kBlock + 16 * static_cast<int>(l);
-    const float *p = src + static_cast<int64_t>(row) * ld_src + c0;
-    float v[16];
-    if (kVec && live && c0 + 16 <= cols) {
+    q.live = it < trips && item < n_items;
+    q.row = q.live ? item / nb : 0;
+    q.b = q.live ? item - q.row * nb : 0;
+    q.c0 = static_cast<int>(q.b) * kBlock + 16 * static_cast<int>(l);
+    return q;
+  };
+  // Issues the loads of one item: 16 source values and, for the requantiser, the
+  // 16 old codes and the old scale.  Elements past `cols` read as zero.
+  auto fetch = [&](const QuantItem &q, float (&v)[16], uint2 &old, float &Mold) {
+    const float *p = src + static_cast<int64_t>(q.row) * ld_src + q.c0;
+    old = make_uint2(kZeroWord, kZeroWord);
+    Mold = 0.0f;
+    if (kRequant && q.live) {
+      old = *reinterpret_cast<const uint2 *>(codes + static_cast<int64_t>(q.row) * (ld / 2) + (q.c0 >> 1));
+      Mold = absmax[static_cast<int64_t>(q.row) * nb + q.b];
+    }
+    if (kVec && q.live && q.c0 + 16 <= cols) {
 #pragma unroll
       for (int k = 0; k < 4; ++k) {
         const float4 a = __ldg(reinterpret_cast<const float4 *>(p) + k);
@@ -46,108 +67,56 @@ nf4_quantize_kernel(const float *__restrict__ src, int64_t ld_src, uint8_t *__re
       }
     } else {
 #pragma unroll
-      for (int j = 0; j < 16; ++j) v[j] = (live && c0 + j < cols) ? __ldg(p + j) : 0.0f;
+      for (int j = 0; j < 16; ++j) v[j] = (q.live && q.c0 + j < cols) ? __ldg(p + j) : 0.0f;
     }
-    float m = 0.0f;
-#pragma unroll
-    for (int j = 0; j < 16; ++j) m = fmaxf(m, fabsf(v[j]));
-    m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 1));
-    m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 2));
-    if (!live) continue;
+  };
 
-    uint2 w = make_uint2(kZeroWord, kZeroWord);
-    if (m > 0.0f) {
-      const Nf4Divisor d = nf4_divisor(m);
-      const float lo[8] = {v[0], v[1], v[2], v[3], v[4], v[5], v[6], v[7]};
-      const float hi[8] = {v[8], v[9], v[10], v[11], v[12], v[13], v[14], v[15]};
-      if (d.exact) {
-        w.x = nf4_quantize8<true>(tab, lo, d);
-        w.y = nf4_quantize8<true>(tab, hi, d);
-      } else {
-        w.x = nf4_quantize8<false>(tab, lo, d);
-        w.y = nf4_quantize8<false>(tab, hi, d);
-      }
-    }
-    uint8_t *crow = codes + static_cast<int64_t>(row) * (ld / 2) + (c0 >> 1);
-    *reinterpret_cast<uint2 *>(crow) = w;
-    if (l == 0) absmax[static_cast<int64_t>(row) * nb + b] = m;
-  }
-}
-
-// ---------------------------------------------------------------------------
-// requantise: W_q <- q_NF4(deq32(W_q) + s * delta), in place (the streaming half
-// of the two-pass merge).  Same thread layout as the quantiser: four threads per
-// block, 16 elements each (four 128-bit loads of delta, one 64-bit load and one
-// 64-bit store of codes).
-// ---------------------------------------------------------------------------
-template <bool kVec>
-__global__ void __launch_bounds__(kQThreads)
-nf4_requantize_kernel(const float *__restrict__ delta, int64_t ld_delta, float s, uint8_t *__restrict__ codes,
-                      float *__restrict__ absmax, int rows, int cols, int ld) {
-  __shared__ Nf4Tables tab;
-  nf4_tables_init(tab, threadIdx.x);
-  __syncthreads();
-
-  const uint32_t nb = static_cast<uint32_t>(ld / kBlock);
-  const uint32_t n_items = static_cast<uint32_t>(rows) * nb;
-  const uint32_t l = threadIdx.x & 3;
-  const uint32_t group0 = (blockIdx.x * kQThreads + threadIdx.x) >> 2;
-  const uint32_t stride = (gridDim.x * kQThreads) >> 2;
-  const uint32_t trips = (n_items + stride - 1) / stride;  // uniform: idle groups still shuffle
-
+  QuantItem cur = item_of(0);
+  float v[16], Mold;
+  uint2 old;
+  fetch(cur, v, old, Mold);
+#pragma unroll 1
   for (uint32_t it = 0; it < trips; ++it) {
-    const uint32_t item = group0 + it * stride;
-    const bool live = item < n_items;
-    const uint32_t row = live ? item / nb : 0;
-    const uint32_t b = live ? item - row * nb : 0;
-    const int c0 = static_cast<int>(b) * kBlock + 16 * static_cast<int>(l);
-    const float *p = delta + static_cast<int64_t>(row) * ld_delta + c0;
-    uint8_t *crow = codes + static_cast<int64_t>(row) * (ld / 2) + (c0 >> 1);
-    float *mp = absmax + static_cast<int64_t>(row) * nb + b;
-    float v[16];
-    uint2 old = make_uint2(kZeroWord, kZeroWord);
-    float Mold = 0.0f;
-    if (live) {
-      old = *reinterpret_cast<const uint2 *>(crow);
-      Mold = *mp;
-    }
-    if (kVec && live && c0 + 16 <= cols) {
-#pragma unroll
-      for (int k = 0; k < 4; ++k) {
-        const float4 a = __ldg(reinterpret_cast<const float4 *>(p) + k);
-        v[4 * k] = a.x; v[4 * k + 1] = a.y; v[4 * k + 2] = a.z; v[4 * k + 3] = a.w;
-      }
-    } else {
-#pragma unroll
-      for (int j = 0; j < 16; ++j) v[j] = (live && c0 + j < cols) ? __ldg(p + j) : 0.0f;  // padding: no update
-    }
+    const QuantItem nxt = item_of(it + 1);
+    float vn[16], Mn;
+    uint2 oldn;
+    fetch(nxt, vn, oldn, Mn);  // in flight while this item is quantised
+
     float m = 0.0f;
 #pragma unroll
     for (int j = 0; j < 16; ++j) {
-      const uint32_t code = ((j < 8 ? old.x : old.y) >> (4 * (j & 7))) & 15u;
-      v[j] = fmaf(s, v[j], Mold * tab.level[code]);
+      if (kRequant) {
+        const uint32_t code = ((j < 8 ? old.x : old.y) >> (4 * (j & 7))) & 15u;
+        v[j] = fmaf(s, v[j], Mold * tab.level[code]);
+      }
       m = fmaxf(m, fabsf(v[j]));
     }
-    // every thread of the block has read the old scale before lane 0 replaces it
+    // (requantiser: every thread of the block has read the old scale by now - the
+    // shuffles need its value - so lane 0 may replace it below)
     m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 1));
     m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 2));
-    if (!live) continue;
-
-    uint2 w = make_uint2(kZeroWord, kZeroWord);
-    if (m > 0.0f) {
-      const Nf4Divisor d = nf4_divisor(m);
-      const float lo[8] = {v[0], v[1], v[2], v[3], v[4], v[5], v[6], v[7]};
-      const float hi[8] = {v[8], v[9], v[10], v[11], v[12], v[13], v[14], v[15]};
-      if (d.exact) {
-        w.x = nf4_quantize8<true>(tab, lo, d);
-        w.y = nf4_quantize8<true>(tab, hi, d);
-      } else {
-        w.x = nf4_quantize8<false>(tab, lo, d);
-        w.y = nf4_quantize8<false>(tab, hi, d);
+    if (cur.live) {
+      uint2 w = make_uint2(kZeroWord, kZeroWord);
+      if (m > 0.0f) {
+        const Nf4Divisor d = nf4_divisor(m);
+        const float lo[8] = {v[0], v[1], v[2], v[3], v[4], v[5], v[6], v[7]};
+        const float hi[8] = {v[8], v[9], v[10], v[11], v[12], v[13], v[14], v[15]};
+        if (d.exact) {
+          w.x = nf4_quantize8<true>(tab, lo, d);
+          w.y = nf4_quantize8<true>(tab, hi, d);
+        } else {
+          w.x = nf4_quantize8<false>(tab, lo, d);
+          w.y = nf4_quantize8<false>(tab, hi, d);
+        }
       }
+      *reinterpret_cast<uint2 *>(codes + static_cast<int64_t>(cur.row) * (ld / 2) + (cur.c0 >> 1)) = w;
+      if (l == 0) absmax[static_cast<int64_t>(cur.row) * nb + cur.b] = m;
     }
-    *reinterpret_cast<uint2 *>(crow) = w;
-    if (l == 0) *mp = m;
+    cur = nxt;
+    old = oldn;
+    Mold = Mn;
+#pragma unroll
+    for (int j = 0; j < 16; ++j) v[j] = vn[j];
   }
 }
 
@@ -170,35 +139,48 @@ nf4_dequantize_kernel(const uint8_t *__restrict__ codes, const float *__restrict
   const uint32_t nb = static_cast<uint32_t>(ld / kBlock);
   const uint32_t n_items = static_cast<uint32_t>(rows) * wpr;  // (host checks < 2^31)
   const uint32_t stride = gridDim.x * kQThreads;
-  for (uint32_t base = blockIdx.x * kQThreads + threadIdx.x; base < n_items; base += kDqUnroll * stride) {
-    uint32_t w[kDqUnroll], row[kDqUnroll];
-    int c0[kDqUnroll];
-    float M[kDqUnroll];
-    bool live[kDqUnroll];
-#pragma unroll
-    for (int u = 0; u < kDqUnroll; ++u) {
-      const uint32_t item = base + u * stride;
-      live[u] = item < n_items;
-      row[u] = live[u] ? item / wpr : 0;
-      const uint32_t h = live[u] ? item - row[u] * wpr : 0;
-      c0[u] = static_cast<int>(h) * 8;
-      live[u] = live[u] && c0[u] < cols;
-      w[u] = kZeroWord;
-      M[u] = 0.0f;
-      if (live[u]) {
-        w[u] = __ldg(reinterpret_cast<const uint32_t *>(codes + static_cast<int64_t>(row[u]) * (ld / 2)) + h);
-        M[u] = __ldg(absmax + static_cast<int64_t>(row[u]) * nb + (h >> 3));
-      }
+  const uint32_t first = blockIdx.x * kQThreads + threadIdx.x;
+
+  struct Word {
+    uint32_t w, row;
+    int c0;
+    float M;
+    bool live;
+  };
+  auto fetch = [&](uint32_t item) {
+    Word q;
+    q.live = item < n_items;
+    q.row = q.live ? item / wpr : 0;
+    const uint32_t h = q.live ? item - q.row * wpr : 0;
+    q.c0 = static_cast<int>(h) * 8;
+    q.live = q.live && q.c0 < cols;
+    q.w = kZeroWord;
+    q.M = 0.0f;
+    if (q.live) {
+      q.w = __ldg(reinterpret_cast<const uint32_t *>(codes + static_cast<int64_t>(q.row) * (ld / 2)) + h);
+      q.M = __ldg(absmax + static_cast<int64_t>(q.row) * nb + (h >> 3));
     }
+    return q;
+  };
+
+  Word cur[kDqUnroll];
+#pragma unroll
+  for (int u = 0; u < kDqUnroll; ++u) cur[u] = fetch(first + u * stride);
+#pragma unroll 1
+  for (uint32_t base = first; base < n_items; base += kDqUnroll * stride) {
+    Word nxt[kDqUnroll];  // in flight while this trip's words are expanded
+#pragma unroll
+    for (int u = 0; u < kDqUnroll; ++u) nxt[u] = fetch(base + (kDqUnroll + u) * stride);
 #pragma unroll
     for (int u = 0; u < kDqUnroll; ++u) {
-      if (!live[u]) continue;
+      const Word &q = cur[u];
+      if (!q.live) continue;
       float v[8];
 #pragma unroll
-      for (int j = 0; j < 8; ++j) v[j] = M[u] * tab.level[(w[u] >> (4 * j)) & 15u];
-      const bool full = kVec && (c0[u] + 8 <= cols);
+      for (int j = 0; j < 8; ++j) v[j] = q.M * tab.level[(q.w >> (4 * j)) & 15u];
+      const bool full = kVec && (q.c0 + 8 <= cols);
       if (kBf16) {
-        __nv_bfloat16 *o = reinterpret_cast<__nv_bfloat16 *>(dst) + static_cast<int64_t>(row[u]) * ld_dst + c0[u];
+        __nv_bfloat16 *o = reinterpret_cast<__nv_bfloat16 *>(dst) + static_cast<int64_t>(q.row) * ld_dst + q.c0;
         if (full) {
           uint4 pk;
           pk.x = pack_bf16x2(v[0], v[1]);
@@ -209,20 +191,22 @@ nf4_dequantize_kernel(const uint8_t *__restrict__ codes, const float *__restrict
         } else {
 #pragma unroll
           for (int j = 0; j < 8; ++j)
-            if (c0[u] + j < cols) o[j] = __float2bfloat16_rn(v[j]);
+            if (q.c0 + j < cols) o[j] = __float2bfloat16_rn(v[j]);
         }
       } else {
-        float *o = reinterpret_cast<float *>(dst) + static_cast<int64_t>(row[u]) * ld_dst + c0[u];
+        float *o = reinterpret_cast<float *>(dst) + static_cast<int64_t>(q.row) * ld_dst + q.c0;
         if (full) {
           reinterpret_cast<float4 *>(o)[0] = make_float4(v[0], v[1], v[2], v[3]);
           reinterpret_cast<float4 *>(o)[1] = make_float4(v[4], v[5], v[6], v[7]);
         } else {
 #pragma unroll
           for (int j = 0; j < 8; ++j)
-            if (c0[u] + j < cols) o[j] = v[j];
+            if (q.c0 + j < cols) o[j] = v[j];
         }
       }
     }
+#pragma unroll
+    for (int u = 0; u < kDqUnroll; ++u) cur[u] = nxt[u];
   }
 }
 
@@ -253,8 +237,8 @@ extern "C" loqt_status loqt_nf4_quantize(const float *src, int64_t ld_src, loqt_
   if (items >= (1ll << 30)) return LOQT_ERR_UNSUPPORTED;  // 32-bit block indices in the kernel
   const bool vec = (reinterpret_cast<uintptr_t>(src) & 15u) == 0 && (ld_src % 4) == 0;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
-  auto kernel = vec ? nf4_quantize_kernel<true> : nf4_quantize_kernel<false>;
-  kernel<<<grid_for(kernel, items * 4), kQThreads, 0, s>>>(src, ld_src, dst.codes, dst.absmax, dst.rows, dst.cols, dst.ld);
+  auto kernel = vec ? nf4_quantize_kernel<true, false> : nf4_quantize_kernel<false, false>;
+  kernel<<<grid_for(kernel, items * 4), kQThreads, 0, s>>>(src, ld_src, 1.0f, dst.codes, dst.absmax, dst.rows, dst.cols, dst.ld);
   count_launch();
   return cudaGetLastError() == cudaSuccess ? LOQT_OK : LOQT_ERR_CUDA;
 }
@@ -289,7 +273,7 @@ extern "C" loqt_status loqt_nf4_requantize(const float *delta, int64_t ld_delta,
   if (items >= (1ll << 30)) return LOQT_ERR_UNSUPPORTED;  // 32-bit block indices in the kernel
   const bool vec = (reinterpret_cast<uintptr_t>(delta) & 15u) == 0 && (ld_delta % 4) == 0;
   cudaStream_t stm = static_cast<cudaStream_t>(stream);
-  auto kernel = vec ? nf4_requantize_kernel<true> : nf4_requantize_kernel<false>;
+  auto kernel = vec ? nf4_quantize_kernel<true, true> : nf4_quantize_kernel<false, true>;
   kernel<<<grid_for(kernel, items * 4), kQThreads, 0, stm>>>(delta, ld_delta, s, Wq.codes, Wq.absmax, Wq.rows, Wq.cols, Wq.ld);
   count_launch();
   return cudaGetLastError() == cudaSuccess ? LOQT_OK : LOQT_ERR_CUDA;
