@@ -101,17 +101,28 @@ struct SmemLayout {
   static constexpr int kBNL = TWO ? BN / 2 : BN;  // B rows staged by this CTA
   static constexpr int kABytes = kBM * kBK * 2;
   static constexpr int kBBytes = kBNL * kBK * 2;
-  static constexpr int kCodeBytes = 8192;  // up to 256 blocks x 32 bytes
-  static constexpr int kStageBytes = kABytes + kBBytes + kCodeBytes;
-  static constexpr int kStages = (225 * 1024 / kStageBytes) < 6 ? (225 * 1024 / kStageBytes) : 6;
-  static constexpr int kBarOffset = kStages * kStageBytes;
-  // full[S], empty[S], codes[S], tfull[2], tempty[2], drain
-  static constexpr int kNumBars = 3 * kStages + 5;
+  static constexpr int kCodeBytes = 8192;  // one code tile: up to 256 blocks x 32 bytes
+  // Packed codes travel in a ring of their own, kCodeLead stages ahead of the
+  // operand ring, so that a freed operand slot can be dequantised into at once
+  // instead of waiting for its codes to arrive.
+  static constexpr int kStageBytes = kABytes + kBBytes;
+  // The code ring is at least as deep as the operand ring (a staging group that has
+  // seen operand slot `it` released may then conclude that the codes of stage
+  // `it - kCodeStages` were consumed, which keeps its parity test unambiguous).
+  static constexpr int stages_for(int s) { return s * kStageBytes + (s > 4 ? s : 4) * kCodeBytes <= 225 * 1024; }
+  static constexpr int kStages = stages_for(6) ? 6 : stages_for(5) ? 5 : stages_for(4) ? 4 : stages_for(3) ? 3 : 2;
+  static constexpr int kCodeStages = kStages > 4 ? kStages : 4;
+  static constexpr int kCodeLead = 2;
+  static constexpr int kCodeOffset = kStages * kStageBytes;
+  static constexpr int kBarOffset = kCodeOffset + kCodeStages * kCodeBytes;
+  // full[S], empty[S], cfull[C], cempty[C], tfull[2], tempty[2], drain
+  static constexpr int kNumBars = 2 * kStages + 2 * kCodeStages + 5;
   static constexpr int kMiscOffset = kBarOffset + kNumBars * 8;
   static constexpr int kTablesOffset = kMiscOffset + 16;
   static constexpr int kTotal = kTablesOffset + static_cast<int>(sizeof(Nf4Tables));
   static constexpr int kDynamicBytes = kTotal + 1024;  // slack for 1024-byte alignment
   static_assert(kStages >= 3, "pipeline too shallow");
+  static_assert(kCodeStages >= kStages && kCodeLead + 2 <= kCodeStages, "code ring too shallow");
   static_assert(kDynamicBytes <= 232448, "exceeds the 227 KiB shared memory of one CTA");
   static_assert(kBM * 32 <= kCodeBytes && kBNL * 32 <= kCodeBytes, "code tile too large");
   static_assert(!TWO || BN == 256, "pairs run 256-wide tiles");
@@ -325,10 +336,12 @@ loqt_gemm_kernel(const __grid_constant__ TensorMaps maps, const GemmParams p) {
   const uint32_t bar0 = smem_base + L::kBarOffset;
   auto full_bar = [&](int s) { return bar0 + 8u * s; };
   auto empty_bar = [&](int s) { return bar0 + 8u * (kStages + s); };
-  auto codes_bar = [&](int s) { return bar0 + 8u * (2 * kStages + s); };
-  auto tfull_bar = [&](int a) { return bar0 + 8u * (3 * kStages + a); };
-  auto tempty_bar = [&](int a) { return bar0 + 8u * (3 * kStages + 2 + a); };
-  const uint32_t drain_bar = bar0 + 8u * (3 * kStages + 4);
+  constexpr int kCodeStages = L::kCodeStages;
+  auto cfull_bar = [&](int c) { return bar0 + 8u * (2 * kStages + c); };
+  auto cempty_bar = [&](int c) { return bar0 + 8u * (2 * kStages + kCodeStages + c); };
+  auto tfull_bar = [&](int a) { return bar0 + 8u * (2 * kStages + 2 * kCodeStages + a); };
+  auto tempty_bar = [&](int a) { return bar0 + 8u * (2 * kStages + 2 * kCodeStages + 2 + a); };
+  const uint32_t drain_bar = bar0 + 8u * (2 * kStages + 2 * kCodeStages + 4);
   volatile uint32_t *misc = reinterpret_cast<volatile uint32_t *>(smem_gen + L::kMiscOffset);
   volatile uint32_t *tmem_slot = misc;       // written by tcgen05.alloc
   volatile uint32_t *abort_flag = misc + 1;  // raised by any role whose wait expired
@@ -369,7 +382,10 @@ loqt_gemm_kernel(const __grid_constant__ TensorMaps maps, const GemmParams p) {
       // the dequant warps of every CTA of the pair
       ptx::mbar_init(full_bar(s), 1 + (p.has_nf4 ? kGroupWarps * (TWO ? 2 : 1) : 0));
       ptx::mbar_init(empty_bar(s), 1);
-      ptx::mbar_init(codes_bar(s), 1);
+    }
+    for (int c = 0; c < kCodeStages; ++c) {
+      ptx::mbar_init(cfull_bar(c), 1);             // the producer (with the tile's bytes, if any)
+      ptx::mbar_init(cempty_bar(c), kGroupWarps);  // the staging group that used the tile
     }
     for (int a = 0; a < 2; ++a) {
       ptx::mbar_init(tfull_bar(a), 1);
@@ -477,20 +493,24 @@ loqt_gemm_kernel(const __grid_constant__ TensorMaps maps, const GemmParams p) {
     }
     const int s = cur.it % kStages;
     const uint32_t ph = (cur.it / kStages) & 1u;
-    // First the slot's release (the same event the producer waits for): groups share
-    // slots, and a group that ran a whole ring ahead of the others would otherwise
-    // test the code barrier two phases early and read "already complete".  Then the
-    // code tile of this stage.
+    // First the operand slot's release (the same event the producer waits for), then
+    // the code tile of this stage.  The order matters: once stage `it - kStages` has
+    // been consumed, every stage up to `it - kCodeStages` has been staged, so the code
+    // barrier cannot still be in the phase two uses back, which a parity test would
+    // read as "already complete".
+    const int cs = cur.it % kCodeStages;
+    const uint32_t cph = (cur.it / kCodeStages) & 1u;
     if (!ptx::mbar_wait<TWO>(empty_bar(s), ph ^ 1u, abort_flag, p.status)) return false;
-    if (!ptx::mbar_wait(codes_bar(s), ph, abort_flag, p.status)) return false;
+    if (!ptx::mbar_wait(cfull_bar(cs), cph, abort_flag, p.status)) return false;
     const uint32_t stage_base = smem_base + s * L::kStageBytes;
-    const uint32_t code_base = stage_base + L::kABytes + L::kBBytes;
+    const uint32_t code_base = smem_base + L::kCodeOffset + cs * L::kCodeBytes;
     deq_store<0>(cur.g, task0, stage_base, code_base);
     if (kTwoRows) deq_store<1>(cur.g, task1, stage_base, code_base);
     if (TWO) ptx::fence_proxy_async_all();
     else ptx::fence_proxy_async_smem();
     __syncwarp();
     if (lane == 0) {
+      ptx::mbar_arrive(cempty_bar(cs));  // code tile read: the producer may refill it
       if (TWO && !leader) ptx::mbar_arrive_cluster(ptx::map_to_cta(full_bar(s), 0));
       else ptx::mbar_arrive(full_bar(s));
     }
@@ -509,8 +529,60 @@ loqt_gemm_kernel(const __grid_constant__ TensorMaps maps, const GemmParams p) {
         ptx::prefetch_tensormap(p.seg[s].a_kind <= OP_TMA_MN ? &maps.a[s] : &maps.ca[s]);
         ptx::prefetch_tensormap(p.seg[s].b_kind <= OP_TMA_MN ? &maps.b[s] : &maps.cb[s]);
       }
-      uint32_t it = 0;
+      // Code tiles run kCodeLead stages ahead of the operands: a second cursor over
+      // the same sequence of stages.
+      struct CodeCursor {
+        int u, kb, kb_hi, m_blk, n_blk;
+        uint32_t it;
+        bool valid;
+      };
+      auto cc_open = [&](CodeCursor &c) {
+        while (c.u < sched.units) {
+          int split, lo;
+          sched.unit(c.u, c.m_blk, c.n_blk, split, lo, c.kb_hi);
+          c.kb = lo;
+          if (c.kb < c.kb_hi) return true;
+          c.u += gridDim.x;
+        }
+        return false;
+      };
       bool ok = true;
+      // Posts the code tile of the cursor's stage (or an empty completion when the
+      // stage has no NF4 operand) and moves the cursor on.
+      auto issue_codes = [&](CodeCursor &c) {
+        const int cs = c.it % kCodeStages;
+        const uint32_t cph = (c.it / kCodeStages) & 1u;
+        if (!(ok = ptx::mbar_wait(cempty_bar(cs), cph ^ 1u, abort_flag, p.status))) return;
+        const int sidx = c.kb < sched.kb_seg0 ? 0 : 1;
+        const int k0 = (sidx == 0 ? c.kb : c.kb - sched.kb_seg0) * kBK;
+        const Segment &sg = p.seg[sidx];
+        const int n_row0 = c.n_blk * BN + (TWO ? static_cast<int>(rank) * kBNL : 0);
+        const uint32_t c_dst = smem_base + L::kCodeOffset + cs * L::kCodeBytes;
+        if (sg.a_kind == OP_NF4_K) {
+          ptx::mbar_arrive_expect_tx(cfull_bar(cs), kBM * 32);
+          ptx::tma_load_2d(c_dst, &maps.ca[sidx], cfull_bar(cs), k0 >> 1, c.m_blk * kBM);
+        } else if (sg.b_kind == OP_NF4_K) {
+          ptx::mbar_arrive_expect_tx(cfull_bar(cs), kBNL * 32);
+          ptx::tma_load_2d(c_dst, &maps.cb[sidx], cfull_bar(cs), k0 >> 1, n_row0);
+        } else if (sg.b_kind == OP_NF4_MN) {
+          ptx::mbar_arrive_expect_tx(cfull_bar(cs), kBNL * 32);
+          ptx::tma_load_2d(c_dst, &maps.cb[sidx], cfull_bar(cs), n_row0 >> 1, k0);
+        } else {
+          ptx::mbar_arrive(cfull_bar(cs));  // nothing to dequantise in this stage
+        }
+        ++c.it;
+        if (++c.kb >= c.kb_hi) {
+          c.u += gridDim.x;
+          c.valid = cc_open(c);
+        }
+      };
+      CodeCursor cc;
+      cc.u = blockIdx.x;
+      cc.it = 0;
+      cc.valid = p.has_nf4 && cc_open(cc);
+      for (int i = 0; ok && i < L::kCodeLead && cc.valid; ++i) issue_codes(cc);
+
+      uint32_t it = 0;
       for (int u = blockIdx.x; ok && u < sched.units; u += gridDim.x) {
         int m_blk, n_blk, split, kb_lo, kb_hi;
         sched.unit(u, m_blk, n_blk, split, kb_lo, kb_hi);
@@ -528,22 +600,6 @@ loqt_gemm_kernel(const __grid_constant__ TensorMaps maps, const GemmParams p) {
           const Segment &sg = p.seg[sidx];
           const uint32_t a_dst = smem_base + s * L::kStageBytes;
           const uint32_t b_dst = a_dst + L::kABytes;
-          const uint32_t c_dst = b_dst + L::kBBytes;
-          // packed codes of the stage's NF4 operand (if any) -> this CTA's code tile
-          if (p.has_nf4) {
-            if (sg.a_kind == OP_NF4_K) {
-              ptx::mbar_arrive_expect_tx(codes_bar(s), kBM * 32);
-              ptx::tma_load_2d(c_dst, &maps.ca[sidx], codes_bar(s), k0 >> 1, m_blk * kBM);
-            } else if (sg.b_kind == OP_NF4_K) {
-              ptx::mbar_arrive_expect_tx(codes_bar(s), kBNL * 32);
-              ptx::tma_load_2d(c_dst, &maps.cb[sidx], codes_bar(s), k0 >> 1, n_row0);
-            } else if (sg.b_kind == OP_NF4_MN) {
-              ptx::mbar_arrive_expect_tx(codes_bar(s), kBNL * 32);
-              ptx::tma_load_2d(c_dst, &maps.cb[sidx], codes_bar(s), n_row0 >> 1, k0);
-            } else {
-              ptx::mbar_arrive(codes_bar(s));  // nothing to dequantise in this stage
-            }
-          }
           uint32_t bytes = 0;
           if (sg.a_kind <= OP_TMA_MN) bytes += L::kABytes;
           if (sg.b_kind <= OP_TMA_MN) bytes += L::kBBytes;
@@ -566,6 +622,10 @@ loqt_gemm_kernel(const __grid_constant__ TensorMaps maps, const GemmParams p) {
           } else if (sg.b_kind == OP_TMA_MN) {
 #pragma unroll
             for (int j = 0; j < kBNL / 64; ++j) load(b_dst + j * 8192, &maps.b[sidx], n_row0 + 64 * j, k0);
+          }
+          if (cc.valid) {
+            issue_codes(cc);
+            if (!ok) break;
           }
         }
       }
