@@ -18,14 +18,20 @@
 // accumulators but stages only half of the B tile (128 of the 256 N rows), and
 // one thread of the leader CTA issues M = 256 instructions that drive both SMs'
 // tensor cores.  Per SM this halves the dequantisation work, the B bytes written
-// to shared memory and the B bytes the tensor core reads from it.  Barriers the
-// MMA thread waits on live in the leader; the follower arrives on them through
-// the cluster's shared-memory window, and the leader forwards "slot free" and
-// "accumulator ready" to the follower the same way.
+// to shared memory and the B bytes the tensor core reads from it - and shared
+// memory bandwidth is what bounds a single CTA here (per 256 x 256 x 64 stage the
+// tensor core reads 96 KiB, TMA writes 40 KiB and the dequant warps move 40 KiB
+// through a 128 B/clk port).  Barriers the MMA thread waits on live in the
+// leader; the follower arrives on them through the cluster's shared-memory
+// window.  "Slot free" and "accumulator ready" reach both CTAs at once: the
+// commit that signals them is delivered to the same barrier in each CTA.
 //
-// Warp roles (448 threads): warp 0 TMA producer, warp 1 MMA issuer + TMEM
-// owner, warps 2-5 epilogue (one per TMEM lane quarter), warps 6-13 NF4
-// dequantisation.  One CTA per SM.
+// Warp roles (480 threads): warp 0 TMA producer of the bf16 operands, warp 1
+// MMA issuer + TMEM owner, warps 2-5 epilogue (one per TMEM lane quarter), warps
+// 6-13 NF4 dequantisation, warp 14 TMA producer of the packed codes (a producer
+// thread spends several hundred cycles per stage on its chain of barrier and
+// copy instructions; one thread for both rings was the pipeline's bottleneck).
+// One CTA per SM.
 #pragma once
 #include <type_traits>
 #include "nf4_dequant.cuh"
@@ -36,10 +42,11 @@ namespace loqt {
 constexpr int kHM = 128;      // rows of one MMA (M of tcgen05.mma)
 constexpr int kBK = 64;       // K elements per pipeline stage (one 128-byte swizzle row of bf16)
 constexpr int kUmmaK = 16;    // K of one tcgen05.mma for 16-bit inputs
-constexpr int kNumThreads = 448;
+constexpr int kNumThreads = 480;
 constexpr int kEpiWarp0 = 2;  // warps 2..5
 constexpr int kDeqWarp0 = 6;  // warps 6..13
 constexpr int kDeqWarps = 8;
+constexpr int kCodeWarp = 14;  // one thread: TMA producer of the packed NF4 codes
 
 // Operand kinds
 enum : int {
@@ -102,8 +109,8 @@ struct SmemLayout {
   static constexpr int kABytes = kBM * kBK * 2;
   static constexpr int kBBytes = kBNL * kBK * 2;
   static constexpr int kCodeBytes = 8192;  // one code tile: up to 256 blocks x 32 bytes
-  // Packed codes travel in a ring of their own, kCodeLead stages ahead of the
-  // operand ring, so that a freed operand slot can be dequantised into at once
+  // Packed codes travel in a ring of their own with their own producer, ahead of
+  // the operand ring, so that a freed operand slot can be dequantised into at once
   // instead of waiting for its codes to arrive.
   static constexpr int kStageBytes = kABytes + kBBytes;
   // The code ring is at least as deep as the operand ring (a staging group that has
@@ -112,7 +119,6 @@ struct SmemLayout {
   static constexpr int stages_for(int s) { return s * kStageBytes + (s > 4 ? s : 4) * kCodeBytes <= 225 * 1024; }
   static constexpr int kStages = stages_for(6) ? 6 : stages_for(5) ? 5 : stages_for(4) ? 4 : stages_for(3) ? 3 : 2;
   static constexpr int kCodeStages = kStages > 4 ? kStages : 4;
-  static constexpr int kCodeLead = 2;
   static constexpr int kCodeOffset = kStages * kStageBytes;
   static constexpr int kBarOffset = kCodeOffset + kCodeStages * kCodeBytes;
   // full[S], empty[S], cfull[C], cempty[C], tfull[2], tempty[2], drain
@@ -122,7 +128,7 @@ struct SmemLayout {
   static constexpr int kTotal = kTablesOffset + static_cast<int>(sizeof(Nf4Tables));
   static constexpr int kDynamicBytes = kTotal + 1024;  // slack for 1024-byte alignment
   static_assert(kStages >= 3, "pipeline too shallow");
-  static_assert(kCodeStages >= kStages && kCodeLead + 2 <= kCodeStages, "code ring too shallow");
+  static_assert(kCodeStages >= kStages, "code ring too shallow");
   static_assert(kDynamicBytes <= 232448, "exceeds the 227 KiB shared memory of one CTA");
   static_assert(kBM * 32 <= kCodeBytes && kBNL * 32 <= kCodeBytes, "code tile too large");
   static_assert(!TWO || BN == 256, "pairs run 256-wide tiles");
@@ -351,9 +357,8 @@ loqt_gemm_kernel(const __grid_constant__ TensorMaps maps, const GemmParams p) {
   const int lane = threadIdx.x & 31;
   const Sched sched(p, kBM, BN);
   // TWO: rank 0 of the pair is the leader (issues the MMAs, owns the barriers the
-  // MMA thread waits on); `peer` is the other CTA's rank.
+  // MMA thread waits on).
   const uint32_t rank = TWO ? ptx::cluster_ctarank() : 0u;
-  const uint32_t peer = rank ^ 1u;
   const bool leader = (rank == 0);
   // The requantising epilogue of the merge is the heaviest one, so dequant warps
   // that have nothing to stage join it in groups of four (one warp per TMEM lane
@@ -506,8 +511,7 @@ loqt_gemm_kernel(const __grid_constant__ TensorMaps maps, const GemmParams p) {
     const uint32_t code_base = smem_base + L::kCodeOffset + cs * L::kCodeBytes;
     deq_store<0>(cur.g, task0, stage_base, code_base);
     if (kTwoRows) deq_store<1>(cur.g, task1, stage_base, code_base);
-    if (TWO) ptx::fence_proxy_async_all();
-    else ptx::fence_proxy_async_smem();
+    ptx::fence_proxy_async_smem();  // (pairs too: the writes are to this CTA's own shared memory)
     __syncwarp();
     if (lane == 0) {
       ptx::mbar_arrive(cempty_bar(cs));  // code tile read: the producer may refill it
@@ -529,59 +533,7 @@ loqt_gemm_kernel(const __grid_constant__ TensorMaps maps, const GemmParams p) {
         ptx::prefetch_tensormap(p.seg[s].a_kind <= OP_TMA_MN ? &maps.a[s] : &maps.ca[s]);
         ptx::prefetch_tensormap(p.seg[s].b_kind <= OP_TMA_MN ? &maps.b[s] : &maps.cb[s]);
       }
-      // Code tiles run kCodeLead stages ahead of the operands: a second cursor over
-      // the same sequence of stages.
-      struct CodeCursor {
-        int u, kb, kb_hi, m_blk, n_blk;
-        uint32_t it;
-        bool valid;
-      };
-      auto cc_open = [&](CodeCursor &c) {
-        while (c.u < sched.units) {
-          int split, lo;
-          sched.unit(c.u, c.m_blk, c.n_blk, split, lo, c.kb_hi);
-          c.kb = lo;
-          if (c.kb < c.kb_hi) return true;
-          c.u += gridDim.x;
-        }
-        return false;
-      };
       bool ok = true;
-      // Posts the code tile of the cursor's stage (or an empty completion when the
-      // stage has no NF4 operand) and moves the cursor on.
-      auto issue_codes = [&](CodeCursor &c) {
-        const int cs = c.it % kCodeStages;
-        const uint32_t cph = (c.it / kCodeStages) & 1u;
-        if (!(ok = ptx::mbar_wait(cempty_bar(cs), cph ^ 1u, abort_flag, p.status))) return;
-        const int sidx = c.kb < sched.kb_seg0 ? 0 : 1;
-        const int k0 = (sidx == 0 ? c.kb : c.kb - sched.kb_seg0) * kBK;
-        const Segment &sg = p.seg[sidx];
-        const int n_row0 = c.n_blk * BN + (TWO ? static_cast<int>(rank) * kBNL : 0);
-        const uint32_t c_dst = smem_base + L::kCodeOffset + cs * L::kCodeBytes;
-        if (sg.a_kind == OP_NF4_K) {
-          ptx::mbar_arrive_expect_tx(cfull_bar(cs), kBM * 32);
-          ptx::tma_load_2d(c_dst, &maps.ca[sidx], cfull_bar(cs), k0 >> 1, c.m_blk * kBM);
-        } else if (sg.b_kind == OP_NF4_K) {
-          ptx::mbar_arrive_expect_tx(cfull_bar(cs), kBNL * 32);
-          ptx::tma_load_2d(c_dst, &maps.cb[sidx], cfull_bar(cs), k0 >> 1, n_row0);
-        } else if (sg.b_kind == OP_NF4_MN) {
-          ptx::mbar_arrive_expect_tx(cfull_bar(cs), kBNL * 32);
-          ptx::tma_load_2d(c_dst, &maps.cb[sidx], cfull_bar(cs), n_row0 >> 1, k0);
-        } else {
-          ptx::mbar_arrive(cfull_bar(cs));  // nothing to dequantise in this stage
-        }
-        ++c.it;
-        if (++c.kb >= c.kb_hi) {
-          c.u += gridDim.x;
-          c.valid = cc_open(c);
-        }
-      };
-      CodeCursor cc;
-      cc.u = blockIdx.x;
-      cc.it = 0;
-      cc.valid = p.has_nf4 && cc_open(cc);
-      for (int i = 0; ok && i < L::kCodeLead && cc.valid; ++i) issue_codes(cc);
-
       uint32_t it = 0;
       for (int u = blockIdx.x; ok && u < sched.units; u += gridDim.x) {
         int m_blk, n_blk, split, kb_lo, kb_hi;
@@ -592,9 +544,6 @@ loqt_gemm_kernel(const __grid_constant__ TensorMaps maps, const GemmParams p) {
           const int s = it % kStages;
           const uint32_t ph = (it / kStages) & 1u;
           if (!(ok = ptx::mbar_wait<TWO>(empty_bar(s), ph ^ 1u, abort_flag, p.status))) break;
-          // the MMA thread frees a slot on the leader's barrier; pass it on
-          // (only real releases: the first pass over the ring waits for nothing)
-          if (TWO && leader && it >= static_cast<uint32_t>(kStages)) ptx::mbar_arrive_cluster(ptx::map_to_cta(empty_bar(s), peer));
           const int sidx = kb < sched.kb_seg0 ? 0 : 1;
           const int k0 = (sidx == 0 ? kb : kb - sched.kb_seg0) * kBK;
           const Segment &sg = p.seg[sidx];
@@ -622,10 +571,6 @@ loqt_gemm_kernel(const __grid_constant__ TensorMaps maps, const GemmParams p) {
           } else if (sg.b_kind == OP_TMA_MN) {
 #pragma unroll
             for (int j = 0; j < kBNL / 64; ++j) load(b_dst + j * 8192, &maps.b[sidx], n_row0 + 64 * j, k0);
-          }
-          if (cc.valid) {
-            issue_codes(cc);
-            if (!ok) break;
           }
         }
       }
@@ -677,11 +622,11 @@ loqt_gemm_kernel(const __grid_constant__ TensorMaps maps, const GemmParams p) {
             }
           }
           // stage reusable (in both CTAs) once these MMAs have read it
-          if (TWO) ptx::mma_commit_pair(empty_bar(s));
+          if (TWO) ptx::mma_commit_pair_both(empty_bar(s));
           else ptx::mma_commit(empty_bar(s));
         }
         if (ok) {
-          if (TWO) ptx::mma_commit_pair(tfull_bar(acc));
+          if (TWO) ptx::mma_commit_pair_both(tfull_bar(acc));
           else ptx::mma_commit(tfull_bar(acc));
         }
       }
@@ -689,6 +634,64 @@ loqt_gemm_kernel(const __grid_constant__ TensorMaps maps, const GemmParams p) {
       if (TWO) ptx::mma_commit_pair(drain_bar);
       else ptx::mma_commit(drain_bar);
       ptx::mbar_wait<TWO>(drain_bar, 0, abort_flag, p.status);
+    }
+  }
+  // =========================================================== code producer
+  else if (warp == kCodeWarp) {
+    if (lane == 0 && p.has_nf4) {
+      // A cursor over the same sequence of stages as the operand producer's; the
+      // ring's depth bounds how far the codes run ahead.
+      struct CodeCursor {
+        int u, kb, kb_hi, m_blk, n_blk;
+        uint32_t it;
+        bool valid;
+      };
+      auto cc_open = [&](CodeCursor &c) {
+        while (c.u < sched.units) {
+          int split, lo;
+          sched.unit(c.u, c.m_blk, c.n_blk, split, lo, c.kb_hi);
+          c.kb = lo;
+          if (c.kb < c.kb_hi) return true;
+          c.u += gridDim.x;
+        }
+        return false;
+      };
+      bool ok = true;
+      // Posts the code tile of the cursor's stage (or an empty completion when the
+      // stage has no NF4 operand) and moves the cursor on.
+      auto issue_codes = [&](CodeCursor &c) {
+        const int cs = c.it % kCodeStages;
+        const uint32_t cph = (c.it / kCodeStages) & 1u;
+        if (!(ok = ptx::mbar_wait(cempty_bar(cs), cph ^ 1u, abort_flag, p.status))) return;
+        const int sidx = c.kb < sched.kb_seg0 ? 0 : 1;
+        const int k0 = (sidx == 0 ? c.kb : c.kb - sched.kb_seg0) * kBK;
+        const Segment &sg = p.seg[sidx];
+        const int n_row0 = c.n_blk * BN + (TWO ? static_cast<int>(rank) * kBNL : 0);
+        const uint32_t c_dst = smem_base + L::kCodeOffset + cs * L::kCodeBytes;
+        if (sg.a_kind == OP_NF4_K) {
+          ptx::mbar_arrive_expect_tx(cfull_bar(cs), kBM * 32);
+          ptx::tma_load_2d(c_dst, &maps.ca[sidx], cfull_bar(cs), k0 >> 1, c.m_blk * kBM);
+        } else if (sg.b_kind == OP_NF4_K) {
+          ptx::mbar_arrive_expect_tx(cfull_bar(cs), kBNL * 32);
+          ptx::tma_load_2d(c_dst, &maps.cb[sidx], cfull_bar(cs), k0 >> 1, n_row0);
+        } else if (sg.b_kind == OP_NF4_MN) {
+          ptx::mbar_arrive_expect_tx(cfull_bar(cs), kBNL * 32);
+          ptx::tma_load_2d(c_dst, &maps.cb[sidx], cfull_bar(cs), n_row0 >> 1, k0);
+        } else {
+          ptx::mbar_arrive(cfull_bar(cs));  // nothing to dequantise in this stage
+        }
+        ++c.it;
+        if (++c.kb >= c.kb_hi) {
+          c.u += gridDim.x;
+          c.valid = cc_open(c);
+        }
+      };
+      CodeCursor cc;
+      cc.u = blockIdx.x;
+      cc.it = 0;
+      cc.valid = p.has_nf4 && cc_open(cc);
+      while (ok && cc.valid) issue_codes(cc);
+
     }
   }
   // =========================================================== epilogue
@@ -703,8 +706,6 @@ loqt_gemm_kernel(const __grid_constant__ TensorMaps maps, const GemmParams p) {
       const uint32_t acc = tile % kAccBufs;
       const uint32_t acc_ph = (tile / kAccBufs) & 1u;
       if (!(ok = ptx::mbar_wait<TWO>(tfull_bar(acc), acc_ph, abort_flag, p.status))) break;
-      // the MMA thread signals the leader's barrier; one leader warp passes it on
-      if (TWO && leader && warp == kEpiWarp0 && lane == 0) ptx::mbar_arrive_cluster(ptx::map_to_cta(tfull_bar(acc), peer));
       ptx::tc_fence_after();
       const int n_base = n_blk * BN;
 #pragma unroll 1

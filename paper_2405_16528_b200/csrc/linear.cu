@@ -93,7 +93,7 @@ constexpr double kCyclesFixed = 3000.0;
 
 // Run eligible products as tcgen05 CTA pairs (cta_group::2).
 #ifndef LOQT_USE_PAIRS
-#define LOQT_USE_PAIRS 0
+#define LOQT_USE_PAIRS 1
 #endif
 constexpr bool kUsePairs = LOQT_USE_PAIRS != 0;
 
