@@ -366,7 +366,7 @@ loqt_gemm_kernel(const __grid_constant__ TensorMaps maps, const GemmParams p) {
   // arriving by TMA both groups help; with an NF4 A operand (128-row tiles) one
   // group stages and the other helps.  The 64-column blocks of a tile are dealt
   // to the epilogue groups round-robin, continuing across tiles.
-  const bool requant_helpers = !TWO && (MH == 1) && (p.epi == EPI_REQUANT);
+  const bool requant_helpers = (MH == 1) && (p.epi == EPI_REQUANT);
   const int epi_groups = requant_helpers ? (p.has_nf4 ? 2 : 3) : 1;
   // The dequant warps work as two groups of four that take the K stages of a
   // tile in turn, so that one group's barrier, fence and bookkeeping time is

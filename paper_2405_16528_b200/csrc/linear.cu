@@ -158,13 +158,23 @@ static loqt_status launch_cfg(const GemmCall &c, cudaStream_t stream) {
 
 // Tile selection.  Candidates: BN in {256, 128}, rows per CTA 128 (two TMEM
 // buffers, overlapped epilogue) or 256 (one buffer, every staged B tile used by
-// two MMA passes).  A stage costs the larger of its tensor time and - when the B
-// operand is NF4 - its dequantisation time (one pass over BN blocks per stage,
-// whatever the tile height); the single-buffered tile adds an exposed epilogue.
+// two MMA passes).  A stage costs the larger of its tensor / shared-memory time
+// and - when the B operand is NF4 - its dequantisation time (one pass over the
+// CTA's B rows per stage, whatever the tile height); the single-buffered tile
+// adds an exposed epilogue.
 // Estimated time = waves x (stages x stage cost + exposed epilogue); smallest wins.
 struct TileCfg {
   int bn, mh;
+  bool two;
 };
+
+// Two CTAs on neighbouring M tiles can run as a tcgen05 pair when tiles pair up
+// exactly: 256-wide tiles, an even number of M tiles (so both CTAs of a pair
+// have the same N tile) and no split-K.
+static bool pair_ok(const GemmCall &c, int bn, int mh) {
+  const int mt = (c.p.M + mh * kHM - 1) / (mh * kHM);
+  return kUsePairs && bn == 256 && (mt % 2 == 0) && c.p.splits == 1;
+}
 
 static TileCfg pick_tile(const GemmCall &c) {
   const int sms = sm_count();
@@ -172,10 +182,10 @@ static TileCfg pick_tile(const GemmCall &c) {
   int kb = 0;
   for (int s = 0; s < c.p.num_segs; ++s) kb += (c.p.seg[s].K + kBK - 1) / kBK;
   if (c.p.splits > 1) kb = c.p.kb_per_split;
-  const TileCfg cands[4] = {{256, 1}, {256, 2}, {128, 1}, {128, 2}};
-  TileCfg best = {256, 1};
+  const TileCfg cands[4] = {{256, 1, false}, {256, 2, false}, {128, 1, false}, {128, 2, false}};
+  TileCfg best = {256, 1, false};
   double best_t = 1e300;
-  for (const TileCfg &t : cands) {
+  for (TileCfg t : cands) {
     if (t.mh == 2 && (c.p.M <= kHM || c.p.epi == EPI_REQUANT)) continue;  // the merge epilogue wants 128-row tiles
     if (t.bn == 256 && c.p.N <= 128) continue;
     const int units = ((c.p.M + t.mh * kHM - 1) / (t.mh * kHM)) * ((c.p.N + t.bn - 1) / t.bn) * c.p.splits;
@@ -190,6 +200,10 @@ static TileCfg pick_tile(const GemmCall &c) {
       best = t;
     }
   }
+  // The costs above are those of single CTAs; a 256-wide choice then runs as pairs
+  // where it can (measured faster for every product but the merge, whose epilogue
+  // - not its main loop - sets the pace).
+  best.two = pair_ok(c, best.bn, best.mh) && c.p.epi != EPI_REQUANT;
   return best;
 }
 
@@ -198,13 +212,7 @@ static loqt_status launch(GemmCall &c, cudaStream_t stream) {
   for (int s = 0; s < c.p.num_segs; ++s)
     if (c.p.seg[s].a_kind >= OP_NF4_K || c.p.seg[s].b_kind >= OP_NF4_K) c.p.has_nf4 = 1;
   const TileCfg t = pick_tile(c);
-  // Two CTAs on neighbouring M tiles can run as a tcgen05 pair when tiles pair up
-  // exactly: 256-wide tiles, an even number of M tiles (so both CTAs of a pair
-  // have the same N tile), no split-K, and not the merge (its epilogue wants all
-  // twelve worker warps of a CTA).
-  const int mt = (c.p.M + t.mh * kHM - 1) / (t.mh * kHM);
-  const bool two = kUsePairs && t.bn == 256 && (mt % 2 == 0) && c.p.splits == 1 && c.p.epi != EPI_REQUANT;
-  if (two) return t.mh == 2 ? launch_cfg<256, 2, true>(c, stream) : launch_cfg<256, 1, true>(c, stream);
+  if (t.two) return t.mh == 2 ? launch_cfg<256, 2, true>(c, stream) : launch_cfg<256, 1, true>(c, stream);
   if (t.bn == 256) return t.mh == 2 ? launch_cfg<256, 2, false>(c, stream) : launch_cfg<256, 1, false>(c, stream);
   return t.mh == 2 ? launch_cfg<128, 2, false>(c, stream) : launch_cfg<128, 1, false>(c, stream);
 }
