@@ -215,3 +215,34 @@ def nf4_requantize(wq, delta, s, cols):
     W32 = nf4_dequantize(wq[0], wq[1], cols).astype(np.float64)
     d = np.asarray(delta, dtype=np.float32).astype(np.float64)
     return nf4_quantize((W32 + float(s) * d).astype(np.float32))
+
+
+def loqt_compensate(W, P, steps):
+    """Error-compensated initialisation of (Q, B) for a fixed projection P
+    (Section 2.5 "Compensating for Quantization Errors"; Algorithm 2, the loop
+    over compensation steps; appendix "Choice of Quantization Method": B =
+    P^+ (W - Q)).  Alternating minimisation of || Q + P B - W ||:
+
+        B_0 = 0
+        for c = 1..steps:   Q_c = q_NF4( W - P B_{c-1} )
+                            B_c = P^+ ( W - deq(Q_c) )
+
+    P has orthonormal columns, so P^+ = P^T.  Precisions follow the hot path:
+    W and W - P B are 32-bit (the quantiser's input), P, the residual
+    W - deq(Q_c) and B enter the matrix products as 16-bit operands (one rounding
+    each), sums in float64.
+
+    W: fp32 [out, in]; P: fp32 [out, r].  Returns ((codes, absmax) of Q_steps,
+    B_steps as fp32 holding bf16 values [r, in])."""
+    W = np.asarray(W, dtype=np.float32)
+    out, inn = W.shape
+    Pb = bf16_round(np.asarray(P, dtype=np.float32)).astype(np.float64)
+    W64 = W.astype(np.float64)
+    B = np.zeros((Pb.shape[1], inn), dtype=np.float32)
+    q = None
+    for _ in range(int(steps)):
+        what = (W64 - Pb @ B.astype(np.float64)).astype(np.float32)
+        q = nf4_quantize(what)
+        resid = bf16_round((W - nf4_dequantize(q[0], q[1], inn)).astype(np.float32))
+        B = bf16_round((Pb.T @ resid.astype(np.float64)).astype(np.float32))
+    return q, B

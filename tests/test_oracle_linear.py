@@ -211,3 +211,67 @@ def test_requantize_equals_merge_for_rank_one(s):
     c, m = O.nf4_requantize(wq, delta, s, inn)
     rc, rm = O.loqt_merge_requant(wq, pq, B, s, (out, inn, r))
     assert np.array_equal(c, rc) and np.array_equal(m, rm)
+
+
+# ---- error-compensated initialisation (Section 2.5, Algorithm 2)
+def _ortho(seed, out, r):
+    return synth.orthonormal(seed, ("P", out, r), out, r).numpy()
+
+
+def test_compensate_first_step_is_the_least_squares_fit():
+    # After one step Q = q(W) exactly, and B is the minimiser of ||Q + P B - W||
+    # over B: numpy's least-squares routine on the same 16-bit P gives it.
+    out, inn, r = 96, 128, 24
+    W = synth.normal(31, ("W",), (out, inn), 0.02).numpy()
+    P = _ortho(31, out, r)
+    (c, m), B = O.loqt_compensate(W, P, 1)
+    rc, rm = O.nf4_quantize(W)
+    assert np.array_equal(c, rc) and np.array_equal(m, rm)
+    Pb = O.bf16_round(P).astype(np.float64)
+    resid = W.astype(np.float64) - O.nf4_dequantize(c, m, inn)
+    ls = np.linalg.lstsq(Pb, resid, rcond=None)[0]
+    assert np.abs(B - ls).max() <= 2.0 ** -7 * np.abs(ls).max()   # two 16-bit roundings
+    # a sign slip (B = P^+ (Q - W)) would give -ls
+    assert np.abs(B + ls).max() > 0.5 * np.abs(ls).max()
+
+
+def test_compensate_reduces_the_error_as_the_projection_predicts():
+    # With B the least-squares fit for Q = q(W), the error W - (Q + P B) is the part
+    # of W - Q outside the span of P: its squared norm drops by about r / out for a
+    # quantisation error that is spread evenly over directions.  Further steps
+    # re-quantise the corrected weights and keep lowering the error (Section 2.5:
+    # "iteratively refine").
+    out, inn, r = 128, 256, 32
+    W = synth.normal(32, ("W",), (out, inn), 0.02).numpy()
+    P = _ortho(32, out, r)
+    Pb = O.bf16_round(P).astype(np.float64)
+    e0 = np.linalg.norm(W - O.nf4_dequantize(*O.nf4_quantize(W), inn)) ** 2
+    errs = []
+    for steps in (1, 2, 3, 5):
+        (c, m), B = O.loqt_compensate(W, P, steps)
+        errs.append(np.linalg.norm(W.astype(np.float64) - O.nf4_dequantize(c, m, inn) - Pb @ B.astype(np.float64)) ** 2)
+    assert (1 - 1.3 * r / out) * e0 < errs[0] < (1 - 0.7 * r / out) * e0
+    assert all(b < a for a, b in zip(errs, errs[1:]))
+
+
+def test_compensate_representable_weights_need_no_correction():
+    out, inn, r = 64, 128, 16
+    W0 = synth.normal(33, ("W",), (out, inn), 0.02).numpy()
+    q0 = O.nf4_quantize(W0)
+    W = O.nf4_dequantize(q0[0], q0[1], inn)      # exactly representable
+    (c, m), B = O.loqt_compensate(W, _ortho(33, out, r), 3)
+    assert np.array_equal(c, q0[0]) and np.array_equal(m, q0[1]) and not B.any()
+
+
+def test_compensate_later_steps_use_the_corrected_weights():
+    # Step 2 quantises W - P B_1, not W: feeding that matrix to the quantiser by hand
+    # must give the same codes.
+    out, inn, r = 96, 192, 24
+    W = synth.normal(34, ("W",), (out, inn), 0.02).numpy()
+    P = _ortho(34, out, r)
+    _, B1 = O.loqt_compensate(W, P, 1)
+    (c2, m2), _ = O.loqt_compensate(W, P, 2)
+    what = (W.astype(np.float64) - O.bf16_round(P).astype(np.float64) @ B1.astype(np.float64)).astype(np.float32)
+    rc, rm = O.nf4_quantize(what)
+    assert np.array_equal(c2, rc) and np.array_equal(m2, rm)
+    assert not np.array_equal(c2, O.nf4_quantize(W)[0])
