@@ -217,7 +217,7 @@ def nf4_requantize(wq, delta, s, cols):
     return nf4_quantize((W32 + float(s) * d).astype(np.float32))
 
 
-def loqt_compensate(W, P, steps):
+def loqt_compensate(W, P, steps, B0=None):
     """Error-compensated initialisation of (Q, B) for a fixed projection P
     (Section 2.5 "Compensating for Quantization Errors"; Algorithm 2, the loop
     over compensation steps; appendix "Choice of Quantization Method": B =
@@ -233,12 +233,14 @@ def loqt_compensate(W, P, steps):
     each), sums in float64.
 
     W: fp32 [out, in]; P: fp32 [out, r].  Returns ((codes, absmax) of Q_steps,
-    B_steps as fp32 holding bf16 values [r, in])."""
+    B_steps as fp32 holding bf16 values [r, in]).  B0 (bf16 values, [r, in])
+    replaces the zero start of Algorithm 2, so that a test can check one step
+    from any state."""
     W = np.asarray(W, dtype=np.float32)
     out, inn = W.shape
     Pb = bf16_round(np.asarray(P, dtype=np.float32)).astype(np.float64)
     W64 = W.astype(np.float64)
-    B = np.zeros((Pb.shape[1], inn), dtype=np.float32)
+    B = np.zeros((Pb.shape[1], inn), dtype=np.float32) if B0 is None else bf16_round(np.asarray(B0, dtype=np.float32))
     q = None
     for _ in range(int(steps)):
         what = (W64 - Pb @ B.astype(np.float64)).astype(np.float32)
