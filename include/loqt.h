@@ -69,7 +69,7 @@ typedef struct {
 } loqt_nf4_mat;
 
 /* Operation selector for loqt_workspace_bytes(). */
-enum { LOQT_OP_FWD = 0, LOQT_OP_BWD = 1, LOQT_OP_MERGE = 2, LOQT_OP_MERGE_SPLIT = 3 };
+enum { LOQT_OP_FWD = 0, LOQT_OP_BWD = 1, LOQT_OP_MERGE = 2, LOQT_OP_MERGE_SPLIT = 3, LOQT_OP_COMPENSATE = 4 };
 
 /*
  * q_NF4 (Section 5.1, first two displayed equations): per block M = max|w|,
@@ -155,6 +155,24 @@ loqt_status loqt_nf4_requantize(const float *delta, int64_t ld_delta, float s, l
  */
 loqt_status loqt_merge_requant_split(loqt_nf4_mat Wq, loqt_nf4_mat Pq, const void *B, int64_t ldb,
                                      float s, void *ws, size_t ws_bytes, void *stream);
+
+/*
+ * Error-compensated initialisation of a layer for a new projection P
+ * (Section 2.5 "Compensating for Quantization Errors"; Algorithm 2, the loop over
+ * compensation steps; appendix: B = P^+ (W - Q)).  Alternating minimisation of
+ * || Q + P B - W || with P fixed:
+ *     B_0 = 0;   for c = 1..steps:   Q_c = q_NF4( W - P B_{c-1} ),   B_c = P^T ( W - deq(Q_c) )
+ *   W  : fp32 [out][ldw] on the device (the full-precision weights to approximate),
+ *        16-byte aligned, ldw % 4 == 0.
+ *   P  : fp32 [out][ldp], orthonormal columns (so that P^+ = P^T).
+ *   Wq : receives Q_steps;  Pq : receives q_NF4(P);  B : receives B_steps as bf16 [r][ldb].
+ * W and W - P B are 32-bit; P, the residual W - deq(Q_c) and B enter the
+ * tensor-core products as bf16, sums in fp32.  1 <= steps <= 16 (the paper uses
+ * at most five).  Workspace: loqt_workspace_bytes(LOQT_OP_COMPENSATE, out, in, r, 0).
+ */
+loqt_status loqt_compensated_init(const float *W, int64_t ldw, const float *P, int64_t ldp,
+                                  int32_t steps, loqt_nf4_mat Wq, loqt_nf4_mat Pq, void *B,
+                                  int64_t ldb, void *ws, size_t ws_bytes, void *stream);
 
 /*
  * The same merge for n independent matrices in one call (a whole model at a

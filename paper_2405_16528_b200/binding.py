@@ -16,13 +16,13 @@ import torch
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libloqt.so")
 
-LOQT_OP_FWD, LOQT_OP_BWD, LOQT_OP_MERGE, LOQT_OP_MERGE_SPLIT = 0, 1, 2, 3
+LOQT_OP_FWD, LOQT_OP_BWD, LOQT_OP_MERGE, LOQT_OP_MERGE_SPLIT, LOQT_OP_COMPENSATE = 0, 1, 2, 3, 4
 BLOCK = 64
 
 EXPORTS = (
     "loqt_nf4_quantize", "loqt_nf4_dequantize", "loqt_linear_fwd", "loqt_linear_bwd",
     "loqt_merge_requant", "loqt_merge_requant_many", "loqt_merge_requant_split", "loqt_nf4_requantize",
-    "loqt_linear_fwd_static", "loqt_workspace_bytes",
+    "loqt_compensated_init", "loqt_linear_fwd_static", "loqt_workspace_bytes",
     "loqt_device_status", "loqt_launch_count", "loqt_status_string",
 )
 
@@ -67,6 +67,8 @@ def lib():
     L.loqt_merge_requant.argtypes = [M, M, vp, i64, f32, vp, sz, vp]
     L.loqt_merge_requant_split.argtypes = [M, M, vp, i64, f32, vp, sz, vp]
     L.loqt_nf4_requantize.argtypes = [vp, i64, f32, M, vp]
+    L.loqt_compensated_init.argtypes = [vp, i64, vp, i64, i32, M, M, vp, i64, vp, sz, vp]
+    L.loqt_compensated_init.restype = ctypes.c_int
     L.loqt_merge_requant_many.argtypes = [i32, ctypes.POINTER(M), ctypes.POINTER(M), ctypes.POINTER(vp), ctypes.POINTER(i64), f32, vp, sz, vp]
     L.loqt_workspace_bytes.argtypes = [ctypes.c_int, i32, i32, i32, i32]
     L.loqt_workspace_bytes.restype = sz
@@ -221,6 +223,22 @@ def loqt_nf4_requantize(delta: torch.Tensor, s: float, Wq: NF4Tensor) -> NF4Tens
     _check(lib().loqt_nf4_requantize(_dev(delta, torch.float32), delta.stride(0), float(s), Wq.view(), _stream()),
            "loqt_nf4_requantize")
     return Wq
+
+
+def loqt_compensated_init(W: torch.Tensor, P: torch.Tensor, steps: int, ws: torch.Tensor | None = None):
+    """Returns (Wq, Pq, B): Q_steps, q_NF4(P) and the bf16 factor B_steps."""
+    out, inn = W.shape
+    r = P.shape[1]
+    Wq, Pq = NF4Tensor.empty(out, inn, W.device), NF4Tensor.empty(out, r, W.device)
+    ldb = (inn + 7) // 8 * 8
+    B = torch.empty((r, ldb), dtype=torch.bfloat16, device=W.device)[:, :inn]
+    if ws is None:
+        ws = new_workspace(loqt_workspace_bytes(LOQT_OP_COMPENSATE, out, inn, r, 0), W.device)
+    _check(lib().loqt_compensated_init(_dev(W, torch.float32), W.stride(0), _dev(P, torch.float32), P.stride(0), int(steps),
+                                       Wq.view(), Pq.view(), B.data_ptr(), B.stride(0), ws.data_ptr(), ws.numel(),
+                                       _stream()), "loqt_compensated_init")
+    loqt_device_status(ws)
+    return Wq, Pq, B
 
 
 def merge_many_workspace_bytes(Wqs, Pqs, group: int = 8) -> int:

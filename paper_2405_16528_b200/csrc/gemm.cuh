@@ -59,7 +59,7 @@ enum : int {
 // Epilogue kinds
 enum : int {
   EPI_BF16 = 0,     // out bf16 = alpha * D
-  EPI_F32 = 1,      // out fp32 = (accumulate ? out : 0) + D          (splits == 1)
+  EPI_F32 = 1,      // out fp32 = (addend, or out when accumulating, or 0) + alpha * D   (splits == 1)
   EPI_PARTIAL = 2,  // partial[split] fp32 = D                        (splits > 1)
   EPI_REQUANT = 3,  // W_q <- q_NF4(deq32(W_q) + alpha * D), in place (merge)
 };
@@ -87,6 +87,8 @@ struct GemmParams {
   int64_t ld_out;   // elements
   float alpha;
   int accumulate;
+  const float *addend;  // EPI_F32: out = addend + alpha * D when set (16-byte aligned rows)
+  int64_t ld_addend;
   uint8_t *wq_codes;  // EPI_REQUANT: W_q updated in place ([M][wq_ld/2], [M][wq_ld/64])
   float *wq_absmax;
   int wq_ld;
@@ -793,28 +795,37 @@ loqt_gemm_kernel(const __grid_constant__ TensorMaps maps, const GemmParams p) {
             } else {
               float *o;
               const int64_t ldo = p.ld_out;
-              bool acc_out = false;
+              const float *base = nullptr;  // what the product is added to
+              float scale = 1.0f;
+              bool base_vec = true;
               if (p.epi == EPI_PARTIAL) {
                 o = reinterpret_cast<float *>(p.out) + (static_cast<int64_t>(split) * p.M + row) * ldo + c0;
               } else {
                 o = reinterpret_cast<float *>(p.out) + static_cast<int64_t>(row) * ldo + c0;
-                acc_out = p.accumulate != 0;
+                scale = p.alpha;
+                if (p.addend != nullptr) {
+                  base = p.addend + static_cast<int64_t>(row) * p.ld_addend + c0;
+                  base_vec = (p.ld_addend & 3) == 0;
+                } else if (p.accumulate != 0) {
+                  base = o;
+                }
               }
-              if (full && (ldo & 3) == 0) {
+              if (full && (ldo & 3) == 0 && base_vec) {
 #pragma unroll
                 for (int g = 0; g < 8; ++g) {
-                  float4 f = make_float4(__uint_as_float(d[4 * g]), __uint_as_float(d[4 * g + 1]),
-                                         __uint_as_float(d[4 * g + 2]), __uint_as_float(d[4 * g + 3]));
-                  if (acc_out) {
-                    const float4 old = reinterpret_cast<float4 *>(o)[g];
-                    f.x += old.x; f.y += old.y; f.z += old.z; f.w += old.w;
-                  }
+                  float4 b4 = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+                  if (base != nullptr) b4 = reinterpret_cast<const float4 *>(base)[g];
+                  float4 f;
+                  f.x = fmaf(scale, __uint_as_float(d[4 * g]), b4.x);
+                  f.y = fmaf(scale, __uint_as_float(d[4 * g + 1]), b4.y);
+                  f.z = fmaf(scale, __uint_as_float(d[4 * g + 2]), b4.z);
+                  f.w = fmaf(scale, __uint_as_float(d[4 * g + 3]), b4.w);
                   reinterpret_cast<float4 *>(o)[g] = f;
                 }
               } else {
 #pragma unroll
                 for (int e = 0; e < 32; ++e)
-                  if (c0 + e < p.N) o[e] = (acc_out ? o[e] : 0.0f) + __uint_as_float(d[e]);
+                  if (c0 + e < p.N) o[e] = fmaf(scale, __uint_as_float(d[e]), base != nullptr ? base[e] : 0.0f);
               }
             }
             __syncwarp();

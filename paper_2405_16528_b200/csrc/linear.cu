@@ -236,6 +236,38 @@ static void db_splits(int r, int in, int T, int &splits, int &kb_per_split) {
   splits = (kb_total + kb_per_split - 1) / kb_per_split;
 }
 
+// out[M x N] (fp32) = (accumulate ? out : 0) + A^T B with A stored [K][M] and B stored
+// [K][N] (both bf16, K outermost), split over K when the tiles alone would not
+// fill the GPU; the partial sums are then added in a fixed order.
+static loqt_status gemm_tn_f32(const void *a, int64_t lda, const void *b, int64_t ldb, int M, int N, int K, float *out,
+                               int64_t ld_out, int accumulate, float *partial, uint32_t *status, cudaStream_t stm) {
+  GemmCall c{};
+  c.p.M = M; c.p.N = N; c.p.num_segs = 1;
+  c.p.seg[0].K = K; c.p.seg[0].a_kind = OP_TMA_MN; c.p.seg[0].b_kind = OP_TMA_MN;
+  c.a[0] = {a, lda}; c.b[0] = {b, ldb};
+  int splits = 1, kbps = 1;
+  db_splits(M, N, K, splits, kbps);
+  c.p.splits = splits; c.p.kb_per_split = kbps; c.p.status = status; c.p.alpha = 1.0f;
+  const int64_t ldp = (static_cast<int64_t>(N) + 3) / 4 * 4;
+  if (splits == 1) {
+    c.p.epi = EPI_F32; c.p.out = out; c.p.ld_out = ld_out; c.p.accumulate = accumulate;
+  } else {
+    c.p.epi = EPI_PARTIAL; c.p.out = partial; c.p.ld_out = ldp;
+  }
+  loqt_status st;
+  if ((st = launch(c, stm)) != LOQT_OK) return st;
+  if (splits > 1) {
+    const int64_t total = static_cast<int64_t>(M) * N;
+    int64_t blocks = (total + 255) / 256;
+    const int64_t cap = static_cast<int64_t>(sm_count()) * 8;
+    if (blocks > cap) blocks = cap;
+    splitk_reduce_kernel<<<static_cast<int>(blocks), 256, 0, stm>>>(partial, splits, M, N, ldp, out, ld_out, accumulate);
+    count_launch();
+    if (cudaGetLastError() != cudaSuccess) return LOQT_ERR_CUDA;
+  }
+  return LOQT_OK;
+}
+
 }  // namespace loqt
 
 using namespace loqt;
@@ -254,6 +286,15 @@ extern "C" size_t loqt_workspace_bytes(int op, int32_t out, int32_t in, int32_t 
   // two-pass merge: the fp32 product P-hat B, out x roundup(in, 64)
   if (op == LOQT_OP_MERGE_SPLIT)
     total += align256(static_cast<size_t>(out > 0 ? out : 0) * ((static_cast<size_t>(in > 0 ? in : 0) + 63) / 64 * 64) * 4);
+  // error-compensated initialisation: bf16 P, bf16 residual, fp32 corrected weights, fp32 B (+ split-K partials)
+  if (op == LOQT_OP_COMPENSATE) {
+    const size_t o = static_cast<size_t>(out > 0 ? out : 0), ld64 = (static_cast<size_t>(in > 0 ? in : 0) + 63) / 64 * 64;
+    const size_t ld4 = (static_cast<size_t>(in > 0 ? in : 0) + 3) / 4 * 4;
+    total += align256(o * ld_lowrank(r) * 2) + align256(o * ld64 * 2) + align256(o * ld64 * 4) + align256(static_cast<size_t>(r) * ld4 * 4);
+    int splits = 1, kbps = 1;
+    db_splits(r, in, out > 0 ? out : 1, splits, kbps);
+    if (splits > 1) total += align256(static_cast<size_t>(splits) * r * ld4 * 4);
+  }
   return total;
 }
 
@@ -350,30 +391,7 @@ extern "C" loqt_status loqt_linear_bwd(loqt_nf4_mat Wq, loqt_nf4_mat Pq, const v
   }
 
   // dB = v'^T x               (r x in; K = T; both operands stored K-outermost)
-  GemmCall c3{};
-  c3.p.M = r; c3.p.N = in; c3.p.num_segs = 1;
-  c3.p.seg[0].K = T; c3.p.seg[0].a_kind = OP_TMA_MN; c3.p.seg[0].b_kind = OP_TMA_MN;
-  c3.a[0] = {v, ldv}; c3.b[0] = {x, ldx};
-  int splits = 1, kbps = 1;
-  db_splits(r, in, T, splits, kbps);
-  c3.p.splits = splits; c3.p.kb_per_split = kbps; c3.p.status = status; c3.p.alpha = 1.0f;
-  const int64_t ldp = (static_cast<int64_t>(in) + 3) / 4 * 4;
-  if (splits == 1) {
-    c3.p.epi = EPI_F32; c3.p.out = dB; c3.p.ld_out = lddb; c3.p.accumulate = accumulate_dB;
-  } else {
-    c3.p.epi = EPI_PARTIAL; c3.p.out = partial; c3.p.ld_out = ldp;
-  }
-  if ((st = launch(c3, stm)) != LOQT_OK) return st;
-  if (splits > 1) {
-    const int64_t total = static_cast<int64_t>(r) * in;
-    int64_t blocks = (total + 255) / 256;
-    const int64_t cap = static_cast<int64_t>(sm_count()) * 8;
-    if (blocks > cap) blocks = cap;
-    splitk_reduce_kernel<<<static_cast<int>(blocks), 256, 0, stm>>>(partial, splits, r, in, ldp, dB, lddb, accumulate_dB);
-    count_launch();
-    if (cudaGetLastError() != cudaSuccess) return LOQT_ERR_CUDA;
-  }
-  return LOQT_OK;
+  return gemm_tn_f32(v, ldv, x, ldx, r, in, T, dB, lddb, accumulate_dB, partial, status, stm);
 }
 
 // The merge of one matrix, in two launches.  `phat` is scratch for deq(P_q).
@@ -466,6 +484,60 @@ extern "C" loqt_status loqt_merge_requant_many(int32_t n, const loqt_nf4_mat *Wq
       if ((st = merge_product(Wq[i], Pq[i], base + static_cast<size_t>(i - g0) * slot, B[i], ldb[i], s,
                               static_cast<uint32_t *>(ws), stm)) != LOQT_OK)
         return st;
+  }
+  return LOQT_OK;
+}
+
+// ---------------------------------------------------------------------------
+// Error-compensated initialisation (Section 2.5; Algorithm 2, compensation loop)
+// ---------------------------------------------------------------------------
+extern "C" loqt_status loqt_compensated_init(const float *W, int64_t ldw, const float *P, int64_t ldp, int32_t steps,
+                                             loqt_nf4_mat Wq, loqt_nf4_mat Pq, void *B, int64_t ldb, void *ws,
+                                             size_t ws_bytes, void *stream) {
+  loqt_status st;
+  if ((st = validate_nf4(Wq)) != LOQT_OK) return st;
+  if ((st = validate_nf4(Pq)) != LOQT_OK) return st;
+  if (Pq.rows != Wq.rows || steps < 1 || steps > 16) return LOQT_ERR_INVALID_ARG;
+  const int out = Wq.rows, in = Wq.cols, r = Pq.cols;
+  if (W == nullptr || P == nullptr || ldw < in || ldp < r) return LOQT_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(W) & 15u) != 0 || (ldw & 3) != 0 || (reinterpret_cast<uintptr_t>(P) & 3u) != 0)
+    return LOQT_ERR_ALIGNMENT;
+  if ((st = check_bf16(B, ldb, in)) != LOQT_OK) return st;
+  if ((st = check_ws(ws, ws_bytes, loqt_workspace_bytes(LOQT_OP_COMPENSATE, out, in, r, 0))) != LOQT_OK) return st;
+  if ((st = check_arch()) != LOQT_OK) return st;
+  cudaStream_t stm = static_cast<cudaStream_t>(stream);
+  uint32_t *status = static_cast<uint32_t *>(ws);
+
+  const int64_t ldr = ld_lowrank(r), ld64 = (static_cast<int64_t>(in) + 63) / 64 * 64, ld4 = (static_cast<int64_t>(in) + 3) / 4 * 4;
+  uint8_t *cursor = static_cast<uint8_t *>(ws) + 256;
+  void *phat = cursor;                                        cursor += align256(static_cast<size_t>(out) * ldr * 2);
+  void *resid = cursor;                                       cursor += align256(static_cast<size_t>(out) * ld64 * 2);
+  float *what = reinterpret_cast<float *>(cursor);            cursor += align256(static_cast<size_t>(out) * ld64 * 4);
+  float *b32 = reinterpret_cast<float *>(cursor);             cursor += align256(static_cast<size_t>(r) * ld4 * 4);
+  float *partial = reinterpret_cast<float *>(cursor);
+
+  // P_q = q(P); the products below use bf16(P), the unquantised projection (Algorithm 2)
+  if ((st = loqt_nf4_quantize(P, ldp, Pq, stream)) != LOQT_OK) return st;
+  if ((st = convert_f32_bf16(P, ldp, phat, ldr, out, r, stm)) != LOQT_OK) return st;
+
+  for (int c = 1; c <= steps; ++c) {
+    // Q_c = q(W - P B_{c-1}) (B_0 = 0), residual = bf16(W - deq(Q_c))
+    const float *src = (c == 1) ? W : what;
+    const int64_t ld_src = (c == 1) ? ldw : ld64;
+    if ((st = nf4_quantize_residual(src, ld_src, W, ldw, Wq, resid, ld64, stm)) != LOQT_OK) return st;
+    // B_c = P^T residual   (r x in; K = out; both operands stored K-outermost), then to bf16
+    if ((st = gemm_tn_f32(phat, ldr, resid, ld64, r, in, out, b32, ld4, 0, partial, status, stm)) != LOQT_OK) return st;
+    if ((st = convert_f32_bf16(b32, ld4, B, ldb, r, in, stm)) != LOQT_OK) return st;
+    if (c == steps) break;
+    // corrected weights for the next step: W - P B_c   (out x in; K = r), fp32
+    GemmCall g{};
+    g.p.M = out; g.p.N = in; g.p.num_segs = 1;
+    g.p.seg[0].K = r; g.p.seg[0].a_kind = OP_TMA_K; g.p.seg[0].b_kind = OP_TMA_MN;
+    g.a[0] = {phat, ldr}; g.b[0] = {B, ldb};
+    g.p.splits = 1;
+    g.p.epi = EPI_F32; g.p.out = what; g.p.ld_out = ld64; g.p.alpha = -1.0f; g.p.addend = W; g.p.ld_addend = ldw;
+    g.p.status = status;
+    if ((st = launch(g, stm)) != LOQT_OK) return st;
   }
   return LOQT_OK;
 }

@@ -14,6 +14,9 @@ constexpr int kQThreads = 256;
 // quantise:   fp32 [rows][ld_src] -> codes [rows][ld/2], absmax [rows][ld/64]
 // requantise: W_q <- q_NF4(deq32(W_q) + s * src), in place (the streaming half of
 //             the two-pass merge)
+// residual:   quantise `src` and also write bf16(ref - deq32(codes)) for every real
+//             element (the error-compensation step: `ref` is the weight matrix
+//             the quantised one should approximate, `src` what is quantised)
 // Four threads share one block of 64 weights; each owns 16 consecutive elements
 // (four 128-bit loads, one 64-bit store of 16 codes; the requantiser also loads
 // its 16 old codes and the block's old scale).
@@ -24,10 +27,14 @@ struct QuantItem {
   bool live;
 };
 
-template <bool kVec, bool kRequant>
+enum : int { kQuantise = 0, kRequantise = 1, kQuantiseResidual = 2 };
+
+template <bool kVec, int kMode>
 __global__ void __launch_bounds__(kQThreads)
 nf4_quantize_kernel(const float *__restrict__ src, int64_t ld_src, float s, uint8_t *__restrict__ codes,
-                    float *__restrict__ absmax, int rows, int cols, int ld) {
+                    float *__restrict__ absmax, int rows, int cols, int ld, const float *__restrict__ ref,
+                    int64_t ld_ref, __nv_bfloat16 *__restrict__ resid, int64_t ld_resid) {
+  constexpr bool kRequant = (kMode == kRequantise);
   __shared__ Nf4Tables tab;
   nf4_tables_init(tab, threadIdx.x);
   __syncthreads();
@@ -111,6 +118,33 @@ nf4_quantize_kernel(const float *__restrict__ src, int64_t ld_src, float s, uint
       }
       *reinterpret_cast<uint2 *>(codes + static_cast<int64_t>(cur.row) * (ld / 2) + (cur.c0 >> 1)) = w;
       if (l == 0) absmax[static_cast<int64_t>(cur.row) * nb + cur.b] = m;
+      if (kMode == kQuantiseResidual && cur.c0 < cols) {
+        const float *rp = ref + static_cast<int64_t>(cur.row) * ld_ref + cur.c0;
+        __nv_bfloat16 *dp = resid + static_cast<int64_t>(cur.row) * ld_resid + cur.c0;
+        const bool full = kVec && (cur.c0 + 16 <= cols);
+        float e[16];
+#pragma unroll
+        for (int j = 0; j < 16; ++j) {
+          const uint32_t code = ((j < 8 ? w.x : w.y) >> (4 * (j & 7))) & 15u;
+          const float t = (full || cur.c0 + j < cols) ? (ref == src ? v[j] : __ldg(rp + j)) : 0.0f;
+          e[j] = __fsub_rn(t, __fmul_rn(m, tab.level[code]));  // two roundings, as the definition has them
+        }
+        if (full) {
+#pragma unroll
+          for (int g = 0; g < 2; ++g) {
+            uint4 pk;
+            pk.x = pack_bf16x2(e[8 * g + 0], e[8 * g + 1]);
+            pk.y = pack_bf16x2(e[8 * g + 2], e[8 * g + 3]);
+            pk.z = pack_bf16x2(e[8 * g + 4], e[8 * g + 5]);
+            pk.w = pack_bf16x2(e[8 * g + 6], e[8 * g + 7]);
+            reinterpret_cast<uint4 *>(dp)[g] = pk;
+          }
+        } else {
+#pragma unroll
+          for (int j = 0; j < 16; ++j)
+            if (cur.c0 + j < cols) dp[j] = __float2bfloat16_rn(e[j]);
+        }
+      }
     }
     cur = nxt;
     old = oldn;
@@ -223,6 +257,43 @@ static int grid_for(Kernel kernel, int64_t threads_needed) {
   return static_cast<int>(blocks);
 }
 
+// fp32 -> bf16 (round to nearest even), row-major with leading dimensions.
+__global__ void __launch_bounds__(kQThreads)
+convert_f32_bf16_kernel(const float *__restrict__ src, int64_t ld_src, __nv_bfloat16 *__restrict__ dst, int64_t ld_dst,
+                        int rows, int cols) {
+  const int64_t total = static_cast<int64_t>(rows) * cols;
+  const int64_t stride = static_cast<int64_t>(gridDim.x) * kQThreads;
+  for (int64_t i = static_cast<int64_t>(blockIdx.x) * kQThreads + threadIdx.x; i < total; i += stride) {
+    const int r = static_cast<int>(i / cols);
+    const int c = static_cast<int>(i - static_cast<int64_t>(r) * cols);
+    dst[static_cast<int64_t>(r) * ld_dst + c] = __float2bfloat16_rn(__ldg(src + static_cast<int64_t>(r) * ld_src + c));
+  }
+}
+
+loqt_status convert_f32_bf16(const float *src, int64_t ld_src, void *dst, int64_t ld_dst, int rows, int cols,
+                             cudaStream_t stream) {
+  const int64_t total = static_cast<int64_t>(rows) * cols;
+  if (total <= 0) return LOQT_OK;
+  convert_f32_bf16_kernel<<<grid_for(convert_f32_bf16_kernel, total), kQThreads, 0, stream>>>(
+      src, ld_src, static_cast<__nv_bfloat16 *>(dst), ld_dst, rows, cols);
+  count_launch();
+  return cudaGetLastError() == cudaSuccess ? LOQT_OK : LOQT_ERR_CUDA;
+}
+
+// dst <- q_NF4(src); resid <- bf16(ref - deq32(dst)).  ref may equal src.
+loqt_status nf4_quantize_residual(const float *src, int64_t ld_src, const float *ref, int64_t ld_ref, loqt_nf4_mat dst,
+                                  void *resid, int64_t ld_resid, cudaStream_t stream) {
+  const int64_t items = static_cast<int64_t>(dst.rows) * (dst.ld / kBlock);
+  if (items >= (1ll << 30)) return LOQT_ERR_UNSUPPORTED;
+  const bool vec = ((reinterpret_cast<uintptr_t>(src) | reinterpret_cast<uintptr_t>(ref) | reinterpret_cast<uintptr_t>(resid)) & 15u) == 0 &&
+                   (ld_src % 4) == 0 && (ld_ref % 4) == 0 && (ld_resid % 8) == 0;
+  auto kernel = vec ? nf4_quantize_kernel<true, kQuantiseResidual> : nf4_quantize_kernel<false, kQuantiseResidual>;
+  kernel<<<grid_for(kernel, items * 4), kQThreads, 0, stream>>>(src, ld_src, 1.0f, dst.codes, dst.absmax, dst.rows, dst.cols, dst.ld, ref,
+                                                                ld_ref, static_cast<__nv_bfloat16 *>(resid), ld_resid);
+  count_launch();
+  return cudaGetLastError() == cudaSuccess ? LOQT_OK : LOQT_ERR_CUDA;
+}
+
 }  // namespace loqt
 
 using namespace loqt;
@@ -237,8 +308,9 @@ extern "C" loqt_status loqt_nf4_quantize(const float *src, int64_t ld_src, loqt_
   if (items >= (1ll << 30)) return LOQT_ERR_UNSUPPORTED;  // 32-bit block indices in the kernel
   const bool vec = (reinterpret_cast<uintptr_t>(src) & 15u) == 0 && (ld_src % 4) == 0;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
-  auto kernel = vec ? nf4_quantize_kernel<true, false> : nf4_quantize_kernel<false, false>;
-  kernel<<<grid_for(kernel, items * 4), kQThreads, 0, s>>>(src, ld_src, 1.0f, dst.codes, dst.absmax, dst.rows, dst.cols, dst.ld);
+  auto kernel = vec ? nf4_quantize_kernel<true, kQuantise> : nf4_quantize_kernel<false, kQuantise>;
+  kernel<<<grid_for(kernel, items * 4), kQThreads, 0, s>>>(src, ld_src, 1.0f, dst.codes, dst.absmax, dst.rows, dst.cols, dst.ld, nullptr, 0,
+                                                           nullptr, 0);
   count_launch();
   return cudaGetLastError() == cudaSuccess ? LOQT_OK : LOQT_ERR_CUDA;
 }
@@ -273,8 +345,9 @@ extern "C" loqt_status loqt_nf4_requantize(const float *delta, int64_t ld_delta,
   if (items >= (1ll << 30)) return LOQT_ERR_UNSUPPORTED;  // 32-bit block indices in the kernel
   const bool vec = (reinterpret_cast<uintptr_t>(delta) & 15u) == 0 && (ld_delta % 4) == 0;
   cudaStream_t stm = static_cast<cudaStream_t>(stream);
-  auto kernel = vec ? nf4_quantize_kernel<true, true> : nf4_quantize_kernel<false, true>;
-  kernel<<<grid_for(kernel, items * 4), kQThreads, 0, stm>>>(delta, ld_delta, s, Wq.codes, Wq.absmax, Wq.rows, Wq.cols, Wq.ld);
+  auto kernel = vec ? nf4_quantize_kernel<true, kRequantise> : nf4_quantize_kernel<false, kRequantise>;
+  kernel<<<grid_for(kernel, items * 4), kQThreads, 0, stm>>>(delta, ld_delta, s, Wq.codes, Wq.absmax, Wq.rows, Wq.cols, Wq.ld, nullptr, 0,
+                                                             nullptr, 0);
   count_launch();
   return cudaGetLastError() == cudaSuccess ? LOQT_OK : LOQT_ERR_CUDA;
 }
