@@ -203,6 +203,37 @@ def time_nf4_kernels(device, peaks, rows=16384, cols=8192, iters=10):
     }
 
 
+def time_compensated_init(device, peaks, cfg, seed, steps=5, iters=5):
+    """Error-compensated initialisation (Section 2.5) of one matrix of the
+    configuration's first shape: `steps` rounds of quantise + residual, B = P^T residual
+    and W - P B.  Flops counted: (2 steps - 1) products of 2 out in r."""
+    import torch
+
+    from paper_2405_16528_b200 import binding as L
+    from paper_2405_16528_b200 import synth
+
+    _, out, inn, _ = next(iter(cfg.shapes()))
+    r = cfg.r
+    W = synth.normal(seed, ("ci", "W"), (out, inn), 0.02, torch.float32, device)
+    P = synth.orthonormal(seed, ("ci", "P"), out, r, device)
+    ws = L.new_workspace(L.loqt_workspace_bytes(L.LOQT_OP_COMPENSATE, out, inn, r, 0), device)
+    for _ in range(2):
+        L.loqt_compensated_init(W, P, steps, ws=ws)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(iters):
+        L.loqt_compensated_init(W, P, steps, ws=ws)
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / iters
+    flops = (2 * steps - 1) * 2.0 * out * inn * r
+    tf = flops / (ms * 1e-3) / 1e12
+    return {
+        "shape": [out, inn], "r": r, "steps": steps, "ms": round(ms, 4), "tflops": round(tf, 1),
+        "pct_bf16_peak_burst": round(100 * tf / peaks["bf16_tflops"], 1), "of": peaks["source"],
+    }
+
+
 def run_per_shape(args):
     """Diagnostic: median time of forward, backward and merge for one matrix of
     each distinct shape of the configuration, L2 flushed between calls."""
@@ -393,6 +424,7 @@ def run_ours(args, rank, world, local_rank):
 
     peaks = load_peaks()
     nf4 = time_nf4_kernels(device, peaks)
+    comp = time_compensated_init(device, peaks, cfg, args.seed)
     tflops = world * flops_step / (ms_fb * 1e-3) / 1e12
     merge_gbs = world * merge_bytes_step / (ms_mg * 1e-3) / 1e9
     merge_tflops = world * merge_flops_step / (ms_mg * 1e-3) / 1e12
@@ -455,6 +487,7 @@ def run_ours(args, rank, world, local_rank):
             "steps": e2e_steps,
         },
         "nf4_stream": nf4,
+        "compensated_init": comp,
         "gpu_launches": int(launches),
         "clocks": clocks,
         "wall_s_timed": round(t_wall, 3),
