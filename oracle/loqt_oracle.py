@@ -248,3 +248,26 @@ def loqt_compensate(W, P, steps, B0=None):
         resid = bf16_round((W - nf4_dequantize(q[0], q[1], inn)).astype(np.float32))
         B = bf16_round((Pb.T @ resid.astype(np.float64)).astype(np.float32))
     return q, B
+
+
+def adam_step(B, g, m, v, step, lr, beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=0.0):
+    """One optimiser step on the trainable factor, B <- B - rho(G^B) (Algorithm 1,
+    the update line; Section 2.1: rho is Adam; hyper-parameter tables: AdamW,
+    optimiser states in BF16).  Adam as published by Kingma & Ba (Algorithm 1
+    there) with the decoupled weight decay of Loshchilov & Hutter:
+
+        m <- beta1 m + (1 - beta1) g          v <- beta2 v + (1 - beta2) g^2
+        mhat = m / (1 - beta1^t)              vhat = v / (1 - beta2^t)
+        B <- B - lr ( mhat / (sqrt(vhat) + eps) + weight_decay B )
+
+    B, m, v hold bf16 values, g is fp32; everything is evaluated in float64 and
+    B, m, v are rounded to bf16 once at the end.  Returns (B, m, v) as fp32 arrays
+    holding bf16 values."""
+    B64 = np.asarray(B, dtype=np.float64)
+    g64 = np.asarray(g, dtype=np.float32).astype(np.float64)
+    m64 = beta1 * np.asarray(m, dtype=np.float64) + (1.0 - beta1) * g64
+    v64 = beta2 * np.asarray(v, dtype=np.float64) + (1.0 - beta2) * g64 * g64
+    mhat = m64 / (1.0 - beta1 ** step)
+    vhat = v64 / (1.0 - beta2 ** step)
+    Bn = B64 - lr * (mhat / (np.sqrt(vhat) + eps) + weight_decay * B64)
+    return bf16_round(Bn.astype(np.float32)), bf16_round(m64.astype(np.float32)), bf16_round(v64.astype(np.float32))
