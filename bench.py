@@ -203,6 +203,30 @@ def time_nf4_kernels(device, peaks, rows=16384, cols=8192, iters=10):
     }
 
 
+def time_adam_step(device, peaks, rows=16384, cols=8192, iters=10):
+    """The fused optimiser step on a factor larger than L2: 4 (gradient) + 3 x (2 + 2)
+    (B and the two bf16 moments, read and written) = 16 bytes per element."""
+    import torch
+
+    from paper_2405_16528_b200 import binding as L
+
+    B = torch.randn((rows, cols), device=device, dtype=torch.float32).mul_(1e-2).to(torch.bfloat16)
+    g = torch.randn((rows, cols), device=device, dtype=torch.float32).mul_(1e-3)
+    m, v = torch.zeros_like(B), torch.zeros_like(B)
+    for step in range(1, 4):
+        L.loqt_adam_step(B, g, m, v, step, 1e-3)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(iters):
+        L.loqt_adam_step(B, g, m, v, 4 + i, 1e-3)
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / iters
+    gbs = rows * cols * 16 / (ms * 1e-3) / 1e9
+    return {"shape": [rows, cols], "ms": round(ms, 4), "gb_s": round(gbs, 1), "pct_hbm": round(100 * gbs / peaks["hbm_gbs"], 1),
+            "of": peaks["source"]}
+
+
 def time_compensated_init(device, peaks, cfg, seed, steps=5, iters=5):
     """Error-compensated initialisation (Section 2.5) of one matrix of the
     configuration's first shape: `steps` rounds of quantise + residual, B = P^T residual
@@ -425,6 +449,7 @@ def run_ours(args, rank, world, local_rank):
     peaks = load_peaks()
     nf4 = time_nf4_kernels(device, peaks)
     comp = time_compensated_init(device, peaks, cfg, args.seed)
+    adam = time_adam_step(device, peaks)
     tflops = world * flops_step / (ms_fb * 1e-3) / 1e12
     merge_gbs = world * merge_bytes_step / (ms_mg * 1e-3) / 1e9
     merge_tflops = world * merge_flops_step / (ms_mg * 1e-3) / 1e12
@@ -488,6 +513,7 @@ def run_ours(args, rank, world, local_rank):
         },
         "nf4_stream": nf4,
         "compensated_init": comp,
+        "adam_step": adam,
         "gpu_launches": int(launches),
         "clocks": clocks,
         "wall_s_timed": round(t_wall, 3),

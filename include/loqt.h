@@ -175,6 +175,27 @@ loqt_status loqt_compensated_init(const float *W, int64_t ldw, const float *P, i
                                   int64_t ldb, void *ws, size_t ws_bytes, void *stream);
 
 /*
+ * One optimiser step on the trainable factor (Algorithm 1, update line
+ * B <- B - rho(G^B); rho = Adam, Section 2.1; optimiser states in BF16 per the
+ * hyper-parameter appendix).  Adam as published by Kingma & Ba, with decoupled
+ * weight decay:
+ *     m <- beta1 m + (1 - beta1) g;   v <- beta2 v + (1 - beta2) g^2
+ *     B <- B - lr ( (m / (1 - beta1^step)) / (sqrt(v / (1 - beta2^step)) + eps) + weight_decay B )
+ *   B  : bf16 [r][ldb], updated in place;  dB : fp32 [r][lddb], the gradient from loqt_linear_bwd;
+ *   m, v : bf16 [r][ld_state], updated in place (zero before the first step).
+ * fp32 arithmetic, one rounding of B, m, v to bf16.  step counts from 1.  The
+ * hyper-parameters are carried as fp32: beta = 0.999 means the fp32 number nearest
+ * to it, also inside 1 - beta.
+ */
+typedef struct {
+  float lr, beta1, beta2, eps, weight_decay;
+  int32_t step;
+} loqt_adam_params;
+
+loqt_status loqt_adam_step(void *B, int64_t ldb, const float *dB, int64_t lddb, void *m, void *v,
+                           int64_t ld_state, int32_t r, int32_t in, loqt_adam_params hp, void *stream);
+
+/*
  * The same merge for n independent matrices in one call (a whole model at a
  * merge step).  Wq, Pq, B, ldb are HOST arrays of length n; the workspace is
  * shared and must satisfy the largest matrix.  A workspace of 256 + k times the

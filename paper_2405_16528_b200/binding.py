@@ -22,13 +22,20 @@ BLOCK = 64
 EXPORTS = (
     "loqt_nf4_quantize", "loqt_nf4_dequantize", "loqt_linear_fwd", "loqt_linear_bwd",
     "loqt_merge_requant", "loqt_merge_requant_many", "loqt_merge_requant_split", "loqt_nf4_requantize",
-    "loqt_compensated_init", "loqt_linear_fwd_static", "loqt_workspace_bytes",
+    "loqt_compensated_init", "loqt_adam_step", "loqt_linear_fwd_static", "loqt_workspace_bytes",
     "loqt_device_status", "loqt_launch_count", "loqt_status_string",
 )
 
 
 class LoqtError(RuntimeError):
     pass
+
+
+class loqt_adam_params(ctypes.Structure):
+    _fields_ = [
+        ("lr", ctypes.c_float), ("beta1", ctypes.c_float), ("beta2", ctypes.c_float), ("eps", ctypes.c_float),
+        ("weight_decay", ctypes.c_float), ("step", ctypes.c_int32),
+    ]
 
 
 class loqt_nf4_mat(ctypes.Structure):
@@ -69,6 +76,8 @@ def lib():
     L.loqt_nf4_requantize.argtypes = [vp, i64, f32, M, vp]
     L.loqt_compensated_init.argtypes = [vp, i64, vp, i64, i32, M, M, vp, i64, vp, sz, vp]
     L.loqt_compensated_init.restype = ctypes.c_int
+    L.loqt_adam_step.argtypes = [vp, i64, vp, i64, vp, vp, i64, i32, i32, loqt_adam_params, vp]
+    L.loqt_adam_step.restype = ctypes.c_int
     L.loqt_merge_requant_many.argtypes = [i32, ctypes.POINTER(M), ctypes.POINTER(M), ctypes.POINTER(vp), ctypes.POINTER(i64), f32, vp, sz, vp]
     L.loqt_workspace_bytes.argtypes = [ctypes.c_int, i32, i32, i32, i32]
     L.loqt_workspace_bytes.restype = sz
@@ -239,6 +248,17 @@ def loqt_compensated_init(W: torch.Tensor, P: torch.Tensor, steps: int, ws: torc
                                        _stream()), "loqt_compensated_init")
     loqt_device_status(ws)
     return Wq, Pq, B
+
+
+def loqt_adam_step(B: torch.Tensor, dB: torch.Tensor, m: torch.Tensor, v: torch.Tensor, step: int, lr: float,
+                   beta1: float = 0.9, beta2: float = 0.999, eps: float = 1e-8, weight_decay: float = 0.0) -> None:
+    """In-place optimiser step on B (bf16) and its bf16 moments m, v from the fp32 gradient dB."""
+    if m.shape != B.shape or v.shape != B.shape or m.stride(0) != v.stride(0):
+        raise LoqtError("B, m and v must have the same shape, m and v the same row stride")
+    hp = loqt_adam_params(lr, beta1, beta2, eps, weight_decay, int(step))
+    _check(lib().loqt_adam_step(_dev(B, torch.bfloat16), B.stride(0), _dev(dB, torch.float32), dB.stride(0),
+                                _dev(m, torch.bfloat16), _dev(v, torch.bfloat16), m.stride(0), B.shape[0], B.shape[1], hp,
+                                _stream()), "loqt_adam_step")
 
 
 def merge_many_workspace_bytes(Wqs, Pqs, group: int = 8) -> int:
