@@ -271,3 +271,11 @@ def adam_step(B, g, m, v, step, lr, beta1=0.9, beta2=0.999, eps=1e-8, weight_dec
     vhat = v64 / (1.0 - beta2 ** step)
     Bn = B64 - lr * (mhat / (np.sqrt(vhat) + eps) + weight_decay * B64)
     return bf16_round(Bn.astype(np.float32)), bf16_round(m64.astype(np.float32)), bf16_round(v64.astype(np.float32))
+
+
+def full_gradient(x, dy):
+    """G^W = dy^T x, the full-rank gradient of the layer's weight (out x in) that is
+    formed only at merge steps to find the next projection (Section 2.1, the
+    gradient G^W of Eq. for W's update; Algorithm 1, the line that computes G^W
+    before Initialize; Algorithm 2 takes its SVD).  Sums in float64."""
+    return np.asarray(dy, dtype=np.float64).T @ np.asarray(x, dtype=np.float64)

@@ -275,3 +275,19 @@ def test_compensate_later_steps_use_the_corrected_weights():
     rc, rm = O.nf4_quantize(what)
     assert np.array_equal(c2, rc) and np.array_equal(m2, rm)
     assert not np.array_equal(c2, O.nf4_quantize(W)[0])
+
+
+def test_full_gradient_is_the_dense_weight_gradient_and_projects_to_dB():
+    # G^W is what autograd gives for the dense layer y = x W^T, and the factor's
+    # gradient is its projection: dB = s P^T G^W (Section 2, "Equivalence of
+    # Gradient Updates").
+    out, inn, r, T = 48, 80, 8, 24
+    wq, pq, B, x, dy = _layer(61, out, inn, r, T)
+    G = O.full_gradient(x, dy)
+    Wt = torch.zeros((out, inn), dtype=torch.float64, requires_grad=True)
+    (torch.tensor(x, dtype=torch.float64) @ Wt.T * torch.tensor(dy, dtype=torch.float64)).sum().backward()
+    assert np.allclose(G, Wt.grad.numpy(), rtol=1e-12, atol=1e-12)
+    s = 0.5
+    _, dB = O.loqt_backward(wq, pq, B, s, x, dy, (out, inn, r))
+    P = O.nf4_dequantize_bf16(pq[0], pq[1], r).astype(np.float64)
+    assert np.allclose(dB, s * P.T @ G, rtol=1e-10, atol=1e-12)
