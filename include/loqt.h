@@ -69,7 +69,7 @@ typedef struct {
 } loqt_nf4_mat;
 
 /* Operation selector for loqt_workspace_bytes(). */
-enum { LOQT_OP_FWD = 0, LOQT_OP_BWD = 1, LOQT_OP_MERGE = 2, LOQT_OP_MERGE_SPLIT = 3, LOQT_OP_COMPENSATE = 4 };
+enum { LOQT_OP_FWD = 0, LOQT_OP_BWD = 1, LOQT_OP_MERGE = 2, LOQT_OP_MERGE_SPLIT = 3, LOQT_OP_COMPENSATE = 4, LOQT_OP_FULL_GRADIENT = 5 };
 
 /*
  * q_NF4 (Section 5.1, first two displayed equations): per block M = max|w|,
@@ -155,6 +155,19 @@ loqt_status loqt_nf4_requantize(const float *delta, int64_t ld_delta, float s, l
  */
 loqt_status loqt_merge_requant_split(loqt_nf4_mat Wq, loqt_nf4_mat Pq, const void *B, int64_t ldb,
                                      float s, void *ws, size_t ws_bytes, void *stream);
+
+/*
+ * Full-rank gradient of the layer's weight, formed only at merge steps to find
+ * the next projection (Algorithm 1: G^W is computed before Initialize; Algorithm
+ * 2 takes its leading singular vectors):
+ *     G = dy^T x        (fp32 [out][ldg]; overwritten, or added to when accumulate != 0)
+ *   x : bf16 [T][ldx],  dy : bf16 [T][lddy].  bf16 products, fp32 accumulation,
+ * split over T with a fixed-order reduction when the tiles alone would not fill
+ * the GPU.  Workspace: loqt_workspace_bytes(LOQT_OP_FULL_GRADIENT, out, in, 0, T).
+ */
+loqt_status loqt_full_gradient(const void *x, int64_t ldx, const void *dy, int64_t lddy, int32_t T,
+                               int32_t out, int32_t in, float *G, int64_t ldg, int accumulate,
+                               void *ws, size_t ws_bytes, void *stream);
 
 /*
  * Error-compensated initialisation of a layer for a new projection P

@@ -16,13 +16,13 @@ import torch
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libloqt.so")
 
-LOQT_OP_FWD, LOQT_OP_BWD, LOQT_OP_MERGE, LOQT_OP_MERGE_SPLIT, LOQT_OP_COMPENSATE = 0, 1, 2, 3, 4
+LOQT_OP_FWD, LOQT_OP_BWD, LOQT_OP_MERGE, LOQT_OP_MERGE_SPLIT, LOQT_OP_COMPENSATE, LOQT_OP_FULL_GRADIENT = 0, 1, 2, 3, 4, 5
 BLOCK = 64
 
 EXPORTS = (
     "loqt_nf4_quantize", "loqt_nf4_dequantize", "loqt_linear_fwd", "loqt_linear_bwd",
     "loqt_merge_requant", "loqt_merge_requant_many", "loqt_merge_requant_split", "loqt_nf4_requantize",
-    "loqt_compensated_init", "loqt_adam_step", "loqt_linear_fwd_static", "loqt_workspace_bytes",
+    "loqt_compensated_init", "loqt_full_gradient", "loqt_adam_step", "loqt_linear_fwd_static", "loqt_workspace_bytes",
     "loqt_device_status", "loqt_launch_count", "loqt_status_string",
 )
 
@@ -76,6 +76,8 @@ def lib():
     L.loqt_nf4_requantize.argtypes = [vp, i64, f32, M, vp]
     L.loqt_compensated_init.argtypes = [vp, i64, vp, i64, i32, M, M, vp, i64, vp, sz, vp]
     L.loqt_compensated_init.restype = ctypes.c_int
+    L.loqt_full_gradient.argtypes = [vp, i64, vp, i64, i32, i32, i32, vp, i64, ctypes.c_int, vp, sz, vp]
+    L.loqt_full_gradient.restype = ctypes.c_int
     L.loqt_adam_step.argtypes = [vp, i64, vp, i64, vp, vp, i64, i32, i32, loqt_adam_params, vp]
     L.loqt_adam_step.restype = ctypes.c_int
     L.loqt_merge_requant_many.argtypes = [i32, ctypes.POINTER(M), ctypes.POINTER(M), ctypes.POINTER(vp), ctypes.POINTER(i64), f32, vp, sz, vp]
@@ -248,6 +250,22 @@ def loqt_compensated_init(W: torch.Tensor, P: torch.Tensor, steps: int, ws: torc
                                        _stream()), "loqt_compensated_init")
     loqt_device_status(ws)
     return Wq, Pq, B
+
+
+def loqt_full_gradient(x: torch.Tensor, dy: torch.Tensor, G: torch.Tensor | None = None, accumulate: bool = False,
+                       ws: torch.Tensor | None = None) -> torch.Tensor:
+    """G^W = dy^T x (fp32 [out, in])."""
+    T, inn = x.shape
+    out = dy.shape[1]
+    if G is None:
+        ld = (inn + 3) // 4 * 4
+        G = torch.empty((out, ld), dtype=torch.float32, device=x.device)[:, :inn]
+    if ws is None:
+        ws = new_workspace(loqt_workspace_bytes(LOQT_OP_FULL_GRADIENT, out, inn, 0, T), x.device)
+    _check(lib().loqt_full_gradient(_dev(x, torch.bfloat16), x.stride(0), _dev(dy, torch.bfloat16), dy.stride(0), T, out, inn,
+                                    _dev(G, torch.float32), G.stride(0), int(accumulate), ws.data_ptr(), ws.numel(),
+                                    _stream()), "loqt_full_gradient")
+    return G
 
 
 def loqt_adam_step(B: torch.Tensor, dB: torch.Tensor, m: torch.Tensor, v: torch.Tensor, step: int, lr: float,

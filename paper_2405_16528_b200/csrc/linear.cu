@@ -295,6 +295,12 @@ extern "C" size_t loqt_workspace_bytes(int op, int32_t out, int32_t in, int32_t 
     db_splits(r, in, out > 0 ? out : 1, splits, kbps);
     if (splits > 1) total += align256(static_cast<size_t>(splits) * r * ld4 * 4);
   }
+  // full-rank gradient: split-K partials only (K = T)
+  if (op == LOQT_OP_FULL_GRADIENT) {
+    int splits = 1, kbps = 1;
+    db_splits(out, in, T > 0 ? T : 1, splits, kbps);
+    if (splits > 1) total += align256(static_cast<size_t>(splits) * out * ((static_cast<size_t>(in) + 3) / 4 * 4) * 4);
+  }
   return total;
 }
 
@@ -486,6 +492,26 @@ extern "C" loqt_status loqt_merge_requant_many(int32_t n, const loqt_nf4_mat *Wq
         return st;
   }
   return LOQT_OK;
+}
+
+// ---------------------------------------------------------------------------
+// Full-rank gradient at merge steps (Algorithm 1: G^W before Initialize)
+// ---------------------------------------------------------------------------
+extern "C" loqt_status loqt_full_gradient(const void *x, int64_t ldx, const void *dy, int64_t lddy, int32_t T, int32_t out,
+                                          int32_t in, float *G, int64_t ldg, int accumulate, void *ws, size_t ws_bytes,
+                                          void *stream) {
+  loqt_status st;
+  if (T <= 0 || out <= 0 || in <= 0) return LOQT_ERR_INVALID_ARG;
+  if ((st = check_bf16(x, ldx, in)) != LOQT_OK) return st;
+  if ((st = check_bf16(dy, lddy, out)) != LOQT_OK) return st;
+  if (G == nullptr || ldg < in) return LOQT_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(G) & 15u) != 0) return LOQT_ERR_ALIGNMENT;
+  if ((st = check_ws(ws, ws_bytes, loqt_workspace_bytes(LOQT_OP_FULL_GRADIENT, out, in, 0, T))) != LOQT_OK) return st;
+  if ((st = check_arch()) != LOQT_OK) return st;
+  float *partial = reinterpret_cast<float *>(static_cast<uint8_t *>(ws) + 256);
+  // G = dy^T x   (out x in; K = T; both operands stored K-outermost)
+  return gemm_tn_f32(dy, lddy, x, ldx, out, in, T, G, ldg, accumulate, partial, static_cast<uint32_t *>(ws),
+                     static_cast<cudaStream_t>(stream));
 }
 
 // ---------------------------------------------------------------------------

@@ -119,6 +119,19 @@ def test_requantize_bit_exact(shape, s):
     assert np.array_equal(got_c, ref_c) and np.array_equal(got_m, ref_m)
 
 
+@pytest.mark.parametrize("shape", SHAPES)
+def test_full_gradient(shape):
+    out, inn, r, T = shape
+    h, d = _setup(18, out, inn, r, T)
+    ref = O.full_gradient(h["x"], h["dy"])
+    G = L.loqt_full_gradient(d["x"], d["dy"])
+    check_close(f32(G), ref, f"G^W {shape}")
+    first = G.clone()
+    L.loqt_full_gradient(d["x"], d["dy"], G=G, accumulate=True)
+    check_close(f32(G), 2 * ref, f"G^W accumulated {shape}")
+    assert torch.equal(L.loqt_full_gradient(d["x"], d["dy"]), first)   # fixed reduction order
+
+
 def test_merge_zero_B_leaves_weights_untouched():
     out, inn, r = 256, 320, 32
     h, d = _setup(13, out, inn, r, 8)
