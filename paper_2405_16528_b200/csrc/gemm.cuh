@@ -104,7 +104,9 @@ struct TensorMaps {
   CUtensorMap cb[2];
 };
 
-template <int BN, int MH, bool TWO>
+// NF4: the kernel variant that stages NF4 operands (code ring, dequant warps); the
+// variant without spends that shared memory on a deeper operand ring.
+template <int BN, int MH, bool TWO, bool NF4>
 struct SmemLayout {
   static constexpr int kBM = MH * kHM;
   static constexpr int kBNL = TWO ? BN / 2 : BN;  // B rows staged by this CTA
@@ -118,9 +120,9 @@ struct SmemLayout {
   // The code ring is at least as deep as the operand ring (a staging group that has
   // seen operand slot `it` released may then conclude that the codes of stage
   // `it - kCodeStages` were consumed, which keeps its parity test unambiguous).
-  static constexpr int stages_for(int s) { return s * kStageBytes + (s > 4 ? s : 4) * kCodeBytes <= 225 * 1024; }
-  static constexpr int kStages = stages_for(6) ? 6 : stages_for(5) ? 5 : stages_for(4) ? 4 : stages_for(3) ? 3 : 2;
-  static constexpr int kCodeStages = kStages > 4 ? kStages : 4;
+  static constexpr int stages_for(int s) { return s * kStageBytes + (NF4 ? (s > 4 ? s : 4) * kCodeBytes : 0) <= 225 * 1024; }
+  static constexpr int kStages = (!NF4 && stages_for(7)) ? 7 : stages_for(6) ? 6 : stages_for(5) ? 5 : stages_for(4) ? 4 : stages_for(3) ? 3 : 2;
+  static constexpr int kCodeStages = !NF4 ? 0 : (kStages > 4 ? kStages : 4);
   static constexpr int kCodeOffset = kStages * kStageBytes;
   static constexpr int kBarOffset = kCodeOffset + kCodeStages * kCodeBytes;
   // full[S], empty[S], cfull[C], cempty[C], tfull[2], tempty[2], drain
@@ -130,7 +132,7 @@ struct SmemLayout {
   static constexpr int kTotal = kTablesOffset + static_cast<int>(sizeof(Nf4Tables));
   static constexpr int kDynamicBytes = kTotal + 1024;  // slack for 1024-byte alignment
   static_assert(kStages >= 3, "pipeline too shallow");
-  static_assert(kCodeStages >= kStages, "code ring too shallow");
+  static_assert(!NF4 || kCodeStages >= kStages, "code ring too shallow");
   static_assert(kDynamicBytes <= 232448, "exceeds the 227 KiB shared memory of one CTA");
   static_assert(kBM * 32 <= kCodeBytes && kBNL * 32 <= kCodeBytes, "code tile too large");
   static_assert(!TWO || BN == 256, "pairs run 256-wide tiles");
@@ -329,10 +331,10 @@ __device__ __forceinline__ void deq_store(const DeqGeom &g, const DeqTask &task,
 // ---------------------------------------------------------------------------
 // The kernel
 // ---------------------------------------------------------------------------
-template <int BN, int MH, bool TWO>
+template <int BN, int MH, bool TWO, bool NF4>
 __global__ void __launch_bounds__(kNumThreads, 1)
 loqt_gemm_kernel(const __grid_constant__ TensorMaps maps, const GemmParams p) {
-  using L = SmemLayout<BN, MH, TWO>;
+  using L = SmemLayout<BN, MH, TWO, NF4>;
   constexpr int kStages = L::kStages;
   constexpr int kBM = L::kBM;
   constexpr int kBNL = L::kBNL;
@@ -345,6 +347,7 @@ loqt_gemm_kernel(const __grid_constant__ TensorMaps maps, const GemmParams p) {
   auto full_bar = [&](int s) { return bar0 + 8u * s; };
   auto empty_bar = [&](int s) { return bar0 + 8u * (kStages + s); };
   constexpr int kCodeStages = L::kCodeStages;
+  constexpr int kCodeRing = kCodeStages > 0 ? kCodeStages : 1;  // (no code ring in kernels without NF4 operands)
   auto cfull_bar = [&](int c) { return bar0 + 8u * (2 * kStages + c); };
   auto cempty_bar = [&](int c) { return bar0 + 8u * (2 * kStages + kCodeStages + c); };
   auto tfull_bar = [&](int a) { return bar0 + 8u * (2 * kStages + 2 * kCodeStages + a); };
@@ -369,7 +372,7 @@ loqt_gemm_kernel(const __grid_constant__ TensorMaps maps, const GemmParams p) {
   // group stages and the other helps.  The 64-column blocks of a tile are dealt
   // to the epilogue groups round-robin, continuing across tiles.
   const bool requant_helpers = (MH == 1) && (p.epi == EPI_REQUANT);
-  const int epi_groups = requant_helpers ? (p.has_nf4 ? 2 : 3) : 1;
+  const int epi_groups = requant_helpers ? (NF4 ? 2 : 3) : 1;
   // The dequant warps work as two groups of four that take the K stages of a
   // tile in turn, so that one group's barrier, fence and bookkeeping time is
   // covered by the other's table lookups (the dequantisation is bound by the
@@ -379,7 +382,7 @@ loqt_gemm_kernel(const __grid_constant__ TensorMaps maps, const GemmParams p) {
   // loop of single-accumulator kernels, was measured 5 % slower: with three stages
   // in the ring a third group only waits for a slot.)
   constexpr int kGroupWarps = kDeqWarps / 2;
-  const int deq_groups = !p.has_nf4 ? 0 : (requant_helpers ? 1 : 2);
+  const int deq_groups = !NF4 ? 0 : (requant_helpers ? 1 : 2);
   const int deq_grp = (warp - kDeqWarp0) / kGroupWarps;
   constexpr uint32_t kTmemCols = 2 * BN;
 
@@ -387,7 +390,7 @@ loqt_gemm_kernel(const __grid_constant__ TensorMaps maps, const GemmParams p) {
     for (int s = 0; s < kStages; ++s) {
       // arrivals: the leader's TMA producer (which also posts the follower's bytes) and
       // the dequant warps of every CTA of the pair
-      ptx::mbar_init(full_bar(s), 1 + (p.has_nf4 ? kGroupWarps * (TWO ? 2 : 1) : 0));
+      ptx::mbar_init(full_bar(s), 1 + (NF4 ? kGroupWarps * (TWO ? 2 : 1) : 0));
       ptx::mbar_init(empty_bar(s), 1);
     }
     for (int c = 0; c < kCodeStages; ++c) {
@@ -463,7 +466,7 @@ loqt_gemm_kernel(const __grid_constant__ TensorMaps maps, const GemmParams p) {
     c.u += gridDim.x;
     return cur_open(c);
   };
-  auto cur_mine = [&](const Cursor &c) { return (c.kb - c.kb_lo) % deq_groups == deq_grp; };
+  auto cur_mine = [&](const Cursor &c) { return (c.kb - c.kb_lo) % (NF4 ? deq_groups : 1) == deq_grp; };
   auto cur_next_mine = [&](Cursor &c) {  // to this group's next stage
     do {
       if (!cur_advance(c)) return false;
@@ -505,8 +508,8 @@ loqt_gemm_kernel(const __grid_constant__ TensorMaps maps, const GemmParams p) {
     // been consumed, every stage up to `it - kCodeStages` has been staged, so the code
     // barrier cannot still be in the phase two uses back, which a parity test would
     // read as "already complete".
-    const int cs = cur.it % kCodeStages;
-    const uint32_t cph = (cur.it / kCodeStages) & 1u;
+    const int cs = cur.it % kCodeRing;
+    const uint32_t cph = (cur.it / kCodeRing) & 1u;
     if (!ptx::mbar_wait<TWO>(empty_bar(s), ph ^ 1u, abort_flag, p.status)) return false;
     if (!ptx::mbar_wait(cfull_bar(cs), cph, abort_flag, p.status)) return false;
     const uint32_t stage_base = smem_base + s * L::kStageBytes;
@@ -640,7 +643,7 @@ loqt_gemm_kernel(const __grid_constant__ TensorMaps maps, const GemmParams p) {
   }
   // =========================================================== code producer
   else if (warp == kCodeWarp) {
-    if (lane == 0 && p.has_nf4) {
+    if (lane == 0 && NF4) {
       // A cursor over the same sequence of stages as the operand producer's; the
       // ring's depth bounds how far the codes run ahead.
       struct CodeCursor {
@@ -662,8 +665,8 @@ loqt_gemm_kernel(const __grid_constant__ TensorMaps maps, const GemmParams p) {
       // Posts the code tile of the cursor's stage (or an empty completion when the
       // stage has no NF4 operand) and moves the cursor on.
       auto issue_codes = [&](CodeCursor &c) {
-        const int cs = c.it % kCodeStages;
-        const uint32_t cph = (c.it / kCodeStages) & 1u;
+        const int cs = c.it % kCodeRing;
+        const uint32_t cph = (c.it / kCodeRing) & 1u;
         if (!(ok = ptx::mbar_wait(cempty_bar(cs), cph ^ 1u, abort_flag, p.status))) return;
         const int sidx = c.kb < sched.kb_seg0 ? 0 : 1;
         const int k0 = (sidx == 0 ? c.kb : c.kb - sched.kb_seg0) * kBK;
@@ -691,7 +694,7 @@ loqt_gemm_kernel(const __grid_constant__ TensorMaps maps, const GemmParams p) {
       CodeCursor cc;
       cc.u = blockIdx.x;
       cc.it = 0;
-      cc.valid = p.has_nf4 && cc_open(cc);
+      cc.valid = NF4 && cc_open(cc);
       while (ok && cc.valid) issue_codes(cc);
 
     }
@@ -843,7 +846,7 @@ loqt_gemm_kernel(const __grid_constant__ TensorMaps maps, const GemmParams p) {
   }
   // =========================================================== NF4 dequant
   else {
-    if (p.has_nf4 && warp < kDeqWarp0 + kGroupWarps * deq_groups) {
+    if (NF4 && warp < kDeqWarp0 + kGroupWarps * deq_groups) {
       deq_begin();
       while (deq_have && deq_step()) {
       }

@@ -97,9 +97,9 @@ constexpr double kCyclesFixed = 3000.0;
 #endif
 constexpr bool kUsePairs = LOQT_USE_PAIRS != 0;
 
-template <int BN, int MH, bool TWO>
+template <int BN, int MH, bool TWO, bool NF4>
 static loqt_status launch_cfg(const GemmCall &c, cudaStream_t stream) {
-  using L = SmemLayout<BN, MH, TWO>;
+  using L = SmemLayout<BN, MH, TWO, NF4>;
   constexpr int BNL = L::kBNL;  // B rows one CTA stages
   TensorMaps maps;
   memset(&maps, 0, sizeof(maps));
@@ -122,7 +122,7 @@ static loqt_status launch_cfg(const GemmCall &c, cudaStream_t stream) {
         return LOQT_ERR_CUDA;
     }
   }
-  auto kernel = loqt_gemm_kernel<BN, MH, TWO>;
+  auto kernel = loqt_gemm_kernel<BN, MH, TWO, NF4>;
   if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kDynamicBytes) != cudaSuccess)
     return LOQT_ERR_CUDA;
   const int mt = (c.p.M + L::kBM - 1) / L::kBM, nt = (c.p.N + BN - 1) / BN;
@@ -207,14 +207,20 @@ static TileCfg pick_tile(const GemmCall &c) {
   return best;
 }
 
+template <bool NF4>
+static loqt_status launch_tile(const GemmCall &c, const TileCfg &t, cudaStream_t stream) {
+  if (t.two) return t.mh == 2 ? launch_cfg<256, 2, true, NF4>(c, stream) : launch_cfg<256, 1, true, NF4>(c, stream);
+  if (t.bn == 256) return t.mh == 2 ? launch_cfg<256, 2, false, NF4>(c, stream) : launch_cfg<256, 1, false, NF4>(c, stream);
+  return t.mh == 2 ? launch_cfg<128, 2, false, NF4>(c, stream) : launch_cfg<128, 1, false, NF4>(c, stream);
+}
+
 static loqt_status launch(GemmCall &c, cudaStream_t stream) {
   c.p.has_nf4 = 0;
   for (int s = 0; s < c.p.num_segs; ++s)
     if (c.p.seg[s].a_kind >= OP_NF4_K || c.p.seg[s].b_kind >= OP_NF4_K) c.p.has_nf4 = 1;
   const TileCfg t = pick_tile(c);
-  if (t.two) return t.mh == 2 ? launch_cfg<256, 2, true>(c, stream) : launch_cfg<256, 1, true>(c, stream);
-  if (t.bn == 256) return t.mh == 2 ? launch_cfg<256, 2, false>(c, stream) : launch_cfg<256, 1, false>(c, stream);
-  return t.mh == 2 ? launch_cfg<128, 2, false>(c, stream) : launch_cfg<128, 1, false>(c, stream);
+  if (c.p.has_nf4) return launch_tile<true>(c, t, stream);
+  return launch_tile<false>(c, t, stream);
 }
 
 // ---------------------------------------------------------------------------
