@@ -501,7 +501,7 @@ def run_ours(args, rank, world, local_rank):
             # DRAM read + write bytes of the five forward/backward launches (u, y, v, dx, dB) of one
             # 4096 x 4096 matrix, from the committed ncu capture; the algorithmic bytes of the same five
             # launches are 332.4e6 (part of y and dx is still in L2 when the kernels end)
-            "traffic": 274.1e6,
+            "traffic": 266.6e6,
             "traffic_of": "ncu dram bytes, 5 fwd+bwd launches of one 4096x4096 matrix (algorithmic 332.4e6)",
         },
         "e2e": {
