@@ -279,3 +279,44 @@ def full_gradient(x, dy):
     gradient G^W of Eq. for W's update; Algorithm 1, the line that computes G^W
     before Initialize; Algorithm 2 takes its SVD).  Sums in float64."""
     return np.asarray(dy, dtype=np.float64).T @ np.asarray(x, dtype=np.float64)
+
+
+# ----------------------------------------------------------------------------
+# Right-side variant  (Section 2.1, Eq. for the one-sided projection: "we compute
+# P^T G if m <= n and G Q otherwise"; Section 2.2: "if m > n the same reasoning
+# holds for Q^T").  The adapter sits on the input side:
+#     W = deq(W_q) + s B deq(Q_q),   B out x r trainable (bf16),   Q r x in frozen NF4.
+# ----------------------------------------------------------------------------
+def _operands_right(wq, qq, B, out_in_r):
+    out, inn, r = out_in_r
+    W = nf4_dequantize_bf16(wq[0], wq[1], inn).astype(np.float64)  # out x in
+    Q = nf4_dequantize_bf16(qq[0], qq[1], inn).astype(np.float64)  # r x in
+    Bm = np.asarray(B, dtype=np.float64)
+    assert W.shape == (out, inn) and Q.shape == (r, inn) and Bm.shape == (out, r)
+    return W, Q, Bm
+
+
+def loqt_forward_right(wq, qq, B, s, x, shape):
+    """y = x W^T + s (x Q^T) B^T, float64, factored order."""
+    W, Q, Bm = _operands_right(wq, qq, B, shape)
+    x = np.asarray(x, dtype=np.float64)
+    return x @ W.T + float(s) * ((x @ Q.T) @ Bm.T)
+
+
+def loqt_backward_right(wq, qq, B, s, x, dy, shape):
+    """Gradients of L = <y, dy>:  dx = dy W + s (dy B) Q;  dB = s dy^T (x Q^T)
+    (= s G^W Q^T with G^W = dy^T x).  Returns (dx [T, in], dB [out, r])."""
+    W, Q, Bm = _operands_right(wq, qq, B, shape)
+    x = np.asarray(x, dtype=np.float64)
+    dy = np.asarray(dy, dtype=np.float64)
+    dx = dy @ W + float(s) * ((dy @ Bm) @ Q)
+    dB = float(s) * (dy.T @ (x @ Q.T))
+    return dx, dB
+
+
+def loqt_merge_values_right(wq, qq, B, s, shape) -> np.ndarray:
+    """fl32( deq32(W_q) + s * B @ Q_BF16 ): the quantiser's input at a merge."""
+    out, inn, r = shape
+    W32 = nf4_dequantize(wq[0], wq[1], inn).astype(np.float64)
+    Q = nf4_dequantize_bf16(qq[0], qq[1], inn).astype(np.float64)
+    return (W32 + float(s) * (np.asarray(B, dtype=np.float64) @ Q)).astype(np.float32)

@@ -291,3 +291,52 @@ def test_full_gradient_is_the_dense_weight_gradient_and_projects_to_dB():
     _, dB = O.loqt_backward(wq, pq, B, s, x, dy, (out, inn, r))
     P = O.nf4_dequantize_bf16(pq[0], pq[1], r).astype(np.float64)
     assert np.allclose(dB, s * P.T @ G, rtol=1e-10, atol=1e-12)
+
+
+# ---- right-side variant (Section 2.1: G Q for m > n)
+def _layer_right(seed, out, inn, r, T):
+    W = synth.normal(seed, ("W",), (out, inn), 0.02).numpy()
+    Qm = synth.orthonormal(seed, ("Q",), inn, r).numpy().T.copy()      # r x in, orthonormal rows
+    B = synth.normal(seed, ("B",), (out, r), 1e-2, torch.bfloat16).to(torch.float32).numpy()
+    x = synth.normal(seed, ("x",), (T, inn), 1.0, torch.bfloat16).to(torch.float32).numpy()
+    dy = synth.normal(seed, ("dy",), (T, out), 1.0, torch.bfloat16).to(torch.float32).numpy()
+    return O.nf4_quantize(W), O.nf4_quantize(Qm), B, x, dy
+
+
+@pytest.mark.parametrize("shape", [(80, 48, 8, 12), (64, 40, 16, 7)])
+def test_right_variant_equals_the_dense_layer(shape):
+    out, inn, r, T = shape
+    s = 0.5
+    wq, qq, B, x, dy = _layer_right(71, out, inn, r, T)
+    W = O.nf4_dequantize_bf16(*wq, inn).astype(np.float64)
+    Q = O.nf4_dequantize_bf16(*qq, inn).astype(np.float64)
+    Weff = W + s * B.astype(np.float64) @ Q
+    y = O.loqt_forward_right(wq, qq, B, s, x, (out, inn, r))
+    assert np.allclose(y, x.astype(np.float64) @ Weff.T, rtol=1e-11, atol=1e-12)
+    # gradients by autograd on the dense parametrisation W + s B Q
+    Bt = torch.tensor(B, dtype=torch.float64, requires_grad=True)
+    xt = torch.tensor(x, dtype=torch.float64, requires_grad=True)
+    yt = xt @ (torch.tensor(W) + s * Bt @ torch.tensor(Q)).T
+    (yt * torch.tensor(dy, dtype=torch.float64)).sum().backward()
+    dx, dB = O.loqt_backward_right(wq, qq, B, s, x, dy, (out, inn, r))
+    assert np.allclose(dx, xt.grad.numpy(), rtol=1e-10, atol=1e-12)
+    assert np.allclose(dB, Bt.grad.numpy(), rtol=1e-10, atol=1e-12)
+    # the projection identity of the right side: dB = s G^W Q^T
+    assert np.allclose(dB, s * O.full_gradient(x, dy) @ Q.T, rtol=1e-10, atol=1e-12)
+
+
+def test_right_variant_is_the_left_variant_of_the_transposed_layer():
+    # W^T = W_q^T + s Q^T B^T: a left-side layer with P = Q^T and factor B^T.  With
+    # square blocks of identical scales out of reach, the check uses the dequantised
+    # matrices directly: the two merged weight matrices are transposes of each other.
+    out, inn, r, T = 64, 128, 8, 4
+    s = 0.25
+    wq, qq, B, x, dy = _layer_right(72, out, inn, r, T)
+    vw = O.loqt_merge_values_right(wq, qq, B, s, (out, inn, r))
+    W32 = O.nf4_dequantize(*wq, inn).astype(np.float64)
+    Q = O.nf4_dequantize_bf16(*qq, inn).astype(np.float64)
+    ref = (W32.T + s * Q.T @ B.astype(np.float64).T).T.astype(np.float32)
+    assert np.array_equal(vw, ref)
+    # B = 0 leaves the quantised weights untouched
+    c, m = O.nf4_quantize(O.loqt_merge_values_right(wq, qq, np.zeros_like(B), 1.0, (out, inn, r)))
+    assert np.array_equal(c, wq[0]) and np.array_equal(m, wq[1])
