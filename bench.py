@@ -304,12 +304,24 @@ def run_per_shape(args):
         delta = torch.randn((out, Wq.ld), dtype=torch.float32, device="cuda")[:, :inn] * 1e-3
         tr = timeit(lambda: L.loqt_nf4_requantize(delta, 1.0, Wc))
         requant_bytes = out * inn * 4 + 2 * synth.nf4_bytes(out, inn)
+        right = {}
+        if out > inn:
+            # the right-side variant the paper prescribes for tall matrices: Q is r x in, B out x r
+            Qq = L.loqt_nf4_quantize(synth.orthonormal(args.seed, ("Q", out, inn), inn, r, "cuda").T.contiguous())
+            Br = synth.normal(args.seed, ("Br", out, inn), (out, r), cfg.sigma_B, torch.bfloat16, "cuda")
+            trf = timeit(lambda: L.loqt_linear_fwd_right(Wq, Qq, Br, 1.0, x))
+            trb = timeit(lambda: L.loqt_linear_bwd_right(Wq, Qq, Br, 1.0, x, dy))
+            trm = timeit(lambda: L.loqt_merge_requant_right(Wc, Qq, Br, 1.0))
+            flops_r = 4.0 * T * inn * out + 2.0 * T * r * (2 * inn + 3 * out)
+            right = {"right_fwd_ms": round(trf, 4), "right_bwd_ms": round(trb, 4), "right_merge_ms": round(trm, 4),
+                     "right_fwdbwd_tflops": round(flops_r / (trf + trb) / 1e9, 1)}
         L.loqt_device_status(ws)
         res[f"{out}x{inn}"] = {
             "fwd_ms": round(tf, 4), "bwd_ms": round(tb, 4), "merge_ms": round(tm, 4), "merge_split_ms": round(ts, 4),
             "fwdbwd_tflops": round(synth.fwd_bwd_flops(out, inn, r, T) / (tf + tb) / 1e9, 1),
             "merge_gb_s": round(synth.merge_bytes(out, inn, r) / tm / 1e6, 1),
             "requant_stage_ms": round(tr, 4), "requant_stage_gb_s": round(requant_bytes / tr / 1e6, 1),
+            **right,
         }
     print(json.dumps({"per_shape": res, "config": cfg.name}), flush=True)
 

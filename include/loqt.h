@@ -69,7 +69,8 @@ typedef struct {
 } loqt_nf4_mat;
 
 /* Operation selector for loqt_workspace_bytes(). */
-enum { LOQT_OP_FWD = 0, LOQT_OP_BWD = 1, LOQT_OP_MERGE = 2, LOQT_OP_MERGE_SPLIT = 3, LOQT_OP_COMPENSATE = 4, LOQT_OP_FULL_GRADIENT = 5 };
+enum { LOQT_OP_FWD = 0, LOQT_OP_BWD = 1, LOQT_OP_MERGE = 2, LOQT_OP_MERGE_SPLIT = 3, LOQT_OP_COMPENSATE = 4, LOQT_OP_FULL_GRADIENT = 5,
+       LOQT_OP_FWD_RIGHT = 6, LOQT_OP_BWD_RIGHT = 7, LOQT_OP_MERGE_RIGHT = 8 };
 
 /*
  * q_NF4 (Section 5.1, first two displayed equations): per block M = max|w|,
@@ -154,6 +155,30 @@ loqt_status loqt_nf4_requantize(const float *delta, int64_t ld_delta, float s, l
  * and serves callers that already hold the product.
  */
 loqt_status loqt_merge_requant_split(loqt_nf4_mat Wq, loqt_nf4_mat Pq, const void *B, int64_t ldb,
+                                     float s, void *ws, size_t ws_bytes, void *stream);
+
+/*
+ * Right-side variant of the layer, for matrices with more rows than columns
+ * (Section 2.1: "we compute P^T G if m <= n and G Q otherwise"; Section 2.2: "if
+ * m > n the same reasoning holds for Q^T").  The frozen projection sits on the
+ * input side and the trainable factor is tall:
+ *     W = deq(W_q) + s B deq(Q_q)      Wq : out x in,  Qq : r x in (NF4, blocks along in),
+ *                                     B  : bf16 [out][ldb] (out x r)
+ *   forward   y  = x deq(W_q)^T + s (x deq(Q_q)^T) B^T
+ *   backward  dx = dy deq(W_q) + s (dy B) deq(Q_q);   dB = s dy^T (x deq(Q_q)^T)   (fp32 [out][lddb])
+ *   merge     W_q <- q_NF4( deq(W_q) + s B deq(Q_q) )   in place
+ * Arguments, precisions and error behaviour as for loqt_linear_fwd / _bwd /
+ * loqt_merge_requant; workspaces from loqt_workspace_bytes(LOQT_OP_FWD_RIGHT /
+ * LOQT_OP_BWD_RIGHT / LOQT_OP_MERGE_RIGHT, out, in, r, T).
+ */
+loqt_status loqt_linear_fwd_right(loqt_nf4_mat Wq, loqt_nf4_mat Qq, const void *B, int64_t ldb, float s,
+                                  const void *x, int64_t ldx, int32_t T, void *y, int64_t ldy,
+                                  void *ws, size_t ws_bytes, void *stream);
+loqt_status loqt_linear_bwd_right(loqt_nf4_mat Wq, loqt_nf4_mat Qq, const void *B, int64_t ldb, float s,
+                                  const void *x, int64_t ldx, const void *dy, int64_t lddy, int32_t T,
+                                  void *dx, int64_t lddx, float *dB, int64_t lddb, int accumulate_dB,
+                                  void *ws, size_t ws_bytes, void *stream);
+loqt_status loqt_merge_requant_right(loqt_nf4_mat Wq, loqt_nf4_mat Qq, const void *B, int64_t ldb,
                                      float s, void *ws, size_t ws_bytes, void *stream);
 
 /*

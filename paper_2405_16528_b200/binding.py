@@ -17,12 +17,14 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libloqt.so")
 
 LOQT_OP_FWD, LOQT_OP_BWD, LOQT_OP_MERGE, LOQT_OP_MERGE_SPLIT, LOQT_OP_COMPENSATE, LOQT_OP_FULL_GRADIENT = 0, 1, 2, 3, 4, 5
+LOQT_OP_FWD_RIGHT, LOQT_OP_BWD_RIGHT, LOQT_OP_MERGE_RIGHT = 6, 7, 8
 BLOCK = 64
 
 EXPORTS = (
     "loqt_nf4_quantize", "loqt_nf4_dequantize", "loqt_linear_fwd", "loqt_linear_bwd",
     "loqt_merge_requant", "loqt_merge_requant_many", "loqt_merge_requant_split", "loqt_nf4_requantize",
-    "loqt_compensated_init", "loqt_full_gradient", "loqt_adam_step", "loqt_linear_fwd_static", "loqt_workspace_bytes",
+    "loqt_compensated_init", "loqt_full_gradient", "loqt_adam_step",
+    "loqt_linear_fwd_right", "loqt_linear_bwd_right", "loqt_merge_requant_right", "loqt_linear_fwd_static", "loqt_workspace_bytes",
     "loqt_device_status", "loqt_launch_count", "loqt_status_string",
 )
 
@@ -76,6 +78,11 @@ def lib():
     L.loqt_nf4_requantize.argtypes = [vp, i64, f32, M, vp]
     L.loqt_compensated_init.argtypes = [vp, i64, vp, i64, i32, M, M, vp, i64, vp, sz, vp]
     L.loqt_compensated_init.restype = ctypes.c_int
+    L.loqt_linear_fwd_right.argtypes = L.loqt_linear_fwd.argtypes
+    L.loqt_linear_bwd_right.argtypes = L.loqt_linear_bwd.argtypes
+    L.loqt_merge_requant_right.argtypes = L.loqt_merge_requant.argtypes
+    for name in ("loqt_linear_fwd_right", "loqt_linear_bwd_right", "loqt_merge_requant_right"):
+        getattr(L, name).restype = ctypes.c_int
     L.loqt_full_gradient.argtypes = [vp, i64, vp, i64, i32, i32, i32, vp, i64, ctypes.c_int, vp, sz, vp]
     L.loqt_full_gradient.restype = ctypes.c_int
     L.loqt_adam_step.argtypes = [vp, i64, vp, i64, vp, vp, i64, i32, i32, loqt_adam_params, vp]
@@ -250,6 +257,42 @@ def loqt_compensated_init(W: torch.Tensor, P: torch.Tensor, steps: int, ws: torc
                                        _stream()), "loqt_compensated_init")
     loqt_device_status(ws)
     return Wq, Pq, B
+
+
+def loqt_linear_fwd_right(Wq: NF4Tensor, Qq: NF4Tensor, B: torch.Tensor, s: float, x: torch.Tensor) -> torch.Tensor:
+    """Right-side variant: y = x deq(W_q)^T + s (x deq(Q_q)^T) B^T; B is out x r."""
+    T = x.shape[0]
+    y = torch.empty((T, (Wq.rows + 7) // 8 * 8), dtype=torch.bfloat16, device=x.device)[:, : Wq.rows]
+    ws = new_workspace(loqt_workspace_bytes(LOQT_OP_FWD_RIGHT, Wq.rows, Wq.cols, Qq.rows, T), x.device)
+    _check(lib().loqt_linear_fwd_right(Wq.view(), Qq.view(), _dev(B, torch.bfloat16), B.stride(0), float(s),
+                                       _dev(x, torch.bfloat16), x.stride(0), T, y.data_ptr(), y.stride(0),
+                                       ws.data_ptr(), ws.numel(), _stream()), "loqt_linear_fwd_right")
+    loqt_device_status(ws)
+    return y
+
+
+def loqt_linear_bwd_right(Wq: NF4Tensor, Qq: NF4Tensor, B: torch.Tensor, s: float, x: torch.Tensor, dy: torch.Tensor,
+                          dB: torch.Tensor | None = None, accumulate_dB: bool = False):
+    """Right-side variant: returns (dx [T, in] bf16, dB [out, r] fp32)."""
+    T, r = x.shape[0], Qq.rows
+    dx = torch.empty((T, (Wq.cols + 7) // 8 * 8), dtype=torch.bfloat16, device=x.device)[:, : Wq.cols]
+    if dB is None:
+        dB = torch.empty((Wq.rows, (r + 3) // 4 * 4), dtype=torch.float32, device=x.device)[:, :r]
+    ws = new_workspace(loqt_workspace_bytes(LOQT_OP_BWD_RIGHT, Wq.rows, Wq.cols, r, T), x.device)
+    _check(lib().loqt_linear_bwd_right(Wq.view(), Qq.view(), _dev(B, torch.bfloat16), B.stride(0), float(s),
+                                       _dev(x, torch.bfloat16), x.stride(0), _dev(dy, torch.bfloat16), dy.stride(0), T,
+                                       dx.data_ptr(), dx.stride(0), _dev(dB, torch.float32), dB.stride(0),
+                                       int(accumulate_dB), ws.data_ptr(), ws.numel(), _stream()), "loqt_linear_bwd_right")
+    loqt_device_status(ws)
+    return dx, dB
+
+
+def loqt_merge_requant_right(Wq: NF4Tensor, Qq: NF4Tensor, B: torch.Tensor, s: float) -> NF4Tensor:
+    ws = new_workspace(loqt_workspace_bytes(LOQT_OP_MERGE_RIGHT, Wq.rows, Wq.cols, Qq.rows, 0), B.device)
+    _check(lib().loqt_merge_requant_right(Wq.view(), Qq.view(), _dev(B, torch.bfloat16), B.stride(0), float(s),
+                                          ws.data_ptr(), ws.numel(), _stream()), "loqt_merge_requant_right")
+    loqt_device_status(ws)
+    return Wq
 
 
 def loqt_full_gradient(x: torch.Tensor, dy: torch.Tensor, G: torch.Tensor | None = None, accumulate: bool = False,

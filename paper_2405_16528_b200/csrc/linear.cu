@@ -301,6 +301,16 @@ extern "C" size_t loqt_workspace_bytes(int op, int32_t out, int32_t in, int32_t 
     db_splits(r, in, out > 0 ? out : 1, splits, kbps);
     if (splits > 1) total += align256(static_cast<size_t>(splits) * r * ld4 * 4);
   }
+  // right-side variant: u (T x r) in forward; u, v (T x r) and the split-K partials of dB (out x r) in backward;
+  // deq(Q_q) as bf16 (r x roundup(in, 64)) in the merge
+  if (op == LOQT_OP_FWD_RIGHT) total += align256(static_cast<size_t>(T > 0 ? T : 0) * ld_lowrank(r) * 2);
+  if (op == LOQT_OP_BWD_RIGHT) {
+    total += 2 * align256(static_cast<size_t>(T > 0 ? T : 0) * ld_lowrank(r) * 2);
+    int splits = 1, kbps = 1;
+    db_splits(out, r, T > 0 ? T : 1, splits, kbps);
+    if (splits > 1) total += align256(static_cast<size_t>(splits) * out * ((static_cast<size_t>(r) + 3) / 4 * 4) * 4);
+  }
+  if (op == LOQT_OP_MERGE_RIGHT) total += align256(static_cast<size_t>(r > 0 ? r : 0) * ((static_cast<size_t>(in > 0 ? in : 0) + 63) / 64 * 64) * 2);
   // full-rank gradient: split-K partials only (K = T)
   if (op == LOQT_OP_FULL_GRADIENT) {
     int splits = 1, kbps = 1;
@@ -498,6 +508,127 @@ extern "C" loqt_status loqt_merge_requant_many(int32_t n, const loqt_nf4_mat *Wq
         return st;
   }
   return LOQT_OK;
+}
+
+// ---------------------------------------------------------------------------
+// Right-side variant: W = deq(W_q) + s B deq(Q_q)   (Section 2.1: G Q for m > n)
+//   Wq : out x in,  Qq : r x in (NF4, blocks along in),  B : bf16 [out][ldb] (out x r)
+// Every product is a configuration of the same engine.
+// ---------------------------------------------------------------------------
+static loqt_status check_layer_right(const loqt_nf4_mat &Wq, const loqt_nf4_mat &Qq, const void *B, int64_t ldb) {
+  loqt_status st;
+  if ((st = validate_nf4(Wq)) != LOQT_OK) return st;
+  if ((st = validate_nf4(Qq)) != LOQT_OK) return st;
+  if (Qq.cols != Wq.cols) return LOQT_ERR_INVALID_ARG;
+  return check_bf16(B, ldb, Qq.rows);
+}
+
+// u = s * x deq(Q_q)^T   (T x r; K = in, Q_q blocks along K)
+static loqt_status right_u(const loqt_nf4_mat &Qq, float s, const void *x, int64_t ldx, int T, void *u, int64_t ldu,
+                           uint32_t *status, cudaStream_t stm) {
+  GemmCall c{};
+  c.p.M = T; c.p.N = Qq.rows; c.p.num_segs = 1;
+  c.p.seg[0].K = Qq.cols; c.p.seg[0].a_kind = OP_TMA_K; c.p.seg[0].b_kind = OP_NF4_K; c.p.seg[0].b_nf4 = nf4_src(Qq);
+  c.a[0] = {x, ldx};
+  c.p.splits = 1;
+  c.p.epi = EPI_BF16; c.p.out = u; c.p.ld_out = ldu; c.p.alpha = s; c.p.status = status;
+  return launch(c, stm);
+}
+
+extern "C" loqt_status loqt_linear_fwd_right(loqt_nf4_mat Wq, loqt_nf4_mat Qq, const void *B, int64_t ldb, float s,
+                                             const void *x, int64_t ldx, int32_t T, void *y, int64_t ldy, void *ws,
+                                             size_t ws_bytes, void *stream) {
+  loqt_status st;
+  if ((st = check_layer_right(Wq, Qq, B, ldb)) != LOQT_OK) return st;
+  if (T <= 0) return LOQT_ERR_INVALID_ARG;
+  const int out = Wq.rows, in = Wq.cols, r = Qq.rows;
+  if ((st = check_bf16(x, ldx, in)) != LOQT_OK) return st;
+  if ((st = check_bf16(y, ldy, out)) != LOQT_OK) return st;
+  if ((st = check_ws(ws, ws_bytes, loqt_workspace_bytes(LOQT_OP_FWD_RIGHT, out, in, r, T))) != LOQT_OK) return st;
+  if ((st = check_arch()) != LOQT_OK) return st;
+  cudaStream_t stm = static_cast<cudaStream_t>(stream);
+  uint32_t *status = static_cast<uint32_t *>(ws);
+  void *u = static_cast<uint8_t *>(ws) + 256;
+  const int64_t ldu = ld_lowrank(r);
+  if ((st = right_u(Qq, s, x, ldx, T, u, ldu, status, stm)) != LOQT_OK) return st;
+  // y = x deq(W_q)^T + u B^T    (K = in, then K = r; B is K-major over r)
+  GemmCall c{};
+  c.p.M = T; c.p.N = out; c.p.num_segs = 2;
+  c.p.seg[0].K = in; c.p.seg[0].a_kind = OP_TMA_K; c.p.seg[0].b_kind = OP_NF4_K; c.p.seg[0].b_nf4 = nf4_src(Wq);
+  c.p.seg[1].K = r; c.p.seg[1].a_kind = OP_TMA_K; c.p.seg[1].b_kind = OP_TMA_K;
+  c.a[0] = {x, ldx}; c.a[1] = {u, ldu}; c.b[1] = {B, ldb};
+  c.p.splits = 1;
+  c.p.epi = EPI_BF16; c.p.out = y; c.p.ld_out = ldy; c.p.alpha = 1.0f; c.p.status = status;
+  return launch(c, stm);
+}
+
+extern "C" loqt_status loqt_linear_bwd_right(loqt_nf4_mat Wq, loqt_nf4_mat Qq, const void *B, int64_t ldb, float s,
+                                             const void *x, int64_t ldx, const void *dy, int64_t lddy, int32_t T, void *dx,
+                                             int64_t lddx, float *dB, int64_t lddb, int accumulate_dB, void *ws,
+                                             size_t ws_bytes, void *stream) {
+  loqt_status st;
+  if ((st = check_layer_right(Wq, Qq, B, ldb)) != LOQT_OK) return st;
+  if (T <= 0) return LOQT_ERR_INVALID_ARG;
+  const int out = Wq.rows, in = Wq.cols, r = Qq.rows;
+  if ((st = check_bf16(x, ldx, in)) != LOQT_OK) return st;
+  if ((st = check_bf16(dy, lddy, out)) != LOQT_OK) return st;
+  if (dx != nullptr && (st = check_bf16(dx, lddx, in)) != LOQT_OK) return st;
+  if (dB == nullptr || lddb < r) return LOQT_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(dB) & 15u) != 0) return LOQT_ERR_ALIGNMENT;
+  if ((st = check_ws(ws, ws_bytes, loqt_workspace_bytes(LOQT_OP_BWD_RIGHT, out, in, r, T))) != LOQT_OK) return st;
+  if ((st = check_arch()) != LOQT_OK) return st;
+  cudaStream_t stm = static_cast<cudaStream_t>(stream);
+  uint32_t *status = static_cast<uint32_t *>(ws);
+  const int64_t ldt = ld_lowrank(r);
+  const size_t tr_bytes = align256(static_cast<size_t>(T) * ldt * 2);
+  void *u = static_cast<uint8_t *>(ws) + 256;
+  void *v = static_cast<uint8_t *>(u) + tr_bytes;
+  float *partial = reinterpret_cast<float *>(static_cast<uint8_t *>(v) + tr_bytes);
+
+  // u = s * x deq(Q_q)^T, recomputed (the forward's copy is not kept)
+  if ((st = right_u(Qq, s, x, ldx, T, u, ldt, status, stm)) != LOQT_OK) return st;
+  if (dx != nullptr) {
+    // v = s * dy B             (T x r; K = out; B stored [K][N])
+    GemmCall c1{};
+    c1.p.M = T; c1.p.N = r; c1.p.num_segs = 1;
+    c1.p.seg[0].K = out; c1.p.seg[0].a_kind = OP_TMA_K; c1.p.seg[0].b_kind = OP_TMA_MN;
+    c1.a[0] = {dy, lddy}; c1.b[0] = {B, ldb};
+    c1.p.splits = 1;
+    c1.p.epi = EPI_BF16; c1.p.out = v; c1.p.ld_out = ldt; c1.p.alpha = s; c1.p.status = status;
+    if ((st = launch(c1, stm)) != LOQT_OK) return st;
+    // dx = dy deq(W_q) + v deq(Q_q)   (K = out with W_q blocks along N = in, then K = r with Q_q blocks along N = in)
+    GemmCall c2{};
+    c2.p.M = T; c2.p.N = in; c2.p.num_segs = 2;
+    c2.p.seg[0].K = out; c2.p.seg[0].a_kind = OP_TMA_K; c2.p.seg[0].b_kind = OP_NF4_MN; c2.p.seg[0].b_nf4 = nf4_src(Wq);
+    c2.p.seg[1].K = r; c2.p.seg[1].a_kind = OP_TMA_K; c2.p.seg[1].b_kind = OP_NF4_MN; c2.p.seg[1].b_nf4 = nf4_src(Qq);
+    c2.a[0] = {dy, lddy}; c2.a[1] = {v, ldt};
+    c2.p.splits = 1;
+    c2.p.epi = EPI_BF16; c2.p.out = dx; c2.p.ld_out = lddx; c2.p.alpha = 1.0f; c2.p.status = status;
+    if ((st = launch(c2, stm)) != LOQT_OK) return st;
+  }
+  // dB = dy^T u              (out x r; K = T; both operands stored K-outermost; u carries s)
+  return gemm_tn_f32(dy, lddy, u, ldt, out, r, T, dB, lddb, accumulate_dB, partial, status, stm);
+}
+
+extern "C" loqt_status loqt_merge_requant_right(loqt_nf4_mat Wq, loqt_nf4_mat Qq, const void *B, int64_t ldb, float s,
+                                                void *ws, size_t ws_bytes, void *stream) {
+  loqt_status st;
+  if ((st = check_layer_right(Wq, Qq, B, ldb)) != LOQT_OK) return st;
+  const int out = Wq.rows, in = Wq.cols, r = Qq.rows;
+  if ((st = check_ws(ws, ws_bytes, loqt_workspace_bytes(LOQT_OP_MERGE_RIGHT, out, in, r, 0))) != LOQT_OK) return st;
+  if ((st = check_arch()) != LOQT_OK) return st;
+  cudaStream_t stm = static_cast<cudaStream_t>(stream);
+  // Q-hat = bf16(deq(Q_q)), once; then Delta = B Q-hat (out x in; K = r) requantised in the epilogue
+  void *qhat = static_cast<uint8_t *>(ws) + 256;
+  if ((st = loqt_nf4_dequantize(Qq, qhat, Qq.ld, 1, stream)) != LOQT_OK) return st;
+  GemmCall c{};
+  c.p.M = out; c.p.N = in; c.p.num_segs = 1;
+  c.p.seg[0].K = r; c.p.seg[0].a_kind = OP_TMA_K; c.p.seg[0].b_kind = OP_TMA_MN;
+  c.a[0] = {B, ldb}; c.b[0] = {qhat, Qq.ld};
+  c.p.splits = 1;
+  c.p.epi = EPI_REQUANT; c.p.alpha = s; c.p.status = static_cast<uint32_t *>(ws);
+  c.p.wq_codes = Wq.codes; c.p.wq_absmax = Wq.absmax; c.p.wq_ld = Wq.ld;
+  return launch(c, stm);
 }
 
 // ---------------------------------------------------------------------------
