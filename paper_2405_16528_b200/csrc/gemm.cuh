@@ -28,10 +28,8 @@
 //
 // Warp roles (480 threads): warp 0 TMA producer of the bf16 operands, warp 1
 // MMA issuer + TMEM owner, warps 2-5 epilogue (one per TMEM lane quarter), warps
-// 6-13 NF4 dequantisation, warp 14 TMA producer of the packed codes (a producer
-// thread spends several hundred cycles per stage on its chain of barrier and
-// copy instructions; one thread for both rings was the pipeline's bottleneck).
-// One CTA per SM.
+// 6-13 NF4 dequantisation, warp 14 TMA producer of the packed codes (their ring
+// runs ahead of the operands', so it has a thread of its own).  One CTA per SM.
 #pragma once
 #include <type_traits>
 #include "nf4_dequant.cuh"

@@ -210,7 +210,7 @@ __device__ __forceinline__ void mma_bf16_ss_pair(uint32_t d_tmem, uint64_t a_des
       : "memory");
 }
 // The same arrival delivered to the barrier at this shared-memory offset in both
-// CTAs of the pair (a commit, not a load: no data is multicast).
+// CTAs of the pair (only the completion signal goes to both; operand copies never do).
 __device__ __forceinline__ void mma_commit_pair_both(uint32_t bar) {
   const uint16_t mask = 3;
   asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;" ::"r"(bar),
