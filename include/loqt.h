@@ -159,9 +159,10 @@ loqt_status loqt_merge_requant_split(loqt_nf4_mat Wq, loqt_nf4_mat Pq, const voi
 
 /*
  * Right-side variant of the layer, for matrices with more rows than columns
- * (Section 2.1: "we compute P^T G if m <= n and G Q otherwise"; Section 2.2: "if
- * m > n the same reasoning holds for Q^T").  The frozen projection sits on the
- * input side and the trainable factor is tall:
+ * (Section 2.1, the one-sided projection equation and the paragraph after it:
+ * the gradient is projected from the right, G Q, when the matrix is taller than
+ * wide, and the adapter derivation carries over with Q^T).  The frozen projection
+ * sits on the input side and the trainable factor is tall:
  *     W = deq(W_q) + s B deq(Q_q)      Wq : out x in,  Qq : r x in (NF4, blocks along in),
  *                                     B  : bf16 [out][ldb] (out x r)
  *   forward   y  = x deq(W_q)^T + s (x deq(Q_q)^T) B^T
@@ -293,6 +294,40 @@ loqt_status loqt_device_status(const void *ws, void *stream);
 /* Number of kernels this library has launched in this process (all entry
  * points, all streams); monotone, for instrumentation. */
 uint64_t loqt_launch_count(void);
+
+/*
+ * Testing and tuning hooks of the product engine.  (No counterpart in the
+ * paper: every product of Section 2 and the merge of Section 2.4 run through one
+ * GEMM kernel that exists in several tile shapes, picked per product by a cost
+ * model.)
+ *
+ * loqt_set_tile_override forces a tile shape for every later product of this
+ * process that supports it: bn = 128 or 256 output columns per tile, rows = 128
+ * or 256 token rows per CTA, pair = 1 to run two CTAs as one tcgen05 pair
+ * (needs bn = 256, else LOQT_ERR_UNSUPPORTED).  Products that cannot run the
+ * forced shape keep the automatic choice: split-K products never pair, and the
+ * merge runs single 128-row tiles only.  bn = 0 restores the automatic choice.
+ * The override is process-global and not synchronised with concurrent calls.
+ *
+ * loqt_variant_launches returns how often the kernel instantiation
+ * (bn, rows, pair, nf4) has been launched so far; nf4 = 1 counts the variant
+ * that dequantises NF4 operands in its main loop, 0 the one fed by TMA alone.
+ */
+loqt_status loqt_set_tile_override(int32_t bn, int32_t rows, int32_t pair);
+uint64_t loqt_variant_launches(int32_t bn, int32_t rows, int32_t pair, int32_t nf4);
+
+/*
+ * Self-test of the bounded device-side wait (no counterpart in the paper).
+ * Every wait inside the kernels gives up after a time limit, sets the status
+ * word of the workspace and lets the kernel drain and return.  This call
+ * launches a one-warp kernel that runs the same wait routine on a barrier
+ * nothing ever arrives on, with a limit of limit_us microseconds (1..100000),
+ * so that afterwards loqt_device_status(ws) reports LOQT_ERR_TIMEOUT and the
+ * context stays usable.  ws: at least 256 bytes, 256-byte aligned; word 0 is
+ * the status word, word 2 receives the number of lanes whose wait completed
+ * (must be 0), word 3 the CTA's abort flag (must be 1).
+ */
+loqt_status loqt_selftest_wait_timeout(void *ws, size_t ws_bytes, uint32_t limit_us, void *stream);
 
 const char *loqt_status_string(loqt_status st);
 

@@ -29,7 +29,7 @@ from __future__ import annotations
 
 import numpy as np
 
-BLOCK = 64  # Section 5.1: "blocks of 64 weights"
+BLOCK = 64  # Section 5.1: the block length of the NF4 quantiser
 
 # NF4 levels q_1..q_16 (ascending).  The paper defers to QLoRA for the values
 # (Section 5.1); these are the 16 fp32 numbers published there: 8 positive and
@@ -282,9 +282,10 @@ def full_gradient(x, dy):
 
 
 # ----------------------------------------------------------------------------
-# Right-side variant  (Section 2.1, Eq. for the one-sided projection: "we compute
-# P^T G if m <= n and G Q otherwise"; Section 2.2: "if m > n the same reasoning
-# holds for Q^T").  The adapter sits on the input side:
+# Right-side variant  (Section 2.1, the one-sided projection equation and the
+# paragraph after it: a matrix taller than wide is projected from the right,
+# G Q, and the adapter derivation carries over with Q^T).  The adapter sits on
+# the input side:
 #     W = deq(W_q) + s B deq(Q_q),   B out x r trainable (bf16),   Q r x in frozen NF4.
 # ----------------------------------------------------------------------------
 def _operands_right(wq, qq, B, out_in_r):

@@ -26,6 +26,7 @@ EXPORTS = (
     "loqt_compensated_init", "loqt_full_gradient", "loqt_adam_step",
     "loqt_linear_fwd_right", "loqt_linear_bwd_right", "loqt_merge_requant_right", "loqt_linear_fwd_static", "loqt_workspace_bytes",
     "loqt_device_status", "loqt_launch_count", "loqt_status_string",
+    "loqt_set_tile_override", "loqt_variant_launches", "loqt_selftest_wait_timeout",
 )
 
 
@@ -93,6 +94,12 @@ def lib():
     L.loqt_device_status.argtypes = [vp, vp]
     L.loqt_launch_count.argtypes = []
     L.loqt_launch_count.restype = ctypes.c_uint64
+    L.loqt_set_tile_override.argtypes = [i32, i32, i32]
+    L.loqt_set_tile_override.restype = ctypes.c_int
+    L.loqt_variant_launches.argtypes = [i32, i32, i32, i32]
+    L.loqt_variant_launches.restype = ctypes.c_uint64
+    L.loqt_selftest_wait_timeout.argtypes = [vp, sz, ctypes.c_uint32, vp]
+    L.loqt_selftest_wait_timeout.restype = ctypes.c_int
     L.loqt_status_string.argtypes = [ctypes.c_int]
     L.loqt_status_string.restype = ctypes.c_char_p
     for name in ("loqt_nf4_quantize", "loqt_nf4_dequantize", "loqt_linear_fwd", "loqt_linear_bwd",
@@ -350,3 +357,18 @@ def loqt_device_status(ws: torch.Tensor) -> None:
 
 def loqt_launch_count() -> int:
     return int(lib().loqt_launch_count())
+
+
+def loqt_set_tile_override(bn: int, rows: int = 128, pair: bool = False) -> None:
+    """Forces a tile shape for later products (bn = 0: automatic again)."""
+    _check(lib().loqt_set_tile_override(int(bn), int(rows), int(bool(pair))), "loqt_set_tile_override")
+
+
+def loqt_variant_launches(bn: int, rows: int, pair: bool, nf4: bool) -> int:
+    return int(lib().loqt_variant_launches(int(bn), int(rows), int(bool(pair)), int(bool(nf4))))
+
+
+def loqt_selftest_wait_timeout(ws: torch.Tensor, limit_us: int = 1000) -> None:
+    """Launches the wait self-test; the outcome is read with loqt_device_status(ws)."""
+    _check(lib().loqt_selftest_wait_timeout(ws.data_ptr(), ws.numel(), int(limit_us), _stream()),
+           "loqt_selftest_wait_timeout")

@@ -159,8 +159,12 @@ __device__ __forceinline__ uint32_t make_idesc(int m, int bn, bool a_mn, bool b_
 struct Sched {
   int mt, nt, units;
   int kb_seg0, kb_total, splits, kb_per_split;
-  __device__ __forceinline__ Sched(const GemmParams &p, int bm, int bn) {
+  // `pairs`: CTAs 2k and 2k+1 of the grid share every N tile, so the M tiles are
+  // counted in twos; an odd count gets one tile past the matrix (its loads read
+  // zeros, its rows are never stored).
+  __device__ __forceinline__ Sched(const GemmParams &p, int bm, int bn, bool pairs) {
     mt = (p.M + bm - 1) / bm;
+    if (pairs) mt = (mt + 1) & ~1;
     nt = (p.N + bn - 1) / bn;
     splits = p.splits;
     kb_per_split = p.kb_per_split;
@@ -358,7 +362,7 @@ loqt_gemm_kernel(const __grid_constant__ TensorMaps maps, const GemmParams p) {
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
-  const Sched sched(p, kBM, BN);
+  const Sched sched(p, kBM, BN, TWO);
   // TWO: rank 0 of the pair is the leader (issues the MMAs, owns the barriers the
   // MMA thread waits on).
   const uint32_t rank = TWO ? ptx::cluster_ctarank() : 0u;

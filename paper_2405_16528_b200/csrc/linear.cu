@@ -1,5 +1,6 @@
 // Host side of the LoQT linear layer: argument checks, TMA descriptors, kernel
 // launches for forward, backward and merge (paper Section 2, Algorithm 1).
+#include <atomic>
 #include <mutex>
 
 #include "gemm.cuh"
@@ -97,6 +98,14 @@ constexpr double kCyclesFixed = 3000.0;
 #endif
 constexpr bool kUsePairs = LOQT_USE_PAIRS != 0;
 
+// Launches per kernel variant (instrumentation: tests ask which instantiation a
+// call ran) and the tile override of loqt_set_tile_override().
+static std::atomic<uint64_t> g_variant_launches[16];
+static std::atomic<int> g_force_bn{0}, g_force_mh{0}, g_force_pair{0};
+static int variant_index(int bn, int mh, bool two, bool nf4) {
+  return (bn == 256 ? 1 : 0) | (mh == 2 ? 2 : 0) | (two ? 4 : 0) | (nf4 ? 8 : 0);
+}
+
 template <int BN, int MH, bool TWO, bool NF4>
 static loqt_status launch_cfg(const GemmCall &c, cudaStream_t stream) {
   using L = SmemLayout<BN, MH, TWO, NF4>;
@@ -125,7 +134,9 @@ static loqt_status launch_cfg(const GemmCall &c, cudaStream_t stream) {
   auto kernel = loqt_gemm_kernel<BN, MH, TWO, NF4>;
   if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kDynamicBytes) != cudaSuccess)
     return LOQT_ERR_CUDA;
-  const int mt = (c.p.M + L::kBM - 1) / L::kBM, nt = (c.p.N + BN - 1) / BN;
+  int mt = (c.p.M + L::kBM - 1) / L::kBM;
+  if (TWO) mt = (mt + 1) & ~1;  // pairs count M tiles in twos (see Sched)
+  const int nt = (c.p.N + BN - 1) / BN;
   const int units = mt * nt * c.p.splits;
   int grid = units < sm_count() ? units : sm_count();
   cudaLaunchConfig_t cfg;
@@ -139,6 +150,7 @@ static loqt_status launch_cfg(const GemmCall &c, cudaStream_t stream) {
   ++nattr;
   if (TWO) {
     grid &= ~1;  // whole pairs (`units` is even in this mode)
+    if (grid < 2) grid = 2;
     attr[nattr].id = cudaLaunchAttributeClusterDimension;
     attr[nattr].val.clusterDim.x = 2;
     attr[nattr].val.clusterDim.y = 1;
@@ -153,6 +165,7 @@ static loqt_status launch_cfg(const GemmCall &c, cudaStream_t stream) {
   cfg.stream = stream;
   const cudaError_t err = cudaLaunchKernelEx(&cfg, kernel, maps, c.p);
   count_launch();
+  g_variant_launches[variant_index(BN, MH, TWO, NF4)].fetch_add(1, std::memory_order_relaxed);
   return (err == cudaSuccess && cudaGetLastError() == cudaSuccess) ? LOQT_OK : LOQT_ERR_CUDA;
 }
 
@@ -204,6 +217,18 @@ static TileCfg pick_tile(const GemmCall &c) {
   // where it can (measured faster for every product but the merge, whose epilogue
   // - not its main loop - sets the pace).
   best.two = pair_ok(c, best.bn, best.mh) && c.p.epi != EPI_REQUANT;
+  // A tile forced by loqt_set_tile_override() replaces the choice wherever the
+  // kernel supports it for this product: pairs need 256-wide tiles and no split-K
+  // (an odd number of M tiles is rounded up by one empty tile), and the merge
+  // epilogue runs on single 128-row tiles only.
+  const int fbn = g_force_bn.load(std::memory_order_relaxed);
+  if (fbn != 0) {
+    const int fmh = g_force_mh.load(std::memory_order_relaxed);
+    const bool fpair = g_force_pair.load(std::memory_order_relaxed) != 0;
+    const bool merge = c.p.epi == EPI_REQUANT;
+    const bool ok = !(merge && (fmh == 2 || fpair)) && !(fpair && (fbn != 256 || c.p.splits != 1 || !kUsePairs));
+    if (ok) best = TileCfg{fbn, fmh, fpair};
+  }
   return best;
 }
 
@@ -229,11 +254,11 @@ static loqt_status launch(GemmCall &c, cudaStream_t stream) {
 static size_t align256(size_t v) { return (v + 255) & ~static_cast<size_t>(255); }
 static int64_t ld_lowrank(int r) { return (static_cast<int64_t>(r) + 63) / 64 * 64; }  // bf16 T x r scratch
 
-// Split-K factor of the dB product (M = r, N = in, K = T), for a 148-SM part.
+// Split-K factor of the dB product (M = r, N = in, K = T): enough splits to give every SM a tile.
 static void db_splits(int r, int in, int T, int &splits, int &kb_per_split) {
   const int tiles = ((r + kHM - 1) / kHM) * ((in + (in > 128 ? 255 : 127)) / (in > 128 ? 256 : 128));
   const int kb_total = (T + kBK - 1) / kBK;
-  int want = 148 / (tiles > 0 ? tiles : 1);
+  int want = sm_count() / (tiles > 0 ? tiles : 1);
   if (want < 1) want = 1;
   if (want > 16) want = 16;
   const int max_by_k = kb_total / 4 > 0 ? kb_total / 4 : 1;  // at least 4 k-blocks per split
@@ -334,15 +359,22 @@ static loqt_status check_ws(const void *ws, size_t ws_bytes, size_t need) {
   return LOQT_OK;
 }
 
+// Argument checks of the forward, shared by its two entry points.
+static loqt_status check_fwd_args(const loqt_nf4_mat &Wq, const loqt_nf4_mat &Pq, const void *B, int64_t ldb, const void *x,
+                                  int64_t ldx, int32_t T, const void *y, int64_t ldy) {
+  loqt_status st;
+  if ((st = check_layer(Wq, Pq, B, ldb)) != LOQT_OK) return st;
+  if (T <= 0) return LOQT_ERR_INVALID_ARG;
+  if ((st = check_bf16(x, ldx, Wq.cols)) != LOQT_OK) return st;
+  return check_bf16(y, ldy, Wq.rows);
+}
+
 extern "C" loqt_status loqt_linear_fwd(loqt_nf4_mat Wq, loqt_nf4_mat Pq, const void *B, int64_t ldb, float s,
                                        const void *x, int64_t ldx, int32_t T, void *y, int64_t ldy, void *ws,
                                        size_t ws_bytes, void *stream) {
   loqt_status st;
-  if ((st = check_layer(Wq, Pq, B, ldb)) != LOQT_OK) return st;
-  if (T <= 0) return LOQT_ERR_INVALID_ARG;
+  if ((st = check_fwd_args(Wq, Pq, B, ldb, x, ldx, T, y, ldy)) != LOQT_OK) return st;
   const int out = Wq.rows, in = Wq.cols, r = Pq.cols;
-  if ((st = check_bf16(x, ldx, in)) != LOQT_OK) return st;
-  if ((st = check_bf16(y, ldy, out)) != LOQT_OK) return st;
   if ((st = check_ws(ws, ws_bytes, loqt_workspace_bytes(LOQT_OP_FWD, out, in, r, T))) != LOQT_OK) return st;
   if ((st = check_arch()) != LOQT_OK) return st;
   cudaStream_t stm = static_cast<cudaStream_t>(stream);
@@ -706,6 +738,27 @@ extern "C" loqt_status loqt_compensated_init(const float *W, int64_t ldw, const 
 }
 
 // ---------------------------------------------------------------------------
+// Tile override and per-variant launch counts (testing and tuning hooks)
+// ---------------------------------------------------------------------------
+extern "C" loqt_status loqt_set_tile_override(int32_t bn, int32_t rows, int32_t pair) {
+  if (bn == 0) {
+    g_force_bn.store(0, std::memory_order_relaxed);
+    return LOQT_OK;
+  }
+  if ((bn != 128 && bn != 256) || (rows != 128 && rows != 256) || (pair != 0 && pair != 1)) return LOQT_ERR_INVALID_ARG;
+  if (pair != 0 && (bn != 256 || !kUsePairs)) return LOQT_ERR_UNSUPPORTED;
+  g_force_mh.store(rows / kHM, std::memory_order_relaxed);
+  g_force_pair.store(pair, std::memory_order_relaxed);
+  g_force_bn.store(bn, std::memory_order_relaxed);
+  return LOQT_OK;
+}
+
+extern "C" uint64_t loqt_variant_launches(int32_t bn, int32_t rows, int32_t pair, int32_t nf4) {
+  if ((bn != 128 && bn != 256) || (rows != 128 && rows != 256)) return 0;
+  return g_variant_launches[variant_index(bn, rows / kHM, pair != 0, nf4 != 0)].load(std::memory_order_relaxed);
+}
+
+// ---------------------------------------------------------------------------
 // Forward without any caller-provided scratch (see loqt_linear_fwd_static in loqt.h)
 // ---------------------------------------------------------------------------
 namespace loqt {
@@ -741,10 +794,12 @@ static loqt_status static_scratch_for_current_device(void **out) {
 extern "C" loqt_status loqt_linear_fwd_static(loqt_nf4_mat Wq, loqt_nf4_mat Pq, const void *B, int64_t ldb, float s,
                                               const void *x, int64_t ldx, int32_t T, void *y, int64_t ldy,
                                               int check_device_status, void *stream) {
-  if (T <= 0 || Pq.cols <= 0) return LOQT_ERR_INVALID_ARG;
+  // Every argument check comes before the first thing enqueued: a rejected call
+  // must leave the shared status word as it was.
+  loqt_status st;
+  if ((st = check_fwd_args(Wq, Pq, B, ldb, x, ldx, T, y, ldy)) != LOQT_OK) return st;
   const size_t need = loqt_workspace_bytes(LOQT_OP_FWD, Wq.rows, Wq.cols, Pq.cols, T);
   if (need > kStaticScratchBytes) return LOQT_ERR_WORKSPACE;  // T * roundup(r, 64) * 2 bytes exceeds the built-in scratch
-  loqt_status st;
   if ((st = check_arch()) != LOQT_OK) return st;
   void *scratch = nullptr;
   if ((st = static_scratch_for_current_device(&scratch)) != LOQT_OK) return st;

@@ -62,7 +62,7 @@ def test_merge(shape, sigma_B):
     mag = np.abs(h["B"]).astype(np.float64) @ Qh
     ulp = np.spacing(np.abs(ref_m).astype(np.float32)).astype(np.float64)
     bound = (np.ceil(r / 16) + 1) * 2.0 ** -23 * abs(s) * mag + np.repeat(ulp, 64, axis=1)[:, :inn]
-    n_diff, max_ulp = check_merge(got_c, got_m, ref_c, ref_m, vw, inn, bound, f"merge {shape}")
+    n_diff, max_ulp, hist = check_merge(got_c, got_m, ref_c, ref_m, vw, inn, bound, f"merge {shape}")
     assert np.all(got_c[:, inn:] == 7)
 
 

@@ -340,3 +340,39 @@ def test_right_variant_is_the_left_variant_of_the_transposed_layer():
     # B = 0 leaves the quantised weights untouched
     c, m = O.nf4_quantize(O.loqt_merge_values_right(wq, qq, np.zeros_like(B), 1.0, (out, inn, r)))
     assert np.array_equal(c, wq[0]) and np.array_equal(m, wq[1])
+
+
+@pytest.mark.parametrize("shape", [(40, 100, 8), (64, 128, 16)])
+def test_right_merge_equals_the_dense_sum_built_entry_by_entry(shape):
+    """The right variant's merged matrix, formed without any oracle routine:
+    W enters as the unrounded fp32 product M * q, Q as that product rounded to
+    bf16 (torch's conversion), each entry's sum over r evaluated exactly
+    (math.fsum) and rounded once to fp32.  A wrong operand precision for Q or W
+    changes low-order bits of many entries and fails the bit-for-bit comparison."""
+    import math
+
+    out, inn, r = shape
+    s = 0.5
+    wq, qq, B, _, _ = _layer_right(73, out, inn, r, 2)
+    B = (B * 3.0).astype(np.float32)      # large enough to move values across fp32 roundings
+    B = O.bf16_round(B)
+    lv = O.NF4_LEVELS
+    bf = lambda v: float(torch.tensor(float(v), dtype=torch.float32).to(torch.bfloat16))
+    Q = [[bf(np.float32(qq[1][k, i // 64]) * lv[qq[0][k, i]]) for i in range(inn)] for k in range(r)]
+    ref = np.zeros((out, inn), dtype=np.float32)
+    for o in range(out):
+        for i in range(inn):
+            w32 = float(np.float32(wq[1][o, i // 64]) * lv[wq[0][o, i]])
+            # s = 0.5 and the bf16 x bf16 products are exact in float64, so fsum sees the exact terms
+            ref[o, i] = np.float32(math.fsum([w32] + [s * float(B[o, k]) * Q[k][i] for k in range(r)]))
+    vw = O.loqt_merge_values_right(wq, qq, B, s, (out, inn, r))
+    # float64 accumulation of <= 16 terms of this size differs from the exact sum by far less than
+    # half an fp32 ulp except at rounding ties; allow the two roundings to disagree on at most a few
+    # entries, and then only by one fp32 ulp
+    diff = vw != ref
+    assert diff.mean() < 2e-3
+    assert np.all(np.abs(vw[diff] - ref[diff]) <= np.spacing(np.abs(ref[diff])))
+    # the same construction with Q left unrounded (fp32) is visibly different: the pin has teeth
+    Q32 = np.array([[float(np.float32(qq[1][k, i // 64]) * lv[qq[0][k, i]]) for i in range(inn)] for k in range(r)])
+    wrong = (O.nf4_dequantize(*wq, inn).astype(np.float64) + s * B.astype(np.float64) @ Q32).astype(np.float32)
+    assert np.mean(wrong != vw) > 0.2

@@ -9,14 +9,17 @@ keeps the forward's scratch in a fixed 8 MiB array of its own.
 This file is named so that pytest collects it last.  It calls the entry point
 through the C ABI twice in a row with different inputs (the shared array still
 holds the first call's intermediate when the second starts) and compares each
-result with the ordinary entry point's on the same inputs.
+result with the ordinary entry point's on the same inputs, and with the CPU
+oracle's forward.
 """
+import numpy as np
 import pytest
 import torch
 
+from oracle import loqt_oracle as O
 from paper_2405_16528_b200 import binding as L
 from paper_2405_16528_b200 import synth
-from tests.gpu_util import MAX_REL, MEAN_REL
+from tests.gpu_util import MAX_REL, MEAN_REL, check_close, f32, from_dev_nf4
 
 pytestmark = pytest.mark.gpu
 
@@ -42,12 +45,24 @@ def test_static_forward_matches_workspace_forward_twice():
         Wq, Pq, B, x = _layer(seed, out, inn, r, T)
         ref = L.loqt_linear_fwd(Wq, Pq, B, s, x)
         y = torch.full((T, out), float("nan"), dtype=torch.bfloat16, device="cuda")
-        before = torch.cuda.memory_allocated()
-        L.loqt_linear_fwd_static(Wq, Pq, B, s, x, y)
-        assert torch.cuda.memory_allocated() == before, "the static entry point must not allocate through torch"
+        if call == 0:
+            # the first call on a device looks up the scratch array's address; let the context settle
+            # before the free-memory readings below
+            L.loqt_linear_fwd_static(Wq, Pq, B, s, x, y)
+            y.fill_(float("nan"))
         torch.cuda.synchronize()
+        before = torch.cuda.memory_allocated()
+        free_before, _ = torch.cuda.mem_get_info()
+        L.loqt_linear_fwd_static(Wq, Pq, B, s, x, y)
+        torch.cuda.synchronize()
+        free_after, _ = torch.cuda.mem_get_info()
+        assert torch.cuda.memory_allocated() == before, "the static entry point must not allocate through torch"
+        # the driver's own count of free device memory sees an allocation made inside the library too
+        assert free_after >= free_before, f"device memory shrank by {free_before - free_after} bytes during the call"
         _compare(y, ref)
         assert torch.equal(y, ref), f"call {call}: same kernels, same inputs, different bits"
+        oracle_y = O.loqt_forward(from_dev_nf4(Wq), from_dev_nf4(Pq), f32(B), s, f32(x), (out, inn, r))
+        check_close(f32(y), oracle_y, f"static forward, call {call}")
 
 
 def test_static_forward_rejects_oversized_problems():
