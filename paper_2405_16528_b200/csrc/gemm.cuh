@@ -94,17 +94,21 @@ struct GemmParams {
   int has_nf4;       // any NF4 operand in any segment
 };
 
-// a/b: bf16 operands; ca/cb: packed NF4 codes viewed as a byte matrix.
+// a/b: bf16 operands; ca/cb: packed NF4 codes viewed as a byte matrix; wq: the
+// packed codes of the matrix a merge updates, one output tile per box.
 struct TensorMaps {
   CUtensorMap a[2];
   CUtensorMap b[2];
   CUtensorMap ca[2];
   CUtensorMap cb[2];
+  CUtensorMap wq;
 };
 
 // NF4: the kernel variant that stages NF4 operands (code ring, dequant warps); the
 // variant without spends that shared memory on a deeper operand ring.
-template <int BN, int MH, bool TWO, bool NF4>
+// REQ: the merge kernel (requantising epilogue): two buffers hold the packed codes
+// of the output tiles' W_q blocks on their way from and to global memory.
+template <int BN, int MH, bool TWO, bool NF4, bool REQ = false>
 struct SmemLayout {
   static constexpr int kBM = MH * kHM;
   static constexpr int kBNL = TWO ? BN / 2 : BN;  // B rows staged by this CTA
@@ -118,13 +122,18 @@ struct SmemLayout {
   // The code ring is at least as deep as the operand ring (a staging group that has
   // seen operand slot `it` released may then conclude that the codes of stage
   // `it - kCodeStages` were consumed, which keeps its parity test unambiguous).
-  static constexpr int stages_for(int s) { return s * kStageBytes + (NF4 ? (s > 4 ? s : 4) * kCodeBytes : 0) <= 225 * 1024; }
+  static constexpr int kWTileBytes = REQ ? kHM * (BN / 2) : 0;  // codes of 128 rows x BN columns of W_q
+  static constexpr int kWBufs = REQ ? 2 : 0;
+  static constexpr int stages_for(int s) {
+    return s * kStageBytes + (NF4 ? (s > 4 ? s : 4) * kCodeBytes : 0) + kWBufs * kWTileBytes <= 225 * 1024;
+  }
   static constexpr int kStages = (!NF4 && stages_for(7)) ? 7 : stages_for(6) ? 6 : stages_for(5) ? 5 : stages_for(4) ? 4 : stages_for(3) ? 3 : 2;
   static constexpr int kCodeStages = !NF4 ? 0 : (kStages > 4 ? kStages : 4);
   static constexpr int kCodeOffset = kStages * kStageBytes;
-  static constexpr int kBarOffset = kCodeOffset + kCodeStages * kCodeBytes;
-  // full[S], empty[S], cfull[C], cempty[C], tfull[2], tempty[2], drain
-  static constexpr int kNumBars = 2 * kStages + 2 * kCodeStages + 5;
+  static constexpr int kWOffset = kCodeOffset + kCodeStages * kCodeBytes;  // (a multiple of 1024)
+  static constexpr int kBarOffset = kWOffset + kWBufs * kWTileBytes;
+  // full[S], empty[S], cfull[C], cempty[C], tfull[2], tempty[2], drain, wfull[2], wdone[2]
+  static constexpr int kNumBars = 2 * kStages + 2 * kCodeStages + 5 + 2 * kWBufs;
   static constexpr int kMiscOffset = kBarOffset + kNumBars * 8;
   static constexpr int kTablesOffset = kMiscOffset + 16;
   static constexpr int kTotal = kTablesOffset + static_cast<int>(sizeof(Nf4Tables));
@@ -134,6 +143,7 @@ struct SmemLayout {
   static_assert(kDynamicBytes <= 232448, "exceeds the 227 KiB shared memory of one CTA");
   static_assert(kBM * 32 <= kCodeBytes && kBNL * 32 <= kCodeBytes, "code tile too large");
   static_assert(!TWO || BN == 256, "pairs run 256-wide tiles");
+  static_assert(!REQ || (MH == 1 && !TWO && !NF4), "the merge runs single 128-row tiles fed by TMA");
 };
 
 // Shared-memory matrix descriptor (tcgen05), 128-byte swizzle.
@@ -333,10 +343,10 @@ __device__ __forceinline__ void deq_store(const DeqGeom &g, const DeqTask &task,
 // ---------------------------------------------------------------------------
 // The kernel
 // ---------------------------------------------------------------------------
-template <int BN, int MH, bool TWO, bool NF4>
+template <int BN, int MH, bool TWO, bool NF4, bool REQ>
 __global__ void __launch_bounds__(kNumThreads, 1)
 loqt_gemm_kernel(const __grid_constant__ TensorMaps maps, const GemmParams p) {
-  using L = SmemLayout<BN, MH, TWO, NF4>;
+  using L = SmemLayout<BN, MH, TWO, NF4, REQ>;
   constexpr int kStages = L::kStages;
   constexpr int kBM = L::kBM;
   constexpr int kBNL = L::kBNL;
@@ -355,6 +365,8 @@ loqt_gemm_kernel(const __grid_constant__ TensorMaps maps, const GemmParams p) {
   auto tfull_bar = [&](int a) { return bar0 + 8u * (2 * kStages + 2 * kCodeStages + a); };
   auto tempty_bar = [&](int a) { return bar0 + 8u * (2 * kStages + 2 * kCodeStages + 2 + a); };
   const uint32_t drain_bar = bar0 + 8u * (2 * kStages + 2 * kCodeStages + 4);
+  auto wfull_bar = [&](int b) { return bar0 + 8u * (2 * kStages + 2 * kCodeStages + 5 + b); };
+  auto wdone_bar = [&](int b) { return bar0 + 8u * (2 * kStages + 2 * kCodeStages + 7 + b); };
   volatile uint32_t *misc = reinterpret_cast<volatile uint32_t *>(smem_gen + L::kMiscOffset);
   volatile uint32_t *tmem_slot = misc;       // written by tcgen05.alloc
   volatile uint32_t *abort_flag = misc + 1;  // raised by any role whose wait expired
@@ -367,14 +379,12 @@ loqt_gemm_kernel(const __grid_constant__ TensorMaps maps, const GemmParams p) {
   // MMA thread waits on).
   const uint32_t rank = TWO ? ptx::cluster_ctarank() : 0u;
   const bool leader = (rank == 0);
-  // The requantising epilogue of the merge is the heaviest one, so dequant warps
-  // that have nothing to stage join it in groups of four (one warp per TMEM lane
-  // quarter: warps 6-9 and 10-13 cover quarters 2,3,0,1).  With both operands
-  // arriving by TMA both groups help; with an NF4 A operand (128-row tiles) one
-  // group stages and the other helps.  The 64-column blocks of a tile are dealt
-  // to the epilogue groups round-robin, continuing across tiles.
-  const bool requant_helpers = (MH == 1) && (p.epi == EPI_REQUANT);
-  const int epi_groups = requant_helpers ? (NF4 ? 2 : 3) : 1;
+  // The requantising epilogue of the merge is the heaviest one, and its kernel has
+  // nothing to dequantise in the main loop, so the dequant warps join it as two
+  // more groups of four (one warp per TMEM lane quarter: warps 6-9 and 10-13
+  // cover quarters 2,3,0,1).  The 64-column blocks of a tile are dealt to the
+  // three groups round-robin, continuing across tiles.
+  constexpr int epi_groups = REQ ? 3 : 1;
   // The dequant warps work as two groups of four that take the K stages of a
   // tile in turn, so that one group's barrier, fence and bookkeeping time is
   // covered by the other's table lookups (the dequantisation is bound by the
@@ -384,7 +394,7 @@ loqt_gemm_kernel(const __grid_constant__ TensorMaps maps, const GemmParams p) {
   // loop of single-accumulator kernels, was measured 5 % slower: with three stages
   // in the ring a third group only waits for a slot.)
   constexpr int kGroupWarps = kDeqWarps / 2;
-  const int deq_groups = !NF4 ? 0 : (requant_helpers ? 1 : 2);
+  constexpr int deq_groups = NF4 ? 2 : 0;
   const int deq_grp = (warp - kDeqWarp0) / kGroupWarps;
   constexpr uint32_t kTmemCols = 2 * BN;
 
@@ -404,10 +414,16 @@ loqt_gemm_kernel(const __grid_constant__ TensorMaps maps, const GemmParams p) {
       ptx::mbar_init(tempty_bar(a), 4 * epi_groups * (TWO ? 2 : 1));
     }
     ptx::mbar_init(drain_bar, 1);
+    if (REQ) {
+      for (int b = 0; b < 2; ++b) {
+        ptx::mbar_init(wfull_bar(b), 1);                // the mover (with the tile's bytes)
+        ptx::mbar_init(wdone_bar(b), 4 * epi_groups);   // every epilogue warp, once per tile
+      }
+    }
     *abort_flag = 0;
     ptx::fence_barrier_init();
   }
-  if (p.epi == EPI_REQUANT) nf4_tables_init(tables, threadIdx.x);
+  if (REQ) nf4_tables_init(tables, threadIdx.x);
   if (warp == 1) {
     if (TWO) {
       ptx::tmem_alloc_pair(smem_u32(const_cast<uint32_t *>(tmem_slot)), kTmemCols);
@@ -645,6 +661,43 @@ loqt_gemm_kernel(const __grid_constant__ TensorMaps maps, const GemmParams p) {
   }
   // =========================================================== code producer
   else if (warp == kCodeWarp) {
+    if (lane == 0 && REQ) {
+      // Mover of the merge: brings the packed codes of each output tile's W_q blocks
+      // into shared memory ahead of the tile's epilogue (one bulk copy of whole
+      // 128-byte rows instead of a 32-byte access per thread and block) and writes
+      // the requantised codes back once every epilogue warp is done with the tile.
+      // Buffer b = tile & 1.  Before a buffer is loaded again, the bulk store that
+      // last read it has finished reading.
+      ptx::prefetch_tensormap(&maps.wq);
+      bool ok = true;
+      uint32_t tile = 0;
+      int pm = 0, pn = 0;  // the previous tile's block coordinates
+      for (int u = blockIdx.x; ok && u < sched.units; u += gridDim.x, ++tile) {
+        int m_blk, n_blk, split, kb_lo, kb_hi;
+        sched.unit(u, m_blk, n_blk, split, kb_lo, kb_hi);
+        const uint32_t b = tile & 1u;
+        ptx::bulk_wait_group_read<0>();
+        ptx::mbar_arrive_expect_tx(wfull_bar(b), L::kWTileBytes);
+        ptx::tma_load_2d(smem_base + L::kWOffset + b * L::kWTileBytes, &maps.wq, wfull_bar(b), n_blk * (BN / 2), m_blk * kHM);
+        if (tile > 0) {
+          const uint32_t pb = (tile - 1) & 1u;
+          if (!(ok = ptx::mbar_wait(wdone_bar(pb), ((tile - 1) >> 1) & 1u, abort_flag, p.status))) break;
+          ptx::tma_store_2d(&maps.wq, smem_base + L::kWOffset + pb * L::kWTileBytes, pn * (BN / 2), pm * kHM);
+          ptx::bulk_commit_group();
+        }
+        pm = m_blk;
+        pn = n_blk;
+      }
+      if (ok && tile > 0) {
+        const uint32_t pb = (tile - 1) & 1u;
+        if (ptx::mbar_wait(wdone_bar(pb), ((tile - 1) >> 1) & 1u, abort_flag, p.status)) {
+          ptx::tma_store_2d(&maps.wq, smem_base + L::kWOffset + pb * L::kWTileBytes, pn * (BN / 2), pm * kHM);
+          ptx::bulk_commit_group();
+        }
+      }
+      // every store has left shared memory and reached global memory before the CTA ends
+      ptx::bulk_wait_group<0>();
+    }
     if (lane == 0 && NF4) {
       // A cursor over the same sequence of stages as the operand producer's; the
       // ring's depth bounds how far the codes run ahead.
@@ -721,39 +774,59 @@ loqt_gemm_kernel(const __grid_constant__ TensorMaps maps, const GemmParams p) {
         const bool row_ok = row < p.M;
         const uint32_t t_row = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + acc * (MH * BN) + h * BN;
 
-        if (p.epi == EPI_REQUANT) {
-          // One NF4 block of W_q per 64 accumulator columns of this thread's row.
+        if constexpr (REQ) {
+          // One NF4 block of W_q per 64 accumulator columns of this thread's row.  The
+          // tile's old codes wait in shared memory (rows of BN / 2 bytes, TMA-swizzled:
+          // 16-byte chunk ^= row & 7 for 128-byte rows, (row >> 1) & 3 for 64-byte rows);
+          // the new codes replace them there and the mover stores the tile.
+          const uint32_t wb = tile & 1u;
+          if (!(ok = ptx::mbar_wait(wfull_bar(wb), (tile >> 1) & 1u, abort_flag, p.status))) break;
+          const int row_t = q * 32 + lane;  // row inside the tile
+          const uint32_t w_row = smem_base + L::kWOffset + wb * L::kWTileBytes + static_cast<uint32_t>(row_t) * (BN / 2);
+          const uint32_t w_key = (BN == 256) ? static_cast<uint32_t>(row_t & 7) : static_cast<uint32_t>((row_t >> 1) & 3);
 #pragma unroll 1
           for (int jb = 0; jb < BN / 64; ++jb) {
-            if (static_cast<int>((tile * (BN / 64) + jb) % epi_groups) != grp) continue;
+            const uint32_t seq = tile * (BN / 64) + jb;  // position in this CTA's sequence of blocks
+            if (static_cast<int>(seq % epi_groups) != grp) continue;
+            const int c0 = n_base + jb * 64;
+            const bool live = row_ok && c0 < p.wq_ld;
+            float *mp = p.wq_absmax + static_cast<int64_t>(row) * (p.wq_ld >> 6) + (c0 >> 6);
+            float Mold = 0.0f;
+            if (live) Mold = *mp;  // in flight while the accumulator is read
+            const uint32_t a0 = w_row + (((2u * jb) ^ w_key) << 4), a1 = w_row + (((2u * jb + 1u) ^ w_key) << 4);
+            const uint4 ca = ld_shared_v4(a0), cb = ld_shared_v4(a1);
             uint32_t d0[32], d1[32];
             ptx::tmem_ld32(t_row + jb * 64, d0);
             ptx::tmem_ld32(t_row + jb * 64 + 32, d1);
             ptx::tmem_ld_wait();
-            const int c0 = n_base + jb * 64;
-            if (row_ok && c0 < p.wq_ld) {
-              uint4 *cp = reinterpret_cast<uint4 *>(p.wq_codes + static_cast<int64_t>(row) * (p.wq_ld >> 1) + (c0 >> 1));
-              float *mp = p.wq_absmax + static_cast<int64_t>(row) * (p.wq_ld >> 6) + (c0 >> 6);
-              const uint4 ca = *cp, cb = *(cp + 1);
-              const float Mold = *mp;
+            if (live) {
               const uint32_t w[8] = {ca.x, ca.y, ca.z, ca.w, cb.x, cb.y, cb.z, cb.w};
-              float v[64];
-              float Mnew = 0.0f;
+              // v = deq32(old) + alpha * delta, two elements per packed instruction; four
+              // running maxima keep the dependent chain of the block maximum short.
+              float2 v[32];
+              float mx[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+              const float2 a2 = make_float2(p.alpha, p.alpha), m2 = make_float2(Mold, Mold);
 #pragma unroll
-              for (int e = 0; e < 64; ++e) {
-                const float deq = Mold * tables.level[(w[e >> 3] >> (4 * (e & 7))) & 15u];
-                const float delta = __uint_as_float(e < 32 ? d0[e] : d1[e - 32]);
-                v[e] = fmaf(p.alpha, delta, deq);
-                Mnew = fmaxf(Mnew, fabsf(v[e]));
+              for (int e = 0; e < 32; ++e) {
+                const uint32_t word = w[e >> 2];
+                const float2 lv = make_float2(tables.level[(word >> (8 * (e & 3))) & 15u],
+                                              tables.level[(word >> (8 * (e & 3) + 4)) & 15u]);
+                const float2 delta = make_float2(__uint_as_float(e < 16 ? d0[2 * e] : d1[2 * e - 32]),
+                                                 __uint_as_float(e < 16 ? d0[2 * e + 1] : d1[2 * e - 31]));
+                v[e] = __ffma2_rn(a2, delta, __fmul2_rn(m2, lv));
+                mx[e & 3] = fmaxf(mx[e & 3], fmaxf(fabsf(v[e].x), fabsf(v[e].y)));
               }
+              const float Mnew = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
               uint32_t o[8];
               const Nf4Divisor dv = nf4_divisor(Mnew);
               auto quantise_block = [&](auto exact) {
 #pragma unroll
                 for (int g = 0; g < 8; ++g) {
-                  const float vv[8] = {v[8 * g], v[8 * g + 1], v[8 * g + 2], v[8 * g + 3],
-                                       v[8 * g + 4], v[8 * g + 5], v[8 * g + 6], v[8 * g + 7]};
-                  o[g] = nf4_quantize8<decltype(exact)::value>(tables, vv, dv);
+                  uint32_t word = 0;
+#pragma unroll
+                  for (int h2 = 0; h2 < 4; ++h2)
+                    word |= nf4_code2(tables, nf4_normalise2<decltype(exact)::value>(dv, v[4 * g + h2])) << (8 * h2);
+                  o[g] = word;
                 }
               };
               if (!(Mnew > 0.0f)) {
@@ -764,12 +837,16 @@ loqt_gemm_kernel(const __grid_constant__ TensorMaps maps, const GemmParams p) {
               } else {
                 quantise_block(std::false_type{});
               }
-              *cp = make_uint4(o[0], o[1], o[2], o[3]);
-              *(cp + 1) = make_uint4(o[4], o[5], o[6], o[7]);
+              st_shared_v4(a0, make_uint4(o[0], o[1], o[2], o[3]));
+              st_shared_v4(a1, make_uint4(o[4], o[5], o[6], o[7]));
               *mp = Mnew;
             }
             __syncwarp();
           }
+          // this warp's blocks of the tile are in place: visible to the bulk store, then signalled
+          ptx::fence_proxy_async_smem();
+          __syncwarp();
+          if (lane == 0) ptx::mbar_arrive(wdone_bar(wb));
         } else {
 #pragma unroll 1
           for (int cb = 0; cb < BN / 32; ++cb) {

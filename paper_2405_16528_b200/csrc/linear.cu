@@ -106,9 +106,9 @@ static int variant_index(int bn, int mh, bool two, bool nf4) {
   return (bn == 256 ? 1 : 0) | (mh == 2 ? 2 : 0) | (two ? 4 : 0) | (nf4 ? 8 : 0);
 }
 
-template <int BN, int MH, bool TWO, bool NF4>
+template <int BN, int MH, bool TWO, bool NF4, bool REQ = false>
 static loqt_status launch_cfg(const GemmCall &c, cudaStream_t stream) {
-  using L = SmemLayout<BN, MH, TWO, NF4>;
+  using L = SmemLayout<BN, MH, TWO, NF4, REQ>;
   constexpr int BNL = L::kBNL;  // B rows one CTA stages
   TensorMaps maps;
   memset(&maps, 0, sizeof(maps));
@@ -131,7 +131,13 @@ static loqt_status launch_cfg(const GemmCall &c, cudaStream_t stream) {
         return LOQT_ERR_CUDA;
     }
   }
-  auto kernel = loqt_gemm_kernel<BN, MH, TWO, NF4>;
+  if (REQ) {
+    // W_q's packed codes, one box = the 128 rows x BN columns an output tile updates
+    const Nf4Src wq{c.p.wq_codes, c.p.wq_absmax, c.p.M, c.p.N, c.p.wq_ld};
+    if (!make_code_map(&maps.wq, wq, BN / 2, kHM, BN == 256 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B))
+      return LOQT_ERR_CUDA;
+  }
+  auto kernel = loqt_gemm_kernel<BN, MH, TWO, NF4, REQ>;
   if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kDynamicBytes) != cudaSuccess)
     return LOQT_ERR_CUDA;
   int mt = (c.p.M + L::kBM - 1) / L::kBM;
@@ -234,6 +240,11 @@ static TileCfg pick_tile(const GemmCall &c) {
 
 template <bool NF4>
 static loqt_status launch_tile(const GemmCall &c, const TileCfg &t, cudaStream_t stream) {
+  if (c.p.epi == EPI_REQUANT) {
+    // the merge kernel: single 128-row tiles, both operands by TMA
+    if (NF4 || t.two || t.mh != 1) return LOQT_ERR_UNSUPPORTED;
+    return t.bn == 256 ? launch_cfg<256, 1, false, false, true>(c, stream) : launch_cfg<128, 1, false, false, true>(c, stream);
+  }
   if (t.two) return t.mh == 2 ? launch_cfg<256, 2, true, NF4>(c, stream) : launch_cfg<256, 1, true, NF4>(c, stream);
   if (t.bn == 256) return t.mh == 2 ? launch_cfg<256, 2, false, NF4>(c, stream) : launch_cfg<256, 1, false, NF4>(c, stream);
   return t.mh == 2 ? launch_cfg<128, 2, false, NF4>(c, stream) : launch_cfg<128, 1, false, NF4>(c, stream);
