@@ -59,7 +59,6 @@ enum : int {
   EPI_BF16 = 0,     // out bf16 = alpha * D
   EPI_F32 = 1,      // out fp32 = (addend, or out when accumulating, or 0) + alpha * D   (splits == 1)
   EPI_PARTIAL = 2,  // partial[split] fp32 = D                        (splits > 1)
-  EPI_REQUANT = 3,  // W_q <- q_NF4(deq32(W_q) + alpha * D), in place (merge)
 };
 
 struct Nf4Src {
@@ -87,21 +86,16 @@ struct GemmParams {
   int accumulate;
   const float *addend;  // EPI_F32: out = addend + alpha * D when set (16-byte aligned rows)
   int64_t ld_addend;
-  uint8_t *wq_codes;  // EPI_REQUANT: W_q updated in place ([M][wq_ld/2], [M][wq_ld/64])
-  float *wq_absmax;
-  int wq_ld;
   uint32_t *status;  // device status word
   int has_nf4;       // any NF4 operand in any segment
 };
 
-// a/b: bf16 operands; ca/cb: packed NF4 codes viewed as a byte matrix; wq: the
-// packed codes of the matrix a merge updates, one output tile per box.
+// a/b: bf16 operands; ca/cb: packed NF4 codes viewed as a byte matrix.
 struct TensorMaps {
   CUtensorMap a[2];
   CUtensorMap b[2];
   CUtensorMap ca[2];
   CUtensorMap cb[2];
-  CUtensorMap wq;
 };
 
 // NF4: the kernel variant that stages NF4 operands (code ring, dequant warps); the
@@ -343,10 +337,10 @@ __device__ __forceinline__ void deq_store(const DeqGeom &g, const DeqTask &task,
 // ---------------------------------------------------------------------------
 // The kernel
 // ---------------------------------------------------------------------------
-template <int BN, int MH, bool TWO, bool NF4, bool REQ>
+template <int BN, int MH, bool TWO, bool NF4>
 __global__ void __launch_bounds__(kNumThreads, 1)
 loqt_gemm_kernel(const __grid_constant__ TensorMaps maps, const GemmParams p) {
-  using L = SmemLayout<BN, MH, TWO, NF4, REQ>;
+  using L = SmemLayout<BN, MH, TWO, NF4>;
   constexpr int kStages = L::kStages;
   constexpr int kBM = L::kBM;
   constexpr int kBNL = L::kBNL;
@@ -365,12 +359,9 @@ loqt_gemm_kernel(const __grid_constant__ TensorMaps maps, const GemmParams p) {
   auto tfull_bar = [&](int a) { return bar0 + 8u * (2 * kStages + 2 * kCodeStages + a); };
   auto tempty_bar = [&](int a) { return bar0 + 8u * (2 * kStages + 2 * kCodeStages + 2 + a); };
   const uint32_t drain_bar = bar0 + 8u * (2 * kStages + 2 * kCodeStages + 4);
-  auto wfull_bar = [&](int b) { return bar0 + 8u * (2 * kStages + 2 * kCodeStages + 5 + b); };
-  auto wdone_bar = [&](int b) { return bar0 + 8u * (2 * kStages + 2 * kCodeStages + 7 + b); };
   volatile uint32_t *misc = reinterpret_cast<volatile uint32_t *>(smem_gen + L::kMiscOffset);
   volatile uint32_t *tmem_slot = misc;       // written by tcgen05.alloc
   volatile uint32_t *abort_flag = misc + 1;  // raised by any role whose wait expired
-  Nf4Tables &tables = *reinterpret_cast<Nf4Tables *>(smem_gen + L::kTablesOffset);
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
@@ -379,12 +370,6 @@ loqt_gemm_kernel(const __grid_constant__ TensorMaps maps, const GemmParams p) {
   // MMA thread waits on).
   const uint32_t rank = TWO ? ptx::cluster_ctarank() : 0u;
   const bool leader = (rank == 0);
-  // The requantising epilogue of the merge is the heaviest one, and its kernel has
-  // nothing to dequantise in the main loop, so the dequant warps join it as two
-  // more groups of four (one warp per TMEM lane quarter: warps 6-9 and 10-13
-  // cover quarters 2,3,0,1).  The 64-column blocks of a tile are dealt to the
-  // three groups round-robin, continuing across tiles.
-  constexpr int epi_groups = REQ ? 3 : 1;
   // The dequant warps work as two groups of four that take the K stages of a
   // tile in turn, so that one group's barrier, fence and bookkeeping time is
   // covered by the other's table lookups (the dequantisation is bound by the
@@ -411,19 +396,12 @@ loqt_gemm_kernel(const __grid_constant__ TensorMaps maps, const GemmParams p) {
     }
     for (int a = 0; a < 2; ++a) {
       ptx::mbar_init(tfull_bar(a), 1);
-      ptx::mbar_init(tempty_bar(a), 4 * epi_groups * (TWO ? 2 : 1));
+      ptx::mbar_init(tempty_bar(a), 4 * (TWO ? 2 : 1));  // the four epilogue warps (of each CTA of a pair)
     }
     ptx::mbar_init(drain_bar, 1);
-    if (REQ) {
-      for (int b = 0; b < 2; ++b) {
-        ptx::mbar_init(wfull_bar(b), 1);                // the mover (with the tile's bytes)
-        ptx::mbar_init(wdone_bar(b), 4 * epi_groups);   // every epilogue warp, once per tile
-      }
-    }
     *abort_flag = 0;
     ptx::fence_barrier_init();
   }
-  if (REQ) nf4_tables_init(tables, threadIdx.x);
   if (warp == 1) {
     if (TWO) {
       ptx::tmem_alloc_pair(smem_u32(const_cast<uint32_t *>(tmem_slot)), kTmemCols);
@@ -661,43 +639,6 @@ loqt_gemm_kernel(const __grid_constant__ TensorMaps maps, const GemmParams p) {
   }
   // =========================================================== code producer
   else if (warp == kCodeWarp) {
-    if (lane == 0 && REQ) {
-      // Mover of the merge: brings the packed codes of each output tile's W_q blocks
-      // into shared memory ahead of the tile's epilogue (one bulk copy of whole
-      // 128-byte rows instead of a 32-byte access per thread and block) and writes
-      // the requantised codes back once every epilogue warp is done with the tile.
-      // Buffer b = tile & 1.  Before a buffer is loaded again, the bulk store that
-      // last read it has finished reading.
-      ptx::prefetch_tensormap(&maps.wq);
-      bool ok = true;
-      uint32_t tile = 0;
-      int pm = 0, pn = 0;  // the previous tile's block coordinates
-      for (int u = blockIdx.x; ok && u < sched.units; u += gridDim.x, ++tile) {
-        int m_blk, n_blk, split, kb_lo, kb_hi;
-        sched.unit(u, m_blk, n_blk, split, kb_lo, kb_hi);
-        const uint32_t b = tile & 1u;
-        ptx::bulk_wait_group_read<0>();
-        ptx::mbar_arrive_expect_tx(wfull_bar(b), L::kWTileBytes);
-        ptx::tma_load_2d(smem_base + L::kWOffset + b * L::kWTileBytes, &maps.wq, wfull_bar(b), n_blk * (BN / 2), m_blk * kHM);
-        if (tile > 0) {
-          const uint32_t pb = (tile - 1) & 1u;
-          if (!(ok = ptx::mbar_wait(wdone_bar(pb), ((tile - 1) >> 1) & 1u, abort_flag, p.status))) break;
-          ptx::tma_store_2d(&maps.wq, smem_base + L::kWOffset + pb * L::kWTileBytes, pn * (BN / 2), pm * kHM);
-          ptx::bulk_commit_group();
-        }
-        pm = m_blk;
-        pn = n_blk;
-      }
-      if (ok && tile > 0) {
-        const uint32_t pb = (tile - 1) & 1u;
-        if (ptx::mbar_wait(wdone_bar(pb), ((tile - 1) >> 1) & 1u, abort_flag, p.status)) {
-          ptx::tma_store_2d(&maps.wq, smem_base + L::kWOffset + pb * L::kWTileBytes, pn * (BN / 2), pm * kHM);
-          ptx::bulk_commit_group();
-        }
-      }
-      // every store has left shared memory and reached global memory before the CTA ends
-      ptx::bulk_wait_group<0>();
-    }
     if (lane == 0 && NF4) {
       // A cursor over the same sequence of stages as the operand producer's; the
       // ring's depth bounds how far the codes run ahead.
@@ -755,9 +696,8 @@ loqt_gemm_kernel(const __grid_constant__ TensorMaps maps, const GemmParams p) {
     }
   }
   // =========================================================== epilogue
-  else if (warp < kDeqWarp0 || warp >= kDeqWarp0 + kGroupWarps * (3 - epi_groups)) {
+  else if (warp < kDeqWarp0) {
     const int q = warp & 3;  // TMEM lane quarter this warp may access
-    const int grp = warp < kDeqWarp0 ? 0 : epi_groups - 1 - (kDeqWarp0 + kDeqWarps - 1 - warp) / kGroupWarps;
     uint32_t tile = 0;
     bool ok = true;
     for (int u = blockIdx.x; ok && u < sched.units; u += gridDim.x, ++tile) {
@@ -773,81 +713,7 @@ loqt_gemm_kernel(const __grid_constant__ TensorMaps maps, const GemmParams p) {
         const int row = m_blk * kBM + h * kHM + q * 32 + lane;
         const bool row_ok = row < p.M;
         const uint32_t t_row = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + acc * (MH * BN) + h * BN;
-
-        if constexpr (REQ) {
-          // One NF4 block of W_q per 64 accumulator columns of this thread's row.  The
-          // tile's old codes wait in shared memory (rows of BN / 2 bytes, TMA-swizzled:
-          // 16-byte chunk ^= row & 7 for 128-byte rows, (row >> 1) & 3 for 64-byte rows);
-          // the new codes replace them there and the mover stores the tile.
-          const uint32_t wb = tile & 1u;
-          if (!(ok = ptx::mbar_wait(wfull_bar(wb), (tile >> 1) & 1u, abort_flag, p.status))) break;
-          const int row_t = q * 32 + lane;  // row inside the tile
-          const uint32_t w_row = smem_base + L::kWOffset + wb * L::kWTileBytes + static_cast<uint32_t>(row_t) * (BN / 2);
-          const uint32_t w_key = (BN == 256) ? static_cast<uint32_t>(row_t & 7) : static_cast<uint32_t>((row_t >> 1) & 3);
-#pragma unroll 1
-          for (int jb = 0; jb < BN / 64; ++jb) {
-            const uint32_t seq = tile * (BN / 64) + jb;  // position in this CTA's sequence of blocks
-            if (static_cast<int>(seq % epi_groups) != grp) continue;
-            const int c0 = n_base + jb * 64;
-            const bool live = row_ok && c0 < p.wq_ld;
-            float *mp = p.wq_absmax + static_cast<int64_t>(row) * (p.wq_ld >> 6) + (c0 >> 6);
-            float Mold = 0.0f;
-            if (live) Mold = *mp;  // in flight while the accumulator is read
-            const uint32_t a0 = w_row + (((2u * jb) ^ w_key) << 4), a1 = w_row + (((2u * jb + 1u) ^ w_key) << 4);
-            const uint4 ca = ld_shared_v4(a0), cb = ld_shared_v4(a1);
-            uint32_t d0[32], d1[32];
-            ptx::tmem_ld32(t_row + jb * 64, d0);
-            ptx::tmem_ld32(t_row + jb * 64 + 32, d1);
-            ptx::tmem_ld_wait();
-            if (live) {
-              const uint32_t w[8] = {ca.x, ca.y, ca.z, ca.w, cb.x, cb.y, cb.z, cb.w};
-              // v = deq32(old) + alpha * delta, two elements per packed instruction; four
-              // running maxima keep the dependent chain of the block maximum short.
-              float2 v[32];
-              float mx[4] = {0.0f, 0.0f, 0.0f, 0.0f};
-              const float2 a2 = make_float2(p.alpha, p.alpha), m2 = make_float2(Mold, Mold);
-#pragma unroll
-              for (int e = 0; e < 32; ++e) {
-                const uint32_t word = w[e >> 2];
-                const float2 lv = make_float2(tables.level[(word >> (8 * (e & 3))) & 15u],
-                                              tables.level[(word >> (8 * (e & 3) + 4)) & 15u]);
-                const float2 delta = make_float2(__uint_as_float(e < 16 ? d0[2 * e] : d1[2 * e - 32]),
-                                                 __uint_as_float(e < 16 ? d0[2 * e + 1] : d1[2 * e - 31]));
-                v[e] = __ffma2_rn(a2, delta, __fmul2_rn(m2, lv));
-                mx[e & 3] = fmaxf(mx[e & 3], fmaxf(fabsf(v[e].x), fabsf(v[e].y)));
-              }
-              const float Mnew = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
-              uint32_t o[8];
-              const Nf4Divisor dv = nf4_divisor(Mnew);
-              auto quantise_block = [&](auto exact) {
-#pragma unroll
-                for (int g = 0; g < 8; ++g) {
-                  uint32_t word = 0;
-#pragma unroll
-                  for (int h2 = 0; h2 < 4; ++h2)
-                    word |= nf4_code2(tables, nf4_normalise2<decltype(exact)::value>(dv, v[4 * g + h2])) << (8 * h2);
-                  o[g] = word;
-                }
-              };
-              if (!(Mnew > 0.0f)) {
-#pragma unroll
-                for (int g = 0; g < 8; ++g) o[g] = kZeroWord;
-              } else if (dv.exact) {
-                quantise_block(std::true_type{});
-              } else {
-                quantise_block(std::false_type{});
-              }
-              st_shared_v4(a0, make_uint4(o[0], o[1], o[2], o[3]));
-              st_shared_v4(a1, make_uint4(o[4], o[5], o[6], o[7]));
-              *mp = Mnew;
-            }
-            __syncwarp();
-          }
-          // this warp's blocks of the tile are in place: visible to the bulk store, then signalled
-          ptx::fence_proxy_async_smem();
-          __syncwarp();
-          if (lane == 0) ptx::mbar_arrive(wdone_bar(wb));
-        } else {
+        {
 #pragma unroll 1
           for (int cb = 0; cb < BN / 32; ++cb) {
             uint32_t d[32];

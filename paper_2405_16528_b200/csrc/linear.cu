@@ -3,7 +3,7 @@
 #include <atomic>
 #include <mutex>
 
-#include "gemm.cuh"
+#include "merge.cuh"
 
 namespace loqt {
 
@@ -106,9 +106,9 @@ static int variant_index(int bn, int mh, bool two, bool nf4) {
   return (bn == 256 ? 1 : 0) | (mh == 2 ? 2 : 0) | (two ? 4 : 0) | (nf4 ? 8 : 0);
 }
 
-template <int BN, int MH, bool TWO, bool NF4, bool REQ = false>
+template <int BN, int MH, bool TWO, bool NF4>
 static loqt_status launch_cfg(const GemmCall &c, cudaStream_t stream) {
-  using L = SmemLayout<BN, MH, TWO, NF4, REQ>;
+  using L = SmemLayout<BN, MH, TWO, NF4>;
   constexpr int BNL = L::kBNL;  // B rows one CTA stages
   TensorMaps maps;
   memset(&maps, 0, sizeof(maps));
@@ -131,13 +131,7 @@ static loqt_status launch_cfg(const GemmCall &c, cudaStream_t stream) {
         return LOQT_ERR_CUDA;
     }
   }
-  if (REQ) {
-    // W_q's packed codes, one box = the 128 rows x BN columns an output tile updates
-    const Nf4Src wq{c.p.wq_codes, c.p.wq_absmax, c.p.M, c.p.N, c.p.wq_ld};
-    if (!make_code_map(&maps.wq, wq, BN / 2, kHM, BN == 256 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B))
-      return LOQT_ERR_CUDA;
-  }
-  auto kernel = loqt_gemm_kernel<BN, MH, TWO, NF4, REQ>;
+  auto kernel = loqt_gemm_kernel<BN, MH, TWO, NF4>;
   if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kDynamicBytes) != cudaSuccess)
     return LOQT_ERR_CUDA;
   int mt = (c.p.M + L::kBM - 1) / L::kBM;
@@ -205,7 +199,7 @@ static TileCfg pick_tile(const GemmCall &c) {
   TileCfg best = {256, 1, false};
   double best_t = 1e300;
   for (TileCfg t : cands) {
-    if (t.mh == 2 && (c.p.M <= kHM || c.p.epi == EPI_REQUANT)) continue;  // the merge epilogue wants 128-row tiles
+    if (t.mh == 2 && c.p.M <= kHM) continue;
     if (t.bn == 256 && c.p.N <= 128) continue;
     const int units = ((c.p.M + t.mh * kHM - 1) / (t.mh * kHM)) * ((c.p.N + t.bn - 1) / t.bn) * c.p.splits;
     const double waves = (units + sms - 1) / sms;
@@ -220,19 +214,16 @@ static TileCfg pick_tile(const GemmCall &c) {
     }
   }
   // The costs above are those of single CTAs; a 256-wide choice then runs as pairs
-  // where it can (measured faster for every product but the merge, whose epilogue
-  // - not its main loop - sets the pace).
-  best.two = pair_ok(c, best.bn, best.mh) && c.p.epi != EPI_REQUANT;
+  // where it can (measured faster).
+  best.two = pair_ok(c, best.bn, best.mh);
   // A tile forced by loqt_set_tile_override() replaces the choice wherever the
   // kernel supports it for this product: pairs need 256-wide tiles and no split-K
-  // (an odd number of M tiles is rounded up by one empty tile), and the merge
-  // epilogue runs on single 128-row tiles only.
+  // (an odd number of M tiles is rounded up by one empty tile).
   const int fbn = g_force_bn.load(std::memory_order_relaxed);
   if (fbn != 0) {
     const int fmh = g_force_mh.load(std::memory_order_relaxed);
     const bool fpair = g_force_pair.load(std::memory_order_relaxed) != 0;
-    const bool merge = c.p.epi == EPI_REQUANT;
-    const bool ok = !(merge && (fmh == 2 || fpair)) && !(fpair && (fbn != 256 || c.p.splits != 1 || !kUsePairs));
+    const bool ok = !(fpair && (fbn != 256 || c.p.splits != 1 || !kUsePairs));
     if (ok) best = TileCfg{fbn, fmh, fpair};
   }
   return best;
@@ -240,11 +231,7 @@ static TileCfg pick_tile(const GemmCall &c) {
 
 template <bool NF4>
 static loqt_status launch_tile(const GemmCall &c, const TileCfg &t, cudaStream_t stream) {
-  if (c.p.epi == EPI_REQUANT) {
-    // the merge kernel: single 128-row tiles, both operands by TMA
-    if (NF4 || t.two || t.mh != 1) return LOQT_ERR_UNSUPPORTED;
-    return t.bn == 256 ? launch_cfg<256, 1, false, false, true>(c, stream) : launch_cfg<128, 1, false, false, true>(c, stream);
-  }
+
   if (t.two) return t.mh == 2 ? launch_cfg<256, 2, true, NF4>(c, stream) : launch_cfg<256, 1, true, NF4>(c, stream);
   if (t.bn == 256) return t.mh == 2 ? launch_cfg<256, 2, false, NF4>(c, stream) : launch_cfg<256, 1, false, NF4>(c, stream);
   return t.mh == 2 ? launch_cfg<128, 2, false, NF4>(c, stream) : launch_cfg<128, 1, false, NF4>(c, stream);
@@ -459,7 +446,9 @@ extern "C" loqt_status loqt_linear_bwd(loqt_nf4_mat Wq, loqt_nf4_mat Pq, const v
   return gemm_tn_f32(v, ldv, x, ldx, r, in, T, dB, lddb, accumulate_dB, partial, status, stm);
 }
 
-// The merge of one matrix, in two launches.  `phat` is scratch for deq(P_q).
+// ---------------------------------------------------------------------------
+// Merge: staging of the dequantised factor, then the batched merge kernel
+// ---------------------------------------------------------------------------
 static size_t merge_scratch_bytes(const loqt_nf4_mat &Pq) {
   return align256(static_cast<size_t>(Pq.rows) * ld_lowrank(Pq.cols) * 2);
 }
@@ -469,29 +458,116 @@ static loqt_status merge_stage(const loqt_nf4_mat &Pq, void *phat, cudaStream_t 
   return loqt_nf4_dequantize(Pq, phat, ld_lowrank(Pq.cols), 1, stm);
 }
 
-// Delta = P-hat B  (out x in; K = r, both operands by TMA), requantised in the epilogue.
-static loqt_status merge_product(const loqt_nf4_mat &Wq, const loqt_nf4_mat &Pq, const void *phat, const void *B,
-                                 int64_t ldb, float s, uint32_t *status, cudaStream_t stm) {
-  GemmCall c{};
-  c.p.M = Wq.rows; c.p.N = Wq.cols; c.p.num_segs = 1;
-  c.p.seg[0].K = Pq.cols; c.p.seg[0].a_kind = OP_TMA_K; c.p.seg[0].b_kind = OP_TMA_MN;
-  c.a[0] = {phat, ld_lowrank(Pq.cols)}; c.b[0] = {B, ldb};
-  c.p.splits = 1;
-  c.p.epi = EPI_REQUANT; c.p.alpha = s; c.p.status = status;
-  c.p.wq_codes = Wq.codes; c.p.wq_absmax = Wq.absmax; c.p.wq_ld = Wq.ld;
-  return launch(c, stm);
+// One matrix of a batched merge: W_q <- q(deq32(W_q) + alpha * A Bm) with A bf16
+// [M][K] (K contiguous) and Bm bf16 [K][N] (N contiguous).
+struct MergeItem {
+  loqt_nf4_mat Wq;
+  Bf16Operand a, b;
+  int K;
+  float alpha;
+};
+
+template <int BN>
+static loqt_status launch_merge(const MergeItem *items, int n, uint32_t *status, cudaStream_t stream) {
+  using L = SmemLayout<BN, 1, false, false, true>;
+  MergeBatch mb;
+  memset(&mb, 0, sizeof(mb));
+  int tiles = 0;
+  for (int i = 0; i < n; ++i) {
+    const MergeItem &it = items[i];
+    const int M = it.Wq.rows, N = it.Wq.cols;
+    if (!make_map(&mb.a[i], it.a.ptr, it.K, M, it.a.ld, kBK, kHM)) return LOQT_ERR_CUDA;
+    if (!make_map(&mb.b[i], it.b.ptr, N, it.K, it.b.ld, 64, kBK)) return LOQT_ERR_CUDA;
+    // W_q's packed codes, one box = the 128 rows x BN columns an output tile updates
+    if (!make_code_map(&mb.wq[i], nf4_src(it.Wq), BN / 2, kHM, BN == 256 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B))
+      return LOQT_ERR_CUDA;
+    MergeProblem &pr = mb.prob[i];
+    pr.wq_absmax = it.Wq.absmax;
+    pr.M = M; pr.N = N; pr.K = it.K; pr.wq_ld = it.Wq.ld;
+    pr.tile0 = tiles;
+    pr.mt = (M + kHM - 1) / kHM;
+    pr.alpha = it.alpha;
+    tiles += pr.mt * ((N + BN - 1) / BN);
+  }
+  mb.count = n;
+  mb.tiles = tiles;
+  mb.status = status;
+  auto kernel = loqt_merge_kernel<BN>;
+  if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kDynamicBytes) != cudaSuccess)
+    return LOQT_ERR_CUDA;
+  cudaLaunchConfig_t cfg;
+  memset(&cfg, 0, sizeof(cfg));
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;  // the prologue may overlap the staging kernel's tail
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  cfg.gridDim = dim3(tiles < sm_count() ? tiles : sm_count());
+  cfg.blockDim = dim3(kNumThreads);
+  cfg.dynamicSmemBytes = L::kDynamicBytes;
+  cfg.stream = stream;
+  const cudaError_t err = cudaLaunchKernelEx(&cfg, kernel, mb);
+  count_launch();
+  g_variant_launches[variant_index(BN, 1, false, false)].fetch_add(1, std::memory_order_relaxed);
+  return (err == cudaSuccess && cudaGetLastError() == cudaSuccess) ? LOQT_OK : LOQT_ERR_CUDA;
+}
+
+// Up to kMergeBatchMax matrices in one persistent launch.  256-wide tiles unless
+// every matrix is at most 128 columns wide or 128-wide tiles are forced.
+static loqt_status merge_batch(const MergeItem *items, int n, uint32_t *status, cudaStream_t stream) {
+  if (n <= 0) return LOQT_OK;
+  if (n > kMergeBatchMax) return LOQT_ERR_INVALID_ARG;
+  bool wide = false;
+  for (int i = 0; i < n; ++i) wide = wide || items[i].Wq.cols > 128;
+  const int fbn = g_force_bn.load(std::memory_order_relaxed);
+  if (fbn != 0) wide = (fbn == 256);
+  return wide ? launch_merge<256>(items, n, status, stream) : launch_merge<128>(items, n, status, stream);
+}
+
+extern "C" loqt_status loqt_merge_requant_many(int32_t n, const loqt_nf4_mat *Wq, const loqt_nf4_mat *Pq,
+                                               const void *const *B, const int64_t *ldb, float s, void *ws,
+                                               size_t ws_bytes, void *stream) {
+  if (n < 0 || (n > 0 && (Wq == nullptr || Pq == nullptr || B == nullptr || ldb == nullptr))) return LOQT_ERR_INVALID_ARG;
+  loqt_status st;
+  size_t slot = 0;
+  for (int i = 0; i < n; ++i) {
+    if ((st = check_layer(Wq[i], Pq[i], B[i], ldb[i])) != LOQT_OK) return st;
+    const size_t need = merge_scratch_bytes(Pq[i]);
+    if (need > slot) slot = need;
+  }
+  if ((st = check_ws(ws, ws_bytes, 256 + slot)) != LOQT_OK) return st;
+  if ((st = check_arch()) != LOQT_OK) return st;
+  if (n == 0) return LOQT_OK;
+  cudaStream_t stm = static_cast<cudaStream_t>(stream);
+  // Matrices are taken in batches: as many as the workspace holds dequantised
+  // factors for (packed back to back) and one launch carries.  A batch's factors
+  // are staged by one launch, its merges run in one persistent launch.
+  uint8_t *base = static_cast<uint8_t *>(ws) + 256;
+  const size_t room = ws_bytes - 256;
+  for (int g0 = 0; g0 < n;) {
+    StageItem stage[kMergeBatchMax];
+    MergeItem items[kMergeBatchMax];
+    size_t used = 0;
+    int g1 = g0;
+    while (g1 < n && g1 - g0 < kMergeBatchMax && used + merge_scratch_bytes(Pq[g1]) <= room) {
+      void *phat = base + used;
+      const int64_t ldp = ld_lowrank(Pq[g1].cols);
+      stage[g1 - g0] = StageItem{Pq[g1], phat, ldp};
+      items[g1 - g0] = MergeItem{Wq[g1], {phat, ldp}, {B[g1], ldb[g1]}, Pq[g1].cols, s};
+      used += merge_scratch_bytes(Pq[g1]);
+      ++g1;
+    }
+    if ((st = nf4_dequantize_bf16_batch(stage, g1 - g0, stm)) != LOQT_OK) return st;
+    if ((st = merge_batch(items, g1 - g0, static_cast<uint32_t *>(ws), stm)) != LOQT_OK) return st;
+    g0 = g1;
+  }
+  return LOQT_OK;
 }
 
 extern "C" loqt_status loqt_merge_requant(loqt_nf4_mat Wq, loqt_nf4_mat Pq, const void *B, int64_t ldb, float s,
                                           void *ws, size_t ws_bytes, void *stream) {
-  loqt_status st;
-  if ((st = check_layer(Wq, Pq, B, ldb)) != LOQT_OK) return st;
-  if ((st = check_ws(ws, ws_bytes, 256 + merge_scratch_bytes(Pq))) != LOQT_OK) return st;
-  if ((st = check_arch()) != LOQT_OK) return st;
-  cudaStream_t stm = static_cast<cudaStream_t>(stream);
-  void *phat = static_cast<uint8_t *>(ws) + 256;
-  if ((st = merge_stage(Pq, phat, stm)) != LOQT_OK) return st;
-  return merge_product(Wq, Pq, phat, B, ldb, s, static_cast<uint32_t *>(ws), stm);
+  const int64_t ldb1 = ldb;
+  return loqt_merge_requant_many(1, &Wq, &Pq, &B, &ldb1, s, ws, ws_bytes, stream);
 }
 
 // The same merge in two passes: Delta = P-hat B written as fp32, then the
@@ -517,40 +593,6 @@ extern "C" loqt_status loqt_merge_requant_split(loqt_nf4_mat Wq, loqt_nf4_mat Pq
   c.p.status = static_cast<uint32_t *>(ws);
   if ((st = launch(c, stm)) != LOQT_OK) return st;
   return loqt_nf4_requantize(delta, Wq.ld, s, Wq, stream);
-}
-
-extern "C" loqt_status loqt_merge_requant_many(int32_t n, const loqt_nf4_mat *Wq, const loqt_nf4_mat *Pq,
-                                               const void *const *B, const int64_t *ldb, float s, void *ws,
-                                               size_t ws_bytes, void *stream) {
-  if (n < 0 || (n > 0 && (Wq == nullptr || Pq == nullptr || B == nullptr || ldb == nullptr))) return LOQT_ERR_INVALID_ARG;
-  loqt_status st;
-  size_t slot = 0;
-  for (int i = 0; i < n; ++i) {
-    if ((st = check_layer(Wq[i], Pq[i], B[i], ldb[i])) != LOQT_OK) return st;
-    const size_t need = merge_scratch_bytes(Pq[i]);
-    if (need > slot) slot = need;
-  }
-  if ((st = check_ws(ws, ws_bytes, 256 + slot)) != LOQT_OK) return st;
-  if ((st = check_arch()) != LOQT_OK) return st;
-  if (n == 0) return LOQT_OK;
-  cudaStream_t stm = static_cast<cudaStream_t>(stream);
-  // The workspace holds as many P-hat slots as fit (at most kMergeGroup): a group's
-  // P-hats are staged back to back, then its products run back to back, so that
-  // the short staging kernels do not drain the GPU between every two products.
-  constexpr int kMergeGroup = 8;
-  int slots = static_cast<int>((ws_bytes - 256) / slot);
-  if (slots > kMergeGroup) slots = kMergeGroup;
-  uint8_t *base = static_cast<uint8_t *>(ws) + 256;
-  for (int g0 = 0; g0 < n; g0 += slots) {
-    const int g1 = g0 + slots < n ? g0 + slots : n;
-    for (int i = g0; i < g1; ++i)
-      if ((st = merge_stage(Pq[i], base + static_cast<size_t>(i - g0) * slot, stm)) != LOQT_OK) return st;
-    for (int i = g0; i < g1; ++i)
-      if ((st = merge_product(Wq[i], Pq[i], base + static_cast<size_t>(i - g0) * slot, B[i], ldb[i], s,
-                              static_cast<uint32_t *>(ws), stm)) != LOQT_OK)
-        return st;
-  }
-  return LOQT_OK;
 }
 
 // ---------------------------------------------------------------------------
@@ -663,15 +705,10 @@ extern "C" loqt_status loqt_merge_requant_right(loqt_nf4_mat Wq, loqt_nf4_mat Qq
   cudaStream_t stm = static_cast<cudaStream_t>(stream);
   // Q-hat = bf16(deq(Q_q)), once; then Delta = B Q-hat (out x in; K = r) requantised in the epilogue
   void *qhat = static_cast<uint8_t *>(ws) + 256;
-  if ((st = loqt_nf4_dequantize(Qq, qhat, Qq.ld, 1, stream)) != LOQT_OK) return st;
-  GemmCall c{};
-  c.p.M = out; c.p.N = in; c.p.num_segs = 1;
-  c.p.seg[0].K = r; c.p.seg[0].a_kind = OP_TMA_K; c.p.seg[0].b_kind = OP_TMA_MN;
-  c.a[0] = {B, ldb}; c.b[0] = {qhat, Qq.ld};
-  c.p.splits = 1;
-  c.p.epi = EPI_REQUANT; c.p.alpha = s; c.p.status = static_cast<uint32_t *>(ws);
-  c.p.wq_codes = Wq.codes; c.p.wq_absmax = Wq.absmax; c.p.wq_ld = Wq.ld;
-  return launch(c, stm);
+  const StageItem stage{Qq, qhat, Qq.ld};
+  if ((st = nf4_dequantize_bf16_batch(&stage, 1, stm)) != LOQT_OK) return st;
+  const MergeItem item{Wq, {B, ldb}, {qhat, Qq.ld}, r, s};
+  return merge_batch(&item, 1, static_cast<uint32_t *>(ws), stm);
 }
 
 // ---------------------------------------------------------------------------

@@ -1,0 +1,322 @@
+// The periodic merge of LoQT (paper Section 2.4; Algorithm 1, merge line):
+//
+//   W_q <- q_NF4( deq32(W_q) + alpha * P-hat B )          in place, for a batch of matrices
+//
+// One persistent launch walks the output tiles of every matrix of the batch, so
+// the tiles of the next matrix fill the SMs that the last wave of the previous
+// one would leave idle.  P-hat (out x r, bf16, staged beforehand) and B (r x in,
+// bf16) arrive by TMA; the product of a 128 x BN tile accumulates in one of two
+// TMEM buffers; the epilogue reads it, one 64-column block of one row per
+// thread - which is exactly one NF4 block of W_q - adds the old dequantised
+// values, takes the block maximum, requantises (quantiser of Section 5.1) and
+// writes codes and scale back.
+//
+// Warp roles (480 threads): warp 0 TMA producer, warp 1 MMA issuer and TMEM
+// owner, warps 2-13 epilogue (three groups of four, one warp per TMEM lane
+// quarter; the 64-column blocks are dealt to the groups round-robin, continuing
+// across tiles), warp 14 mover of W_q.  The mover brings the packed codes and
+// the scales of each tile's W_q blocks into shared memory ahead of the tile's
+// epilogue - whole 128-byte rows by one bulk copy instead of a 32-byte access
+// per thread and block - and stores the requantised tile once every epilogue
+// warp is done with it.
+#pragma once
+#include "gemm.cuh"
+
+namespace loqt {
+
+constexpr int kMergeBatchMax = 32;  // matrices per launch (bounded by the kernel parameter space)
+
+struct MergeProblem {
+  float *wq_absmax;  // [M][wq_ld / 64]
+  int M, N, K;       // out, in, r
+  int wq_ld;
+  int tile0;         // position of this matrix's first tile in the launch's sequence of tiles
+  int mt;            // tiles along M (tile = tile0 + n_blk * mt + m_blk)
+  float alpha;
+  int pad_;
+};
+
+struct MergeBatch {
+  CUtensorMap a[kMergeBatchMax];   // P-hat, bf16 [M][K]: box 64 (K) x 128 rows
+  CUtensorMap b[kMergeBatchMax];   // B, bf16 [K][N]: box 64 (N) x 64 (K), an MN-major operand
+  CUtensorMap wq[kMergeBatchMax];  // packed codes of W_q as bytes [M][wq_ld / 2]: box BN / 2 x 128 rows
+  MergeProblem prob[kMergeBatchMax];
+  int count;
+  int tiles;  // of all matrices together
+  uint32_t *status;
+};
+
+template <int BN>
+__global__ void __launch_bounds__(kNumThreads, 1)
+loqt_merge_kernel(const __grid_constant__ MergeBatch mb) {
+  using L = SmemLayout<BN, 1, false, false, true>;
+  constexpr int kStages = L::kStages;
+  constexpr int kEpiGroups = 3;
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t *smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
+
+  const uint32_t bar0 = smem_base + L::kBarOffset;
+  auto full_bar = [&](int s) { return bar0 + 8u * s; };
+  auto empty_bar = [&](int s) { return bar0 + 8u * (kStages + s); };
+  auto tfull_bar = [&](int a) { return bar0 + 8u * (2 * kStages + a); };
+  auto tempty_bar = [&](int a) { return bar0 + 8u * (2 * kStages + 2 + a); };
+  const uint32_t drain_bar = bar0 + 8u * (2 * kStages + 4);
+  auto wfull_bar = [&](int b) { return bar0 + 8u * (2 * kStages + 5 + b); };
+  auto wdone_bar = [&](int b) { return bar0 + 8u * (2 * kStages + 7 + b); };
+  volatile uint32_t *misc = reinterpret_cast<volatile uint32_t *>(smem_gen + L::kMiscOffset);
+  volatile uint32_t *tmem_slot = misc;
+  volatile uint32_t *abort_flag = misc + 1;
+  Nf4Tables &tables = *reinterpret_cast<Nf4Tables *>(smem_gen + L::kTablesOffset);
+
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+  constexpr uint32_t kTmemCols = 2 * BN;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kStages; ++s) {
+      ptx::mbar_init(full_bar(s), 1);
+      ptx::mbar_init(empty_bar(s), 1);
+    }
+    for (int a = 0; a < 2; ++a) {
+      ptx::mbar_init(tfull_bar(a), 1);
+      ptx::mbar_init(tempty_bar(a), 4 * kEpiGroups);
+      ptx::mbar_init(wfull_bar(a), 1);               // the mover, with the tile's bytes
+      ptx::mbar_init(wdone_bar(a), 4 * kEpiGroups);  // every epilogue warp, once per tile
+    }
+    ptx::mbar_init(drain_bar, 1);
+    *abort_flag = 0;
+    ptx::fence_barrier_init();
+  }
+  nf4_tables_init(tables, threadIdx.x);
+  if (warp == 1) {
+    ptx::tmem_alloc(smem_u32(const_cast<uint32_t *>(tmem_slot)), kTmemCols);
+    ptx::tmem_relinquish();
+  }
+  ptx::tc_fence_before();
+  __syncthreads();
+  ptx::tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+  // nothing above touched global data: it may overlap the previous kernel's tail
+  ptx::grid_launch_dependents();
+  ptx::grid_dependency_wait();
+
+  // Where tile g of the launch lies: matrix pi (the search resumes from the
+  // caller's last position: a CTA's tiles come in ascending order) and the tile's
+  // block coordinates inside it.
+  auto locate = [&](int g, int &pi, int &m_blk, int &n_blk) {
+    while (pi + 1 < mb.count && g >= mb.prob[pi + 1].tile0) ++pi;
+    const int local = g - mb.prob[pi].tile0;
+    const int mt = mb.prob[pi].mt;
+    n_blk = local / mt;
+    m_blk = local - n_blk * mt;
+  };
+
+  // =========================================================== TMA producer
+  if (warp == 0) {
+    if (lane == 0) {
+      bool ok = true;
+      uint32_t it = 0;
+      int pi = 0, seen = -1;
+      for (int g = blockIdx.x; ok && g < mb.tiles; g += gridDim.x) {
+        int m_blk, n_blk;
+        locate(g, pi, m_blk, n_blk);
+        if (pi != seen) {
+          ptx::prefetch_tensormap(&mb.a[pi]);
+          ptx::prefetch_tensormap(&mb.b[pi]);
+          seen = pi;
+        }
+        const int kbs = (mb.prob[pi].K + kBK - 1) / kBK;
+        for (int kb = 0; kb < kbs; ++kb, ++it) {
+          const int s = it % kStages;
+          const uint32_t ph = (it / kStages) & 1u;
+          if (!(ok = ptx::mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, mb.status))) break;
+          const uint32_t a_dst = smem_base + s * L::kStageBytes;
+          const uint32_t b_dst = a_dst + L::kABytes;
+          ptx::mbar_arrive_expect_tx(full_bar(s), L::kABytes + L::kBBytes);
+          ptx::tma_load_2d(a_dst, &mb.a[pi], full_bar(s), kb * kBK, m_blk * kHM);
+#pragma unroll
+          for (int j = 0; j < BN / 64; ++j)
+            ptx::tma_load_2d(b_dst + j * 8192, &mb.b[pi], full_bar(s), n_blk * BN + 64 * j, kb * kBK);
+        }
+      }
+      if (!ok) {
+        // give copies already in flight time to land before the shared memory is released
+        const uint64_t t0 = ptx::globaltimer_ns();
+        while (ptx::globaltimer_ns() - t0 < 200000ull) {
+        }
+      }
+    }
+  }
+  // =========================================================== MMA issuer
+  else if (warp == 1) {
+    if (lane == 0) {
+      uint32_t it = 0, tile = 0;
+      bool ok = true;
+      int pi = 0;
+      const uint32_t idesc = make_idesc(kHM, BN, false, true);
+      for (int g = blockIdx.x; ok && g < mb.tiles; g += gridDim.x, ++tile) {
+        int m_blk, n_blk;
+        locate(g, pi, m_blk, n_blk);
+        const int kbs = (mb.prob[pi].K + kBK - 1) / kBK;
+        const uint32_t acc = tile & 1u;
+        if (!(ok = ptx::mbar_wait(tempty_bar(acc), ((tile >> 1) & 1u) ^ 1u, abort_flag, mb.status))) break;
+        ptx::tc_fence_after();
+        const uint32_t d_tmem = tmem_base + acc * BN;
+        for (int kb = 0; kb < kbs; ++kb, ++it) {
+          const int s = it % kStages;
+          const uint32_t ph = (it / kStages) & 1u;
+          if (!(ok = ptx::mbar_wait(full_bar(s), ph, abort_flag, mb.status))) break;
+          ptx::tc_fence_after();
+          const uint32_t a_addr = smem_base + s * L::kStageBytes;
+          const uint64_t a_desc = make_smem_desc(a_addr, false);
+          const uint64_t b_desc = make_smem_desc(a_addr + L::kABytes, true);
+#pragma unroll
+          for (uint32_t k = 0; k < kBK / kUmmaK; ++k)
+            ptx::mma_bf16_ss(d_tmem, a_desc + k * (32u >> 4), b_desc + k * (2048u >> 4), idesc, (kb > 0 || k > 0) ? 1u : 0u);
+          ptx::mma_commit(empty_bar(s));
+        }
+        if (ok) ptx::mma_commit(tfull_bar(acc));
+      }
+      // every MMA issued above has finished before TMEM is freed
+      ptx::mma_commit(drain_bar);
+      ptx::mbar_wait(drain_bar, 0, abort_flag, mb.status);
+    }
+  }
+  // =========================================================== mover of W_q
+  else if (warp == kCodeWarp) {
+    if (lane == 0) {
+      // Buffer b = tile & 1.  Before a buffer is loaded again, the bulk store that
+      // last read it has finished reading (stores complete in the order issued).
+      bool ok = true;
+      uint32_t tile = 0;
+      int pi = 0, prev_pi = 0, pm = 0, pn = 0;
+      auto store_prev = [&]() {
+        const uint32_t pb = (tile - 1) & 1u;
+        if (!(ok = ptx::mbar_wait(wdone_bar(pb), ((tile - 1) >> 1) & 1u, abort_flag, mb.status))) return;
+        ptx::tma_store_2d(&mb.wq[prev_pi], smem_base + L::kWOffset + pb * L::kWTileBytes, pn * (BN / 2), pm * kHM);
+        ptx::bulk_commit_group();
+      };
+      for (int g = blockIdx.x; ok && g < mb.tiles; g += gridDim.x, ++tile) {
+        int m_blk, n_blk;
+        locate(g, pi, m_blk, n_blk);
+        const uint32_t b = tile & 1u;
+        ptx::bulk_wait_group_read<0>();
+        ptx::mbar_arrive_expect_tx(wfull_bar(b), L::kWTileBytes);
+        ptx::tma_load_2d(smem_base + L::kWOffset + b * L::kWTileBytes, &mb.wq[pi], wfull_bar(b), n_blk * (BN / 2), m_blk * kHM);
+        if (tile > 0) store_prev();
+        prev_pi = pi;
+        pm = m_blk;
+        pn = n_blk;
+      }
+      if (ok && tile > 0) store_prev();
+      // every store has left shared memory and reached global memory before the CTA ends
+      ptx::bulk_wait_group<0>();
+    }
+  }
+  // =========================================================== epilogue
+  else {
+    const int q = warp & 3;                   // TMEM lane quarter this warp may access
+    const int grp = (warp - kEpiWarp0) >> 2;  // warps 2-5, 6-9, 10-13
+    uint32_t tile = 0;
+    bool ok = true;
+    int pi = 0;
+    for (int g = blockIdx.x; ok && g < mb.tiles; g += gridDim.x, ++tile) {
+      int m_blk, n_blk;
+      locate(g, pi, m_blk, n_blk);
+      const MergeProblem &pr = mb.prob[pi];
+      const uint32_t acc = tile & 1u;
+      const uint32_t ph = (tile >> 1) & 1u;
+      if (!(ok = ptx::mbar_wait(tfull_bar(acc), ph, abort_flag, mb.status))) break;
+      // the tile's old codes (rows of BN / 2 bytes, TMA-swizzled: 16-byte chunk ^= row & 7
+      // for 128-byte rows, (row >> 1) & 3 for 64-byte rows); the new ones replace them there
+      if (!(ok = ptx::mbar_wait(wfull_bar(acc), ph, abort_flag, mb.status))) break;
+      ptx::tc_fence_after();
+      const int row_t = q * 32 + lane;  // row inside the tile
+      const int row = m_blk * kHM + row_t;
+      const bool row_ok = row < pr.M;
+      const uint32_t t_row = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + acc * BN;
+      const uint32_t w_row = smem_base + L::kWOffset + acc * L::kWTileBytes + static_cast<uint32_t>(row_t) * (BN / 2);
+      const uint32_t w_key = (BN == 256) ? static_cast<uint32_t>(row_t & 7) : static_cast<uint32_t>((row_t >> 1) & 3);
+      const float alpha = pr.alpha;
+#pragma unroll 1
+      for (int jb = 0; jb < BN / 64; ++jb) {
+        const uint32_t seq = tile * (BN / 64) + jb;  // position in this CTA's sequence of blocks
+        if (static_cast<int>(seq % kEpiGroups) != grp) continue;
+        const int c0 = n_blk * BN + jb * 64;
+        const bool live = row_ok && c0 < pr.wq_ld;
+        float *mp = pr.wq_absmax + static_cast<int64_t>(row) * (pr.wq_ld >> 6) + (c0 >> 6);
+        float Mold = 0.0f;
+        if (live) Mold = *mp;  // in flight while the accumulator is read
+        const uint32_t a0 = w_row + (((2u * jb) ^ w_key) << 4), a1 = w_row + (((2u * jb + 1u) ^ w_key) << 4);
+        const uint4 ca = ld_shared_v4(a0), cb = ld_shared_v4(a1);
+        uint32_t d0[32], d1[32];
+        ptx::tmem_ld32(t_row + jb * 64, d0);
+        ptx::tmem_ld32(t_row + jb * 64 + 32, d1);
+        ptx::tmem_ld_wait();
+        if (live) {
+          const uint32_t w[8] = {ca.x, ca.y, ca.z, ca.w, cb.x, cb.y, cb.z, cb.w};
+          // v = deq32(old) + alpha * delta, two elements per packed instruction; four
+          // running maxima keep the dependent chain of the block maximum short
+          float2 v[32];
+          float mx[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+          const float2 a2 = make_float2(alpha, alpha), m2 = make_float2(Mold, Mold);
+#pragma unroll
+          for (int e = 0; e < 32; ++e) {
+            const uint32_t word = w[e >> 2];
+            const float2 lv = make_float2(tables.level[(word >> (8 * (e & 3))) & 15u],
+                                          tables.level[(word >> (8 * (e & 3) + 4)) & 15u]);
+            const float2 delta = make_float2(__uint_as_float(e < 16 ? d0[2 * e] : d1[2 * e - 32]),
+                                             __uint_as_float(e < 16 ? d0[2 * e + 1] : d1[2 * e - 31]));
+            v[e] = __ffma2_rn(a2, delta, __fmul2_rn(m2, lv));
+            mx[e & 3] = fmaxf(mx[e & 3], fmaxf(fabsf(v[e].x), fabsf(v[e].y)));
+          }
+          const float Mnew = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
+          uint32_t o[8];
+          const Nf4Divisor dv = nf4_divisor(Mnew);
+          auto quantise_block = [&](auto exact) {
+#pragma unroll
+            for (int g8 = 0; g8 < 8; ++g8) {
+              uint32_t word = 0;
+#pragma unroll
+              for (int h2 = 0; h2 < 4; ++h2)
+                word |= nf4_code2(tables, nf4_normalise2<decltype(exact)::value>(dv, v[4 * g8 + h2])) << (8 * h2);
+              o[g8] = word;
+            }
+          };
+          if (!(Mnew > 0.0f)) {
+#pragma unroll
+            for (int g8 = 0; g8 < 8; ++g8) o[g8] = kZeroWord;
+          } else if (dv.exact) {
+            quantise_block(std::true_type{});
+          } else {
+            quantise_block(std::false_type{});
+          }
+          st_shared_v4(a0, make_uint4(o[0], o[1], o[2], o[3]));
+          st_shared_v4(a1, make_uint4(o[4], o[5], o[6], o[7]));
+          *mp = Mnew;
+        }
+        __syncwarp();
+      }
+      // This warp's blocks of the tile are in place: made visible to the bulk store,
+      // then signalled; the accumulator goes back to the MMA warp.
+      ptx::fence_proxy_async_smem();
+      ptx::tc_fence_before();
+      __syncwarp();
+      if (lane == 0) {
+        ptx::mbar_arrive(wdone_bar(acc));
+        ptx::mbar_arrive(tempty_bar(acc));
+      }
+    }
+  }
+
+  // =========================================================== teardown
+  ptx::tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    ptx::tc_fence_after();
+    ptx::tmem_dealloc(tmem_base, kTmemCols);
+  }
+}
+
+}  // namespace loqt

@@ -161,19 +161,14 @@ nf4_quantize_kernel(const float *__restrict__ src, int64_t ld_src, float s, uint
 // ---------------------------------------------------------------------------
 constexpr int kDqUnroll = 4;
 
+// Expands the code words first, first + stride, ... of one matrix.
 template <bool kBf16, bool kVec>
-__global__ void __launch_bounds__(kQThreads)
-nf4_dequantize_kernel(const uint8_t *__restrict__ codes, const float *__restrict__ absmax,
-                      void *__restrict__ dst, int64_t ld_dst, int rows, int cols, int ld) {
-  __shared__ Nf4Tables tab;
-  nf4_tables_init(tab, threadIdx.x);
-  __syncthreads();
-
+__device__ __forceinline__ void dequantize_words(const Nf4Tables &tab, const uint8_t *__restrict__ codes,
+                                                 const float *__restrict__ absmax, void *__restrict__ dst, int64_t ld_dst,
+                                                 int rows, int cols, int ld, uint32_t first, uint32_t stride) {
   const uint32_t wpr = static_cast<uint32_t>(ld / 8);  // code words per row
   const uint32_t nb = static_cast<uint32_t>(ld / kBlock);
   const uint32_t n_items = static_cast<uint32_t>(rows) * wpr;  // (host checks < 2^31)
-  const uint32_t stride = gridDim.x * kQThreads;
-  const uint32_t first = blockIdx.x * kQThreads + threadIdx.x;
 
   struct Word {
     uint32_t w, row;
@@ -244,6 +239,46 @@ nf4_dequantize_kernel(const uint8_t *__restrict__ codes, const float *__restrict
   }
 }
 
+template <bool kBf16, bool kVec>
+__global__ void __launch_bounds__(kQThreads)
+nf4_dequantize_kernel(const uint8_t *__restrict__ codes, const float *__restrict__ absmax,
+                      void *__restrict__ dst, int64_t ld_dst, int rows, int cols, int ld) {
+  __shared__ Nf4Tables tab;
+  nf4_tables_init(tab, threadIdx.x);
+  __syncthreads();
+  dequantize_words<kBf16, kVec>(tab, codes, absmax, dst, ld_dst, rows, cols, ld, blockIdx.x * kQThreads + threadIdx.x,
+                                gridDim.x * kQThreads);
+}
+
+// Several matrices to bf16 in one launch (the staging step of a batched merge):
+// the grid is dealt to the matrices in proportion to their sizes, blocks cta0 ..
+// cta0 + ctas - 1 stride over matrix i.
+struct DequantBatch {
+  struct Item {
+    const uint8_t *codes;
+    const float *absmax;
+    void *dst;
+    int64_t ld_dst;
+    int rows, cols, ld;
+    int cta0, ctas;
+  } item[kStageBatchMax];
+  int count;
+};
+
+template <bool kVec>
+__global__ void __launch_bounds__(kQThreads)
+nf4_dequantize_batch_kernel(const __grid_constant__ DequantBatch batch) {
+  __shared__ Nf4Tables tab;
+  nf4_tables_init(tab, threadIdx.x);
+  __syncthreads();
+  int i = 0;
+  while (i + 1 < batch.count && static_cast<int>(blockIdx.x) >= batch.item[i + 1].cta0) ++i;
+  const DequantBatch::Item &m = batch.item[i];
+  const uint32_t local = blockIdx.x - static_cast<uint32_t>(m.cta0);
+  dequantize_words<true, kVec>(tab, m.codes, m.absmax, m.dst, m.ld_dst, m.rows, m.cols, m.ld, local * kQThreads + threadIdx.x,
+                               static_cast<uint32_t>(m.ctas) * kQThreads);
+}
+
 // Grid of a streaming kernel: enough blocks for the work, at most as many as
 // are resident at once (the kernels loop with a grid stride).
 template <typename Kernel>
@@ -290,6 +325,40 @@ loqt_status nf4_quantize_residual(const float *src, int64_t ld_src, const float 
   auto kernel = vec ? nf4_quantize_kernel<true, kQuantiseResidual> : nf4_quantize_kernel<false, kQuantiseResidual>;
   kernel<<<grid_for(kernel, items * 4), kQThreads, 0, stream>>>(src, ld_src, 1.0f, dst.codes, dst.absmax, dst.rows, dst.cols, dst.ld, ref,
                                                                 ld_ref, static_cast<__nv_bfloat16 *>(resid), ld_resid);
+  count_launch();
+  return cudaGetLastError() == cudaSuccess ? LOQT_OK : LOQT_ERR_CUDA;
+}
+
+// dst_i <- bf16(deq(src_i)) for up to kStageBatchMax matrices, one launch.
+loqt_status nf4_dequantize_bf16_batch(const StageItem *items, int n, cudaStream_t stream) {
+  if (n <= 0) return LOQT_OK;
+  if (n > kStageBatchMax) return LOQT_ERR_INVALID_ARG;
+  DequantBatch batch;
+  memset(&batch, 0, sizeof(batch));
+  bool vec = true;
+  int64_t total = 0;
+  for (int i = 0; i < n; ++i) {
+    const loqt_nf4_mat &m = items[i].src;
+    const int64_t words = static_cast<int64_t>(m.rows) * (m.ld / 8);
+    if (words >= (1ll << 31)) return LOQT_ERR_UNSUPPORTED;
+    total += words;
+    vec = vec && (reinterpret_cast<uintptr_t>(items[i].dst) & 15u) == 0 && (items[i].ld_dst % 8) == 0;
+  }
+  auto kernel = vec ? nf4_dequantize_batch_kernel<true> : nf4_dequantize_batch_kernel<false>;
+  const int cap = grid_for(kernel, (total + kDqUnroll - 1) / kDqUnroll);
+  int next = 0;
+  for (int i = 0; i < n; ++i) {
+    const loqt_nf4_mat &m = items[i].src;
+    const int64_t words = static_cast<int64_t>(m.rows) * (m.ld / 8);
+    int64_t ctas = (words * cap + total - 1) / total;                     // share of the grid
+    const int64_t need = (words + kQThreads * kDqUnroll - 1) / (kQThreads * kDqUnroll);  // blocks with work
+    if (ctas > need) ctas = need;
+    if (ctas < 1) ctas = 1;
+    batch.item[i] = {m.codes, m.absmax, items[i].dst, items[i].ld_dst, m.rows, m.cols, m.ld, next, static_cast<int>(ctas)};
+    next += static_cast<int>(ctas);
+  }
+  batch.count = n;
+  kernel<<<next, kQThreads, 0, stream>>>(batch);
   count_launch();
   return cudaGetLastError() == cudaSuccess ? LOQT_OK : LOQT_ERR_CUDA;
 }

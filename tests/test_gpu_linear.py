@@ -141,12 +141,29 @@ def test_merge_zero_B_leaves_weights_untouched():
 
 
 def test_merge_many_matches_single():
-    shapes = [(256, 256, 32), (384, 320, 64), (200, 136, 24)]
-    sets = [_setup(14 + i, o, n, r, 8)[1] for i, (o, n, r) in enumerate(shapes)]
-    singles = [L.loqt_merge_requant(x["Wq"].clone(), x["Pq"], x["B"], 0.5) for x in sets]
-    L.loqt_merge_requant_many([x["Wq"] for x in sets], [x["Pq"] for x in sets], [x["B"] for x in sets], 0.5)
-    for one, x in zip(singles, sets):
-        assert torch.equal(one.codes, x["Wq"].codes) and torch.equal(one.absmax, x["Wq"].absmax)
+    # 18 matrices of mixed shapes (ragged and not, several ranks) through one call: the batched launch walks
+    # the tiles of all of them as one sequence and must leave every matrix exactly as a merge of its own does;
+    # a few are also compared with the oracle.  A small workspace forces the call to split into several batches.
+    shapes = [(256, 256, 32), (384, 320, 64), (200, 136, 24), (512, 1376, 128), (1376, 512, 128), (640, 5461, 96),
+              (130, 70, 8), (128, 256, 64), (1024, 1024, 256), (96, 4096, 48), (2736, 192, 40), (257, 257, 16),
+              (64, 64, 64), (768, 1000, 72), (1000, 768, 200), (5461, 256, 40), (300, 2100, 512), (2048, 640, 320)]
+    sets = [_setup(14 + i, o, n, r, 8) for i, (o, n, r) in enumerate(shapes)]
+    devs = [d for _, d in sets]
+    singles = [L.loqt_merge_requant(x["Wq"].clone(), x["Pq"], x["B"], 0.5) for x in devs]
+    for group in (8, 1):
+        trial = [x["Wq"].clone() for x in devs]
+        ws = L.new_workspace(L.merge_many_workspace_bytes(trial, [x["Pq"] for x in devs], group=group))
+        L.loqt_merge_requant_many(trial, [x["Pq"] for x in devs], [x["B"] for x in devs], 0.5, ws=ws)
+        L.loqt_device_status(ws)
+        for one, got in zip(singles, trial):
+            assert torch.equal(one.codes, got.codes) and torch.equal(one.absmax, got.absmax)
+    for i in (0, 5, 11, 16):
+        (h, d), (o, n, r) = sets[i], shapes[i]
+        vw = O.loqt_merge_values(h["wq"], h["pq"], h["B"], 0.5, (o, n, r))
+        ref_c, ref_m = O.nf4_quantize(vw)
+        got_c, got_m = from_dev_nf4(singles[i])
+        bound, _ = merge_error_bound(h["pq"], h["B"], 0.5, r, ref_m)
+        check_merge(got_c, got_m, ref_c, ref_m, vw, n, bound, f"merge-many {shapes[i]}")
 
 
 def test_forward_special_cases_on_device():
