@@ -414,3 +414,98 @@ def dq_dequantize_absmax(codes: np.ndarray, c1: np.ndarray, offset, shape=None) 
 def dq_bits_per_weight() -> float:
     """Storage of a doubly quantised NF4 matrix per weight, in bits."""
     return 4.0 + 8.0 / BLOCK + 32.0 / (BLOCK * DQ_BLOCK)
+
+
+# ----------------------------------------------------------------------------
+# 8-bit optimiser states  (the paper trains B with "8-bit Adam", citing Dettmers et
+# al., "8-bit Optimizers via Block-wise Quantization": Section 3.2 memory
+# comparison, the 13B run and the continued-pretraining appendix)
+#
+# The paper gives no formulas; the reading taken is that publication's scheme:
+# the two Adam moments are stored as 8-bit codes, quantised block-wise (blocks of
+# 2048 consecutive elements, one fp32 scale = the block's largest magnitude), in
+# the "dynamic tree" data type - a sign bit, then a run of zero bits whose length
+# E is a base-10 exponent, an indicator bit, and the remaining f bits a linear
+# fraction - with the sign bit turned into one more fraction bit for the
+# non-negative second moment.  The fraction's grid inside a decade is this
+# file's reading: magnitude(E, j) = 10^-E * (0.1 + 0.9 * (j + 1) / 2^f), j = 0 ..
+# 2^f - 1, so that a decade's largest value is 10^-E itself and its smallest lies
+# just above the decade below; code 0 is zero.  Read as an integer, the magnitude
+# bits are then 2^f + j: magnitudes ascend with the code.
+# An optimiser step dequantises the moments, updates in 32-bit arithmetic, and
+# quantises them again.
+# ----------------------------------------------------------------------------
+OPT8_BLOCK = 2048
+
+
+def dyn8_codebook(signed: bool) -> np.ndarray:
+    """Magnitudes of the 8-bit dynamic data type as fp32, indexed by the magnitude
+    bits (7 of them when a sign bit is kept, else 8): 128 or 256 ascending values."""
+    bits = 7 if signed else 8
+    c = np.zeros(1 << bits, dtype=np.float64)
+    for f in range(bits):
+        E = bits - 1 - f
+        for j in range(1 << f):
+            c[(1 << f) + j] = (0.1 + 0.9 * (j + 1) / float(1 << f)) * (10.0 ** -E)
+    return c.astype(np.float32)
+
+
+def dyn8_quantize(x: np.ndarray, signed: bool):
+    """Block-wise quantisation of a flat fp32 array to the 8-bit dynamic type.
+    Per block of 2048: M = max |x|; n = fl32(x / M); the magnitude index is the
+    number of midpoints between neighbouring magnitudes that |n| exceeds (so the
+    nearest magnitude, the smaller one on a tie); the sign goes to bit 7 (signed
+    type, never set for a zero magnitude).  Returns (codes uint8 [n], absmax fp32)."""
+    x = np.ascontiguousarray(x, dtype=np.float32).reshape(-1)
+    n_el = x.size
+    nb = (n_el + OPT8_BLOCK - 1) // OPT8_BLOCK
+    c = dyn8_codebook(signed).astype(np.float64)
+    mid = (c[:-1] + c[1:]) / 2.0
+    codes = np.zeros(n_el, dtype=np.uint8)
+    absmax = np.zeros(nb, dtype=np.float32)
+    for b in range(nb):
+        blk = x[b * OPT8_BLOCK : (b + 1) * OPT8_BLOCK]
+        M = np.float32(np.max(np.abs(blk)))
+        absmax[b] = M
+        if not M > 0:
+            continue
+        n = (blk / M).astype(np.float32).astype(np.float64)
+        idx = np.searchsorted(mid, np.abs(n), side="left").astype(np.uint8)  # count of midpoints strictly below |n|
+        if signed:
+            idx = np.where((n < 0) & (idx > 0), idx | 0x80, idx).astype(np.uint8)
+        codes[b * OPT8_BLOCK : b * OPT8_BLOCK + blk.size] = idx
+    return codes, absmax
+
+
+def dyn8_dequantize(codes: np.ndarray, absmax: np.ndarray, signed: bool) -> np.ndarray:
+    """x' = fl32( magnitude[code] * M ), negated when the sign bit is set."""
+    codes = np.asarray(codes, dtype=np.uint8).reshape(-1)
+    c = dyn8_codebook(signed)
+    M = np.repeat(np.asarray(absmax, dtype=np.float32), OPT8_BLOCK)[: codes.size]
+    if signed:
+        mag = (c[codes & 0x7F] * M).astype(np.float32)
+        return np.where(codes & 0x80, -mag, mag).astype(np.float32)
+    return (c[codes] * M).astype(np.float32)
+
+
+def adam8_step(B, g, m8, m_absmax, v8, v_absmax, step, lr, beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=0.0):
+    """One Adam step on B (see adam_step) with the moments held in 8 bits: they are
+    dequantised, updated with the gradient, used for the step on B, and quantised
+    again.  B: bf16 values [r, in]; g: fp32 [r, in]; m8, v8: uint8 [r * in] codes of
+    the row-major flattened moments with one fp32 scale per 2048 elements.
+    Evaluated in float64 from the fp32 dequantised moments; B is rounded once to
+    bf16, the new moments once to fp32 before quantisation.
+    Returns (B, m8, m_absmax, v8, v_absmax)."""
+    shape = np.asarray(B).shape
+    m = dyn8_dequantize(m8, m_absmax, True).astype(np.float64).reshape(shape)
+    v = dyn8_dequantize(v8, v_absmax, False).astype(np.float64).reshape(shape)
+    B64 = np.asarray(B, dtype=np.float64)
+    g64 = np.asarray(g, dtype=np.float32).astype(np.float64)
+    m64 = beta1 * m + (1.0 - beta1) * g64
+    v64 = beta2 * v + (1.0 - beta2) * g64 * g64
+    mhat = m64 / (1.0 - beta1 ** step)
+    vhat = v64 / (1.0 - beta2 ** step)
+    Bn = B64 - lr * (mhat / (np.sqrt(vhat) + eps) + weight_decay * B64)
+    mq = dyn8_quantize(m64.astype(np.float32).reshape(-1), True)
+    vq = dyn8_quantize(v64.astype(np.float32).reshape(-1), False)
+    return bf16_round(Bn.astype(np.float32)), mq[0], mq[1], vq[0], vq[1]
