@@ -326,24 +326,16 @@ def run_per_shape(args):
     print(json.dumps({"per_shape": res, "config": cfg.name}), flush=True)
 
 
-def run_ours(args, rank, world, local_rank):
+def measure_config(args, ci, rank, world, local_rank, dist, device, e2e=True):
+    """Builds the layer set of configuration `ci` on this rank's GPU, runs W warm-up
+    steps and K timed steps (fwd+bwd of every matrix, then one merge of all), and
+    returns the timings (max over ranks) with the clocks sampled meanwhile."""
     import torch
 
     from paper_2405_16528_b200 import binding as L
-    from paper_2405_16528_b200 import build, synth
+    from paper_2405_16528_b200 import synth
 
-    build.build()
-    L.lib()  # fails loudly when the CUDA library is missing
-    torch.cuda.set_device(local_rank)
-    device = torch.device("cuda", local_rank)
-    dist = None
-    if world > 1:
-        import torch.distributed as dist_mod
-
-        dist = dist_mod
-        dist.init_process_group("nccl", device_id=device)
-
-    cfg = synth.CONFIGS[args.config]
+    cfg = synth.CONFIGS[ci]
     if args.layers > 0:
         import dataclasses
 
@@ -404,54 +396,118 @@ def run_ours(args, rank, world, local_rank):
     ms_mg = sum(e[1].elapsed_time(e[2]) for e in ev) / args.steps
     ms_step = sum(e[0].elapsed_time(e[2]) for e in ev) / args.steps
 
-    # ---- end to end: activations come from pinned host memory every step, the
-    # gradient of the trained matrix goes back to the host
-    e2e_steps = max(1, min(args.steps, 2))
-    shapes = {}
-    for m in mats:
-        key = (m["out"], m["in"])
-        if key not in shapes:
-            shapes[key] = {
-                "hx": torch.empty((cfg.T, m["x"].stride(0)), dtype=torch.bfloat16).pin_memory(),
-                "hdy": torch.empty((cfg.T, m["dy"].stride(0)), dtype=torch.bfloat16).pin_memory(),
-                "hdB": torch.empty((cfg.r, m["in"]), dtype=torch.float32).pin_memory(),
-                "dxin": torch.empty((cfg.T, m["x"].stride(0)), dtype=torch.bfloat16, device=device),
-                "ddy": torch.empty((cfg.T, m["dy"].stride(0)), dtype=torch.bfloat16, device=device),
-            }
-            shapes[key]["hx"].normal_()
-            shapes[key]["hdy"].normal_()
-    h2d = d2h = 0
-    for m in mats:
-        sh = shapes[(m["out"], m["in"])]
-        h2d += sh["hx"].numel() * 2 + sh["hdy"].numel() * 2
-        d2h += sh["hdB"].numel() * 4
-
-    def e2e_step():
+    # ---- end to end through the public API with HOST buffers: every step the activations x and the
+    # output gradients dy of every matrix come from pinned host memory, the gradient of the trained
+    # factor goes back to the host, and the merge of all matrices closes the step.  y and dx stay on
+    # the device (in a training step they feed the neighbouring layers there).
+    ms_e2e, h2d, d2h, e2e_steps = 0.0, 0, 0, 0
+    if e2e:
+        e2e_steps = max(1, min(args.steps, 2))
+        shapes = {}
+        for m in mats:
+            key = (m["out"], m["in"])
+            if key not in shapes:
+                shapes[key] = {
+                    "hx": torch.empty((cfg.T, m["x"].stride(0)), dtype=torch.bfloat16).pin_memory(),
+                    "hdy": torch.empty((cfg.T, m["dy"].stride(0)), dtype=torch.bfloat16).pin_memory(),
+                    "hdB": torch.empty((cfg.r, m["in"]), dtype=torch.float32).pin_memory(),
+                    "dxin": torch.empty((cfg.T, m["x"].stride(0)), dtype=torch.bfloat16, device=device),
+                    "ddy": torch.empty((cfg.T, m["dy"].stride(0)), dtype=torch.bfloat16, device=device),
+                }
+                shapes[key]["hx"].normal_()
+                shapes[key]["hdy"].normal_()
         for m in mats:
             sh = shapes[(m["out"], m["in"])]
-            b = bufs[(m["out"], m["in"])]
-            sh["dxin"].copy_(sh["hx"], non_blocking=True)
-            sh["ddy"].copy_(sh["hdy"], non_blocking=True)
-            xin = sh["dxin"][:, : m["in"]]
-            dyin = sh["ddy"][:, : m["out"]]
-            L.loqt_linear_fwd(m["Wq"], m["Pq"], m["B"], s, xin, y=b["y"], ws=ws)
-            L.loqt_linear_bwd(m["Wq"], m["Pq"], m["B"], s, xin, dyin, dx=b["dx"], dB=b["dB"], ws=ws)
-            sh["hdB"].copy_(b["dB"], non_blocking=True)
+            h2d += sh["hx"].numel() * 2 + sh["hdy"].numel() * 2
+            d2h += sh["hdB"].numel() * 4
 
-    e2e_step()
-    sync()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record()
-    for _ in range(e2e_steps):
+        def e2e_step():
+            for m in mats:
+                sh = shapes[(m["out"], m["in"])]
+                b = bufs[(m["out"], m["in"])]
+                sh["dxin"].copy_(sh["hx"], non_blocking=True)
+                sh["ddy"].copy_(sh["hdy"], non_blocking=True)
+                xin = sh["dxin"][:, : m["in"]]
+                dyin = sh["ddy"][:, : m["out"]]
+                L.loqt_linear_fwd(m["Wq"], m["Pq"], m["B"], s, xin, y=b["y"], ws=ws)
+                L.loqt_linear_bwd(m["Wq"], m["Pq"], m["B"], s, xin, dyin, dx=b["dx"], dB=b["dB"], ws=ws)
+                sh["hdB"].copy_(b["dB"], non_blocking=True)
+            merge()
+
         e2e_step()
-    e1.record()
-    sync()
-    ms_e2e = e0.elapsed_time(e1) / e2e_steps
+        sync()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(e2e_steps):
+            e2e_step()
+        e1.record()
+        sync()
+        ms_e2e = e0.elapsed_time(e1) / e2e_steps
+        del shapes
 
     times = torch.tensor([ms_fb, ms_mg, ms_step, ms_e2e], dtype=torch.float64, device=device)
     if dist is not None:
         dist.all_reduce(times, op=dist.ReduceOp.MAX)
     ms_fb, ms_mg, ms_step, ms_e2e = [float(v) for v in times.cpu()]
+    out = {
+        "cfg": cfg, "n_mats": len(mats), "flops_step": flops_step, "merge_bytes_step": merge_bytes_step,
+        "merge_flops_step": merge_flops_step, "ms_fb": ms_fb, "ms_mg": ms_mg, "ms_step": ms_step, "ms_e2e": ms_e2e,
+        "h2d": h2d, "d2h": d2h, "e2e_steps": e2e_steps, "launches": int(launches), "clocks": clocks, "t_wall": t_wall, "s": s,
+    }
+    del mats, bufs, ws, Wqs, Pqs, Bs
+    torch.cuda.empty_cache()
+    return out
+
+
+def merge_report(m, world, peaks):
+    """The merge of one measured configuration: GB/s on its algorithmic bytes (read and
+    write W_q, read P_q, read B), the TFLOP/s of its product, and the share of the roof
+    that binds it, max(tensor time, HBM time)."""
+    gbs = world * m["merge_bytes_step"] / (m["ms_mg"] * 1e-3) / 1e9
+    tf = world * m["merge_flops_step"] / (m["ms_mg"] * 1e-3) / 1e12
+    t_tensor = m["merge_flops_step"] / (peaks["bf16_tflops_sustained"] * 1e12)
+    t_hbm = m["merge_bytes_step"] / (peaks["hbm_gbs"] * 1e9)
+    return {
+        "ms": round(m["ms_mg"], 3),
+        "gb_s": round(gbs, 1),
+        "pct_hbm": round(100 * gbs / world / peaks["hbm_gbs"], 2),
+        "gemm_tflops": round(tf, 1),
+        "binding_roof": "tensor" if t_tensor >= t_hbm else "hbm",
+        "pct_of_binding_roof": round(100 * max(t_tensor, t_hbm) / (m["ms_mg"] * 1e-3), 2),
+        "bytes_per_step": m["merge_bytes_step"],
+    }
+
+
+# DRAM read + write bytes of the forward/backward launches (u, y, v, dx, dB) of ONE attention-shaped
+# matrix, from the ncu capture summarised in profiles/ (None where no capture of the current kernels exists).
+NCU_TRAFFIC = {
+    4: {"bytes": None, "of": "no capture of the current kernels yet (algorithmic 332.4e6 for one 4096x4096 matrix)"},
+}
+
+
+def run_ours(args, rank, world, local_rank):
+    import torch
+
+    from paper_2405_16528_b200 import binding as L
+    from paper_2405_16528_b200 import build, synth
+
+    build.build()
+    L.lib()  # fails loudly when the CUDA library is missing
+    torch.cuda.set_device(local_rank)
+    device = torch.device("cuda", local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+
+        dist = dist_mod
+        dist.init_process_group("nccl", device_id=device)
+
+    main = measure_config(args, args.config, rank, world, local_rank, dist, device)
+    # the second north-star shape set (Llama-1B: odd MLP width 5461, r = 512, T = 8192) in the same run
+    extra = {}
+    for ci in args.also:
+        if ci != args.config:
+            extra[ci] = measure_config(args, ci, rank, world, local_rank, dist, device, e2e=False)
 
     if rank != 0:
         if dist is not None:
@@ -459,13 +515,13 @@ def run_ours(args, rank, world, local_rank):
         return
 
     peaks = load_peaks()
+    cfg = main["cfg"]
     nf4 = time_nf4_kernels(device, peaks)
     comp = time_compensated_init(device, peaks, cfg, args.seed)
     adam = time_adam_step(device, peaks)
-    tflops = world * flops_step / (ms_fb * 1e-3) / 1e12
-    merge_gbs = world * merge_bytes_step / (ms_mg * 1e-3) / 1e9
-    merge_tflops = world * merge_flops_step / (ms_mg * 1e-3) / 1e12
+    tflops = world * main["flops_step"] / (main["ms_fb"] * 1e-3) / 1e12
     per_gpu_tflops = tflops / world
+    traffic = NCU_TRAFFIC.get(args.config, {"bytes": None, "of": "no capture for this configuration"})
     result = {
         "metric": METRIC,
         "value": round(tflops, 2),
@@ -473,35 +529,27 @@ def run_ours(args, rank, world, local_rank):
         "n_gpus": world,
         "steps": args.steps,
         "warmup": args.warmup,
-        "ms_per_step": round(ms_step, 3),
-        "ms_fwd_bwd": round(ms_fb, 3),
-        "ms_merge": round(ms_mg, 3),
+        "ms_per_step": round(main["ms_step"], 3),
+        "ms_fwd_bwd": round(main["ms_fb"], 3),
+        "ms_merge": round(main["ms_mg"], 3),
         "higher_is_better": True,
         "scaling": "weak",
         "vs_baseline": None,
         "dtype": "bf16 x bf16 -> fp32 (NF4 weights)",
         "data": "synthetic",
         "config": {
-            "workload": f"configs[{args.config}] {cfg.name}: {len(mats)} projection matrices, r={cfg.r}, T={cfg.T}",
+            "workload": f"configs[{args.config}] {cfg.name}: {main['n_mats']} projection matrices, r={cfg.r}, T={cfg.T}",
             "step": "fwd+bwd of every matrix, then merge_requant of all",
             "l2": "inputs larger than L2: every matrix has its own weights and activations",
             "replicas": world,
-            "s": s,
+            "s": main["s"],
         },
         "pct_bf16_peak": {
             "burst": round(100 * per_gpu_tflops / peaks["bf16_tflops"], 2),
             "sustained": round(100 * per_gpu_tflops / peaks["bf16_tflops_sustained"], 2),
             "of": peaks["source"],
         },
-        "merge_requant": {
-            "gb_s": round(merge_gbs, 1),
-            "pct_hbm": round(100 * merge_gbs / world / peaks["hbm_gbs"], 2),
-            "gemm_tflops": round(merge_tflops, 1),
-            "pct_of_binding_roof": round(
-                100 * max(merge_flops_step / (peaks["bf16_tflops_sustained"] * 1e12), merge_bytes_step / (peaks["hbm_gbs"] * 1e9))
-                / (ms_mg * 1e-3), 2),
-            "bytes_per_step": merge_bytes_step,
-        },
+        "merge_requant": merge_report(main, world, peaks),
         "roofline": {
             "kernel": "loqt_gemm_kernel (fused NF4-dequant tcgen05 GEMM; all fwd+bwd launches)",
             "bound": "tensor",
@@ -510,26 +558,39 @@ def run_ours(args, rank, world, local_rank):
             "unit": "TFLOP/s",
             "frac": round(per_gpu_tflops / peaks["bf16_tflops_sustained"], 4),
             "peak_kind": f"sustained, of {peaks['source']}",
-            # DRAM read + write bytes of the five forward/backward launches (u, y, v, dx, dB) of one
-            # 4096 x 4096 matrix, from the committed ncu capture; the algorithmic bytes of the same five
-            # launches are 332.4e6 (part of y and dx is still in L2 when the kernels end)
-            "traffic": 266.6e6,
-            "traffic_of": "ncu dram bytes, 5 fwd+bwd launches of one 4096x4096 matrix (algorithmic 332.4e6)",
+            "traffic": traffic["bytes"],
+            "traffic_of": traffic["of"],
         },
         "e2e": {
-            "value": round(world * flops_step / (ms_e2e * 1e-3) / 1e12, 2),
+            "value": round(world * main["flops_step"] / (main["ms_e2e"] * 1e-3) / 1e12, 2),
             "unit": "TFLOP/s",
-            "h2d_bytes_per_step": h2d,
-            "d2h_bytes_per_step": d2h,
-            "steps": e2e_steps,
+            "h2d_bytes_per_step": main["h2d"],
+            "d2h_bytes_per_step": main["d2h"],
+            "steps": main["e2e_steps"],
+            "region": "H2D of x and dy of every matrix from pinned memory, fwd, bwd, D2H of dB, then the merge of all matrices",
+            "left_out": "y and dx are not copied back: they stay on the device for the neighbouring layers",
         },
+        "configs": {},
         "nf4_stream": nf4,
         "compensated_init": comp,
         "adam_step": adam,
-        "gpu_launches": int(launches),
-        "clocks": clocks,
-        "wall_s_timed": round(t_wall, 3),
+        "gpu_launches": main["launches"],
+        "clocks": main["clocks"],
+        "wall_s_timed": round(main["t_wall"], 3),
     }
+    for ci, m in extra.items():
+        tf = m["flops_step"] / (m["ms_fb"] * 1e-3) / 1e12  # per GPU
+        result["configs"][str(ci)] = {
+            "workload": f"configs[{ci}] {m['cfg'].name}: {m['n_mats']} projection matrices, r={m['cfg'].r}, T={m['cfg'].T}",
+            "tflops": round(world * tf, 2),
+            "ms_fwd_bwd": round(m["ms_fb"], 3),
+            "pct_bf16_peak": {"burst": round(100 * tf / peaks["bf16_tflops"], 2),
+                              "sustained": round(100 * tf / peaks["bf16_tflops_sustained"], 2), "of": peaks["source"]},
+            "merge_requant": merge_report(m, world, peaks),
+            "gpu_launches": m["launches"],
+            "clocks": m["clocks"],
+            "roofline_traffic": None,
+        }
     if not args.no_cpu_baseline and world == 1:
         result["cpu_baseline"] = cpu_baseline(cfg, args.seed)
     print(json.dumps(result), flush=True)
@@ -628,6 +689,8 @@ def main():
     ap.add_argument("--seed", type=int, default=0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--layers", type=int, default=0, help="override the layer count (small cases for profiling)")
+    ap.add_argument("--also", type=int, nargs="*", default=[3],
+                    help="further configurations measured (fwd+bwd and merge) after the main one, reported under \"configs\"")
     ap.add_argument("--per-shape", action="store_true", help="diagnostic: time one matrix of each distinct shape and exit")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))

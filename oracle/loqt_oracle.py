@@ -378,8 +378,9 @@ def dq_quantize_absmax(absmax: np.ndarray, offset=None):
     offset: the mean of c2 rounded to fp32 (computed here in float64 unless given;
             any nearby value is a valid encoding parameter, so a caller may pass
             the one another implementation chose).
-    Per block of 256 consecutive scales: d = fl32(c2 - offset); c1 = max |d|;
-    code = E4M3( fl32( fl32(d / c1) * 448 ) ), +0 when c1 = 0.
+    Per block of 256 consecutive scales: d = fl32(c2 - offset); m = max |d|;
+    code = E4M3( fl32( fl32(d / m) * 448 ) ), +0 when m = 0; the stored second-level
+    scale is c1 = fl32(m / 448), the value one E4M3 unit stands for.
     Returns (codes uint8 [n], c1 fp32 [ceil(n / 256)], offset fp32 scalar)."""
     c2 = np.ascontiguousarray(absmax, dtype=np.float32).reshape(-1)
     n = c2.size
@@ -393,7 +394,7 @@ def dq_quantize_absmax(absmax: np.ndarray, offset=None):
     for b in range(nb):
         blk = d[b * DQ_BLOCK : (b + 1) * DQ_BLOCK]
         m = np.float32(np.max(np.abs(blk)))
-        c1[b] = m
+        c1[b] = np.float32(m / np.float32(E4M3_MAX))
         if m > 0:
             t = ((blk / m).astype(np.float32) * np.float32(E4M3_MAX)).astype(np.float32)
             codes[b * DQ_BLOCK : b * DQ_BLOCK + blk.size] = e4m3_encode(t)
@@ -402,10 +403,9 @@ def dq_quantize_absmax(absmax: np.ndarray, offset=None):
 
 def dq_dequantize_absmax(codes: np.ndarray, c1: np.ndarray, offset, shape=None) -> np.ndarray:
     """The scales the layer works with after double quantisation:
-    c2' = fl32( fl32( fl32(E4M3(code) / 448) * c1 ) + offset ), three fp32 roundings
-    in this order (E4M3(code) / 448 is a division by a non-power of two)."""
+    c2' = fl32( fl32( E4M3(code) * c1 ) + offset ), two fp32 roundings."""
     codes = np.asarray(codes, dtype=np.uint8).reshape(-1)
-    q = (e4m3_decode(codes).astype(np.float32) / np.float32(E4M3_MAX)).astype(np.float32)
+    q = e4m3_decode(codes).astype(np.float32)
     scale = np.repeat(np.asarray(c1, dtype=np.float32), DQ_BLOCK)[: codes.size]
     out = ((q * scale).astype(np.float32) + np.float32(offset)).astype(np.float32)
     return out if shape is None else out.reshape(shape)

@@ -56,7 +56,7 @@ def test_round_trip_error_is_within_the_format_bound(n):
     back = O.dq_dequantize_absmax(codes, c1, off)
     d = (c2 - off).astype(np.float64)
     err = np.abs(back.astype(np.float64) - c2.astype(np.float64))
-    scale = np.repeat(c1.astype(np.float64), 256)[:n]
+    scale = np.repeat(c1.astype(np.float64), 256)[:n] * 448.0      # the block's largest centred scale
     # E4M3 keeps 3 mantissa bits: relative half-spacing 2^-4 for normal values, absolute half-spacing
     # 2^-10 below 2^-6 (in units where the block maximum is 448); plus fp32 roundings of the arithmetic
     bound = np.maximum(np.abs(d) * 2.0 ** -4, scale * 2.0 ** -10 / 448.0) + 8 * np.spacing(c2).astype(np.float64)
@@ -77,7 +77,7 @@ def test_representable_scales_round_trip_exactly():
     c2 = np.concatenate([vals, -vals]).astype(np.float32)            # mean exactly 0, max 448
     assert c2.size == 254
     codes, c1, off = O.dq_quantize_absmax(c2)
-    assert off == 0.0 and c1[0] == 448.0
+    assert off == 0.0 and c1[0] == 1.0                             # one E4M3 unit stands for 1.0
     assert np.array_equal(O.dq_dequantize_absmax(codes, c1, off), c2)
     # all-equal scales: everything sits in the offset, codes are +0
     c2 = np.full(300, 0.0371, dtype=np.float32)
