@@ -246,6 +246,50 @@ loqt_status loqt_merge_requant_many(int32_t n, const loqt_nf4_mat *Wq, const loq
                                     size_t ws_bytes, void *stream);
 
 /*
+ * Double quantisation of the block scales (Section 2.4, last paragraph: the
+ * quantiser's own state is quantised a second time, as in QLoRA; the paper gives
+ * no parameters, the scheme taken is QLoRA's: the fp32 scales of a matrix, in row-major order
+ * [rows][ld/64], are centred by their mean and stored as 8-bit floats - OCP FP8
+ * E4M3 - in blocks of 256 with one fp32 second-level scale per block).
+ *   codes8 : [n] bytes, n = rows * ld / 64     c1 : [ceil(n / 256)] fp32
+ *   offset : one fp32 (device memory)          all DEVICE pointers, caller-owned
+ *   encode: offset = mean(c2); per block d = c2 - offset, m = max|d|,
+ *           code = E4M3((d / m) * 448) (nearest, ties to even), c1 = m / 448
+ *   decode: c2' = E4M3(code) * c1 + offset      (each operation rounded to fp32)
+ * Storage per weight: 4 + 8/64 + 32/(64*256) = 4.127 bits instead of 4.5.
+ *
+ * loqt_scales_double_quantize / _dequantize convert between the fp32 scales of
+ * a loqt_nf4_mat and this form (ws: loqt_scales_workspace_bytes() bytes; the
+ * mean is summed in double precision in a fixed order, so results are
+ * reproducible).  loqt_nf4_dequantize_dq, loqt_linear_fwd_dq and
+ * loqt_linear_bwd_dq are loqt_nf4_dequantize, loqt_linear_fwd and
+ * loqt_linear_bwd reading the scales of W_q and P_q from this form inside the
+ * kernels (the absmax pointers of the loqt_nf4_mat arguments are not read and
+ * may be NULL); same arguments, workspaces and error behaviour otherwise.  The
+ * merge works on fp32 scales: expand them, merge, and encode the new ones.
+ */
+typedef struct {
+  uint8_t *codes8;
+  float *c1;
+  float *offset;
+  int64_t n;
+} loqt_dq_scales;
+
+size_t loqt_scales_workspace_bytes(void);
+loqt_status loqt_scales_double_quantize(const float *absmax, loqt_dq_scales dst, void *ws, size_t ws_bytes,
+                                        void *stream);
+loqt_status loqt_scales_double_dequantize(loqt_dq_scales src, float *absmax, void *stream);
+loqt_status loqt_nf4_dequantize_dq(loqt_nf4_mat src, loqt_dq_scales dq, void *dst, int64_t ld_dst,
+                                   int dst_is_bf16, void *stream);
+loqt_status loqt_linear_fwd_dq(loqt_nf4_mat Wq, loqt_dq_scales Wdq, loqt_nf4_mat Pq, loqt_dq_scales Pdq,
+                               const void *B, int64_t ldb, float s, const void *x, int64_t ldx, int32_t T,
+                               void *y, int64_t ldy, void *ws, size_t ws_bytes, void *stream);
+loqt_status loqt_linear_bwd_dq(loqt_nf4_mat Wq, loqt_dq_scales Wdq, loqt_nf4_mat Pq, loqt_dq_scales Pdq,
+                               const void *B, int64_t ldb, float s, const void *x, int64_t ldx,
+                               const void *dy, int64_t lddy, int32_t T, void *dx, int64_t lddx, float *dB,
+                               int64_t lddb, int accumulate_dB, void *ws, size_t ws_bytes, void *stream);
+
+/*
  * Forward for callers that cannot allocate device memory.  (The paper has no
  * counterpart: this is a convenience of this library, not part of the method.)
  *

@@ -27,6 +27,8 @@ EXPORTS = (
     "loqt_linear_fwd_right", "loqt_linear_bwd_right", "loqt_merge_requant_right", "loqt_linear_fwd_static", "loqt_workspace_bytes",
     "loqt_device_status", "loqt_launch_count", "loqt_status_string",
     "loqt_set_tile_override", "loqt_variant_launches", "loqt_selftest_wait_timeout",
+    "loqt_scales_workspace_bytes", "loqt_scales_double_quantize", "loqt_scales_double_dequantize",
+    "loqt_nf4_dequantize_dq", "loqt_linear_fwd_dq", "loqt_linear_bwd_dq",
 )
 
 
@@ -50,6 +52,10 @@ class loqt_nf4_mat(ctypes.Structure):
         ("ld", ctypes.c_int32),
         ("block", ctypes.c_int32),
     ]
+
+
+class loqt_dq_scales(ctypes.Structure):
+    _fields_ = [("codes8", ctypes.c_void_p), ("c1", ctypes.c_void_p), ("offset", ctypes.c_void_p), ("n", ctypes.c_int64)]
 
 
 _lib = None
@@ -100,6 +106,17 @@ def lib():
     L.loqt_variant_launches.restype = ctypes.c_uint64
     L.loqt_selftest_wait_timeout.argtypes = [vp, sz, ctypes.c_uint32, vp]
     L.loqt_selftest_wait_timeout.restype = ctypes.c_int
+    D = loqt_dq_scales
+    L.loqt_scales_workspace_bytes.argtypes = []
+    L.loqt_scales_workspace_bytes.restype = sz
+    L.loqt_scales_double_quantize.argtypes = [vp, D, vp, sz, vp]
+    L.loqt_scales_double_dequantize.argtypes = [D, vp, vp]
+    L.loqt_nf4_dequantize_dq.argtypes = [M, D, vp, i64, ctypes.c_int, vp]
+    L.loqt_linear_fwd_dq.argtypes = [M, D, M, D, vp, i64, f32, vp, i64, i32, vp, i64, vp, sz, vp]
+    L.loqt_linear_bwd_dq.argtypes = [M, D, M, D, vp, i64, f32, vp, i64, vp, i64, i32, vp, i64, vp, i64, ctypes.c_int, vp, sz, vp]
+    for name in ("loqt_scales_double_quantize", "loqt_scales_double_dequantize", "loqt_nf4_dequantize_dq", "loqt_linear_fwd_dq",
+                 "loqt_linear_bwd_dq"):
+        getattr(L, name).restype = ctypes.c_int
     L.loqt_status_string.argtypes = [ctypes.c_int]
     L.loqt_status_string.restype = ctypes.c_char_p
     for name in ("loqt_nf4_quantize", "loqt_nf4_dequantize", "loqt_linear_fwd", "loqt_linear_bwd",
@@ -327,6 +344,79 @@ def loqt_adam_step(B: torch.Tensor, dB: torch.Tensor, m: torch.Tensor, v: torch.
     _check(lib().loqt_adam_step(_dev(B, torch.bfloat16), B.stride(0), _dev(dB, torch.float32), dB.stride(0),
                                 _dev(m, torch.bfloat16), _dev(v, torch.bfloat16), m.stride(0), B.shape[0], B.shape[1], hp,
                                 _stream()), "loqt_adam_step")
+
+
+@dataclass
+class DQScales:
+    """Device storage of the doubly quantised block scales of one NF4 matrix."""
+    codes8: torch.Tensor  # uint8 [n]
+    c1: torch.Tensor      # fp32 [ceil(n / 256)]
+    offset: torch.Tensor  # fp32 [1]
+
+    def view(self) -> loqt_dq_scales:
+        return loqt_dq_scales(self.codes8.data_ptr(), self.c1.data_ptr(), self.offset.data_ptr(), self.codes8.numel())
+
+    @staticmethod
+    def empty(n: int, device="cuda") -> "DQScales":
+        return DQScales(torch.empty((n,), dtype=torch.uint8, device=device),
+                        torch.empty(((n + 255) // 256,), dtype=torch.float32, device=device),
+                        torch.empty((1,), dtype=torch.float32, device=device))
+
+
+def loqt_scales_double_quantize(absmax: torch.Tensor, dst: DQScales | None = None) -> DQScales:
+    """Doubly quantises the fp32 block scales of a matrix (contiguous, row-major)."""
+    if not absmax.is_contiguous():
+        raise LoqtError("the scales must be contiguous")
+    dst = dst if dst is not None else DQScales.empty(absmax.numel(), absmax.device)
+    ws = new_workspace(int(lib().loqt_scales_workspace_bytes()), absmax.device)
+    _check(lib().loqt_scales_double_quantize(_dev(absmax, torch.float32), dst.view(), ws.data_ptr(), ws.numel(), _stream()),
+           "loqt_scales_double_quantize")
+    return dst
+
+
+def loqt_scales_double_dequantize(src: DQScales, shape) -> torch.Tensor:
+    out = torch.empty(shape, dtype=torch.float32, device=src.codes8.device)
+    _check(lib().loqt_scales_double_dequantize(src.view(), out.data_ptr(), _stream()), "loqt_scales_double_dequantize")
+    return out
+
+
+def _codes_only(q: NF4Tensor) -> loqt_nf4_mat:
+    return loqt_nf4_mat(q.codes.data_ptr(), None, q.rows, q.cols, q.ld, BLOCK)
+
+
+def loqt_nf4_dequantize_dq(src: NF4Tensor, dq: DQScales, dtype=torch.float32) -> torch.Tensor:
+    dst = torch.empty((src.rows, src.cols), dtype=dtype, device=src.codes.device)
+    is_bf16 = {torch.float32: 0, torch.bfloat16: 1}[dtype]
+    _check(lib().loqt_nf4_dequantize_dq(_codes_only(src), dq.view(), _dev(dst), dst.stride(0), is_bf16, _stream()),
+           "loqt_nf4_dequantize_dq")
+    return dst
+
+
+def loqt_linear_fwd_dq(Wq: NF4Tensor, Wdq: DQScales, Pq: NF4Tensor, Pdq: DQScales, B: torch.Tensor, s: float, x: torch.Tensor,
+                       y: torch.Tensor | None = None) -> torch.Tensor:
+    T = x.shape[0]
+    if y is None:
+        y = torch.empty((T, (Wq.rows + 7) // 8 * 8), dtype=torch.bfloat16, device=x.device)[:, : Wq.rows]
+    ws = new_workspace(loqt_workspace_bytes(LOQT_OP_FWD, Wq.rows, Wq.cols, Pq.cols, T), x.device)
+    _check(lib().loqt_linear_fwd_dq(_codes_only(Wq), Wdq.view(), _codes_only(Pq), Pdq.view(), _dev(B, torch.bfloat16), B.stride(0),
+                                    float(s), _dev(x, torch.bfloat16), x.stride(0), T, _dev(y, torch.bfloat16), y.stride(0),
+                                    ws.data_ptr(), ws.numel(), _stream()), "loqt_linear_fwd_dq")
+    loqt_device_status(ws)
+    return y
+
+
+def loqt_linear_bwd_dq(Wq: NF4Tensor, Wdq: DQScales, Pq: NF4Tensor, Pdq: DQScales, B: torch.Tensor, s: float, x: torch.Tensor,
+                       dy: torch.Tensor):
+    T = x.shape[0]
+    dx = torch.empty((T, (Wq.cols + 7) // 8 * 8), dtype=torch.bfloat16, device=x.device)[:, : Wq.cols]
+    dB = torch.empty((Pq.cols, (Wq.cols + 3) // 4 * 4), dtype=torch.float32, device=x.device)[:, : Wq.cols]
+    ws = new_workspace(loqt_workspace_bytes(LOQT_OP_BWD, Wq.rows, Wq.cols, Pq.cols, T), x.device)
+    _check(lib().loqt_linear_bwd_dq(_codes_only(Wq), Wdq.view(), _codes_only(Pq), Pdq.view(), _dev(B, torch.bfloat16), B.stride(0),
+                                    float(s), _dev(x, torch.bfloat16), x.stride(0), _dev(dy, torch.bfloat16), dy.stride(0), T,
+                                    dx.data_ptr(), dx.stride(0), dB.data_ptr(), dB.stride(0), 0, ws.data_ptr(), ws.numel(),
+                                    _stream()), "loqt_linear_bwd_dq")
+    loqt_device_status(ws)
+    return dx, dB
 
 
 def merge_many_workspace_bytes(Wqs, Pqs, group: int = 8) -> int:

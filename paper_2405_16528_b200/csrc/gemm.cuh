@@ -61,10 +61,15 @@ enum : int {
   EPI_PARTIAL = 2,  // partial[split] fp32 = D                        (splits > 1)
 };
 
+// absmax: the fp32 block scales, or null when the scales are doubly quantised
+// (paper Section 2.4): then scale i = fl32(fl32(E4M3(absmax8[i]) * c1[i / 256]) + *offset).
 struct Nf4Src {
   const uint8_t *codes;
   const float *absmax;
   int rows, cols, ld;
+  const uint8_t *absmax8;
+  const float *c1;
+  const float *offset;
 };
 
 struct Segment {
@@ -199,8 +204,12 @@ struct DeqGeom {
   uint32_t dst;        // byte offset of the 128-byte operand row inside the stage
   uint32_t sw;         // row index & 7 (swizzle key of the operand row)
   int active;          // 0: this thread has no row inside the matrix (outputs it would feed are discarded)
-  const float *mptr;   // block scale of k-block 0 of the segment
-  int mstride;         // floats between consecutive k-blocks
+  const float *mptr;   // block scale of k-block 0 of the segment (fp32 scales)
+  int64_t midx;        // its index in the matrix's sequence of scales (doubly quantised scales)
+  const uint8_t *m8;   // doubly quantised scales: codes, second-level scales, offset (null otherwise)
+  const float *c1;
+  const float *off;
+  int mstride;         // scales between consecutive k-blocks
   int kb_valid;        // k-blocks of the segment for which the row exists; later ones are the K tail (zeros)
   // A thread of a 256-row tile owns a second block, 128 tasks further on: the same
   // geometry shifted by constant offsets.
@@ -223,6 +232,10 @@ __device__ __forceinline__ DeqGeom deq_geom(const GemmParams &p, int seg_idx, in
   g.src = g.src2 = g.dst = g.sw = 0;
   g.active = 0;
   g.mptr = nullptr;
+  g.midx = 0;
+  g.m8 = nullptr;
+  g.c1 = nullptr;
+  g.off = nullptr;
   g.mstride = 0;
   g.kb_valid = 0;
   g.active2 = g.kb_valid2 = 0;
@@ -248,7 +261,7 @@ __device__ __forceinline__ DeqGeom deq_geom(const GemmParams &p, int seg_idx, in
     g.src2 = g.src + 16;
     if (row >= src.rows) return g;
     g.active = 1;
-    g.mptr = src.absmax + static_cast<int64_t>(row) * nb;
+    g.midx = static_cast<int64_t>(row) * nb;
     g.mstride = 1;
     g.kb_valid = 0x7fffffff;  // padded columns hold the zero level
     // second block: tile row t + 128
@@ -278,7 +291,7 @@ __device__ __forceinline__ DeqGeom deq_geom(const GemmParams &p, int seg_idx, in
     g.src2 = o1 ^ (((o1 >> 7) & mask) << 4);
     if (col0 >= src.ld) return g;
     g.active = 1;
-    g.mptr = src.absmax + static_cast<int64_t>(kk) * nb + (col0 >> 6);
+    g.midx = static_cast<int64_t>(kk) * nb + (col0 >> 6);
     g.mstride = 64 * nb;
     g.kb_valid = src.rows > kk ? (src.rows - kk + 63) >> 6 : 0;  // beyond: the K tail must contribute zero
     // second block (256-row tiles only): same chunk, K-row kk + 32
@@ -287,6 +300,13 @@ __device__ __forceinline__ DeqGeom deq_geom(const GemmParams &p, int seg_idx, in
     g.d2 = 4u * 1024u;
     g.s2 = 32u * RB;
     g.m2 = 32 * nb;
+  }
+  if (src.absmax != nullptr) {
+    g.mptr = src.absmax + g.midx;
+  } else {
+    g.m8 = src.absmax8;
+    g.c1 = src.c1;
+    g.off = src.offset;
   }
   return g;
 }
@@ -298,7 +318,11 @@ __device__ __forceinline__ DeqTask deq_fetch(const DeqGeom &g, int kb_in_seg) {
   const int active = kSecond ? g.active2 : g.active;
   const int valid = kSecond ? g.kb_valid2 : g.kb_valid;
   task.mode = !active ? 0 : (kb_in_seg < valid ? 1 : 2);
-  if (task.mode == 1) task.M = __ldg(g.mptr + static_cast<int64_t>(kb_in_seg) * g.mstride + (kSecond ? g.m2 : 0));
+  if (task.mode == 1) {
+    const int64_t rel = static_cast<int64_t>(kb_in_seg) * g.mstride + (kSecond ? g.m2 : 0);
+    if (g.m8 == nullptr) task.M = __ldg(g.mptr + rel);
+    else task.M = dq_scale(g.m8, g.c1, g.off, g.midx + rel);
+  }
   return task;
 }
 

@@ -67,7 +67,11 @@ static bool map_operand(CUtensorMap *map, int kind, const Bf16Operand &op, int r
   return make_map(map, op.ptr, rows, K, op.ld, 64, kBK);
 }
 
-static Nf4Src nf4_src(const loqt_nf4_mat &m) { return Nf4Src{m.codes, m.absmax, m.rows, m.cols, m.ld}; }
+static Nf4Src nf4_src(const loqt_nf4_mat &m) { return Nf4Src{m.codes, m.absmax, m.rows, m.cols, m.ld, nullptr, nullptr, nullptr}; }
+// The same matrix with doubly quantised scales (m.absmax is not used).
+static Nf4Src nf4_src_dq(const loqt_nf4_mat &m, const loqt_dq_scales &dq) {
+  return Nf4Src{m.codes, nullptr, m.rows, m.cols, m.ld, dq.codes8, dq.c1, dq.offset};
+}
 
 static loqt_status check_bf16(const void *p, int64_t ld, int64_t cols) {
   if (p == nullptr || ld < cols) return LOQT_ERR_INVALID_ARG;
@@ -367,12 +371,11 @@ static loqt_status check_fwd_args(const loqt_nf4_mat &Wq, const loqt_nf4_mat &Pq
   return check_bf16(y, ldy, Wq.rows);
 }
 
-extern "C" loqt_status loqt_linear_fwd(loqt_nf4_mat Wq, loqt_nf4_mat Pq, const void *B, int64_t ldb, float s,
-                                       const void *x, int64_t ldx, int32_t T, void *y, int64_t ldy, void *ws,
-                                       size_t ws_bytes, void *stream) {
+// Forward with both NF4 operands given as engine sources (fp32 or doubly quantised scales).
+static loqt_status fwd_impl(const Nf4Src &W, const Nf4Src &P, const void *B, int64_t ldb, float s, const void *x, int64_t ldx,
+                            int32_t T, void *y, int64_t ldy, void *ws, size_t ws_bytes, void *stream) {
   loqt_status st;
-  if ((st = check_fwd_args(Wq, Pq, B, ldb, x, ldx, T, y, ldy)) != LOQT_OK) return st;
-  const int out = Wq.rows, in = Wq.cols, r = Pq.cols;
+  const int out = W.rows, in = W.cols, r = P.cols;
   if ((st = check_ws(ws, ws_bytes, loqt_workspace_bytes(LOQT_OP_FWD, out, in, r, T))) != LOQT_OK) return st;
   if ((st = check_arch()) != LOQT_OK) return st;
   cudaStream_t stm = static_cast<cudaStream_t>(stream);
@@ -392,27 +395,42 @@ extern "C" loqt_status loqt_linear_fwd(loqt_nf4_mat Wq, loqt_nf4_mat Pq, const v
   // y = x deq(W_q)^T + u deq(P_q)^T    (K = in, then K = r, one accumulator)
   GemmCall c2{};
   c2.p.M = T; c2.p.N = out; c2.p.num_segs = 2;
-  c2.p.seg[0].K = in; c2.p.seg[0].a_kind = OP_TMA_K; c2.p.seg[0].b_kind = OP_NF4_K; c2.p.seg[0].b_nf4 = nf4_src(Wq);
-  c2.p.seg[1].K = r; c2.p.seg[1].a_kind = OP_TMA_K; c2.p.seg[1].b_kind = OP_NF4_K; c2.p.seg[1].b_nf4 = nf4_src(Pq);
+  c2.p.seg[0].K = in; c2.p.seg[0].a_kind = OP_TMA_K; c2.p.seg[0].b_kind = OP_NF4_K; c2.p.seg[0].b_nf4 = W;
+  c2.p.seg[1].K = r; c2.p.seg[1].a_kind = OP_TMA_K; c2.p.seg[1].b_kind = OP_NF4_K; c2.p.seg[1].b_nf4 = P;
   c2.a[0] = {x, ldx}; c2.a[1] = {u, ldu};
   c2.p.splits = 1;
   c2.p.epi = EPI_BF16; c2.p.out = y; c2.p.ld_out = ldy; c2.p.alpha = 1.0f; c2.p.status = status;
   return launch(c2, stm);
 }
 
-extern "C" loqt_status loqt_linear_bwd(loqt_nf4_mat Wq, loqt_nf4_mat Pq, const void *B, int64_t ldb, float s,
-                                       const void *x, int64_t ldx, const void *dy, int64_t lddy, int32_t T, void *dx,
-                                       int64_t lddx, float *dB, int64_t lddb, int accumulate_dB, void *ws,
+extern "C" loqt_status loqt_linear_fwd(loqt_nf4_mat Wq, loqt_nf4_mat Pq, const void *B, int64_t ldb, float s,
+                                       const void *x, int64_t ldx, int32_t T, void *y, int64_t ldy, void *ws,
                                        size_t ws_bytes, void *stream) {
+  loqt_status st;
+  if ((st = check_fwd_args(Wq, Pq, B, ldb, x, ldx, T, y, ldy)) != LOQT_OK) return st;
+  return fwd_impl(nf4_src(Wq), nf4_src(Pq), B, ldb, s, x, ldx, T, y, ldy, ws, ws_bytes, stream);
+}
+
+// Argument checks of the backward, shared by its entry points.
+static loqt_status check_bwd_args(const loqt_nf4_mat &Wq, const loqt_nf4_mat &Pq, const void *B, int64_t ldb, const void *x,
+                                  int64_t ldx, const void *dy, int64_t lddy, int32_t T, const void *dx, int64_t lddx,
+                                  const float *dB, int64_t lddb) {
   loqt_status st;
   if ((st = check_layer(Wq, Pq, B, ldb)) != LOQT_OK) return st;
   if (T <= 0) return LOQT_ERR_INVALID_ARG;
-  const int out = Wq.rows, in = Wq.cols, r = Pq.cols;
-  if ((st = check_bf16(x, ldx, in)) != LOQT_OK) return st;
-  if ((st = check_bf16(dy, lddy, out)) != LOQT_OK) return st;
-  if (dx != nullptr && (st = check_bf16(dx, lddx, in)) != LOQT_OK) return st;
-  if (dB == nullptr || lddb < in) return LOQT_ERR_INVALID_ARG;
+  if ((st = check_bf16(x, ldx, Wq.cols)) != LOQT_OK) return st;
+  if ((st = check_bf16(dy, lddy, Wq.rows)) != LOQT_OK) return st;
+  if (dx != nullptr && (st = check_bf16(dx, lddx, Wq.cols)) != LOQT_OK) return st;
+  if (dB == nullptr || lddb < Wq.cols) return LOQT_ERR_INVALID_ARG;
   if ((reinterpret_cast<uintptr_t>(dB) & 15u) != 0) return LOQT_ERR_ALIGNMENT;
+  return LOQT_OK;
+}
+
+static loqt_status bwd_impl(const Nf4Src &W, const Nf4Src &P, const void *B, int64_t ldb, float s, const void *x, int64_t ldx,
+                            const void *dy, int64_t lddy, int32_t T, void *dx, int64_t lddx, float *dB, int64_t lddb,
+                            int accumulate_dB, void *ws, size_t ws_bytes, void *stream) {
+  loqt_status st;
+  const int out = W.rows, in = W.cols, r = P.cols;
   if ((st = check_ws(ws, ws_bytes, loqt_workspace_bytes(LOQT_OP_BWD, out, in, r, T))) != LOQT_OK) return st;
   if ((st = check_arch()) != LOQT_OK) return st;
   cudaStream_t stm = static_cast<cudaStream_t>(stream);
@@ -424,7 +442,7 @@ extern "C" loqt_status loqt_linear_bwd(loqt_nf4_mat Wq, loqt_nf4_mat Pq, const v
   // v' = s * dy deq(P_q)      (T x r; K = out; P_q read with its blocks along N = r)
   GemmCall c1{};
   c1.p.M = T; c1.p.N = r; c1.p.num_segs = 1;
-  c1.p.seg[0].K = out; c1.p.seg[0].a_kind = OP_TMA_K; c1.p.seg[0].b_kind = OP_NF4_MN; c1.p.seg[0].b_nf4 = nf4_src(Pq);
+  c1.p.seg[0].K = out; c1.p.seg[0].a_kind = OP_TMA_K; c1.p.seg[0].b_kind = OP_NF4_MN; c1.p.seg[0].b_nf4 = P;
   c1.a[0] = {dy, lddy};
   c1.p.splits = 1;
   c1.p.epi = EPI_BF16; c1.p.out = v; c1.p.ld_out = ldv; c1.p.alpha = s; c1.p.status = status;
@@ -434,7 +452,7 @@ extern "C" loqt_status loqt_linear_bwd(loqt_nf4_mat Wq, loqt_nf4_mat Pq, const v
   if (dx != nullptr) {
     GemmCall c2{};
     c2.p.M = T; c2.p.N = in; c2.p.num_segs = 2;
-    c2.p.seg[0].K = out; c2.p.seg[0].a_kind = OP_TMA_K; c2.p.seg[0].b_kind = OP_NF4_MN; c2.p.seg[0].b_nf4 = nf4_src(Wq);
+    c2.p.seg[0].K = out; c2.p.seg[0].a_kind = OP_TMA_K; c2.p.seg[0].b_kind = OP_NF4_MN; c2.p.seg[0].b_nf4 = W;
     c2.p.seg[1].K = r; c2.p.seg[1].a_kind = OP_TMA_K; c2.p.seg[1].b_kind = OP_TMA_MN;
     c2.a[0] = {dy, lddy}; c2.a[1] = {v, ldv}; c2.b[1] = {B, ldb};
     c2.p.splits = 1;
@@ -444,6 +462,56 @@ extern "C" loqt_status loqt_linear_bwd(loqt_nf4_mat Wq, loqt_nf4_mat Pq, const v
 
   // dB = v'^T x               (r x in; K = T; both operands stored K-outermost)
   return gemm_tn_f32(v, ldv, x, ldx, r, in, T, dB, lddb, accumulate_dB, partial, status, stm);
+}
+
+extern "C" loqt_status loqt_linear_bwd(loqt_nf4_mat Wq, loqt_nf4_mat Pq, const void *B, int64_t ldb, float s,
+                                       const void *x, int64_t ldx, const void *dy, int64_t lddy, int32_t T, void *dx,
+                                       int64_t lddx, float *dB, int64_t lddb, int accumulate_dB, void *ws,
+                                       size_t ws_bytes, void *stream) {
+  loqt_status st;
+  if ((st = check_bwd_args(Wq, Pq, B, ldb, x, ldx, dy, lddy, T, dx, lddx, dB, lddb)) != LOQT_OK) return st;
+  return bwd_impl(nf4_src(Wq), nf4_src(Pq), B, ldb, s, x, ldx, dy, lddy, T, dx, lddx, dB, lddb, accumulate_dB, ws, ws_bytes,
+                  stream);
+}
+
+// ---------------------------------------------------------------------------
+// The layer with doubly quantised block scales (Section 2.4: the quantisation state
+// is itself quantised).  The operand staging decodes each block's scale from its
+// 8-bit code; everything else is the forward / backward above.
+// ---------------------------------------------------------------------------
+static loqt_status check_dq(const loqt_nf4_mat &m, const loqt_dq_scales &dq) {
+  if (dq.codes8 == nullptr || dq.c1 == nullptr || dq.offset == nullptr) return LOQT_ERR_INVALID_ARG;
+  if (dq.n != static_cast<int64_t>(m.rows) * (m.ld / kBlock)) return LOQT_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(dq.c1) & 3u) != 0 || (reinterpret_cast<uintptr_t>(dq.offset) & 3u) != 0) return LOQT_ERR_ALIGNMENT;
+  return LOQT_OK;
+}
+// validate_nf4 insists on fp32 scales; a doubly quantised view passes with any non-null stand-in
+static loqt_nf4_mat with_stand_in_scales(loqt_nf4_mat m, const loqt_dq_scales &dq) {
+  if (m.absmax == nullptr) m.absmax = dq.c1;
+  return m;
+}
+
+extern "C" loqt_status loqt_linear_fwd_dq(loqt_nf4_mat Wq, loqt_dq_scales Wdq, loqt_nf4_mat Pq, loqt_dq_scales Pdq, const void *B,
+                                          int64_t ldb, float s, const void *x, int64_t ldx, int32_t T, void *y, int64_t ldy,
+                                          void *ws, size_t ws_bytes, void *stream) {
+  loqt_status st;
+  if ((st = check_fwd_args(with_stand_in_scales(Wq, Wdq), with_stand_in_scales(Pq, Pdq), B, ldb, x, ldx, T, y, ldy)) != LOQT_OK)
+    return st;
+  if ((st = check_dq(Wq, Wdq)) != LOQT_OK || (st = check_dq(Pq, Pdq)) != LOQT_OK) return st;
+  return fwd_impl(nf4_src_dq(Wq, Wdq), nf4_src_dq(Pq, Pdq), B, ldb, s, x, ldx, T, y, ldy, ws, ws_bytes, stream);
+}
+
+extern "C" loqt_status loqt_linear_bwd_dq(loqt_nf4_mat Wq, loqt_dq_scales Wdq, loqt_nf4_mat Pq, loqt_dq_scales Pdq, const void *B,
+                                          int64_t ldb, float s, const void *x, int64_t ldx, const void *dy, int64_t lddy,
+                                          int32_t T, void *dx, int64_t lddx, float *dB, int64_t lddb, int accumulate_dB, void *ws,
+                                          size_t ws_bytes, void *stream) {
+  loqt_status st;
+  if ((st = check_bwd_args(with_stand_in_scales(Wq, Wdq), with_stand_in_scales(Pq, Pdq), B, ldb, x, ldx, dy, lddy, T, dx, lddx, dB,
+                           lddb)) != LOQT_OK)
+    return st;
+  if ((st = check_dq(Wq, Wdq)) != LOQT_OK || (st = check_dq(Pq, Pdq)) != LOQT_OK) return st;
+  return bwd_impl(nf4_src_dq(Wq, Wdq), nf4_src_dq(Pq, Pdq), B, ldb, s, x, ldx, dy, lddy, T, dx, lddx, dB, lddb, accumulate_dB, ws,
+                  ws_bytes, stream);
 }
 
 // ---------------------------------------------------------------------------

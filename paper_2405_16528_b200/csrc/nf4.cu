@@ -162,10 +162,18 @@ nf4_quantize_kernel(const float *__restrict__ src, int64_t ld_src, float s, uint
 constexpr int kDqUnroll = 4;
 
 // Expands the code words first, first + stride, ... of one matrix.
-template <bool kBf16, bool kVec>
+// Doubly quantised scales of a matrix (null codes8: plain fp32 scales are used).
+struct DqScales {
+  const uint8_t *codes8;
+  const float *c1;
+  const float *offset;
+};
+
+template <bool kBf16, bool kVec, bool kDq = false>
 __device__ __forceinline__ void dequantize_words(const Nf4Tables &tab, const uint8_t *__restrict__ codes,
                                                  const float *__restrict__ absmax, void *__restrict__ dst, int64_t ld_dst,
-                                                 int rows, int cols, int ld, uint32_t first, uint32_t stride) {
+                                                 int rows, int cols, int ld, uint32_t first, uint32_t stride,
+                                                 DqScales dq = DqScales{nullptr, nullptr, nullptr}) {
   const uint32_t wpr = static_cast<uint32_t>(ld / 8);  // code words per row
   const uint32_t nb = static_cast<uint32_t>(ld / kBlock);
   const uint32_t n_items = static_cast<uint32_t>(rows) * wpr;  // (host checks < 2^31)
@@ -187,7 +195,8 @@ __device__ __forceinline__ void dequantize_words(const Nf4Tables &tab, const uin
     q.M = 0.0f;
     if (q.live) {
       q.w = __ldg(reinterpret_cast<const uint32_t *>(codes + static_cast<int64_t>(q.row) * (ld / 2)) + h);
-      q.M = __ldg(absmax + static_cast<int64_t>(q.row) * nb + (h >> 3));
+      const int64_t si = static_cast<int64_t>(q.row) * nb + (h >> 3);
+      q.M = kDq ? dq_scale(dq.codes8, dq.c1, dq.offset, si) : __ldg(absmax + si);
     }
     return q;
   };
@@ -248,6 +257,18 @@ nf4_dequantize_kernel(const uint8_t *__restrict__ codes, const float *__restrict
   __syncthreads();
   dequantize_words<kBf16, kVec>(tab, codes, absmax, dst, ld_dst, rows, cols, ld, blockIdx.x * kQThreads + threadIdx.x,
                                 gridDim.x * kQThreads);
+}
+
+// The same with doubly quantised block scales (paper Section 2.4).
+template <bool kBf16, bool kVec>
+__global__ void __launch_bounds__(kQThreads)
+nf4_dequantize_dq_kernel(const uint8_t *__restrict__ codes, DqScales dq, void *__restrict__ dst, int64_t ld_dst, int rows,
+                         int cols, int ld) {
+  __shared__ Nf4Tables tab;
+  nf4_tables_init(tab, threadIdx.x);
+  __syncthreads();
+  dequantize_words<kBf16, kVec, true>(tab, codes, nullptr, dst, ld_dst, rows, cols, ld, blockIdx.x * kQThreads + threadIdx.x,
+                                      gridDim.x * kQThreads, dq);
 }
 
 // Several matrices to bf16 in one launch (the staging step of a batched merge):
@@ -417,6 +438,28 @@ extern "C" loqt_status loqt_nf4_requantize(const float *delta, int64_t ld_delta,
   auto kernel = vec ? nf4_quantize_kernel<true, kRequantise> : nf4_quantize_kernel<false, kRequantise>;
   kernel<<<grid_for(kernel, items * 4), kQThreads, 0, stm>>>(delta, ld_delta, s, Wq.codes, Wq.absmax, Wq.rows, Wq.cols, Wq.ld, nullptr, 0,
                                                              nullptr, 0);
+  count_launch();
+  return cudaGetLastError() == cudaSuccess ? LOQT_OK : LOQT_ERR_CUDA;
+}
+
+extern "C" loqt_status loqt_nf4_dequantize_dq(loqt_nf4_mat src, loqt_dq_scales dq, void *dst, int64_t ld_dst, int dst_is_bf16,
+                                              void *stream) {
+  if (dq.codes8 == nullptr || dq.c1 == nullptr || dq.offset == nullptr) return LOQT_ERR_INVALID_ARG;
+  if (src.absmax == nullptr) src.absmax = dq.c1;  // (not read: the scales come from dq)
+  loqt_status st = validate_nf4(src);
+  if (st != LOQT_OK) return st;
+  if (dq.n != static_cast<int64_t>(src.rows) * (src.ld / kBlock)) return LOQT_ERR_INVALID_ARG;
+  if (dst == nullptr || ld_dst < src.cols) return LOQT_ERR_INVALID_ARG;
+  const uintptr_t a = reinterpret_cast<uintptr_t>(dst);
+  if ((a & (dst_is_bf16 ? 1u : 3u)) != 0) return LOQT_ERR_ALIGNMENT;
+  if ((st = check_arch()) != LOQT_OK) return st;
+  const int64_t items = static_cast<int64_t>(src.rows) * (src.ld / 8);
+  if (items >= (1ll << 31)) return LOQT_ERR_UNSUPPORTED;
+  const bool vec = (a & 15u) == 0 && (ld_dst % (dst_is_bf16 ? 8 : 4)) == 0;
+  auto kernel = dst_is_bf16 ? (vec ? nf4_dequantize_dq_kernel<true, true> : nf4_dequantize_dq_kernel<true, false>)
+                            : (vec ? nf4_dequantize_dq_kernel<false, true> : nf4_dequantize_dq_kernel<false, false>);
+  kernel<<<grid_for(kernel, (items + kDqUnroll - 1) / kDqUnroll), kQThreads, 0, static_cast<cudaStream_t>(stream)>>>(
+      src.codes, DqScales{dq.codes8, dq.c1, dq.offset}, dst, ld_dst, src.rows, src.cols, src.ld);
   count_launch();
   return cudaGetLastError() == cudaSuccess ? LOQT_OK : LOQT_ERR_CUDA;
 }
