@@ -235,6 +235,31 @@ loqt_status loqt_adam_step(void *B, int64_t ldb, const float *dB, int64_t lddb, 
                            int64_t ld_state, int32_t r, int32_t in, loqt_adam_params hp, void *stream);
 
 /*
+ * The same step with the two moments held in 8 bits (the paper trains B with
+ * "8-bit Adam": memory comparison of Section 3.2, the 13B run, the continued
+ * pretraining appendix; it cites Dettmers et al., "8-bit Optimizers via Block-wise
+ * Quantization", whose scheme is taken).  The row-major flattened r x in moments
+ * are cut into blocks of 2048 elements; each block has one fp32 scale (its largest
+ * magnitude) and one code per element in the dynamic tree data type: bit 7 sign,
+ * then a run of E zero bits (a base-10 exponent), an indicator bit and f fraction
+ * bits j: magnitude = 10^-E (0.1 + 0.9 (j + 1) / 2^f) times the block scale; code 0
+ * is zero.  The non-negative second moment uses bit 7 as a further fraction bit.
+ *   st.m8, st.v8 : uint8 [r * in] codes;  st.m_absmax, st.v_absmax : fp32 [ceil(r * in / 2048)]
+ *   (all zero before the first step).  B, dB, hp as for loqt_adam_step.
+ * Per block: dequantise, Adam update in fp32 (as loqt_adam_step), new block
+ * scales, nearest-magnitude quantisation of the new moments.
+ */
+typedef struct {
+  uint8_t *m8;
+  float *m_absmax;
+  uint8_t *v8;
+  float *v_absmax;
+} loqt_adam8_state;
+
+loqt_status loqt_adam8_step(void *B, int64_t ldb, const float *dB, int64_t lddb, loqt_adam8_state st,
+                            int32_t r, int32_t in, loqt_adam_params hp, void *stream);
+
+/*
  * The same merge for n independent matrices in one call (a whole model at a
  * merge step).  Wq, Pq, B, ldb are HOST arrays of length n; the workspace is
  * shared and must satisfy the largest matrix.  A workspace of 256 + k times the

@@ -28,7 +28,7 @@ EXPORTS = (
     "loqt_device_status", "loqt_launch_count", "loqt_status_string",
     "loqt_set_tile_override", "loqt_variant_launches", "loqt_selftest_wait_timeout",
     "loqt_scales_workspace_bytes", "loqt_scales_double_quantize", "loqt_scales_double_dequantize",
-    "loqt_nf4_dequantize_dq", "loqt_linear_fwd_dq", "loqt_linear_bwd_dq",
+    "loqt_nf4_dequantize_dq", "loqt_linear_fwd_dq", "loqt_linear_bwd_dq", "loqt_adam8_step",
 )
 
 
@@ -52,6 +52,10 @@ class loqt_nf4_mat(ctypes.Structure):
         ("ld", ctypes.c_int32),
         ("block", ctypes.c_int32),
     ]
+
+
+class loqt_adam8_state(ctypes.Structure):
+    _fields_ = [("m8", ctypes.c_void_p), ("m_absmax", ctypes.c_void_p), ("v8", ctypes.c_void_p), ("v_absmax", ctypes.c_void_p)]
 
 
 class loqt_dq_scales(ctypes.Structure):
@@ -117,6 +121,8 @@ def lib():
     for name in ("loqt_scales_double_quantize", "loqt_scales_double_dequantize", "loqt_nf4_dequantize_dq", "loqt_linear_fwd_dq",
                  "loqt_linear_bwd_dq"):
         getattr(L, name).restype = ctypes.c_int
+    L.loqt_adam8_step.argtypes = [vp, i64, vp, i64, loqt_adam8_state, i32, i32, loqt_adam_params, vp]
+    L.loqt_adam8_step.restype = ctypes.c_int
     L.loqt_status_string.argtypes = [ctypes.c_int]
     L.loqt_status_string.restype = ctypes.c_char_p
     for name in ("loqt_nf4_quantize", "loqt_nf4_dequantize", "loqt_linear_fwd", "loqt_linear_bwd",
@@ -417,6 +423,20 @@ def loqt_linear_bwd_dq(Wq: NF4Tensor, Wdq: DQScales, Pq: NF4Tensor, Pdq: DQScale
                                     _stream()), "loqt_linear_bwd_dq")
     loqt_device_status(ws)
     return dx, dB
+
+
+def loqt_adam8_step(B: torch.Tensor, dB: torch.Tensor, m8: torch.Tensor, m_absmax: torch.Tensor, v8: torch.Tensor,
+                    v_absmax: torch.Tensor, step: int, lr: float, beta1: float = 0.9, beta2: float = 0.999, eps: float = 1e-8,
+                    weight_decay: float = 0.0) -> None:
+    """In-place optimiser step on B (bf16) with 8-bit block-wise quantised moments
+    (m8, v8: uint8 [r * in]; m_absmax, v_absmax: fp32 [ceil(r * in / 2048)])."""
+    n = B.shape[0] * B.shape[1]
+    if m8.numel() != n or v8.numel() != n or m_absmax.numel() != (n + 2047) // 2048 or v_absmax.numel() != (n + 2047) // 2048:
+        raise LoqtError("moment buffers do not match the shape of B")
+    hp = loqt_adam_params(lr, beta1, beta2, eps, weight_decay, int(step))
+    st = loqt_adam8_state(_dev(m8, torch.uint8), _dev(m_absmax, torch.float32), _dev(v8, torch.uint8), _dev(v_absmax, torch.float32))
+    _check(lib().loqt_adam8_step(_dev(B, torch.bfloat16), B.stride(0), _dev(dB, torch.float32), dB.stride(0), st,
+                                 B.shape[0], B.shape[1], hp, _stream()), "loqt_adam8_step")
 
 
 def merge_many_workspace_bytes(Wqs, Pqs, group: int = 8) -> int:
