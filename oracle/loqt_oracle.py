@@ -509,3 +509,44 @@ def adam8_step(B, g, m8, m_absmax, v8, v_absmax, step, lr, beta1=0.9, beta2=0.99
     mq = dyn8_quantize(m64.astype(np.float32).reshape(-1), True)
     vq = dyn8_quantize(v64.astype(np.float32).reshape(-1), False)
     return bf16_round(Bn.astype(np.float32)), mq[0], mq[1], vq[0], vq[1]
+
+
+# ----------------------------------------------------------------------------
+# The projection P from the full-rank gradient  (Section 2, first paragraph, and
+# Algorithm 2, the SVD lines: P = the first r columns of U in G^W = U S V^T)
+# ----------------------------------------------------------------------------
+def top_r_left_subspace(G: np.ndarray, r: int) -> np.ndarray:
+    """The definition: the r left singular vectors of G with the largest singular
+    values, as the columns of an out x r matrix (numpy's SVD, float64).  Only the
+    spanned subspace is unique (signs, and rotations inside groups of equal
+    singular values, are not)."""
+    U, _, _ = np.linalg.svd(np.asarray(G, dtype=np.float64), full_matrices=False)
+    return U[:, :r]
+
+
+def subspace_iteration(G: np.ndarray, Omega: np.ndarray, iters: int) -> np.ndarray:
+    """An approximation of that subspace by randomised subspace iteration (Halko,
+    Martinsson and Tropp, "Finding structure with randomness", Algorithm 4.4),
+    the route a GPU takes because it consists of matrix products and the
+    orthonormalisation of tall thin matrices:
+
+        Q = orth(G Omega);  repeat iters times:  Z = orth(G^T Q);  Q = orth(G Z)
+
+    Omega: in x r test matrix (the random numbers are an input).  orth() is the Q
+    factor of numpy's QR.  float64 throughout.  Returns Q, out x r with orthonormal
+    columns; its span tends to the top-r left singular subspace as iters grows, at
+    the rate (sigma_{r+1} / sigma_r)^(2 iters + 1)."""
+    G = np.asarray(G, dtype=np.float64)
+    Q, _ = np.linalg.qr(G @ np.asarray(Omega, dtype=np.float64))
+    for _ in range(int(iters)):
+        Z, _ = np.linalg.qr(G.T @ Q)
+        Q, _ = np.linalg.qr(G @ Z)
+    return Q
+
+
+def subspace_sines(P: np.ndarray, Q: np.ndarray) -> np.ndarray:
+    """Sines of the principal angles between the column spaces of P and Q (both
+    with orthonormal columns): the singular values of (I - P P^T) Q."""
+    P = np.asarray(P, dtype=np.float64)
+    Q = np.asarray(Q, dtype=np.float64)
+    return np.linalg.svd(Q - P @ (P.T @ Q), compute_uv=False)
