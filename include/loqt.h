@@ -44,7 +44,8 @@ typedef enum {
   LOQT_ERR_WORKSPACE = 4,   /* workspace missing or smaller than required          */
   LOQT_ERR_CUDA = 5,        /* a CUDA runtime / driver call failed                 */
   LOQT_ERR_TIMEOUT = 6,     /* a bounded device-side wait expired                  */
-  LOQT_ERR_ARCH = 7         /* current device is not compute capability 10.x       */
+  LOQT_ERR_ARCH = 7,        /* current device is not compute capability 10.x       */
+  LOQT_ERR_NUMERIC = 8      /* loqt_projection: an iterate was rank deficient to working precision */
 } loqt_status;
 
 /*
@@ -70,7 +71,7 @@ typedef struct {
 
 /* Operation selector for loqt_workspace_bytes(). */
 enum { LOQT_OP_FWD = 0, LOQT_OP_BWD = 1, LOQT_OP_MERGE = 2, LOQT_OP_MERGE_SPLIT = 3, LOQT_OP_COMPENSATE = 4, LOQT_OP_FULL_GRADIENT = 5,
-       LOQT_OP_FWD_RIGHT = 6, LOQT_OP_BWD_RIGHT = 7, LOQT_OP_MERGE_RIGHT = 8 };
+       LOQT_OP_FWD_RIGHT = 6, LOQT_OP_BWD_RIGHT = 7, LOQT_OP_MERGE_RIGHT = 8, LOQT_OP_PROJECTION = 9 };
 
 /*
  * q_NF4 (Section 5.1, first two displayed equations): per block M = max|w|,
@@ -194,6 +195,36 @@ loqt_status loqt_merge_requant_right(loqt_nf4_mat Wq, loqt_nf4_mat Qq, const voi
 loqt_status loqt_full_gradient(const void *x, int64_t ldx, const void *dy, int64_t lddy, int32_t T,
                                int32_t out, int32_t in, float *G, int64_t ldg, int accumulate,
                                void *ws, size_t ws_bytes, void *stream);
+
+/*
+ * The projection from the full-rank gradient (Section 2.1, the rank-r factorisation
+ * of the gradient; Algorithm 2, the SVD lines: P = the r leading left singular
+ * vectors of G^W).  Only the subspace those vectors span enters the method
+ * (P P^T G), and the library approximates it by randomised subspace iteration
+ * (Halko, Martinsson and Tropp, "Finding structure with randomness", Algorithm 4.4):
+ *     Q = orth(G Omega);   repeat iters times:   Z = orth(G^T Q);   Q = orth(G Z);   P = Q
+ * The span of P tends to the leading subspace at the rate
+ * (sigma_(r+1) / sigma_r)^(2 iters + 1).
+ *   G     : fp32 [out][ldg] on the device (from loqt_full_gradient); 16-byte
+ *           aligned.  It enters the products rounded once to bf16 (the paper
+ *           trains in BF16, so its gradients carry no more).
+ *   Omega : bf16 [in][ldo], the in x r test matrix (independent standard normal
+ *           entries drawn by the caller; the random numbers are an input).
+ *   P     : fp32 [out][ldp], receives out x r with orthonormal columns.
+ *   1 <= r <= min(out, in), r <= 4096;  0 <= iters <= 16.
+ * Products: tcgen05, bf16 operands with fp32 accumulation; an orthonormalised
+ * iterate enters the next product as the sum of two bf16 matrices (value and
+ * rounding remainder), so it carries 16 significant bits.  orth() is Cholesky QR
+ * in double precision (Gram matrix, blocked Cholesky factorisation, triangular
+ * solve).  If an iterate is rank deficient to working precision (G of rank below
+ * r, or cond(G Omega) beyond about 1e7) the factorisation meets a non-positive
+ * pivot: the kernels then finish with that pivot replaced by one, set the
+ * status word, and loqt_device_status() returns LOQT_ERR_NUMERIC; P is then
+ * not a valid basis.  Workspace: loqt_workspace_bytes(LOQT_OP_PROJECTION, out, in, r, 0).
+ */
+loqt_status loqt_projection(const float *G, int64_t ldg, int32_t out, int32_t in, int32_t r,
+                            const void *Omega, int64_t ldo, int32_t iters, float *P, int64_t ldp,
+                            void *ws, size_t ws_bytes, void *stream);
 
 /*
  * Error-compensated initialisation of a layer for a new projection P
@@ -357,7 +388,8 @@ loqt_status loqt_linear_fwd_static(loqt_nf4_mat Wq, loqt_nf4_mat Pq, const void 
 size_t loqt_workspace_bytes(int op, int32_t out, int32_t in, int32_t r, int32_t T);
 
 /* Copies the status word at the start of a workspace back to the host
- * (synchronises `stream`) and maps it to LOQT_OK / LOQT_ERR_TIMEOUT. */
+ * (synchronises `stream`) and maps it to LOQT_OK, LOQT_ERR_TIMEOUT (a bounded wait
+ * expired) or LOQT_ERR_NUMERIC (loqt_projection met a rank-deficient iterate). */
 loqt_status loqt_device_status(const void *ws, void *stream);
 
 /* Number of kernels this library has launched in this process (all entry

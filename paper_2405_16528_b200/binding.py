@@ -17,7 +17,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libloqt.so")
 
 LOQT_OP_FWD, LOQT_OP_BWD, LOQT_OP_MERGE, LOQT_OP_MERGE_SPLIT, LOQT_OP_COMPENSATE, LOQT_OP_FULL_GRADIENT = 0, 1, 2, 3, 4, 5
-LOQT_OP_FWD_RIGHT, LOQT_OP_BWD_RIGHT, LOQT_OP_MERGE_RIGHT = 6, 7, 8
+LOQT_OP_FWD_RIGHT, LOQT_OP_BWD_RIGHT, LOQT_OP_MERGE_RIGHT, LOQT_OP_PROJECTION = 6, 7, 8, 9
 BLOCK = 64
 
 EXPORTS = (
@@ -28,7 +28,7 @@ EXPORTS = (
     "loqt_device_status", "loqt_launch_count", "loqt_status_string",
     "loqt_set_tile_override", "loqt_variant_launches", "loqt_selftest_wait_timeout",
     "loqt_scales_workspace_bytes", "loqt_scales_double_quantize", "loqt_scales_double_dequantize",
-    "loqt_nf4_dequantize_dq", "loqt_linear_fwd_dq", "loqt_linear_bwd_dq", "loqt_adam8_step",
+    "loqt_nf4_dequantize_dq", "loqt_linear_fwd_dq", "loqt_linear_bwd_dq", "loqt_adam8_step", "loqt_projection",
 )
 
 
@@ -96,6 +96,8 @@ def lib():
         getattr(L, name).restype = ctypes.c_int
     L.loqt_full_gradient.argtypes = [vp, i64, vp, i64, i32, i32, i32, vp, i64, ctypes.c_int, vp, sz, vp]
     L.loqt_full_gradient.restype = ctypes.c_int
+    L.loqt_projection.argtypes = [vp, i64, i32, i32, i32, vp, i64, i32, vp, i64, vp, sz, vp]
+    L.loqt_projection.restype = ctypes.c_int
     L.loqt_adam_step.argtypes = [vp, i64, vp, i64, vp, vp, i64, i32, i32, loqt_adam_params, vp]
     L.loqt_adam_step.restype = ctypes.c_int
     L.loqt_merge_requant_many.argtypes = [i32, ctypes.POINTER(M), ctypes.POINTER(M), ctypes.POINTER(vp), ctypes.POINTER(i64), f32, vp, sz, vp]
@@ -339,6 +341,22 @@ def loqt_full_gradient(x: torch.Tensor, dy: torch.Tensor, G: torch.Tensor | None
                                     _dev(G, torch.float32), G.stride(0), int(accumulate), ws.data_ptr(), ws.numel(),
                                     _stream()), "loqt_full_gradient")
     return G
+
+
+def loqt_projection(G: torch.Tensor, Omega: torch.Tensor, iters: int, P: torch.Tensor | None = None,
+                    ws: torch.Tensor | None = None) -> torch.Tensor:
+    """P (fp32 [out, r], orthonormal columns) spanning approximately the r leading left singular vectors of
+    G (fp32 [out, in]) by `iters` rounds of subspace iteration started from Omega (bf16 [in, r])."""
+    out, inn = G.shape
+    r = Omega.shape[1]
+    if P is None:
+        P = torch.empty((out, r), dtype=torch.float32, device=G.device)
+    if ws is None:
+        ws = new_workspace(loqt_workspace_bytes(LOQT_OP_PROJECTION, out, inn, r, 0), G.device)
+    _check(lib().loqt_projection(_dev(G, torch.float32), G.stride(0), out, inn, r, _dev(Omega, torch.bfloat16), Omega.stride(0),
+                                 int(iters), _dev(P, torch.float32), P.stride(0), ws.data_ptr(), ws.numel(), _stream()),
+           "loqt_projection")
+    return P
 
 
 def loqt_adam_step(B: torch.Tensor, dB: torch.Tensor, m: torch.Tensor, v: torch.Tensor, step: int, lr: float,

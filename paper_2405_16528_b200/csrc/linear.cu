@@ -338,6 +338,13 @@ extern "C" size_t loqt_workspace_bytes(int op, int32_t out, int32_t in, int32_t 
     if (splits > 1) total += align256(static_cast<size_t>(splits) * out * ((static_cast<size_t>(r) + 3) / 4 * 4) * 4);
   }
   if (op == LOQT_OP_MERGE_RIGHT) total += align256(static_cast<size_t>(r > 0 ? r : 0) * ((static_cast<size_t>(in > 0 ? in : 0) + 63) / 64 * 64) * 2);
+  // projection: bf16 G, one fp32 iterate, its hi + lo bf16 basis, and the orthonormalisation's scratch
+  if (op == LOQT_OP_PROJECTION) {
+    const size_t o = static_cast<size_t>(out > 0 ? out : 0), i = static_cast<size_t>(in > 0 ? in : 0);
+    const size_t big = o > i ? o : i, ldr = static_cast<size_t>(ld_lowrank(r));
+    total += align256(o * ((i + 63) / 64 * 64) * 2) + align256(big * ldr * 4) + 2 * align256(big * ldr * 2) +
+             orth_workspace_bytes(static_cast<int>(big), r);
+  }
   // full-rank gradient: split-K partials only (K = T)
   if (op == LOQT_OP_FULL_GRADIENT) {
     int splits = 1, kbps = 1;
@@ -797,6 +804,64 @@ extern "C" loqt_status loqt_full_gradient(const void *x, int64_t ldx, const void
   // G = dy^T x   (out x in; K = T; both operands stored K-outermost)
   return gemm_tn_f32(dy, lddy, x, ldx, out, in, T, G, ldg, accumulate, partial, static_cast<uint32_t *>(ws),
                      static_cast<cudaStream_t>(stream));
+}
+
+// ---------------------------------------------------------------------------
+// Projection from the full-rank gradient (Algorithm 2, SVD lines) by randomised
+// subspace iteration: products on the engine, orthonormalisation in subspace.cu
+// ---------------------------------------------------------------------------
+// Y (fp32, M x r) = A (hi + lo)  with the basis given as two bf16 matrices
+// [K][ldq]; A is bf16 G read K-major (A = G: M = out, K = in) or MN-major
+// (A = G^T: M = in, K = out).  Two K segments share the accumulator.
+static loqt_status projection_product(const void *gb, int64_t ldgb, bool transposed, int M, int K, int r, const void *hi,
+                                      const void *lo, int64_t ldq, float *Y, int64_t ldy, uint32_t *status, cudaStream_t stm) {
+  GemmCall c{};
+  c.p.M = M; c.p.N = r; c.p.num_segs = lo != nullptr ? 2 : 1;
+  for (int s = 0; s < c.p.num_segs; ++s) {
+    c.p.seg[s].K = K; c.p.seg[s].a_kind = transposed ? OP_TMA_MN : OP_TMA_K; c.p.seg[s].b_kind = OP_TMA_MN;
+    c.a[s] = {gb, ldgb};
+  }
+  c.b[0] = {hi, ldq};
+  c.b[1] = {lo, ldq};
+  c.p.splits = 1;
+  c.p.epi = EPI_F32; c.p.out = Y; c.p.ld_out = ldy; c.p.alpha = 1.0f; c.p.accumulate = 0; c.p.status = status;
+  return launch(c, stm);
+}
+
+extern "C" loqt_status loqt_projection(const float *G, int64_t ldg, int32_t out, int32_t in, int32_t r, const void *Omega,
+                                       int64_t ldo, int32_t iters, float *P, int64_t ldp, void *ws, size_t ws_bytes,
+                                       void *stream) {
+  loqt_status st;
+  if (out <= 0 || in <= 0 || r <= 0 || r > out || r > in || r > 4096 || iters < 0 || iters > 16) return LOQT_ERR_INVALID_ARG;
+  if (G == nullptr || P == nullptr || ldg < in || ldp < r) return LOQT_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(G) & 15u) != 0 || (reinterpret_cast<uintptr_t>(P) & 3u) != 0) return LOQT_ERR_ALIGNMENT;
+  if ((st = check_bf16(Omega, ldo, r)) != LOQT_OK) return st;
+  if ((st = check_ws(ws, ws_bytes, loqt_workspace_bytes(LOQT_OP_PROJECTION, out, in, r, 0))) != LOQT_OK) return st;
+  if ((st = check_arch()) != LOQT_OK) return st;
+  cudaStream_t stm = static_cast<cudaStream_t>(stream);
+  uint32_t *status = static_cast<uint32_t *>(ws);
+  const int big = out > in ? out : in;
+  const int64_t ldgb = (static_cast<int64_t>(in) + 63) / 64 * 64, ldr = ld_lowrank(r);
+  uint8_t *cursor = static_cast<uint8_t *>(ws) + 256;
+  void *gb = cursor;                                  cursor += align256(static_cast<size_t>(out) * ldgb * 2);
+  float *Y = reinterpret_cast<float *>(cursor);       cursor += align256(static_cast<size_t>(big) * ldr * 4);
+  void *hi = cursor;                                  cursor += align256(static_cast<size_t>(big) * ldr * 2);
+  void *lo = cursor;                                  cursor += align256(static_cast<size_t>(big) * ldr * 2);
+  void *orth_ws = cursor;
+
+  if ((st = convert_f32_bf16(G, ldg, gb, ldgb, out, in, stm)) != LOQT_OK) return st;
+  // Q = orth(G Omega)
+  if ((st = projection_product(gb, ldgb, false, out, in, r, Omega, nullptr, ldo, Y, ldr, status, stm)) != LOQT_OK) return st;
+  if ((st = orthonormalise(Y, ldr, out, r, iters == 0 ? P : nullptr, ldp, hi, lo, ldr, orth_ws, status, stm)) != LOQT_OK) return st;
+  for (int it = 1; it <= iters; ++it) {
+    // Z = orth(G^T Q)
+    if ((st = projection_product(gb, ldgb, true, in, out, r, hi, lo, ldr, Y, ldr, status, stm)) != LOQT_OK) return st;
+    if ((st = orthonormalise(Y, ldr, in, r, nullptr, 0, hi, lo, ldr, orth_ws, status, stm)) != LOQT_OK) return st;
+    // Q = orth(G Z)
+    if ((st = projection_product(gb, ldgb, false, out, in, r, hi, lo, ldr, Y, ldr, status, stm)) != LOQT_OK) return st;
+    if ((st = orthonormalise(Y, ldr, out, r, it == iters ? P : nullptr, ldp, hi, lo, ldr, orth_ws, status, stm)) != LOQT_OK) return st;
+  }
+  return LOQT_OK;
 }
 
 // ---------------------------------------------------------------------------

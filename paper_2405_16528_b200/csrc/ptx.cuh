@@ -52,7 +52,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     if (*abort_flag != 0) return false;
     if (globaltimer_ns() - t0 > limit_ns) {
       *abort_flag = 1;
-      atomicExch(status, kErrTimeout);
+      atomicOr(status, kErrTimeout);
       return false;
     }
   }

@@ -52,6 +52,7 @@ const char *loqt_status_string(loqt_status st) {
     case LOQT_ERR_CUDA: return "CUDA call failed";
     case LOQT_ERR_TIMEOUT: return "device-side wait timed out";
     case LOQT_ERR_ARCH: return "device is not sm_100";
+    case LOQT_ERR_NUMERIC: return "matrix numerically rank deficient (Cholesky pivot not positive)";
   }
   return "unknown status";
 }
@@ -63,7 +64,8 @@ loqt_status loqt_device_status(const void *ws, void *stream) {
   if (cudaMemcpyAsync(&word, ws, sizeof(word), cudaMemcpyDeviceToHost, st) != cudaSuccess)
     return LOQT_ERR_CUDA;
   if (cudaStreamSynchronize(st) != cudaSuccess) return LOQT_ERR_CUDA;
-  return word == 0 ? LOQT_OK : LOQT_ERR_TIMEOUT;
+  if (word & loqt::kErrTimeout) return LOQT_ERR_TIMEOUT;
+  return (word & loqt::kErrNumeric) ? LOQT_ERR_NUMERIC : LOQT_OK;
 }
 
 }  // extern "C"

@@ -48,6 +48,22 @@ def orthonormal(seed, names, rows, cols, device="cpu"):
     return q.to(torch.float32).contiguous()
 
 
+def lowrank_gradient(seed, names, out, inn, r, tail=0.5, noise=1e-3, device="cpu"):
+    """fp32 out x in matrix shaped like a layer's full-rank gradient: a dominant
+    part of rank r (singular values spread linearly over [1, 2]), a tail of
+    min(out, in) - r further directions (singular values from `tail` down to a
+    tenth of it) and dense Gaussian noise of standard deviation `noise`.
+    Singular vectors are Q factors of Gaussian matrices.  Drawn in float64."""
+    g = _gen(seed, names, "cpu")
+    k = min(out, inn)
+    U, _ = torch.linalg.qr(torch.randn((out, k), generator=g, dtype=torch.float64))
+    V, _ = torch.linalg.qr(torch.randn((inn, k), generator=g, dtype=torch.float64))
+    sv = torch.cat([torch.linspace(2.0, 1.0, r, dtype=torch.float64),
+                    float(tail) * torch.linspace(1.0, 0.1, k - r, dtype=torch.float64)])
+    G = (U * sv) @ V.T + float(noise) * torch.randn((out, inn), generator=g, dtype=torch.float64)
+    return G.to(torch.float32).to(device)
+
+
 @dataclass(frozen=True)
 class LayerSet:
     """One benchmark / parity configuration: the distinct projection shapes of a
