@@ -258,6 +258,38 @@ def time_compensated_init(device, peaks, cfg, seed, steps=5, iters=5):
     }
 
 
+def time_projection(device, peaks, cfg, seed, iters=2, reps=3):
+    """The projection step (Algorithm 2, SVD lines) for one matrix of the configuration's first shape:
+    randomised subspace iteration with `iters` rounds from a Gaussian test matrix.  Work counted: the
+    2 iters + 1 products of 2 out in r flops (tensor cores) and, per orthonormalisation, m r^2 (Gram, lower
+    half) + r^3 / 3 (Cholesky) + m r^2 (triangular solve) double-precision flops."""
+    import torch
+
+    from paper_2405_16528_b200 import binding as L
+    from paper_2405_16528_b200 import synth
+
+    _, out, inn, _ = next(iter(cfg.shapes()))
+    r = cfg.r
+    G = synth.normal(seed, ("pj", "G"), (out, inn), 1.0, torch.float32, device)
+    Om = synth.normal(seed, ("pj", "Omega"), (inn, r), 1.0, torch.bfloat16, device)
+    P = torch.empty((out, r), dtype=torch.float32, device=device)
+    ws = L.new_workspace(L.loqt_workspace_bytes(L.LOQT_OP_PROJECTION, out, inn, r, 0), device)
+    for _ in range(2):
+        L.loqt_projection(G, Om, iters, P=P, ws=ws)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(reps):
+        L.loqt_projection(G, Om, iters, P=P, ws=ws)
+    e1.record()
+    torch.cuda.synchronize()
+    L.loqt_device_status(ws)
+    ms = e0.elapsed_time(e1) / reps
+    f64 = sum(2.0 * m * r * r + r ** 3 / 3.0 for m in [out] + [inn, out] * iters)
+    return {"shape": [out, inn], "r": r, "iters": iters, "ms": round(ms, 3),
+            "product_tflops_bf16": round((2 * iters + 1) * 2.0 * out * inn * r / 1e12, 4),
+            "orth_gflops_f64": round(f64 / 1e9, 2), "orth_f64_tflops_if_all_time": round(f64 / (ms * 1e-3) / 1e12, 2)}
+
+
 def run_per_shape(args):
     """Diagnostic: median time of forward, backward and merge for one matrix of
     each distinct shape of the configuration, L2 flushed between calls."""
@@ -481,7 +513,9 @@ def merge_report(m, world, peaks):
 # DRAM read + write bytes of the forward/backward launches (u, y, v, dx, dB) of ONE attention-shaped
 # matrix, from the ncu capture summarised in profiles/ (None where no capture of the current kernels exists).
 NCU_TRAFFIC = {
-    4: {"bytes": None, "of": "no capture of the current kernels yet (algorithmic 332.4e6 for one 4096x4096 matrix)"},
+    4: {"bytes": 266.6e6,
+        "of": "sum of dram__bytes_read + dram__bytes_write over the five launches (u, y, v, dx, dB) of one 4096x4096 matrix, "
+              "r=1024, T=4096 (profiles/loqt_gemm_kernel_llama7b_attention.md); algorithmic bytes of the same launches 332.4e6"},
 }
 
 
@@ -519,6 +553,7 @@ def run_ours(args, rank, world, local_rank):
     nf4 = time_nf4_kernels(device, peaks)
     comp = time_compensated_init(device, peaks, cfg, args.seed)
     adam = time_adam_step(device, peaks)
+    proj = time_projection(device, peaks, cfg, args.seed)
     tflops = world * main["flops_step"] / (main["ms_fb"] * 1e-3) / 1e12
     per_gpu_tflops = tflops / world
     traffic = NCU_TRAFFIC.get(args.config, {"bytes": None, "of": "no capture for this configuration"})
@@ -574,6 +609,7 @@ def run_ours(args, rank, world, local_rank):
         "nf4_stream": nf4,
         "compensated_init": comp,
         "adam_step": adam,
+        "projection": proj,
         "gpu_launches": main["launches"],
         "clocks": main["clocks"],
         "wall_s_timed": round(main["t_wall"], 3),
