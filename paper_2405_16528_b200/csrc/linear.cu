@@ -312,6 +312,8 @@ extern "C" size_t loqt_workspace_bytes(int op, int32_t out, int32_t in, int32_t 
     int splits = 1, kbps = 1;
     db_splits(r, in, T > 0 ? T : 1, splits, kbps);
     if (splits > 1) total += align256(static_cast<size_t>(splits) * r * ((static_cast<size_t>(in) + 3) / 4 * 4) * 4);
+    // bf16(deq(P_q)), out x roundup(r, 64): staged once per backward for v = dy P-hat
+    total += align256(static_cast<size_t>(out > 0 ? out : 0) * ld_lowrank(r) * 2);
   }
   // merge: deq(P_q) as bf16, out x roundup(r, 64)
   if (op == LOQT_OP_MERGE || op == LOQT_OP_MERGE_SPLIT)
@@ -319,11 +321,11 @@ extern "C" size_t loqt_workspace_bytes(int op, int32_t out, int32_t in, int32_t 
   // two-pass merge: the fp32 product P-hat B, out x roundup(in, 64)
   if (op == LOQT_OP_MERGE_SPLIT)
     total += align256(static_cast<size_t>(out > 0 ? out : 0) * ((static_cast<size_t>(in > 0 ? in : 0) + 63) / 64 * 64) * 4);
-  // error-compensated initialisation: bf16 P, bf16 residual, fp32 corrected weights, fp32 B (+ split-K partials)
+  // error-compensated initialisation: bf16 P, bf16 residual, fp32 B (+ split-K partials)
   if (op == LOQT_OP_COMPENSATE) {
     const size_t o = static_cast<size_t>(out > 0 ? out : 0), ld64 = (static_cast<size_t>(in > 0 ? in : 0) + 63) / 64 * 64;
     const size_t ld4 = (static_cast<size_t>(in > 0 ? in : 0) + 3) / 4 * 4;
-    total += align256(o * ld_lowrank(r) * 2) + align256(o * ld64 * 2) + align256(o * ld64 * 4) + align256(static_cast<size_t>(r) * ld4 * 4);
+    total += align256(o * ld_lowrank(r) * 2) + align256(o * ld64 * 2) + align256(static_cast<size_t>(r) * ld4 * 4);
     int splits = 1, kbps = 1;
     db_splits(r, in, out > 0 ? out : 1, splits, kbps);
     if (splits > 1) total += align256(static_cast<size_t>(splits) * r * ld4 * 4);
@@ -433,9 +435,11 @@ static loqt_status check_bwd_args(const loqt_nf4_mat &Wq, const loqt_nf4_mat &Pq
   return LOQT_OK;
 }
 
-static loqt_status bwd_impl(const Nf4Src &W, const Nf4Src &P, const void *B, int64_t ldb, float s, const void *x, int64_t ldx,
-                            const void *dy, int64_t lddy, int32_t T, void *dx, int64_t lddx, float *dB, int64_t lddb,
-                            int accumulate_dB, void *ws, size_t ws_bytes, void *stream) {
+// Pq_fp32: the factor with fp32 scales when it has them (then it is staged as bf16
+// for the product v), null when its scales are doubly quantised.
+static loqt_status bwd_impl(const Nf4Src &W, const Nf4Src &P, const loqt_nf4_mat *Pq_fp32, const void *B, int64_t ldb, float s,
+                            const void *x, int64_t ldx, const void *dy, int64_t lddy, int32_t T, void *dx, int64_t lddx, float *dB,
+                            int64_t lddb, int accumulate_dB, void *ws, size_t ws_bytes, void *stream) {
   loqt_status st;
   const int out = W.rows, in = W.cols, r = P.cols;
   if ((st = check_ws(ws, ws_bytes, loqt_workspace_bytes(LOQT_OP_BWD, out, in, r, T))) != LOQT_OK) return st;
@@ -445,11 +449,27 @@ static loqt_status bwd_impl(const Nf4Src &W, const Nf4Src &P, const void *B, int
   const int64_t ldv = ld_lowrank(r);
   void *v = static_cast<uint8_t *>(ws) + 256;
   float *partial = reinterpret_cast<float *>(static_cast<uint8_t *>(v) + align256(static_cast<size_t>(T) * ldv * 2));
+  int db_split = 1, db_kbps = 1;
+  db_splits(r, in, T, db_split, db_kbps);
+  void *phat = reinterpret_cast<uint8_t *>(partial) +
+               (db_split > 1 ? align256(static_cast<size_t>(db_split) * r * ((static_cast<size_t>(in) + 3) / 4 * 4) * 4) : 0);
 
-  // v' = s * dy deq(P_q)      (T x r; K = out; P_q read with its blocks along N = r)
+  // v' = s * dy deq(P_q)      (T x r; K = out).  With N = r only, dequantising P_q inside
+  // the product would repeat it for every 256 token rows and bind the main loop; the
+  // factor is small (out x r), so it is dequantised once into the workspace (it stays
+  // in L2) and v runs as a plain bf16 product.  With doubly quantised scales P_q is
+  // read in place, its blocks along N = r.
   GemmCall c1{};
   c1.p.M = T; c1.p.N = r; c1.p.num_segs = 1;
-  c1.p.seg[0].K = out; c1.p.seg[0].a_kind = OP_TMA_K; c1.p.seg[0].b_kind = OP_NF4_MN; c1.p.seg[0].b_nf4 = P;
+  c1.p.seg[0].K = out; c1.p.seg[0].a_kind = OP_TMA_K;
+  if (Pq_fp32 != nullptr) {
+    const StageItem stage{*Pq_fp32, phat, ldv};
+    if ((st = nf4_dequantize_bf16_batch(&stage, 1, stm)) != LOQT_OK) return st;
+    c1.p.seg[0].b_kind = OP_TMA_MN;
+    c1.b[0] = {phat, ldv};
+  } else {
+    c1.p.seg[0].b_kind = OP_NF4_MN; c1.p.seg[0].b_nf4 = P;
+  }
   c1.a[0] = {dy, lddy};
   c1.p.splits = 1;
   c1.p.epi = EPI_BF16; c1.p.out = v; c1.p.ld_out = ldv; c1.p.alpha = s; c1.p.status = status;
@@ -477,7 +497,7 @@ extern "C" loqt_status loqt_linear_bwd(loqt_nf4_mat Wq, loqt_nf4_mat Pq, const v
                                        size_t ws_bytes, void *stream) {
   loqt_status st;
   if ((st = check_bwd_args(Wq, Pq, B, ldb, x, ldx, dy, lddy, T, dx, lddx, dB, lddb)) != LOQT_OK) return st;
-  return bwd_impl(nf4_src(Wq), nf4_src(Pq), B, ldb, s, x, ldx, dy, lddy, T, dx, lddx, dB, lddb, accumulate_dB, ws, ws_bytes,
+  return bwd_impl(nf4_src(Wq), nf4_src(Pq), &Pq, B, ldb, s, x, ldx, dy, lddy, T, dx, lddx, dB, lddb, accumulate_dB, ws, ws_bytes,
                   stream);
 }
 
@@ -517,8 +537,8 @@ extern "C" loqt_status loqt_linear_bwd_dq(loqt_nf4_mat Wq, loqt_dq_scales Wdq, l
                            lddb)) != LOQT_OK)
     return st;
   if ((st = check_dq(Wq, Wdq)) != LOQT_OK || (st = check_dq(Pq, Pdq)) != LOQT_OK) return st;
-  return bwd_impl(nf4_src_dq(Wq, Wdq), nf4_src_dq(Pq, Pdq), B, ldb, s, x, ldx, dy, lddy, T, dx, lddx, dB, lddb, accumulate_dB, ws,
-                  ws_bytes, stream);
+  return bwd_impl(nf4_src_dq(Wq, Wdq), nf4_src_dq(Pq, Pdq), nullptr, B, ldb, s, x, ldx, dy, lddy, T, dx, lddx, dB, lddb,
+                  accumulate_dB, ws, ws_bytes, stream);
 }
 
 // ---------------------------------------------------------------------------
@@ -540,9 +560,15 @@ struct MergeItem {
   Bf16Operand a, b;
   int K;
   float alpha;
+  // compensation mode: Wq is only written; the sum starts from the fp32 matrix w32 and
+  // the bf16 residual w32 - deq32(Wq) is written to resid
+  const float *w32 = nullptr;
+  int64_t ld_w32 = 0;
+  void *resid = nullptr;
+  int64_t ld_resid = 0;
 };
 
-template <int BN>
+template <int BN, bool COMP = false>
 static loqt_status launch_merge(const MergeItem *items, int n, uint32_t *status, cudaStream_t stream) {
   using L = SmemLayout<BN, 1, false, false, true>;
   MergeBatch mb;
@@ -562,12 +588,14 @@ static loqt_status launch_merge(const MergeItem *items, int n, uint32_t *status,
     pr.tile0 = tiles;
     pr.mt = (M + kHM - 1) / kHM;
     pr.alpha = it.alpha;
+    pr.w32 = it.w32; pr.ld_w32 = it.ld_w32;
+    pr.resid = static_cast<__nv_bfloat16 *>(it.resid); pr.ld_resid = it.ld_resid;
     tiles += pr.mt * ((N + BN - 1) / BN);
   }
   mb.count = n;
   mb.tiles = tiles;
   mb.status = status;
-  auto kernel = loqt_merge_kernel<BN>;
+  auto kernel = loqt_merge_kernel<BN, COMP>;
   if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kDynamicBytes) != cudaSuccess)
     return LOQT_ERR_CUDA;
   cudaLaunchConfig_t cfg;
@@ -596,6 +624,8 @@ static loqt_status merge_batch(const MergeItem *items, int n, uint32_t *status, 
   for (int i = 0; i < n; ++i) wide = wide || items[i].Wq.cols > 128;
   const int fbn = g_force_bn.load(std::memory_order_relaxed);
   if (fbn != 0) wide = (fbn == 256);
+  const bool comp = items[0].w32 != nullptr;  // a batch is all of one kind
+  if (comp) return wide ? launch_merge<256, true>(items, n, status, stream) : launch_merge<128, true>(items, n, status, stream);
   return wide ? launch_merge<256>(items, n, status, stream) : launch_merge<128>(items, n, status, stream);
 }
 
@@ -888,32 +918,40 @@ extern "C" loqt_status loqt_compensated_init(const float *W, int64_t ldw, const 
   uint8_t *cursor = static_cast<uint8_t *>(ws) + 256;
   void *phat = cursor;                                        cursor += align256(static_cast<size_t>(out) * ldr * 2);
   void *resid = cursor;                                       cursor += align256(static_cast<size_t>(out) * ld64 * 2);
-  float *what = reinterpret_cast<float *>(cursor);            cursor += align256(static_cast<size_t>(out) * ld64 * 4);
   float *b32 = reinterpret_cast<float *>(cursor);             cursor += align256(static_cast<size_t>(r) * ld4 * 4);
   float *partial = reinterpret_cast<float *>(cursor);
 
   // P_q = q(P); the products below use bf16(P), the unquantised projection (Algorithm 2)
   if ((st = loqt_nf4_quantize(P, ldp, Pq, stream)) != LOQT_OK) return st;
   if ((st = convert_f32_bf16(P, ldp, phat, ldr, out, r, stm)) != LOQT_OK) return st;
+  int splits = 1, kbps = 1;
+  db_splits(r, in, out, splits, kbps);
 
   for (int c = 1; c <= steps; ++c) {
-    // Q_c = q(W - P B_{c-1}) (B_0 = 0), residual = bf16(W - deq(Q_c))
-    const float *src = (c == 1) ? W : what;
-    const int64_t ld_src = (c == 1) ? ldw : ld64;
-    if ((st = nf4_quantize_residual(src, ld_src, W, ldw, Wq, resid, ld64, stm)) != LOQT_OK) return st;
-    // B_c = P^T residual   (r x in; K = out; both operands stored K-outermost), then to bf16
-    if ((st = gemm_tn_f32(phat, ldr, resid, ld64, r, in, out, b32, ld4, 0, partial, status, stm)) != LOQT_OK) return st;
-    if ((st = convert_f32_bf16(b32, ld4, B, ldb, r, in, stm)) != LOQT_OK) return st;
-    if (c == steps) break;
-    // corrected weights for the next step: W - P B_c   (out x in; K = r), fp32
-    GemmCall g{};
-    g.p.M = out; g.p.N = in; g.p.num_segs = 1;
-    g.p.seg[0].K = r; g.p.seg[0].a_kind = OP_TMA_K; g.p.seg[0].b_kind = OP_TMA_MN;
-    g.a[0] = {phat, ldr}; g.b[0] = {B, ldb};
-    g.p.splits = 1;
-    g.p.epi = EPI_F32; g.p.out = what; g.p.ld_out = ld64; g.p.alpha = -1.0f; g.p.addend = W; g.p.ld_addend = ldw;
-    g.p.status = status;
-    if ((st = launch(g, stm)) != LOQT_OK) return st;
+    if (c == 1) {
+      // Q_1 = q(W) (B_0 = 0), residual = bf16(W - deq(Q_1)): one streaming pass
+      if ((st = nf4_quantize_residual(W, ldw, W, ldw, Wq, resid, ld64, stm)) != LOQT_OK) return st;
+    } else {
+      // Q_c = q(W - P B_(c-1)), residual = bf16(W - deq(Q_c)): the product P B (out x in; K = r)
+      // with the quantiser and the residual in its epilogue; W - P B is never written
+      MergeItem item{Wq, {phat, ldr}, {B, ldb}, r, -1.0f};
+      item.w32 = W; item.ld_w32 = ldw; item.resid = resid; item.ld_resid = ld64;
+      if ((st = merge_batch(&item, 1, status, stm)) != LOQT_OK) return st;
+    }
+    // B_c = P^T residual   (r x in; K = out; both operands stored K-outermost), rounded to bf16:
+    // in the product's epilogue when one pass over K does it, else after the split-K sum
+    if (splits == 1) {
+      GemmCall g{};
+      g.p.M = r; g.p.N = in; g.p.num_segs = 1;
+      g.p.seg[0].K = out; g.p.seg[0].a_kind = OP_TMA_MN; g.p.seg[0].b_kind = OP_TMA_MN;
+      g.a[0] = {phat, ldr}; g.b[0] = {resid, ld64};
+      g.p.splits = 1; g.p.kb_per_split = 0;
+      g.p.epi = EPI_BF16; g.p.out = B; g.p.ld_out = ldb; g.p.alpha = 1.0f; g.p.status = status;
+      if ((st = launch(g, stm)) != LOQT_OK) return st;
+    } else {
+      if ((st = gemm_tn_f32(phat, ldr, resid, ld64, r, in, out, b32, ld4, 0, partial, status, stm)) != LOQT_OK) return st;
+      if ((st = convert_f32_bf16(b32, ld4, B, ldb, r, in, stm)) != LOQT_OK) return st;
+    }
   }
   return LOQT_OK;
 }

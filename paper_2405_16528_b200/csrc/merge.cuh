@@ -34,6 +34,11 @@ struct MergeProblem {
   int mt;            // tiles along M (tile = tile0 + n_blk * mt + m_blk)
   float alpha;
   int pad_;
+  // compensation mode only (kComp): the fp32 matrix that takes the place of deq32(W_q)
+  // in the sum, and the bf16 residual W - deq32(new codes) written beside the codes
+  const float *w32;       // [M][ld_w32]
+  __nv_bfloat16 *resid;   // [M][ld_resid]
+  int64_t ld_w32, ld_resid;
 };
 
 struct MergeBatch {
@@ -46,7 +51,14 @@ struct MergeBatch {
   uint32_t *status;
 };
 
-template <int BN>
+// kComp = false: the merge above.  kComp = true: one step of the error-compensated
+// initialisation (paper Section 2.5; Algorithm 2, compensation loop) in the same
+// pipeline: the fp32 weights W take the place of deq32(W_q) in the sum,
+//   Q <- q_NF4( W + alpha * A B )        (alpha = -1, A = P, B = B_(c-1)),
+// the codes and scales of Q are written (nothing of W_q is read), and with them
+// the bf16 residual W - deq32(Q) that the next product P^T (W - Q) consumes.  The
+// corrected weights W - P B never exist in memory.
+template <int BN, bool kComp = false>
 __global__ void __launch_bounds__(kNumThreads, 1)
 loqt_merge_kernel(const __grid_constant__ MergeBatch mb) {
   using L = SmemLayout<BN, 1, false, false, true>;
@@ -202,8 +214,14 @@ loqt_merge_kernel(const __grid_constant__ MergeBatch mb) {
         locate(g, pi, m_blk, n_blk);
         const uint32_t b = tile & 1u;
         ptx::bulk_wait_group_read<0>();
-        ptx::mbar_arrive_expect_tx(wfull_bar(b), L::kWTileBytes);
-        ptx::tma_load_2d(smem_base + L::kWOffset + b * L::kWTileBytes, &mb.wq[pi], wfull_bar(b), n_blk * (BN / 2), m_blk * kHM);
+        if (kComp) {
+          // nothing to bring in: the arrival only tells the epilogue that the store which
+          // last read this buffer is done with it
+          ptx::mbar_arrive(wfull_bar(b));
+        } else {
+          ptx::mbar_arrive_expect_tx(wfull_bar(b), L::kWTileBytes);
+          ptx::tma_load_2d(smem_base + L::kWOffset + b * L::kWTileBytes, &mb.wq[pi], wfull_bar(b), n_blk * (BN / 2), m_blk * kHM);
+        }
         if (tile > 0) store_prev();
         prev_pi = pi;
         pm = m_blk;
@@ -246,29 +264,58 @@ loqt_merge_kernel(const __grid_constant__ MergeBatch mb) {
         const int c0 = n_blk * BN + jb * 64;
         const bool live = row_ok && c0 < pr.wq_ld;
         float *mp = pr.wq_absmax + static_cast<int64_t>(row) * (pr.wq_ld >> 6) + (c0 >> 6);
-        float Mold = 0.0f;
-        if (live) Mold = *mp;  // in flight while the accumulator is read
         const uint32_t a0 = w_row + (((2u * jb) ^ w_key) << 4), a1 = w_row + (((2u * jb + 1u) ^ w_key) << 4);
-        const uint4 ca = ld_shared_v4(a0), cb = ld_shared_v4(a1);
+        float Mold = 0.0f;
+        uint4 ca = make_uint4(0, 0, 0, 0), cb = ca;
+        // compensation mode: this thread's 64 weights, read straight from global memory
+        // (256 contiguous bytes per thread; elements beyond the matrix read as zero)
+        float2 v[32];
+        const float *wp = nullptr;
+        bool wide = false;
+        if (kComp) {
+          wp = pr.w32 + static_cast<int64_t>(row) * pr.ld_w32 + c0;
+          wide = live && c0 + 64 <= pr.N && (pr.ld_w32 & 3) == 0 && (reinterpret_cast<uintptr_t>(pr.w32) & 15u) == 0;
+          if (wide) {
+#pragma unroll
+            for (int e = 0; e < 16; ++e) {
+              const float4 t = __ldg(reinterpret_cast<const float4 *>(wp) + e);
+              v[2 * e] = make_float2(t.x, t.y);
+              v[2 * e + 1] = make_float2(t.z, t.w);
+            }
+          } else {
+#pragma unroll
+            for (int e = 0; e < 32; ++e)
+              v[e] = make_float2((live && c0 + 2 * e < pr.N) ? __ldg(wp + 2 * e) : 0.0f,
+                                 (live && c0 + 2 * e + 1 < pr.N) ? __ldg(wp + 2 * e + 1) : 0.0f);
+          }
+        } else {
+          if (live) Mold = *mp;  // in flight while the accumulator is read
+          ca = ld_shared_v4(a0);
+          cb = ld_shared_v4(a1);
+        }
         uint32_t d0[32], d1[32];
         ptx::tmem_ld32(t_row + jb * 64, d0);
         ptx::tmem_ld32(t_row + jb * 64 + 32, d1);
         ptx::tmem_ld_wait();
         if (live) {
           const uint32_t w[8] = {ca.x, ca.y, ca.z, ca.w, cb.x, cb.y, cb.z, cb.w};
-          // v = deq32(old) + alpha * delta, two elements per packed instruction; four
-          // running maxima keep the dependent chain of the block maximum short
-          float2 v[32];
+          // v = deq32(old) + alpha * delta (compensation: W + alpha * delta), two elements
+          // per packed instruction; four running maxima keep the dependent chain of the
+          // block maximum short
           float mx[4] = {0.0f, 0.0f, 0.0f, 0.0f};
           const float2 a2 = make_float2(alpha, alpha), m2 = make_float2(Mold, Mold);
 #pragma unroll
           for (int e = 0; e < 32; ++e) {
-            const uint32_t word = w[e >> 2];
-            const float2 lv = make_float2(tables.level[(word >> (8 * (e & 3))) & 15u],
-                                          tables.level[(word >> (8 * (e & 3) + 4)) & 15u]);
             const float2 delta = make_float2(__uint_as_float(e < 16 ? d0[2 * e] : d1[2 * e - 32]),
                                              __uint_as_float(e < 16 ? d0[2 * e + 1] : d1[2 * e - 31]));
-            v[e] = __ffma2_rn(a2, delta, __fmul2_rn(m2, lv));
+            if (kComp) {
+              v[e] = __ffma2_rn(a2, delta, v[e]);
+            } else {
+              const uint32_t word = w[e >> 2];
+              const float2 lv = make_float2(tables.level[(word >> (8 * (e & 3))) & 15u],
+                                            tables.level[(word >> (8 * (e & 3) + 4)) & 15u]);
+              v[e] = __ffma2_rn(a2, delta, __fmul2_rn(m2, lv));
+            }
             mx[e & 3] = fmaxf(mx[e & 3], fmaxf(fabsf(v[e].x), fabsf(v[e].y)));
           }
           const float Mnew = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
@@ -295,6 +342,47 @@ loqt_merge_kernel(const __grid_constant__ MergeBatch mb) {
           st_shared_v4(a0, make_uint4(o[0], o[1], o[2], o[3]));
           st_shared_v4(a1, make_uint4(o[4], o[5], o[6], o[7]));
           *mp = Mnew;
+          if (kComp) {
+            // residual = bf16( W - fl32(Mnew * q[code]) ): two fp32 roundings, as the definition
+            // has them; W is read again (an L1 / L2 hit) rather than kept in registers
+            __nv_bfloat16 *rp = pr.resid + static_cast<int64_t>(row) * pr.ld_resid + c0;
+            const bool wide_out = wide && (pr.ld_resid & 7) == 0 && (reinterpret_cast<uintptr_t>(pr.resid) & 15u) == 0;
+#pragma unroll
+            for (int g8 = 0; g8 < 8; ++g8) {
+              float2 wv[4];
+              if (wide) {
+                const float4 t0 = __ldg(reinterpret_cast<const float4 *>(wp) + 2 * g8);
+                const float4 t1 = __ldg(reinterpret_cast<const float4 *>(wp) + 2 * g8 + 1);
+                wv[0] = make_float2(t0.x, t0.y); wv[1] = make_float2(t0.z, t0.w);
+                wv[2] = make_float2(t1.x, t1.y); wv[3] = make_float2(t1.z, t1.w);
+              } else {
+#pragma unroll
+                for (int h2 = 0; h2 < 4; ++h2) {
+                  const int c = 8 * g8 + 2 * h2;
+                  wv[h2] = make_float2(c0 + c < pr.N ? __ldg(wp + c) : 0.0f, c0 + c + 1 < pr.N ? __ldg(wp + c + 1) : 0.0f);
+                }
+              }
+              uint32_t pk[4];
+#pragma unroll
+              for (int h2 = 0; h2 < 4; ++h2) {
+                const uint32_t byte = (o[g8] >> (8 * h2)) & 0xFFu;
+                // scalar intrinsics: the packed multiply and add may be contracted into one fused operation
+                const float e_lo = __fsub_rn(wv[h2].x, __fmul_rn(Mnew, tables.level[byte & 15u]));
+                const float e_hi = __fsub_rn(wv[h2].y, __fmul_rn(Mnew, tables.level[byte >> 4]));
+                pk[h2] = pack_bf16x2(e_lo, e_hi);
+              }
+              if (wide_out) {
+                reinterpret_cast<uint4 *>(rp)[g8] = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+              } else {
+#pragma unroll
+                for (int h2 = 0; h2 < 4; ++h2) {
+                  const int c = 8 * g8 + 2 * h2;
+                  if (c0 + c < pr.N) rp[c] = __ushort_as_bfloat16(static_cast<unsigned short>(pk[h2] & 0xFFFFu));
+                  if (c0 + c + 1 < pr.N) rp[c + 1] = __ushort_as_bfloat16(static_cast<unsigned short>(pk[h2] >> 16));
+                }
+              }
+            }
+          }
         }
         __syncwarp();
       }

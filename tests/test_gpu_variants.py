@@ -90,8 +90,9 @@ def test_forward_backward_merge_with_forced_tile(forced_tile, shape):
     dB = torch.full((r, inn), 3.0, dtype=torch.float32, device="cuda")
     L.loqt_linear_bwd(Wq, Pq, B, s, x, dy, dx=dx, dB=dB, ws=ws)
     L.loqt_device_status(ws)
-    nf4_2, _ = _counts(forced_tile)
-    assert nf4_2 == nf4_1 + 2, "v and dx did not run the forced instantiation"
+    nf4_2, bf16_2 = _counts(forced_tile)
+    # dx dequantises W_q in its main loop; v = dy P-hat reads the factor staged as bf16 (the variant without NF4 staging)
+    assert nf4_2 == nf4_1 + 1 and bf16_2 >= bf16_1 + 1, "v and dx did not run the forced instantiation"
     check_close(f32(dx), ref["dx"], f"dx {shape} {_tile_id(forced_tile)}")
     check_close(f32(dB), ref["dB"], f"dB {shape} {_tile_id(forced_tile)}")
 
