@@ -551,6 +551,7 @@ def run_ours(args, rank, world, local_rank):
     peaks = load_peaks()
     cfg = main["cfg"]
     nf4 = time_nf4_kernels(device, peaks)
+    nf4_large = time_nf4_kernels(device, peaks, rows=65536, cols=8192, iters=5)
     comp = time_compensated_init(device, peaks, cfg, args.seed)
     adam = time_adam_step(device, peaks)
     proj = time_projection(device, peaks, cfg, args.seed)
@@ -607,6 +608,7 @@ def run_ours(args, rank, world, local_rank):
         },
         "configs": {},
         "nf4_stream": nf4,
+        "nf4_stream_large": nf4_large,
         "compensated_init": comp,
         "adam_step": adam,
         "projection": proj,

@@ -269,7 +269,7 @@ loqt_merge_kernel(const __grid_constant__ MergeBatch mb) {
         uint4 ca = make_uint4(0, 0, 0, 0), cb = ca;
         // compensation mode: this thread's 64 weights, read straight from global memory
         // (256 contiguous bytes per thread; elements beyond the matrix read as zero)
-        float2 v[32];
+        float2 v[32], wk[32];
         const float *wp = nullptr;
         bool wide = false;
         if (kComp) {
@@ -309,6 +309,7 @@ loqt_merge_kernel(const __grid_constant__ MergeBatch mb) {
             const float2 delta = make_float2(__uint_as_float(e < 16 ? d0[2 * e] : d1[2 * e - 32]),
                                              __uint_as_float(e < 16 ? d0[2 * e + 1] : d1[2 * e - 31]));
             if (kComp) {
+              wk[e] = v[e];  // W itself, for the residual
               v[e] = __ffma2_rn(a2, delta, v[e]);
             } else {
               const uint32_t word = w[e >> 2];
@@ -344,24 +345,13 @@ loqt_merge_kernel(const __grid_constant__ MergeBatch mb) {
           *mp = Mnew;
           if (kComp) {
             // residual = bf16( W - fl32(Mnew * q[code]) ): two fp32 roundings, as the definition
-            // has them; W is read again (an L1 / L2 hit) rather than kept in registers
+            // has them; W comes from the copy kept above (reading it again from global memory,
+            // one row segment per thread, costs more load/store-unit time than the spills do)
             __nv_bfloat16 *rp = pr.resid + static_cast<int64_t>(row) * pr.ld_resid + c0;
             const bool wide_out = wide && (pr.ld_resid & 7) == 0 && (reinterpret_cast<uintptr_t>(pr.resid) & 15u) == 0;
 #pragma unroll
             for (int g8 = 0; g8 < 8; ++g8) {
-              float2 wv[4];
-              if (wide) {
-                const float4 t0 = __ldg(reinterpret_cast<const float4 *>(wp) + 2 * g8);
-                const float4 t1 = __ldg(reinterpret_cast<const float4 *>(wp) + 2 * g8 + 1);
-                wv[0] = make_float2(t0.x, t0.y); wv[1] = make_float2(t0.z, t0.w);
-                wv[2] = make_float2(t1.x, t1.y); wv[3] = make_float2(t1.z, t1.w);
-              } else {
-#pragma unroll
-                for (int h2 = 0; h2 < 4; ++h2) {
-                  const int c = 8 * g8 + 2 * h2;
-                  wv[h2] = make_float2(c0 + c < pr.N ? __ldg(wp + c) : 0.0f, c0 + c + 1 < pr.N ? __ldg(wp + c + 1) : 0.0f);
-                }
-              }
+              const float2 wv[4] = {wk[4 * g8], wk[4 * g8 + 1], wk[4 * g8 + 2], wk[4 * g8 + 3]};
               uint32_t pk[4];
 #pragma unroll
               for (int h2 = 0; h2 < 4; ++h2) {

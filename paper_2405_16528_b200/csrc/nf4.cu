@@ -2,13 +2,51 @@
 //
 // All are HBM-bound: quantise moves 4 + 0.5625 bytes per element, requantise
 // 4 + 2 * 0.5625, dequantise 0.5625 + 2 (bf16) or + 4 (fp32).  Loads and stores
-// are 128-bit where alignment allows, and every thread keeps the next trip's
-// loads in flight while it works on the current one.
+// are 128-bit where alignment allows.  To stay memory-bound the kernels must be
+// frugal with instructions (a few per element), so the work is dealt out row-wise:
+// a thread keeps its position inside the row for the whole kernel and walks down
+// the rows with pointer increments - no division, no 64-bit index arithmetic per
+// item - and it has the loads of several rows in flight before it works on the
+// first.
 #include "common.cuh"
 
 namespace loqt {
 
 constexpr int kQThreads = 256;
+
+// Row-wise distribution of a block's 256 threads: `per_row` threads (a power of two,
+// 2^log2) side by side along a row, 256 / per_row rows per pass; blockIdx.x selects
+// the chunk of the row, blockIdx.y the first rows.
+struct RowDeal {
+  int log2;  // log2 of the threads (or thread groups) a block puts side by side in a row
+  dim3 grid;
+};
+
+// units: work units per row (one per thread or thread group); per_block: units a
+// block holds (256 threads, or 64 groups of four); the grid covers the row in x and
+// as many rows in y as `resident` blocks allow.
+static RowDeal deal_rows(int units, int per_block, int rows, int resident) {
+  RowDeal d;
+  d.log2 = 0;
+  while ((1 << d.log2) < units && (1 << d.log2) < per_block) ++d.log2;
+  const int per_row = 1 << d.log2;
+  const int gx = (units + per_row - 1) / per_row;
+  const int rows_per_pass = per_block / per_row;
+  int gy = (rows + rows_per_pass - 1) / rows_per_pass;
+  int cap = resident / gx;
+  if (cap < 1) cap = 1;
+  if (gy > cap) gy = cap;
+  if (gy > 65535) gy = 65535;
+  d.grid = dim3(static_cast<unsigned>(gx), static_cast<unsigned>(gy > 0 ? gy : 1));
+  return d;
+}
+
+template <typename Kernel>
+static int resident_blocks(Kernel kernel) {
+  int per_sm = 0;
+  if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, kQThreads, 0) != cudaSuccess || per_sm < 1) per_sm = 1;
+  return sm_count() * per_sm;
+}
 
 // ---------------------------------------------------------------------------
 // quantise:   fp32 [rows][ld_src] -> codes [rows][ld/2], absmax [rows][ld/64]
@@ -17,151 +55,169 @@ constexpr int kQThreads = 256;
 // residual:   quantise `src` and also write bf16(ref - deq32(codes)) for every real
 //             element (the error-compensation step: `ref` is the weight matrix
 //             the quantised one should approximate, `src` what is quantised)
-// Four threads share one block of 64 weights; each owns 16 consecutive elements
-// (four 128-bit loads, one 64-bit store of 16 codes; the requantiser also loads
-// its 16 old codes and the block's old scale).
+// Four threads share one block of 64 weights.  Where the whole block lies inside
+// the matrix, thread l loads the 16-byte pieces l, l + 4, l + 8, l + 12 of its 256
+// bytes, so that every load instruction of the group covers 64 contiguous bytes
+// (whole 32-byte sectors); it then owns elements 16 k + 4 l .. + 3, k = 0..3, and
+// the four threads exchange 16-bit pieces of their code words by shuffles so that
+// each stores 8 contiguous bytes of codes.  A block cut short by the matrix edge
+// is read element by element, 16 consecutive elements per thread.  The
+// requantiser also loads its 16 old codes and the block's old scale.
 // ---------------------------------------------------------------------------
-struct QuantItem {
-  uint32_t row, b;
-  int c0;
-  bool live;
-};
-
 enum : int { kQuantise = 0, kRequantise = 1, kQuantiseResidual = 2 };
+
+struct QuantLoad {
+  float v[16];
+  uint2 old;
+  float Mold;
+};
 
 template <bool kVec, int kMode>
 __global__ void __launch_bounds__(kQThreads)
 nf4_quantize_kernel(const float *__restrict__ src, int64_t ld_src, float s, uint8_t *__restrict__ codes,
                     float *__restrict__ absmax, int rows, int cols, int ld, const float *__restrict__ ref,
-                    int64_t ld_ref, __nv_bfloat16 *__restrict__ resid, int64_t ld_resid) {
+                    int64_t ld_ref, __nv_bfloat16 *__restrict__ resid, int64_t ld_resid, int gx_log2) {
   constexpr bool kRequant = (kMode == kRequantise);
   __shared__ Nf4Tables tab;
   nf4_tables_init(tab, threadIdx.x);
   __syncthreads();
 
-  const uint32_t nb = static_cast<uint32_t>(ld / kBlock);
-  const uint32_t n_items = static_cast<uint32_t>(rows) * nb;  // one item = one NF4 block (host checks < 2^30)
-  const uint32_t l = threadIdx.x & 3;                         // lane within the 4-thread group
-  const uint32_t group0 = (blockIdx.x * kQThreads + threadIdx.x) >> 2;
-  const uint32_t stride = (gridDim.x * kQThreads) >> 2;
-  // All threads of a warp run the same trip count: idle groups still take part in the shuffles.
-  const uint32_t trips = (n_items + stride - 1) / stride;
-
-  auto item_of = [&](uint32_t it) {
-    QuantItem q;
-    const uint32_t item = group0 + it * stride;
-    q.live = it < trips && item < n_items;
-    q.row = q.live ? item / nb : 0;
-    q.b = q.live ? item - q.row * nb : 0;
-    q.c0 = static_cast<int>(q.b) * kBlock + 16 * static_cast<int>(l);
-    return q;
+  const int nb = ld / kBlock;
+  const int l = threadIdx.x & 3;          // lane within the 4-thread group
+  const int group = threadIdx.x >> 2;     // 64 groups per block
+  const int gx = group & ((1 << gx_log2) - 1), gy = group >> gx_log2;
+  const int b = (static_cast<int>(blockIdx.x) << gx_log2) + gx;  // NF4 block inside the row
+  const int rows_per_pass = 64 >> gx_log2;
+  const int row_stride = static_cast<int>(gridDim.y) * rows_per_pass;
+  const int row_first = static_cast<int>(blockIdx.y) * rows_per_pass;  // of this block: the same for all its threads
+  const int c0 = b * kBlock + 16 * l;  // first element of this thread's 8 bytes of codes
+  const bool col_live = b < nb;
+  const bool wide = kVec && (b + 1) * kBlock <= cols;  // the whole block is inside the matrix: interleaved ownership
+  // element of the row that v[j] holds
+  auto elem = [&](int j) { return wide ? b * kBlock + 16 * (j >> 2) + 4 * l + (j & 3) : c0 + j; };
+  // Pieces of 16 bits (four codes) change hands inside the group: piece p of thread j
+  // goes to position j of thread p.  Used to turn the old codes of 16 consecutive
+  // elements into those of the interleaved elements and back (the map is its own
+  // inverse).  All lanes of the warp take part.
+  auto exchange = [&](uint2 w) {
+    const unsigned long long w64 = (static_cast<unsigned long long>(w.y) << 32) | w.x;
+    unsigned long long out = 0;
+#pragma unroll
+    for (int d = 0; d < 4; ++d) {
+      const int p = l ^ d;
+      uint32_t piece = static_cast<uint32_t>(w64 >> (16 * p)) & 0xFFFFu;
+      if (d != 0) piece = __shfl_xor_sync(0xffffffffu, piece, d);
+      out |= static_cast<unsigned long long>(piece) << (16 * p);
+    }
+    return make_uint2(static_cast<uint32_t>(out), static_cast<uint32_t>(out >> 32));
   };
+
   // Issues the loads of one item: 16 source values and, for the requantiser, the
   // 16 old codes and the old scale.  Elements past `cols` read as zero.
-  auto fetch = [&](const QuantItem &q, float (&v)[16], uint2 &old, float &Mold) {
-    const float *p = src + static_cast<int64_t>(q.row) * ld_src + q.c0;
-    old = make_uint2(kZeroWord, kZeroWord);
-    Mold = 0.0f;
-    if (kRequant && q.live) {
-      old = *reinterpret_cast<const uint2 *>(codes + static_cast<int64_t>(q.row) * (ld / 2) + (q.c0 >> 1));
-      Mold = absmax[static_cast<int64_t>(q.row) * nb + q.b];
+  auto fetch = [&](int row, QuantLoad &q) {
+    const bool live = col_live && row < rows;
+    q.old = make_uint2(kZeroWord, kZeroWord);
+    q.Mold = 0.0f;
+    if (kRequant && live) {
+      q.old = *reinterpret_cast<const uint2 *>(codes + static_cast<int64_t>(row) * (ld / 2) + (c0 >> 1));
+      q.Mold = absmax[static_cast<int64_t>(row) * nb + b];
     }
-    if (kVec && q.live && q.c0 + 16 <= cols) {
+    const float *p = src + static_cast<int64_t>(row) * ld_src;
+    if (live && wide) {
 #pragma unroll
       for (int k = 0; k < 4; ++k) {
-        const float4 a = __ldg(reinterpret_cast<const float4 *>(p) + k);
-        v[4 * k] = a.x; v[4 * k + 1] = a.y; v[4 * k + 2] = a.z; v[4 * k + 3] = a.w;
+        const float4 a = __ldg(reinterpret_cast<const float4 *>(p + b * kBlock) + 4 * k + l);
+        q.v[4 * k] = a.x; q.v[4 * k + 1] = a.y; q.v[4 * k + 2] = a.z; q.v[4 * k + 3] = a.w;
       }
     } else {
 #pragma unroll
-      for (int j = 0; j < 16; ++j) v[j] = (q.live && q.c0 + j < cols) ? __ldg(p + j) : 0.0f;
+      for (int j = 0; j < 16; ++j) q.v[j] = (live && c0 + j < cols) ? __ldg(p + c0 + j) : 0.0f;
     }
   };
 
-  QuantItem cur = item_of(0);
-  float v[16], Mold;
-  uint2 old;
-  fetch(cur, v, old, Mold);
-#pragma unroll 1
-  for (uint32_t it = 0; it < trips; ++it) {
-    const QuantItem nxt = item_of(it + 1);
-    float vn[16], Mn;
-    uint2 oldn;
-    fetch(nxt, vn, oldn, Mn);  // in flight while this item is quantised
-
+  // Quantises one item whose loads have arrived.  Every thread of a warp calls this
+  // the same number of times (the shuffles need all lanes).
+  auto work = [&](int row, QuantLoad &q) {
+    const bool live = col_live && row < rows;
+    if (kRequant) {
+      const uint2 x = exchange(q.old);
+      if (wide) q.old = x;
+    }
     float m = 0.0f;
 #pragma unroll
     for (int j = 0; j < 16; ++j) {
       if (kRequant) {
-        const uint32_t code = ((j < 8 ? old.x : old.y) >> (4 * (j & 7))) & 15u;
-        v[j] = fmaf(s, v[j], Mold * tab.level[code]);
+        const uint32_t code = ((j < 8 ? q.old.x : q.old.y) >> (4 * (j & 7))) & 15u;
+        q.v[j] = fmaf(s, q.v[j], q.Mold * tab.level[code]);
       }
-      m = fmaxf(m, fabsf(v[j]));
+      m = fmaxf(m, fabsf(q.v[j]));
     }
     // (requantiser: every thread of the block has read the old scale by now - the
     // shuffles need its value - so lane 0 may replace it below)
     m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 1));
     m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 2));
-    if (cur.live) {
-      uint2 w = make_uint2(kZeroWord, kZeroWord);
-      if (m > 0.0f) {
-        const Nf4Divisor d = nf4_divisor(m);
-        const float lo[8] = {v[0], v[1], v[2], v[3], v[4], v[5], v[6], v[7]};
-        const float hi[8] = {v[8], v[9], v[10], v[11], v[12], v[13], v[14], v[15]};
-        if (d.exact) {
-          w.x = nf4_quantize8<true>(tab, lo, d);
-          w.y = nf4_quantize8<true>(tab, hi, d);
-        } else {
-          w.x = nf4_quantize8<false>(tab, lo, d);
-          w.y = nf4_quantize8<false>(tab, hi, d);
-        }
-      }
-      *reinterpret_cast<uint2 *>(codes + static_cast<int64_t>(cur.row) * (ld / 2) + (cur.c0 >> 1)) = w;
-      if (l == 0) absmax[static_cast<int64_t>(cur.row) * nb + cur.b] = m;
-      if (kMode == kQuantiseResidual && cur.c0 < cols) {
-        const float *rp = ref + static_cast<int64_t>(cur.row) * ld_ref + cur.c0;
-        __nv_bfloat16 *dp = resid + static_cast<int64_t>(cur.row) * ld_resid + cur.c0;
-        const bool full = kVec && (cur.c0 + 16 <= cols);
-        float e[16];
-#pragma unroll
-        for (int j = 0; j < 16; ++j) {
-          const uint32_t code = ((j < 8 ? w.x : w.y) >> (4 * (j & 7))) & 15u;
-          const float t = (full || cur.c0 + j < cols) ? (ref == src ? v[j] : __ldg(rp + j)) : 0.0f;
-          e[j] = __fsub_rn(t, __fmul_rn(m, tab.level[code]));  // two roundings, as the definition has them
-        }
-        if (full) {
-#pragma unroll
-          for (int g = 0; g < 2; ++g) {
-            uint4 pk;
-            pk.x = pack_bf16x2(e[8 * g + 0], e[8 * g + 1]);
-            pk.y = pack_bf16x2(e[8 * g + 2], e[8 * g + 3]);
-            pk.z = pack_bf16x2(e[8 * g + 4], e[8 * g + 5]);
-            pk.w = pack_bf16x2(e[8 * g + 6], e[8 * g + 7]);
-            reinterpret_cast<uint4 *>(dp)[g] = pk;
-          }
-        } else {
-#pragma unroll
-          for (int j = 0; j < 16; ++j)
-            if (cur.c0 + j < cols) dp[j] = __float2bfloat16_rn(e[j]);
-        }
+    uint2 w = make_uint2(kZeroWord, kZeroWord);  // codes of v[0..15]
+    if (live && m > 0.0f) {
+      const Nf4Divisor d = nf4_divisor(m);
+      const float lo[8] = {q.v[0], q.v[1], q.v[2], q.v[3], q.v[4], q.v[5], q.v[6], q.v[7]};
+      const float hi[8] = {q.v[8], q.v[9], q.v[10], q.v[11], q.v[12], q.v[13], q.v[14], q.v[15]};
+      if (d.exact) {
+        w.x = nf4_quantize8<true>(tab, lo, d);
+        w.y = nf4_quantize8<true>(tab, hi, d);
+      } else {
+        w.x = nf4_quantize8<false>(tab, lo, d);
+        w.y = nf4_quantize8<false>(tab, hi, d);
       }
     }
-    cur = nxt;
-    old = oldn;
-    Mold = Mn;
+    const uint2 wx = exchange(w);  // (every lane: the shuffles need the whole warp)
+    if (!live) return;
+    *reinterpret_cast<uint2 *>(codes + static_cast<int64_t>(row) * (ld / 2) + (c0 >> 1)) = wide ? wx : w;
+    if (l == 0) absmax[static_cast<int64_t>(row) * nb + b] = m;
+    if (kMode == kQuantiseResidual && c0 < cols) {
+      const float *rp = ref + static_cast<int64_t>(row) * ld_ref;
+      __nv_bfloat16 *dp = resid + static_cast<int64_t>(row) * ld_resid;
+      float e[16];
 #pragma unroll
-    for (int j = 0; j < 16; ++j) v[j] = vn[j];
+      for (int j = 0; j < 16; ++j) {
+        const uint32_t code = ((j < 8 ? w.x : w.y) >> (4 * (j & 7))) & 15u;
+        const float t = (wide || c0 + j < cols) ? (ref == src ? q.v[j] : __ldg(rp + elem(j))) : 0.0f;
+        e[j] = __fsub_rn(t, __fmul_rn(m, tab.level[code]));  // two roundings, as the definition has them
+      }
+      if (wide) {
+#pragma unroll
+        for (int k = 0; k < 4; ++k)  // four runs of four elements, 8 bytes each
+          *reinterpret_cast<uint2 *>(dp + elem(4 * k)) = make_uint2(pack_bf16x2(e[4 * k], e[4 * k + 1]), pack_bf16x2(e[4 * k + 2], e[4 * k + 3]));
+      } else {
+#pragma unroll
+        for (int j = 0; j < 16; ++j)
+          if (c0 + j < cols) dp[c0 + j] = __float2bfloat16_rn(e[j]);
+      }
+    }
+  };
+
+  // Two rows per trip: both rows' loads are issued before the first is worked on.
+  // (Keeping the loads of a further pair in flight costs registers and occupancy and
+  // was measured slower.)
+#pragma unroll 1
+  for (int base = row_first; base < rows; base += 2 * row_stride) {
+    QuantLoad qa, qb;
+    const int ra = base + gy, rb = ra + row_stride;
+    fetch(ra, qa);
+    fetch(rb, qb);
+    work(ra, qa);
+    work(rb, qb);
   }
 }
 
 // ---------------------------------------------------------------------------
 // dequantise: one thread per 8 consecutive elements (one 32-bit word of codes,
-// one 16- or 32-byte store, so that a warp's stores are contiguous), four
-// independent words per trip so that enough loads are in flight.
+// one 16- or 32-byte store, so that a warp's stores are contiguous), the words
+// of four rows in flight per trip.  Two codes are looked up at a time: a byte of
+// the code word indexes a 256-entry table of level pairs, and one packed
+// multiply scales the pair.
 // ---------------------------------------------------------------------------
-constexpr int kDqUnroll = 4;
+constexpr int kDqRows = 4;  // rows a thread has in flight
 
-// Expands the code words first, first + stride, ... of one matrix.
 // Doubly quantised scales of a matrix (null codes8: plain fp32 scales are used).
 struct DqScales {
   const uint8_t *codes8;
@@ -169,111 +225,90 @@ struct DqScales {
   const float *offset;
 };
 
-template <bool kBf16, bool kVec, bool kDq = false>
-__device__ __forceinline__ void dequantize_words(const Nf4Tables &tab, const uint8_t *__restrict__ codes,
-                                                 const float *__restrict__ absmax, void *__restrict__ dst, int64_t ld_dst,
-                                                 int rows, int cols, int ld, uint32_t first, uint32_t stride,
-                                                 DqScales dq = DqScales{nullptr, nullptr, nullptr}) {
-  const uint32_t wpr = static_cast<uint32_t>(ld / 8);  // code words per row
-  const uint32_t nb = static_cast<uint32_t>(ld / kBlock);
-  const uint32_t n_items = static_cast<uint32_t>(rows) * wpr;  // (host checks < 2^31)
+struct Nf4PairTable {
+  float2 pair[256];  // pair[b] = {level[b & 15], level[b >> 4]}
+};
+__device__ __forceinline__ void nf4_pairs_init(Nf4PairTable &t, int tid) {
+  if (tid < 256) t.pair[tid] = make_float2(c_nf4_level[tid & 15], c_nf4_level[tid >> 4]);
+}
 
-  struct Word {
-    uint32_t w, row;
-    int c0;
-    float M;
-    bool live;
-  };
-  auto fetch = [&](uint32_t item) {
-    Word q;
-    q.live = item < n_items;
-    q.row = q.live ? item / wpr : 0;
-    const uint32_t h = q.live ? item - q.row * wpr : 0;
-    q.c0 = static_cast<int>(h) * 8;
-    q.live = q.live && q.c0 < cols;
-    q.w = kZeroWord;
-    q.M = 0.0f;
-    if (q.live) {
-      q.w = __ldg(reinterpret_cast<const uint32_t *>(codes + static_cast<int64_t>(q.row) * (ld / 2)) + h);
-      const int64_t si = static_cast<int64_t>(q.row) * nb + (h >> 3);
-      q.M = kDq ? dq_scale(dq.codes8, dq.c1, dq.offset, si) : __ldg(absmax + si);
-    }
-    return q;
-  };
-
-  Word cur[kDqUnroll];
-#pragma unroll
-  for (int u = 0; u < kDqUnroll; ++u) cur[u] = fetch(first + u * stride);
+// Expands word h (elements 8 h .. 8 h + 7) of rows row0, row0 + row_stride, ...
+template <bool kBf16, bool kVec, bool kDq>
+__device__ __forceinline__ void dequantize_rows(const Nf4PairTable &tab, const uint8_t *__restrict__ codes,
+                                                const float *__restrict__ absmax, DqScales dq, void *__restrict__ dst,
+                                                int64_t ld_dst, int rows, int cols, int ld, int h, int row0, int row_stride) {
+  const int wpr = ld / 8, nb = ld / kBlock;
+  const int c0 = h * 8;
+  if (h >= wpr || c0 >= cols) return;
+  const bool full = kVec && (c0 + 8 <= cols);
 #pragma unroll 1
-  for (uint32_t base = first; base < n_items; base += kDqUnroll * stride) {
-    Word nxt[kDqUnroll];  // in flight while this trip's words are expanded
+  for (int base = row0; base < rows; base += kDqRows * row_stride) {
+    uint32_t w[kDqRows];
+    float M[kDqRows];
 #pragma unroll
-    for (int u = 0; u < kDqUnroll; ++u) nxt[u] = fetch(base + (kDqUnroll + u) * stride);
-#pragma unroll
-    for (int u = 0; u < kDqUnroll; ++u) {
-      const Word &q = cur[u];
-      if (!q.live) continue;
-      float v[8];
-#pragma unroll
-      for (int j = 0; j < 8; ++j) v[j] = q.M * tab.level[(q.w >> (4 * j)) & 15u];
-      const bool full = kVec && (q.c0 + 8 <= cols);
-      if (kBf16) {
-        __nv_bfloat16 *o = reinterpret_cast<__nv_bfloat16 *>(dst) + static_cast<int64_t>(q.row) * ld_dst + q.c0;
-        if (full) {
-          uint4 pk;
-          pk.x = pack_bf16x2(v[0], v[1]);
-          pk.y = pack_bf16x2(v[2], v[3]);
-          pk.z = pack_bf16x2(v[4], v[5]);
-          pk.w = pack_bf16x2(v[6], v[7]);
-          *reinterpret_cast<uint4 *>(o) = pk;
-        } else {
-#pragma unroll
-          for (int j = 0; j < 8; ++j)
-            if (q.c0 + j < cols) o[j] = __float2bfloat16_rn(v[j]);
-        }
-      } else {
-        float *o = reinterpret_cast<float *>(dst) + static_cast<int64_t>(q.row) * ld_dst + q.c0;
-        if (full) {
-          reinterpret_cast<float4 *>(o)[0] = make_float4(v[0], v[1], v[2], v[3]);
-          reinterpret_cast<float4 *>(o)[1] = make_float4(v[4], v[5], v[6], v[7]);
-        } else {
-#pragma unroll
-          for (int j = 0; j < 8; ++j)
-            if (q.c0 + j < cols) o[j] = v[j];
-        }
+    for (int u = 0; u < kDqRows; ++u) {
+      const int row = base + u * row_stride;
+      w[u] = kZeroWord;
+      M[u] = 0.0f;
+      if (row < rows) {
+        w[u] = __ldg(reinterpret_cast<const uint32_t *>(codes) + static_cast<int64_t>(row) * wpr + h);
+        const int64_t si = static_cast<int64_t>(row) * nb + (h >> 3);
+        M[u] = kDq ? dq_scale(dq.codes8, dq.c1, dq.offset, si) : __ldg(absmax + si);
       }
     }
 #pragma unroll
-    for (int u = 0; u < kDqUnroll; ++u) cur[u] = nxt[u];
+    for (int u = 0; u < kDqRows; ++u) {
+      const int row = base + u * row_stride;
+      if (row >= rows) break;
+      const float2 M2 = make_float2(M[u], M[u]);
+      float2 p[4];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) p[j] = __fmul2_rn(M2, tab.pair[(w[u] >> (8 * j)) & 0xFFu]);
+      if (kBf16) {
+        __nv_bfloat16 *o = reinterpret_cast<__nv_bfloat16 *>(dst) + static_cast<int64_t>(row) * ld_dst + c0;
+        if (full) {
+          *reinterpret_cast<uint4 *>(o) = make_uint4(pack_bf16x2(p[0].x, p[0].y), pack_bf16x2(p[1].x, p[1].y),
+                                                     pack_bf16x2(p[2].x, p[2].y), pack_bf16x2(p[3].x, p[3].y));
+        } else {
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            if (c0 + 2 * j < cols) o[2 * j] = __float2bfloat16_rn(p[j].x);
+            if (c0 + 2 * j + 1 < cols) o[2 * j + 1] = __float2bfloat16_rn(p[j].y);
+          }
+        }
+      } else {
+        float *o = reinterpret_cast<float *>(dst) + static_cast<int64_t>(row) * ld_dst + c0;
+        if (full) {
+          reinterpret_cast<float4 *>(o)[0] = make_float4(p[0].x, p[0].y, p[1].x, p[1].y);
+          reinterpret_cast<float4 *>(o)[1] = make_float4(p[2].x, p[2].y, p[3].x, p[3].y);
+        } else {
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            if (c0 + 2 * j < cols) o[2 * j] = p[j].x;
+            if (c0 + 2 * j + 1 < cols) o[2 * j + 1] = p[j].y;
+          }
+        }
+      }
+    }
   }
 }
 
-template <bool kBf16, bool kVec>
+template <bool kBf16, bool kVec, bool kDq>
 __global__ void __launch_bounds__(kQThreads)
-nf4_dequantize_kernel(const uint8_t *__restrict__ codes, const float *__restrict__ absmax,
-                      void *__restrict__ dst, int64_t ld_dst, int rows, int cols, int ld) {
-  __shared__ Nf4Tables tab;
-  nf4_tables_init(tab, threadIdx.x);
+nf4_dequantize_kernel(const uint8_t *__restrict__ codes, const float *__restrict__ absmax, DqScales dq,
+                      void *__restrict__ dst, int64_t ld_dst, int rows, int cols, int ld, int wx_log2) {
+  __shared__ Nf4PairTable tab;
+  nf4_pairs_init(tab, threadIdx.x);
   __syncthreads();
-  dequantize_words<kBf16, kVec>(tab, codes, absmax, dst, ld_dst, rows, cols, ld, blockIdx.x * kQThreads + threadIdx.x,
-                                gridDim.x * kQThreads);
-}
-
-// The same with doubly quantised block scales (paper Section 2.4).
-template <bool kBf16, bool kVec>
-__global__ void __launch_bounds__(kQThreads)
-nf4_dequantize_dq_kernel(const uint8_t *__restrict__ codes, DqScales dq, void *__restrict__ dst, int64_t ld_dst, int rows,
-                         int cols, int ld) {
-  __shared__ Nf4Tables tab;
-  nf4_tables_init(tab, threadIdx.x);
-  __syncthreads();
-  dequantize_words<kBf16, kVec, true>(tab, codes, nullptr, dst, ld_dst, rows, cols, ld, blockIdx.x * kQThreads + threadIdx.x,
-                                      gridDim.x * kQThreads, dq);
+  const int tx = threadIdx.x & ((1 << wx_log2) - 1), ty = threadIdx.x >> wx_log2;
+  const int rows_per_pass = kQThreads >> wx_log2;
+  dequantize_rows<kBf16, kVec, kDq>(tab, codes, absmax, dq, dst, ld_dst, rows, cols, ld, (static_cast<int>(blockIdx.x) << wx_log2) + tx,
+                                    static_cast<int>(blockIdx.y) * rows_per_pass + ty, static_cast<int>(gridDim.y) * rows_per_pass);
 }
 
 // Several matrices to bf16 in one launch (the staging step of a batched merge):
-// the grid is dealt to the matrices in proportion to their sizes, blocks cta0 ..
-// cta0 + ctas - 1 stride over matrix i.
+// the grid is dealt to the matrices in proportion to their sizes; blocks cta0 ..
+// cta0 + ctas - 1 work on matrix i, `chunks` of them side by side along a row.
 struct DequantBatch {
   struct Item {
     const uint8_t *codes;
@@ -281,7 +316,7 @@ struct DequantBatch {
     void *dst;
     int64_t ld_dst;
     int rows, cols, ld;
-    int cta0, ctas;
+    int cta0, ctas, chunks, wx_log2;
   } item[kStageBatchMax];
   int count;
 };
@@ -289,49 +324,63 @@ struct DequantBatch {
 template <bool kVec>
 __global__ void __launch_bounds__(kQThreads)
 nf4_dequantize_batch_kernel(const __grid_constant__ DequantBatch batch) {
-  __shared__ Nf4Tables tab;
-  nf4_tables_init(tab, threadIdx.x);
+  __shared__ Nf4PairTable tab;
+  nf4_pairs_init(tab, threadIdx.x);
   __syncthreads();
   int i = 0;
   while (i + 1 < batch.count && static_cast<int>(blockIdx.x) >= batch.item[i + 1].cta0) ++i;
   const DequantBatch::Item &m = batch.item[i];
-  const uint32_t local = blockIdx.x - static_cast<uint32_t>(m.cta0);
-  dequantize_words<true, kVec>(tab, m.codes, m.absmax, m.dst, m.ld_dst, m.rows, m.cols, m.ld, local * kQThreads + threadIdx.x,
-                               static_cast<uint32_t>(m.ctas) * kQThreads);
+  const int local = static_cast<int>(blockIdx.x) - m.cta0;
+  const int bx = local % m.chunks, by = local / m.chunks;
+  const int tx = threadIdx.x & ((1 << m.wx_log2) - 1), ty = threadIdx.x >> m.wx_log2;
+  const int rows_per_pass = kQThreads >> m.wx_log2;
+  dequantize_rows<true, kVec, false>(tab, m.codes, m.absmax, DqScales{nullptr, nullptr, nullptr}, m.dst, m.ld_dst, m.rows, m.cols, m.ld,
+                                     (bx << m.wx_log2) + tx, by * rows_per_pass + ty, (m.ctas / m.chunks) * rows_per_pass);
 }
 
-// Grid of a streaming kernel: enough blocks for the work, at most as many as
-// are resident at once (the kernels loop with a grid stride).
-template <typename Kernel>
-static int grid_for(Kernel kernel, int64_t threads_needed) {
-  int per_sm = 0;
-  if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, kQThreads, 0) != cudaSuccess || per_sm < 1) per_sm = 1;
-  int64_t blocks = (threads_needed + kQThreads - 1) / kQThreads;
-  const int64_t cap = static_cast<int64_t>(sm_count()) * per_sm;
-  if (blocks > cap) blocks = cap;
-  if (blocks < 1) blocks = 1;
-  return static_cast<int>(blocks);
-}
-
-// fp32 -> bf16 (round to nearest even), row-major with leading dimensions.
+// fp32 -> bf16 (round to nearest even), row-major with leading dimensions: one
+// thread per 8 consecutive elements of a row, rows walked as above.
+template <bool kVec>
 __global__ void __launch_bounds__(kQThreads)
 convert_f32_bf16_kernel(const float *__restrict__ src, int64_t ld_src, __nv_bfloat16 *__restrict__ dst, int64_t ld_dst,
-                        int rows, int cols) {
-  const int64_t total = static_cast<int64_t>(rows) * cols;
-  const int64_t stride = static_cast<int64_t>(gridDim.x) * kQThreads;
-  for (int64_t i = static_cast<int64_t>(blockIdx.x) * kQThreads + threadIdx.x; i < total; i += stride) {
-    const int r = static_cast<int>(i / cols);
-    const int c = static_cast<int>(i - static_cast<int64_t>(r) * cols);
-    dst[static_cast<int64_t>(r) * ld_dst + c] = __float2bfloat16_rn(__ldg(src + static_cast<int64_t>(r) * ld_src + c));
+                        int rows, int cols, int wx_log2) {
+  const int tx = threadIdx.x & ((1 << wx_log2) - 1), ty = threadIdx.x >> wx_log2;
+  const int rows_per_pass = kQThreads >> wx_log2;
+  const int c0 = ((static_cast<int>(blockIdx.x) << wx_log2) + tx) * 8;
+  if (c0 >= cols) return;
+  const bool full = kVec && c0 + 8 <= cols;
+  const int row_stride = static_cast<int>(gridDim.y) * rows_per_pass;
+  for (int row = static_cast<int>(blockIdx.y) * rows_per_pass + ty; row < rows; row += row_stride) {
+    const float *p = src + static_cast<int64_t>(row) * ld_src + c0;
+    __nv_bfloat16 *o = dst + static_cast<int64_t>(row) * ld_dst + c0;
+    if (full) {
+      const float4 a = __ldg(reinterpret_cast<const float4 *>(p)), b = __ldg(reinterpret_cast<const float4 *>(p) + 1);
+      *reinterpret_cast<uint4 *>(o) = make_uint4(pack_bf16x2(a.x, a.y), pack_bf16x2(a.z, a.w), pack_bf16x2(b.x, b.y), pack_bf16x2(b.z, b.w));
+    } else {
+      for (int j = 0; j < 8 && c0 + j < cols; ++j) o[j] = __float2bfloat16_rn(__ldg(p + j));
+    }
   }
 }
 
 loqt_status convert_f32_bf16(const float *src, int64_t ld_src, void *dst, int64_t ld_dst, int rows, int cols,
                              cudaStream_t stream) {
-  const int64_t total = static_cast<int64_t>(rows) * cols;
-  if (total <= 0) return LOQT_OK;
-  convert_f32_bf16_kernel<<<grid_for(convert_f32_bf16_kernel, total), kQThreads, 0, stream>>>(
-      src, ld_src, static_cast<__nv_bfloat16 *>(dst), ld_dst, rows, cols);
+  if (rows <= 0 || cols <= 0) return LOQT_OK;
+  const bool vec = ((reinterpret_cast<uintptr_t>(src) | reinterpret_cast<uintptr_t>(dst)) & 15u) == 0 && (ld_src % 4) == 0 && (ld_dst % 8) == 0;
+  auto kernel = vec ? convert_f32_bf16_kernel<true> : convert_f32_bf16_kernel<false>;
+  const RowDeal d = deal_rows((cols + 7) / 8, kQThreads, rows, resident_blocks(kernel));
+  kernel<<<d.grid, kQThreads, 0, stream>>>(src, ld_src, static_cast<__nv_bfloat16 *>(dst), ld_dst, rows, cols, d.log2);
+  count_launch();
+  return cudaGetLastError() == cudaSuccess ? LOQT_OK : LOQT_ERR_CUDA;
+}
+
+// Launch of the quantiser in one of its three modes.
+template <int kMode>
+static loqt_status launch_quantiser(const float *src, int64_t ld_src, float s, const loqt_nf4_mat &dst, const float *ref, int64_t ld_ref,
+                                    void *resid, int64_t ld_resid, bool vec, cudaStream_t stream) {
+  auto kernel = vec ? nf4_quantize_kernel<true, kMode> : nf4_quantize_kernel<false, kMode>;
+  const RowDeal d = deal_rows(dst.ld / kBlock, kQThreads / 4, dst.rows, resident_blocks(kernel));
+  kernel<<<d.grid, kQThreads, 0, stream>>>(src, ld_src, s, dst.codes, dst.absmax, dst.rows, dst.cols, dst.ld, ref, ld_ref,
+                                           static_cast<__nv_bfloat16 *>(resid), ld_resid, d.log2);
   count_launch();
   return cudaGetLastError() == cudaSuccess ? LOQT_OK : LOQT_ERR_CUDA;
 }
@@ -343,11 +392,7 @@ loqt_status nf4_quantize_residual(const float *src, int64_t ld_src, const float 
   if (items >= (1ll << 30)) return LOQT_ERR_UNSUPPORTED;
   const bool vec = ((reinterpret_cast<uintptr_t>(src) | reinterpret_cast<uintptr_t>(ref) | reinterpret_cast<uintptr_t>(resid)) & 15u) == 0 &&
                    (ld_src % 4) == 0 && (ld_ref % 4) == 0 && (ld_resid % 8) == 0;
-  auto kernel = vec ? nf4_quantize_kernel<true, kQuantiseResidual> : nf4_quantize_kernel<false, kQuantiseResidual>;
-  kernel<<<grid_for(kernel, items * 4), kQThreads, 0, stream>>>(src, ld_src, 1.0f, dst.codes, dst.absmax, dst.rows, dst.cols, dst.ld, ref,
-                                                                ld_ref, static_cast<__nv_bfloat16 *>(resid), ld_resid);
-  count_launch();
-  return cudaGetLastError() == cudaSuccess ? LOQT_OK : LOQT_ERR_CUDA;
+  return launch_quantiser<kQuantiseResidual>(src, ld_src, 1.0f, dst, ref, ld_ref, resid, ld_resid, vec, stream);
 }
 
 // dst_i <- bf16(deq(src_i)) for up to kStageBatchMax matrices, one launch.
@@ -366,20 +411,33 @@ loqt_status nf4_dequantize_bf16_batch(const StageItem *items, int n, cudaStream_
     vec = vec && (reinterpret_cast<uintptr_t>(items[i].dst) & 15u) == 0 && (items[i].ld_dst % 8) == 0;
   }
   auto kernel = vec ? nf4_dequantize_batch_kernel<true> : nf4_dequantize_batch_kernel<false>;
-  const int cap = grid_for(kernel, (total + kDqUnroll - 1) / kDqUnroll);
+  const int resident = resident_blocks(kernel);
   int next = 0;
   for (int i = 0; i < n; ++i) {
     const loqt_nf4_mat &m = items[i].src;
     const int64_t words = static_cast<int64_t>(m.rows) * (m.ld / 8);
-    int64_t ctas = (words * cap + total - 1) / total;                     // share of the grid
-    const int64_t need = (words + kQThreads * kDqUnroll - 1) / (kQThreads * kDqUnroll);  // blocks with work
-    if (ctas > need) ctas = need;
-    if (ctas < 1) ctas = 1;
-    batch.item[i] = {m.codes, m.absmax, items[i].dst, items[i].ld_dst, m.rows, m.cols, m.ld, next, static_cast<int>(ctas)};
-    next += static_cast<int>(ctas);
+    int share = static_cast<int>((words * resident + total - 1) / total);  // this matrix's part of the resident grid
+    if (share < 1) share = 1;
+    const RowDeal d = deal_rows(m.ld / 8, kQThreads, (m.rows + kDqRows - 1) / kDqRows, share);
+    const int chunks = static_cast<int>(d.grid.x), ctas = chunks * static_cast<int>(d.grid.y);
+    batch.item[i] = {m.codes, m.absmax, items[i].dst, items[i].ld_dst, m.rows, m.cols, m.ld, next, ctas, chunks, d.log2};
+    next += ctas;
   }
   batch.count = n;
   kernel<<<next, kQThreads, 0, stream>>>(batch);
+  count_launch();
+  return cudaGetLastError() == cudaSuccess ? LOQT_OK : LOQT_ERR_CUDA;
+}
+
+// One matrix, fp32 or doubly quantised scales, bf16 or fp32 output.
+template <bool kDq>
+static loqt_status launch_dequantiser(const loqt_nf4_mat &src, DqScales dq, void *dst, int64_t ld_dst, int dst_is_bf16, cudaStream_t stream) {
+  const uintptr_t a = reinterpret_cast<uintptr_t>(dst);
+  const bool vec = (a & 15u) == 0 && (ld_dst % (dst_is_bf16 ? 8 : 4)) == 0;
+  auto kernel = dst_is_bf16 ? (vec ? nf4_dequantize_kernel<true, true, kDq> : nf4_dequantize_kernel<true, false, kDq>)
+                            : (vec ? nf4_dequantize_kernel<false, true, kDq> : nf4_dequantize_kernel<false, false, kDq>);
+  const RowDeal d = deal_rows(src.ld / 8, kQThreads, (src.rows + kDqRows - 1) / kDqRows, resident_blocks(kernel));
+  kernel<<<d.grid, kQThreads, 0, stream>>>(src.codes, src.absmax, dq, dst, ld_dst, src.rows, src.cols, src.ld, d.log2);
   count_launch();
   return cudaGetLastError() == cudaSuccess ? LOQT_OK : LOQT_ERR_CUDA;
 }
@@ -395,14 +453,9 @@ extern "C" loqt_status loqt_nf4_quantize(const float *src, int64_t ld_src, loqt_
   if ((reinterpret_cast<uintptr_t>(src) & 3u) != 0) return LOQT_ERR_ALIGNMENT;
   if ((st = check_arch()) != LOQT_OK) return st;
   const int64_t items = static_cast<int64_t>(dst.rows) * (dst.ld / kBlock);
-  if (items >= (1ll << 30)) return LOQT_ERR_UNSUPPORTED;  // 32-bit block indices in the kernel
+  if (items >= (1ll << 30)) return LOQT_ERR_UNSUPPORTED;
   const bool vec = (reinterpret_cast<uintptr_t>(src) & 15u) == 0 && (ld_src % 4) == 0;
-  cudaStream_t s = static_cast<cudaStream_t>(stream);
-  auto kernel = vec ? nf4_quantize_kernel<true, kQuantise> : nf4_quantize_kernel<false, kQuantise>;
-  kernel<<<grid_for(kernel, items * 4), kQThreads, 0, s>>>(src, ld_src, 1.0f, dst.codes, dst.absmax, dst.rows, dst.cols, dst.ld, nullptr, 0,
-                                                           nullptr, 0);
-  count_launch();
-  return cudaGetLastError() == cudaSuccess ? LOQT_OK : LOQT_ERR_CUDA;
+  return launch_quantiser<kQuantise>(src, ld_src, 1.0f, dst, nullptr, 0, nullptr, 0, vec, static_cast<cudaStream_t>(stream));
 }
 
 extern "C" loqt_status loqt_nf4_dequantize(loqt_nf4_mat src, void *dst, int64_t ld_dst, int dst_is_bf16,
@@ -414,15 +467,8 @@ extern "C" loqt_status loqt_nf4_dequantize(loqt_nf4_mat src, void *dst, int64_t 
   if ((a & (dst_is_bf16 ? 1u : 3u)) != 0) return LOQT_ERR_ALIGNMENT;
   if ((st = check_arch()) != LOQT_OK) return st;
   const int64_t items = static_cast<int64_t>(src.rows) * (src.ld / 8);
-  if (items >= (1ll << 31)) return LOQT_ERR_UNSUPPORTED;  // 32-bit word indices in the kernel
-  cudaStream_t s = static_cast<cudaStream_t>(stream);
-  const bool vec = (a & 15u) == 0 && (ld_dst % (dst_is_bf16 ? 8 : 4)) == 0;
-  auto kernel = dst_is_bf16 ? (vec ? nf4_dequantize_kernel<true, true> : nf4_dequantize_kernel<true, false>)
-                            : (vec ? nf4_dequantize_kernel<false, true> : nf4_dequantize_kernel<false, false>);
-  kernel<<<grid_for(kernel, (items + kDqUnroll - 1) / kDqUnroll), kQThreads, 0, s>>>(src.codes, src.absmax, dst, ld_dst, src.rows,
-                                                                                     src.cols, src.ld);
-  count_launch();
-  return cudaGetLastError() == cudaSuccess ? LOQT_OK : LOQT_ERR_CUDA;
+  if (items >= (1ll << 31)) return LOQT_ERR_UNSUPPORTED;
+  return launch_dequantiser<false>(src, DqScales{nullptr, nullptr, nullptr}, dst, ld_dst, dst_is_bf16, static_cast<cudaStream_t>(stream));
 }
 
 extern "C" loqt_status loqt_nf4_requantize(const float *delta, int64_t ld_delta, float s, loqt_nf4_mat Wq, void *stream) {
@@ -432,14 +478,9 @@ extern "C" loqt_status loqt_nf4_requantize(const float *delta, int64_t ld_delta,
   if ((reinterpret_cast<uintptr_t>(delta) & 3u) != 0) return LOQT_ERR_ALIGNMENT;
   if ((st = check_arch()) != LOQT_OK) return st;
   const int64_t items = static_cast<int64_t>(Wq.rows) * (Wq.ld / kBlock);
-  if (items >= (1ll << 30)) return LOQT_ERR_UNSUPPORTED;  // 32-bit block indices in the kernel
+  if (items >= (1ll << 30)) return LOQT_ERR_UNSUPPORTED;
   const bool vec = (reinterpret_cast<uintptr_t>(delta) & 15u) == 0 && (ld_delta % 4) == 0;
-  cudaStream_t stm = static_cast<cudaStream_t>(stream);
-  auto kernel = vec ? nf4_quantize_kernel<true, kRequantise> : nf4_quantize_kernel<false, kRequantise>;
-  kernel<<<grid_for(kernel, items * 4), kQThreads, 0, stm>>>(delta, ld_delta, s, Wq.codes, Wq.absmax, Wq.rows, Wq.cols, Wq.ld, nullptr, 0,
-                                                             nullptr, 0);
-  count_launch();
-  return cudaGetLastError() == cudaSuccess ? LOQT_OK : LOQT_ERR_CUDA;
+  return launch_quantiser<kRequantise>(delta, ld_delta, s, Wq, nullptr, 0, nullptr, 0, vec, static_cast<cudaStream_t>(stream));
 }
 
 extern "C" loqt_status loqt_nf4_dequantize_dq(loqt_nf4_mat src, loqt_dq_scales dq, void *dst, int64_t ld_dst, int dst_is_bf16,
@@ -455,11 +496,5 @@ extern "C" loqt_status loqt_nf4_dequantize_dq(loqt_nf4_mat src, loqt_dq_scales d
   if ((st = check_arch()) != LOQT_OK) return st;
   const int64_t items = static_cast<int64_t>(src.rows) * (src.ld / 8);
   if (items >= (1ll << 31)) return LOQT_ERR_UNSUPPORTED;
-  const bool vec = (a & 15u) == 0 && (ld_dst % (dst_is_bf16 ? 8 : 4)) == 0;
-  auto kernel = dst_is_bf16 ? (vec ? nf4_dequantize_dq_kernel<true, true> : nf4_dequantize_dq_kernel<true, false>)
-                            : (vec ? nf4_dequantize_dq_kernel<false, true> : nf4_dequantize_dq_kernel<false, false>);
-  kernel<<<grid_for(kernel, (items + kDqUnroll - 1) / kDqUnroll), kQThreads, 0, static_cast<cudaStream_t>(stream)>>>(
-      src.codes, DqScales{dq.codes8, dq.c1, dq.offset}, dst, ld_dst, src.rows, src.cols, src.ld);
-  count_launch();
-  return cudaGetLastError() == cudaSuccess ? LOQT_OK : LOQT_ERR_CUDA;
+  return launch_dequantiser<true>(src, DqScales{dq.codes8, dq.c1, dq.offset}, dst, ld_dst, dst_is_bf16, static_cast<cudaStream_t>(stream));
 }
