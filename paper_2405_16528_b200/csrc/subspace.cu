@@ -7,21 +7,31 @@
 // them each m x r iterate Y is replaced by an orthonormal basis of its columns.
 //
 // orth(Y) here is Cholesky QR carried out in double precision on the CUDA
-// cores: S = Y^T Y, S = L L^T, Q = Y L^-T.  The first iterate Y = G Omega of a
-// square Gaussian test block has a condition number of several thousand times
-// sigma_1 / sigma_r; in double precision the Gram matrix keeps its square (up
-// to about 1e14) without losing positive definiteness, so one pass gives a
-// basis orthonormal to 1e-16 cond(Y)^2.  Everything is tiled 64 x 64; no kernel
-// waits on another CTA (one launch per dependent step), and all sums run in a
-// fixed order, so results are reproducible.
+// cores: S = Y^T Y, S = L L^T, X = L^-1, Q = Y X^T.  Double precision because the
+// Gram matrix squares the condition number of Y: with cond(Y) up to 1e6 one pass
+// still gives a basis orthonormal to 1e-4, where single precision would lose
+// positive definiteness beyond cond(Y) of a few thousand.
+//
+//   gram_kernel        S = Y^T Y        128 x 128 tiles of the lower triangle, the rows of Y
+//                                       split among CTAs, partial sums added in a fixed order
+//   chol_panel_kernel  S = L L^T        right-looking, 64 columns per step: the diagonal block
+//   chol_update_kernel                  is factored and inverted in shared memory, the panel
+//                                       below it formed, the trailing matrix updated
+//   block_gemm_kernel  X = L^-1         by doubling: with the diagonal blocks A^-1, B^-1 of size h
+//                                       known, the block below is -B^-1 C A^-1 (two products per
+//                                       level, log2(r / 64) levels)
+//   apply_kernel       Q = Y X^T        one triangular product, 128 x 128 tiles
+//
+// No kernel waits on another CTA (one launch per dependent step), and all sums
+// run in a fixed order, so results are reproducible.
 #include "common.cuh"
 
 namespace loqt {
 
 namespace {
 
-constexpr int kT = 64;        // tile edge
-constexpr int kTP = kT + 1;   // padded row of a shared-memory tile (doubles)
+constexpr int kT = 64;       // tile edge of the factorisation
+constexpr int kTP = kT + 1;  // padded row of a 64-wide shared-memory tile (doubles)
 
 // acc[i][j] += sum_k a[k][row0 + i] * b[k][col0 + j], k < kc; a and b are
 // shared-memory tiles stored k-outermost with padded rows of kTP doubles.
@@ -40,6 +50,37 @@ __device__ __forceinline__ void tile_fma(double (&acc)[4][4], const double *a, c
   }
 }
 
+// The two large products work on 128 x 128 tiles: 256 threads as 16 x 16, each
+// with an 8 x 8 block of the tile in registers.  Thread (ty, tx) owns rows
+// 2 ty + 32 q + e and columns 2 tx + 32 q' + e' (q, q' = 0..3; e, e' = 0, 1), so that
+// a warp's 16-byte loads of the column operand are contiguous and those of the row
+// operand are broadcasts: 64 fused multiply-adds per 8 loads, which leaves the
+// double-precision pipe, not shared memory, as the limit.
+constexpr int kG = 128;      // tile edge
+constexpr int kGP = kG + 2;  // padded row (doubles): rows stay 16-byte aligned
+constexpr int kGK = 16;      // k-chunk staged per step
+constexpr size_t kBigSmem = 2 * 2 * kGK * kGP * sizeof(double);  // two operands, two buffers
+
+__device__ __forceinline__ int own8(int t, int i) { return 2 * t + 32 * (i >> 1) + (i & 1); }
+
+__device__ __forceinline__ void tile_fma8(double (&acc)[8][8], const double *a, const double *b, int ty, int tx) {
+#pragma unroll 2
+  for (int k = 0; k < kGK; ++k) {
+    double2 av[4], bv[4];
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      av[q] = *reinterpret_cast<const double2 *>(a + k * kGP + 2 * ty + 32 * q);
+      bv[q] = *reinterpret_cast<const double2 *>(b + k * kGP + 2 * tx + 32 * q);
+    }
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      const double ai = (i & 1) ? av[i >> 1].y : av[i >> 1].x;
+#pragma unroll
+      for (int j = 0; j < 8; ++j) acc[i][j] = fma(ai, (j & 1) ? bv[j >> 1].y : bv[j >> 1].x, acc[i][j]);
+    }
+  }
+}
+
 // Lower-triangle tile number t -> (bi, bj), bj <= bi.
 __device__ __forceinline__ void lower_tile(int t, int &bi, int &bj) {
   int i = static_cast<int>((sqrtf(8.0f * static_cast<float>(t) + 1.0f) - 1.0f) * 0.5f);
@@ -49,38 +90,77 @@ __device__ __forceinline__ void lower_tile(int t, int &bi, int &bj) {
   bj = t - i * (i + 1) / 2;
 }
 
-// partial[split][rp][rp] (lower tiles only) = sum over this split's rows k of Y[k][i] Y[k][j].
+// partial[split][rp][rp] (128 x 128 tiles of the lower triangle) = sum over this
+// split's rows k of Y[k][i] Y[k][j].  A chunk of 16 rows of Y is staged per step
+// (converted to double), the next chunk's loads are in flight meanwhile.
 __global__ void __launch_bounds__(256)
 gram_kernel(const float *__restrict__ Y, int64_t ldy, int m, int r, int rp, int rows_per_split, double *__restrict__ partial) {
-  __shared__ double As[32 * kTP];
-  __shared__ double Bs[32 * kTP];
+  extern __shared__ __align__(16) double smg[];
   int bi, bj;
   lower_tile(blockIdx.x, bi, bj);
+  const bool diag = bi == bj;
   const int split = blockIdx.y;
   const int k_begin = split * rows_per_split;
   const int k_end = min(m, k_begin + rows_per_split);
   const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
-  double acc[4][4] = {};
-  for (int k0 = k_begin; k0 < k_end; k0 += 32) {
+  // staging: thread -> row kk of the chunk, 8 consecutive columns of the tile
+  const int kk = tid >> 4, i8 = (tid & 15) * 8;
+  const bool vec = (ldy & 3) == 0 && (reinterpret_cast<uintptr_t>(Y) & 15u) == 0;
+  auto fetch = [&](int k0, int tile, float (&v)[8]) {
+    const int row = k0 + kk, col = tile * kG + i8;
 #pragma unroll
-    for (int e = 0; e < 8; ++e) {
-      const int idx = tid + e * 256, kk = idx >> 6, c = idx & 63;
-      const int row = k0 + kk;
-      const int ci = bi * kT + c, cj = bj * kT + c;
-      const bool in_rows = row < k_end;
-      As[kk * kTP + c] = (in_rows && ci < r) ? static_cast<double>(Y[static_cast<int64_t>(row) * ldy + ci]) : 0.0;
-      Bs[kk * kTP + c] = (in_rows && cj < r) ? static_cast<double>(Y[static_cast<int64_t>(row) * ldy + cj]) : 0.0;
+    for (int e = 0; e < 8; ++e) v[e] = 0.0f;
+    if (row >= k_end) return;
+    const float *p = Y + static_cast<int64_t>(row) * ldy + col;
+    if (vec && col + 8 <= r) {
+      const float4 a = __ldg(reinterpret_cast<const float4 *>(p)), b = __ldg(reinterpret_cast<const float4 *>(p) + 1);
+      v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w; v[4] = b.x; v[5] = b.y; v[6] = b.z; v[7] = b.w;
+    } else {
+#pragma unroll
+      for (int e = 0; e < 8; ++e)
+        if (col + e < r) v[e] = __ldg(p + e);
+    }
+  };
+  auto stash = [&](double *dst, const float (&v)[8]) {
+#pragma unroll
+    for (int e = 0; e < 8; e += 2)
+      *reinterpret_cast<double2 *>(dst + kk * kGP + i8 + e) = make_double2(static_cast<double>(v[e]), static_cast<double>(v[e + 1]));
+  };
+  double acc[8][8] = {};
+  float va[8], vb[8];
+  fetch(k_begin, bi, va);
+  if (!diag) fetch(k_begin, bj, vb);
+  int buf = 0;
+  stash(smg, va);
+  if (!diag) stash(smg + kGK * kGP, vb);
+  __syncthreads();
+  for (int k0 = k_begin; k0 < k_end; k0 += kGK) {
+    const bool more = k0 + kGK < k_end;
+    if (more) {
+      fetch(k0 + kGK, bi, va);
+      if (!diag) fetch(k0 + kGK, bj, vb);
+    }
+    const double *a = smg + buf * 2 * kGK * kGP;
+    tile_fma8(acc, a, diag ? a : a + kGK * kGP, ty, tx);
+    if (more) {
+      double *nxt = smg + (buf ^ 1) * 2 * kGK * kGP;
+      stash(nxt, va);
+      if (!diag) stash(nxt + kGK * kGP, vb);
     }
     __syncthreads();
-    tile_fma(acc, As, Bs, ty * 4, tx * 4, 32);
-    __syncthreads();
+    buf ^= 1;
   }
   double *out = partial + static_cast<int64_t>(split) * rp * rp;
 #pragma unroll
-  for (int i = 0; i < 4; ++i)
+  for (int i = 0; i < 8; ++i) {
+    const int row = bi * kG + own8(ty, i);
+    if (row >= rp) continue;
 #pragma unroll
-    for (int j = 0; j < 4; ++j)
-      out[static_cast<int64_t>(bi * kT + ty * 4 + i) * rp + bj * kT + tx * 4 + j] = acc[i][j];
+    for (int j = 0; j < 8; j += 2) {
+      const int col = bj * kG + own8(tx, j);
+      if (col < rp) *reinterpret_cast<double2 *>(out + static_cast<int64_t>(row) * rp + col) = make_double2(acc[i][j], acc[i][j + 1]);
+    }
+  }
 }
 
 // S = sum of the partial Gram matrices in split order, written over split 0;
@@ -91,7 +171,7 @@ __global__ void gram_reduce_kernel(double *__restrict__ partial, int splits, int
   for (int64_t e = blockIdx.x * static_cast<int64_t>(blockDim.x) + threadIdx.x; e < total;
        e += static_cast<int64_t>(gridDim.x) * blockDim.x) {
     const int i = static_cast<int>(e / rp), j = static_cast<int>(e % rp);
-    if (j / kT > i / kT) continue;  // upper tiles are never read
+    if (j / kG > i / kG) continue;  // tiles above the diagonal were not computed and are never read
     double s = 0.0;
     for (int sp = 0; sp < splits; ++sp) s += partial[sp * total + e];
     if (i >= r || j >= r) s = (i == j) ? 1.0 : 0.0;
@@ -99,77 +179,137 @@ __global__ void gram_reduce_kernel(double *__restrict__ partial, int splits, int
   }
 }
 
+// 1 / x to double precision without the divide sequence: hardware estimate, two Newton steps.
+__device__ __forceinline__ double fast_rcp(double x) {
+  double y;
+  asm("rcp.approx.ftz.f64 %0, %1;" : "=d"(y) : "d"(x));
+  y = fma(y, fma(-x, y, 1.0), y);
+  return fma(y, fma(-x, y, 1.0), y);
+}
+
 // Panel step p of the blocked Cholesky factorisation S = L L^T (64 columns at a
 // time, right-looking).  Every CTA factors the 64 x 64 diagonal block S_pp in
-// shared memory and inverts the factor; CTA 0 stores L_pp^-1 (all that is ever
-// needed of the diagonal block; S_pp itself stays as it is, the other CTAs of
-// this launch are still reading it), CTA b > 0 replaces the block S_(p+b),p by
-// L_(p+b),p = S_(p+b),p L_pp^-T.
+// shared memory and inverts the factor; CTA 0 stores L_pp^-1 into the diagonal
+// block of X (all that is ever needed of the diagonal block; S_pp itself stays as
+// it is, the other CTAs of this launch are still reading it), CTA b > 0 replaces
+// the block S_(p+b),p by L_(p+b),p = S_(p+b),p L_pp^-T.
 // A pivot that is not positive (the iterate is rank deficient to working
 // precision) is replaced by one and reported through the status word.
+//
+// The factorisation keeps the lower triangle in registers (its 2080 elements dealt
+// over the 256 threads, nine slots each) and passes only the current column through
+// shared memory: step j subtracts col[i] col[k] / pivot_j from every element (i, k)
+// with k > j, and the owners of column j + 1 publish it for the next step - one
+// barrier per step.  The inverse of the factor is built by doubling: 8 x 8 diagonal
+// blocks by forward substitution, then three levels of X21 = -X22 (L21 X11).
 __global__ void __launch_bounds__(256)
-chol_panel_kernel(double *__restrict__ S, int rp, int p, double *__restrict__ linv, uint32_t *status) {
-  extern __shared__ double sm[];
-  double *D = sm;                  // [64][65] the diagonal block, then its factor
-  double *Xt = sm + kT * kTP;      // [64][65] Xt[c][i] = (L_pp^-1)[i][c]
-  double *As = sm + 2 * kT * kTP;  // [64][65] As[c][a] = S_ip[a][c]
+chol_panel_kernel(double *__restrict__ S, int rp, int p, double *__restrict__ X, uint32_t *status) {
+  extern __shared__ __align__(16) double sm[];
+  double *D = sm;                  // [64][65] the diagonal block, its factor L, finally Xt[c][i] = (L^-1)[i][c]
+  double *Xs = sm + kT * kTP;      // [64][65] L^-1
+  double *As = sm + 2 * kT * kTP;  // [64][65] scratch of the inversion, then As[c][a] = S_ip[a][c]
+  __shared__ double col[2][kT];
+  __shared__ double pivot[kT];
   const int tid = threadIdx.x;
   const int64_t d0 = static_cast<int64_t>(p) * kT;
-  for (int e = tid; e < kT * kT; e += 256) {
-    const int i = e >> 6, j = e & 63;
-    D[i * kTP + j] = (j <= i) ? S[(d0 + i) * rp + d0 + j] : 0.0;
+
+  // ---- factorisation
+  constexpr int kSlots = 9, kLower = kT * (kT + 1) / 2;
+  double val[kSlots];
+  int ei[kSlots], ek[kSlots];
+#pragma unroll
+  for (int q = 0; q < kSlots; ++q) {
+    const int idx = tid + 256 * q;
+    int i = 0, k = 0;
+    if (idx < kLower) lower_tile(idx, i, k);
+    ei[q] = i;
+    ek[q] = idx < kLower ? k : -1;  // -1: empty slot
+    val[q] = idx < kLower ? S[(d0 + i) * rp + d0 + k] : 0.0;
+    if (ek[q] == 0) col[0][i] = val[q];
   }
   __syncthreads();
   for (int j = 0; j < kT; ++j) {
-    if (tid == 0) {
-      double d = D[j * kTP + j];
-      if (!(d > 0.0)) {
-        atomicOr(status, kErrNumeric);
-        d = 1.0;
-      }
-      D[j * kTP + j] = sqrt(d);
+    const double *cur = col[j & 1];
+    double *nxt = col[(j + 1) & 1];
+    double piv = cur[j];
+    if (!(piv > 0.0)) {
+      if (tid == 0) atomicOr(status, kErrNumeric);
+      piv = 1.0;
     }
-    __syncthreads();
-    const double djj = D[j * kTP + j];
-    if (tid > j && tid < kT) D[tid * kTP + j] /= djj;
-    __syncthreads();
-    // trailing update of the block's lower triangle: D[i][k] -= D[i][j] D[k][j], j < k <= i
-    for (int e = tid; e < kT * kT; e += 256) {
-      const int i = e >> 6, k = e & 63;
-      if (k > j && k <= i) D[i * kTP + k] -= D[i * kTP + j] * D[k * kTP + j];
+    if (tid == 0) pivot[j] = piv;
+    const double inv = fast_rcp(piv);
+#pragma unroll
+    for (int q = 0; q < kSlots; ++q) {
+      if (ek[q] > j) {
+        val[q] = fma(-cur[ei[q]] * inv, cur[ek[q]], val[q]);
+        if (ek[q] == j + 1) nxt[ei[q]] = val[q];
+      }
     }
     __syncthreads();
   }
-  // inverse of the lower-triangular factor, one column per thread (forward substitution on a unit vector)
+  // L[i][k] = value / sqrt(pivot_k), L[k][k] = sqrt(pivot_k); zero above the diagonal
+  for (int e = tid; e < kT * kT; e += 256) D[(e >> 6) * kTP + (e & 63)] = 0.0, Xs[(e >> 6) * kTP + (e & 63)] = 0.0;
+  __syncthreads();
+#pragma unroll
+  for (int q = 0; q < kSlots; ++q) {
+    if (ek[q] < 0) continue;
+    const double sq = sqrt(pivot[ek[q]]);
+    D[ei[q] * kTP + ek[q]] = (ei[q] == ek[q]) ? sq : val[q] / sq;
+  }
+  __syncthreads();
+
+  // ---- inverse of the factor
+  // 8 x 8 diagonal blocks: thread (block, column) solves L x = e_c inside its block
   if (tid < kT) {
-    const int c = tid;
-    for (int i = 0; i < kT; ++i) {
-      double x = 0.0;
-      if (i >= c) {
-        double sum = (i == c) ? 1.0 : 0.0;
-        for (int k = c; k < i; ++k) sum -= D[i * kTP + k] * Xt[c * kTP + k];
-        x = sum / D[i * kTP + i];
-      }
-      Xt[c * kTP + i] = x;
+    const int b0 = tid & ~7, c = tid & 7;
+    double x[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      double sum = (i == c) ? 1.0 : 0.0;
+#pragma unroll
+      for (int k = 0; k < 8; ++k)
+        if (k < i && k >= c) sum = fma(-D[(b0 + i) * kTP + b0 + k], x[k], sum);
+      x[i] = (i < c) ? 0.0 : sum / D[(b0 + i) * kTP + b0 + i];
+      Xs[(b0 + i) * kTP + b0 + c] = x[i];
     }
   }
   __syncthreads();
+  // doubling: for every super-block [d, d + 2h): T = L21 X11, then X21 = -X22 T
+  for (int h = 8; h < kT; h *= 2) {
+    const int elems = (kT / (2 * h)) * h * h;
+    for (int e = tid; e < elems; e += 256) {
+      const int z = e / (h * h), a = (e / h) % h, b = e % h, d = 2 * h * z;
+      double sum = 0.0;
+      for (int k = b; k < h; ++k) sum = fma(D[(d + h + a) * kTP + d + k], Xs[(d + k) * kTP + d + b], sum);
+      As[(d + h + a) * kTP + d + b] = sum;
+    }
+    __syncthreads();
+    for (int e = tid; e < elems; e += 256) {
+      const int z = e / (h * h), a = (e / h) % h, b = e % h, d = 2 * h * z;
+      double sum = 0.0;
+      for (int k = 0; k <= a; ++k) sum = fma(Xs[(d + h + a) * kTP + d + h + k], As[(d + h + k) * kTP + d + b], sum);
+      Xs[(d + h + a) * kTP + d + b] = -sum;
+    }
+    __syncthreads();
+  }
   if (blockIdx.x == 0) {
     for (int e = tid; e < kT * kT; e += 256) {
       const int i = e >> 6, j = e & 63;
-      linv[static_cast<int64_t>(p) * kT * kT + e] = Xt[j * kTP + i];
+      X[(d0 + i) * rp + d0 + j] = Xs[i * kTP + j];
     }
     return;
   }
+  // ---- this CTA's block of the panel: L_ip = S_ip L_pp^-T
   const int64_t r0 = static_cast<int64_t>(p + blockIdx.x) * kT;
   for (int e = tid; e < kT * kT; e += 256) {
     const int a = e >> 6, c = e & 63;
     As[c * kTP + a] = S[(r0 + a) * rp + d0 + c];
+    D[c * kTP + a] = Xs[a * kTP + c];  // Xt[c][i] = (L^-1)[i][c]
   }
   __syncthreads();
   const int tx = tid & 15, ty = tid >> 4;
   double acc[4][4] = {};
-  tile_fma(acc, As, Xt, ty * 4, tx * 4, kT);  // sum_c S_ip[a][c] (L_pp^-1)[b][c]
+  tile_fma(acc, As, D, ty * 4, tx * 4, kT);  // sum_c S_ip[a][c] (L_pp^-1)[b][c]
 #pragma unroll
   for (int i = 0; i < 4; ++i)
 #pragma unroll
@@ -203,79 +343,121 @@ chol_update_kernel(double *__restrict__ S, int rp, int p) {
     for (int j = 0; j < 4; ++j) S[(i0 + ty * 4 + i) * rp + j0 + tx * 4 + j] -= acc[i][j];
 }
 
-// Q = Y L^-T by blocks of 64 columns: Q_j = (Y_j - sum_(k<j) Q_k L_jk^T) L_jj^-T.
-// A CTA owns 32 rows of Y and walks the column blocks in order; its rows of Q
-// stay in double precision in `qd` for the later blocks.  Outputs (each
-// optional): Q as fp32, and Q split into two bf16 matrices hi + lo (hi =
-// bf16(Q), lo = bf16(Q - hi)), the form in which the next product consumes it.
-__global__ void __launch_bounds__(128)
-solve_kernel(const float *__restrict__ Y, int64_t ldy, int m, int r, int rp, const double *__restrict__ L,
-             const double *__restrict__ linv, double *__restrict__ qd, float *__restrict__ qf, int64_t ldqf,
-             __nv_bfloat16 *__restrict__ qhi, __nv_bfloat16 *__restrict__ qlo, int64_t ldqb) {
-  extern __shared__ double sm[];
-  double *As = sm;             // [64][65] As[c][a], a < 32
-  double *Bs = sm + kT * kTP;  // [64][65]
-  const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;  // 16 x 8 threads, 4 x 4 outputs each
-  const int64_t row0 = static_cast<int64_t>(blockIdx.x) * 32;
-  const int nb = rp / kT;
-  for (int j = 0; j < nb; ++j) {
-    double acc[4][4] = {};
-    for (int k = 0; k < j; ++k) {
-      for (int e = tid; e < 32 * kT; e += 128) {
-        const int a = e >> 6, c = e & 63;
-        As[c * kTP + a] = (row0 + a < m) ? qd[(row0 + a) * rp + k * kT + c] : 0.0;
-      }
-      for (int e = tid; e < kT * kT; e += 128) {
-        const int b = e >> 6, c = e & 63;
-        Bs[c * kTP + b] = L[static_cast<int64_t>(j * kT + b) * rp + k * kT + c];
-      }
-      __syncthreads();
-      tile_fma(acc, As, Bs, ty * 4, tx * 4, kT);
-      __syncthreads();
+// One product of the inversion by doubling, for every diagonal super-block of
+// size 2 h at once (blockIdx.z): with d0 = 2 h z, the h x h blocks
+//   first  (second == 0):  T(z) = C A         C = L[d0 + h .., d0 ..],  A = X[d0 .., d0 ..]
+//   second (second == 1):  X[d0 + h .., d0 ..] = - B T(z)      B = X[d0 + h .., d0 + h ..]
+// T(z) is kept at the position of the block it leads to.  64 x 64 output tiles, k
+// over the h columns; rows and columns beyond rp count as zero.
+__global__ void __launch_bounds__(256)
+block_gemm_kernel(const double *__restrict__ L, double *__restrict__ X, double *__restrict__ T, int rp, int h, int second) {
+  __shared__ double As[32 * kTP];
+  __shared__ double Bs[32 * kTP];
+  const int d0 = 2 * h * static_cast<int>(blockIdx.z);
+  const int ti = static_cast<int>(blockIdx.y) * kT, tj = static_cast<int>(blockIdx.x) * kT;  // tile origin inside the h x h block
+  if (d0 + h + ti >= rp) return;  // the lower block is cut off by the matrix edge (the whole CTA leaves)
+  const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
+  // left operand M1 (rows d0 + h + ti .., columns m1_col0 + k) and right operand M2 (rows m2_row0 + k, columns d0 + tj ..)
+  const double *M1 = second ? X : L;
+  const double *M2 = second ? T : X;
+  const int64_t m1_row0 = d0 + h + ti, m1_col0 = second ? d0 + h : d0;
+  const int64_t m2_row0 = second ? d0 + h : d0, m2_col0 = d0 + tj;
+  double acc[4][4] = {};
+  for (int k0 = 0; k0 < h; k0 += 32) {
+    for (int e = tid; e < kT * 32; e += 256) {
+      const int a = e >> 5, c = e & 31;  // As[c][a] = M1[row a][k0 + c]
+      const int64_t row = m1_row0 + a, col = m1_col0 + k0 + c;
+      As[c * kTP + a] = (row < rp && col < rp) ? M1[row * rp + col] : 0.0;
     }
-    // T = Y_j - acc, stored k-outermost for the product with L_jj^-T
-#pragma unroll
-    for (int i = 0; i < 4; ++i)
-#pragma unroll
-      for (int jj = 0; jj < 4; ++jj) {
-        const int64_t row = row0 + ty * 4 + i;
-        const int col = j * kT + tx * 4 + jj;
-        const double y = (row < m && col < r) ? static_cast<double>(Y[row * ldy + col]) : 0.0;
-        As[(tx * 4 + jj) * kTP + ty * 4 + i] = y - acc[i][jj];
-      }
-    for (int e = tid; e < kT * kT; e += 128) {
-      const int b = e >> 6, c = e & 63;
-      Bs[c * kTP + b] = linv[static_cast<int64_t>(j) * kT * kT + e];  // Bs[c][b] = (L_jj^-1)[b][c]
+    for (int e = tid; e < kT * 32; e += 256) {
+      const int c = e >> 6, b = e & 63;  // Bs[c][b] = M2[k0 + c][column b]
+      const int64_t row = m2_row0 + k0 + c, col = m2_col0 + b;
+      Bs[c * kTP + b] = (row < rp && col < rp) ? M2[row * rp + col] : 0.0;
     }
     __syncthreads();
-    double q[4][4] = {};
-    tile_fma(q, As, Bs, ty * 4, tx * 4, kT);
-#pragma unroll
-    for (int i = 0; i < 4; ++i)
-#pragma unroll
-      for (int jj = 0; jj < 4; ++jj) {
-        const int64_t row = row0 + ty * 4 + i;
-        const int col = j * kT + tx * 4 + jj;
-        if (row >= m) continue;
-        qd[row * rp + col] = q[i][jj];
-        if (col >= r) continue;
-        const float f = static_cast<float>(q[i][jj]);
-        if (qf != nullptr) qf[row * ldqf + col] = f;
-        if (qhi != nullptr) {
-          const __nv_bfloat16 hi = __float2bfloat16_rn(f);
-          qhi[row * ldqb + col] = hi;
-          qlo[row * ldqb + col] = __float2bfloat16_rn(static_cast<float>(q[i][jj] - static_cast<double>(__bfloat162float(hi))));
-        }
-      }
+    tile_fma(acc, As, Bs, ty * 4, tx * 4, 32);
     __syncthreads();
+  }
+  double *dst = second ? X : T;
+  const int64_t dr0 = d0 + h + ti, dc0 = d0 + tj;
+#pragma unroll
+  for (int i = 0; i < 4; ++i)
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const int64_t row = dr0 + ty * 4 + i, col = dc0 + tx * 4 + j;
+      if (row < rp && col < rp) dst[row * rp + col] = second ? -acc[i][j] : acc[i][j];
+    }
+}
+
+// Q = Y X^T with X = L^-1 lower triangular: Q[a][j] = sum_(c <= j) Y[a][c] X[j][c].
+// 128 x 128 tiles; the tile of column block bj sums over the columns c < 128 (bj + 1).
+// Outputs (each optional): Q as fp32, and Q split into two bf16 matrices hi + lo
+// (hi = bf16(Q), lo = bf16(Q - hi)), the form in which the next product consumes it.
+__global__ void __launch_bounds__(256)
+apply_kernel(const float *__restrict__ Y, int64_t ldy, int m, int r, int rp, const double *__restrict__ X,
+             float *__restrict__ qf, int64_t ldqf, __nv_bfloat16 *__restrict__ qhi, __nv_bfloat16 *__restrict__ qlo, int64_t ldqb) {
+  extern __shared__ __align__(16) double smg[];
+  const int bj = static_cast<int>(gridDim.y) - 1 - static_cast<int>(blockIdx.y);  // longest sums first
+  const int64_t row0 = static_cast<int64_t>(blockIdx.x) * kG;
+  const int j0 = bj * kG;
+  const int k_end = min(rp, j0 + kG);
+  const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
+  // staging: thread -> one row of the tile (a for Y, b for X), 8 consecutive k
+  const int sr = tid >> 1, sk = (tid & 1) * 8;
+  auto fetch = [&](int k0, double (&va)[8], double (&vb)[8]) {
+    const int64_t row = row0 + sr;
+    const int c = k0 + sk;
+#pragma unroll
+    for (int e = 0; e < 8; ++e) va[e] = (row < m && c + e < r) ? static_cast<double>(__ldg(Y + row * ldy + c + e)) : 0.0;
+    const int xr = j0 + sr;
+#pragma unroll
+    for (int e = 0; e < 8; ++e) vb[e] = (xr < rp && c + e < rp) ? X[static_cast<int64_t>(xr) * rp + c + e] : 0.0;
+  };
+  auto stash = [&](double *dst, const double (&va)[8], const double (&vb)[8]) {
+#pragma unroll
+    for (int e = 0; e < 8; ++e) {
+      dst[(sk + e) * kGP + sr] = va[e];
+      dst[kGK * kGP + (sk + e) * kGP + sr] = vb[e];
+    }
+  };
+  double acc[8][8] = {};
+  double va[8], vb[8];
+  fetch(0, va, vb);
+  stash(smg, va, vb);
+  __syncthreads();
+  int buf = 0;
+  for (int k0 = 0; k0 < k_end; k0 += kGK) {
+    const bool more = k0 + kGK < k_end;
+    if (more) fetch(k0 + kGK, va, vb);
+    const double *a = smg + buf * 2 * kGK * kGP;
+    tile_fma8(acc, a, a + kGK * kGP, ty, tx);
+    if (more) stash(smg + (buf ^ 1) * 2 * kGK * kGP, va, vb);
+    __syncthreads();
+    buf ^= 1;
+  }
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    const int64_t row = row0 + own8(ty, i);
+    if (row >= m) continue;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      const int col = j0 + own8(tx, j);
+      if (col >= r) continue;
+      const float f = static_cast<float>(acc[i][j]);
+      if (qf != nullptr) qf[row * ldqf + col] = f;
+      if (qhi != nullptr) {
+        const __nv_bfloat16 hi = __float2bfloat16_rn(f);
+        qhi[row * ldqb + col] = hi;
+        qlo[row * ldqb + col] = __float2bfloat16_rn(static_cast<float>(acc[i][j] - static_cast<double>(__bfloat162float(hi))));
+      }
+    }
   }
 }
 
 constexpr size_t kPanelSmem = 3 * kT * kTP * sizeof(double);
-constexpr size_t kSolveSmem = 2 * kT * kTP * sizeof(double);
 
 int gram_splits(int m, int rp) {
-  const int nb = rp / kT, tiles = nb * (nb + 1) / 2;
+  const int nb = (rp + kG - 1) / kG, tiles = nb * (nb + 1) / 2;
   int splits = sm_count() / tiles;
   if (splits > 16) splits = 16;
   const int by_rows = (m + 255) / 256;
@@ -283,46 +465,60 @@ int gram_splits(int m, int rp) {
   return splits < 1 ? 1 : splits;
 }
 
+size_t up256(size_t v) { return (v + 255) & ~static_cast<size_t>(255); }
+
 }  // namespace
 
 size_t orth_workspace_bytes(int m, int r) {
   const size_t rp = (static_cast<size_t>(r) + kT - 1) / kT * kT;
-  const size_t gram = static_cast<size_t>(gram_splits(m, static_cast<int>(rp))) * rp * rp * sizeof(double);
-  const size_t inv = rp * kT * sizeof(double);
-  const size_t qd = static_cast<size_t>(m) * rp * sizeof(double);
-  auto up = [](size_t v) { return (v + 255) & ~static_cast<size_t>(255); };
-  return up(gram) + up(inv) + up(qd);
+  const size_t sq = rp * rp * sizeof(double);
+  return up256(static_cast<size_t>(gram_splits(m, static_cast<int>(rp))) * sq) + 2 * up256(sq);  // Gram partials / L, X, T
 }
 
 loqt_status orthonormalise(const float *Y, int64_t ldy, int m, int r, float *qf, int64_t ldqf, void *qhi, void *qlo,
                            int64_t ldqb, void *ws, uint32_t *status, cudaStream_t stream) {
   const int rp = (r + kT - 1) / kT * kT, nb = rp / kT;
   const int splits = gram_splits(m, rp);
-  auto up = [](size_t v) { return (v + 255) & ~static_cast<size_t>(255); };
+  const size_t sq = static_cast<size_t>(rp) * rp * sizeof(double);
   uint8_t *cursor = static_cast<uint8_t *>(ws);
   double *S = reinterpret_cast<double *>(cursor);
-  cursor += up(static_cast<size_t>(splits) * rp * rp * sizeof(double));
-  double *linv = reinterpret_cast<double *>(cursor);
-  cursor += up(static_cast<size_t>(rp) * kT * sizeof(double));
-  double *qd = reinterpret_cast<double *>(cursor);
+  cursor += up256(static_cast<size_t>(splits) * sq);
+  double *X = reinterpret_cast<double *>(cursor);
+  cursor += up256(sq);
+  double *T = reinterpret_cast<double *>(cursor);
 
+  // Every kernel of the sequence asks for the same split of the SM's memory between shared
+  // memory and L1: a change of the split between two launches makes the second wait for
+  // the SMs to drain and switch over.
   static bool attr_set = false;
   if (!attr_set) {
-    if (cudaFuncSetAttribute(chol_panel_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kPanelSmem)) != cudaSuccess ||
-        cudaFuncSetAttribute(solve_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kSolveSmem)) != cudaSuccess)
-      return LOQT_ERR_CUDA;
+    bool ok = cudaFuncSetAttribute(chol_panel_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kPanelSmem)) == cudaSuccess &&
+              cudaFuncSetAttribute(gram_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kBigSmem)) == cudaSuccess &&
+              cudaFuncSetAttribute(apply_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kBigSmem)) == cudaSuccess;
+    const int carve = cudaSharedmemCarveoutMaxShared;
+    ok = ok && cudaFuncSetAttribute(chol_panel_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, carve) == cudaSuccess &&
+         cudaFuncSetAttribute(chol_update_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, carve) == cudaSuccess &&
+         cudaFuncSetAttribute(block_gemm_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, carve) == cudaSuccess &&
+         cudaFuncSetAttribute(gram_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, carve) == cudaSuccess &&
+         cudaFuncSetAttribute(gram_reduce_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, carve) == cudaSuccess &&
+         cudaFuncSetAttribute(apply_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, carve) == cudaSuccess;
+    if (!ok) return LOQT_ERR_CUDA;
     attr_set = true;
   }
+  int launches = 0;
+  // S = Y^T Y
   int rows_per_split = (m + splits - 1) / splits;
-  rows_per_split = (rows_per_split + 31) / 32 * 32;
-  const int tiles = nb * (nb + 1) / 2;
-  gram_kernel<<<dim3(tiles, splits), 256, 0, stream>>>(Y, ldy, m, r, rp, rows_per_split, S);
+  rows_per_split = (rows_per_split + kGK - 1) / kGK * kGK;
+  const int gb = (rp + kG - 1) / kG;
+  gram_kernel<<<dim3(gb * (gb + 1) / 2, splits), 256, kBigSmem, stream>>>(Y, ldy, m, r, rp, rows_per_split, S);
   int blocks = static_cast<int>((static_cast<int64_t>(rp) * rp + 255) / 256);
   if (blocks > sm_count() * 8) blocks = sm_count() * 8;
   gram_reduce_kernel<<<blocks, 256, 0, stream>>>(S, splits, r, rp);
-  int launches = 2;
+  launches += 2;
+  // S = L L^T (L's blocks below the diagonal replace S's), X's diagonal blocks = the inverses of L's
+  if (cudaMemsetAsync(X, 0, sq, stream) != cudaSuccess) return LOQT_ERR_CUDA;
   for (int p = 0; p < nb; ++p) {
-    chol_panel_kernel<<<nb - p, 256, kPanelSmem, stream>>>(S, rp, p, linv, status);
+    chol_panel_kernel<<<nb - p, 256, kPanelSmem, stream>>>(S, rp, p, X, status);
     ++launches;
     const int n = nb - p - 1;
     if (n > 0) {
@@ -330,8 +526,16 @@ loqt_status orthonormalise(const float *Y, int64_t ldy, int m, int r, float *qf,
       ++launches;
     }
   }
-  solve_kernel<<<(m + 31) / 32, 128, kSolveSmem, stream>>>(Y, ldy, m, r, rp, S, linv, qd, qf, ldqf,
-                                                           static_cast<__nv_bfloat16 *>(qhi), static_cast<__nv_bfloat16 *>(qlo), ldqb);
+  // X = L^-1 by doubling the size of the inverted diagonal blocks
+  for (int h = kT; h < rp; h *= 2) {
+    const int supers = (rp + 2 * h - 1) / (2 * h), ht = h / kT;
+    block_gemm_kernel<<<dim3(ht, ht, supers), 256, 0, stream>>>(S, X, T, rp, h, 0);
+    block_gemm_kernel<<<dim3(ht, ht, supers), 256, 0, stream>>>(S, X, T, rp, h, 1);
+    launches += 2;
+  }
+  // Q = Y X^T
+  apply_kernel<<<dim3((m + kG - 1) / kG, gb), 256, kBigSmem, stream>>>(Y, ldy, m, r, rp, X, qf, ldqf, static_cast<__nv_bfloat16 *>(qhi),
+                                                                       static_cast<__nv_bfloat16 *>(qlo), ldqb);
   count_launch(launches + 1);
   return cudaGetLastError() == cudaSuccess ? LOQT_OK : LOQT_ERR_CUDA;
 }
