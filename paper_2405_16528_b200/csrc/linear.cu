@@ -95,6 +95,7 @@ constexpr double kNarrowTilePenalty = 1.15;  // N = 128 passes move more operand
 constexpr double kCyclesDequantRow = 3.3;
 constexpr double kCyclesEpilogueRow = 400.0;
 constexpr double kCyclesFixed = 3000.0;
+constexpr double kPairGain = 0.85;  // stage time of a CTA pair relative to two single CTAs (measured)
 
 // Run eligible products as tcgen05 CTA pairs (cta_group::2).
 #ifndef LOQT_USE_PAIRS
@@ -211,14 +212,14 @@ static TileCfg pick_tile(const GemmCall &c) {
     const double deq = b_nf4 ? kCyclesDequantRow * t.bn : 0.0;
     const double stage = mma > deq ? mma : deq;
     const double epi = (t.mh == 2 ? 1.0 : 0.25) * kCyclesEpilogueRow * t.mh * t.bn / 32.0;
-    const double cost = waves * (kb * stage + epi + kCyclesFixed);
+    double cost = waves * (kb * stage + epi + kCyclesFixed);
+    if (t.bn == 256 && pair_ok(c, 256, t.mh)) cost *= kPairGain;  // it will run as CTA pairs
     if (cost < best_t) {
       best_t = cost;
       best = t;
     }
   }
-  // The costs above are those of single CTAs; a 256-wide choice then runs as pairs
-  // where it can (measured faster).
+  // a 256-wide choice runs as pairs where it can
   best.two = pair_ok(c, best.bn, best.mh);
   // A tile forced by loqt_set_tile_override() replaces the choice wherever the
   // kernel supports it for this product: pairs need 256-wide tiles and no split-K
