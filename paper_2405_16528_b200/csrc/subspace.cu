@@ -33,16 +33,19 @@ namespace {
 constexpr int kT = 64;       // tile edge of the factorisation
 constexpr int kTP = kT + 1;  // padded row of a 64-wide shared-memory tile (doubles)
 
-// acc[i][j] += sum_k a[k][row0 + i] * b[k][col0 + j], k < kc; a and b are
+// 64 x 64 tiles, 256 threads as 16 x 16: thread (ty, tx) owns rows ty + 16 i and
+// columns tx + 16 j (a warp's loads of the column operand are then 16 consecutive
+// doubles, free of bank conflicts, and its stores to global memory contiguous).
+// acc[i][j] += sum_k a[k][ty + 16 i] * b[k][tx + 16 j], k < kc; a and b are
 // shared-memory tiles stored k-outermost with padded rows of kTP doubles.
-__device__ __forceinline__ void tile_fma(double (&acc)[4][4], const double *a, const double *b, int row0, int col0, int kc) {
+__device__ __forceinline__ void tile_fma(double (&acc)[4][4], const double *a, const double *b, int ty, int tx, int kc) {
 #pragma unroll 4
   for (int k = 0; k < kc; ++k) {
     double av[4], bv[4];
 #pragma unroll
-    for (int i = 0; i < 4; ++i) av[i] = a[k * kTP + row0 + i];
+    for (int i = 0; i < 4; ++i) av[i] = a[k * kTP + ty + 16 * i];
 #pragma unroll
-    for (int j = 0; j < 4; ++j) bv[j] = b[k * kTP + col0 + j];
+    for (int j = 0; j < 4; ++j) bv[j] = b[k * kTP + tx + 16 * j];
 #pragma unroll
     for (int i = 0; i < 4; ++i)
 #pragma unroll
@@ -179,11 +182,14 @@ __global__ void gram_reduce_kernel(double *__restrict__ partial, int splits, int
   }
 }
 
-// 1 / x to double precision without the divide sequence: hardware estimate, two Newton steps.
+// 1 / x without the divide sequence: the hardware estimate (20 bits) and one Newton step
+// give a relative error of about 1e-12, ample for an elimination multiplier here (the
+// basis it leads to is rounded to single precision), and keep the chain of dependent
+// double-precision operations per elimination step short: that chain, 64 times per
+// panel, is what the factorisation waits on.
 __device__ __forceinline__ double fast_rcp(double x) {
   double y;
   asm("rcp.approx.ftz.f64 %0, %1;" : "=d"(y) : "d"(x));
-  y = fma(y, fma(-x, y, 1.0), y);
   return fma(y, fma(-x, y, 1.0), y);
 }
 
@@ -241,13 +247,14 @@ chol_panel_kernel(double *__restrict__ S, int rp, int p, double *__restrict__ X,
 #pragma unroll
     for (int q = 0; q < kSlots; ++q) {
       if (ek[q] > j) {
-        val[q] = fma(-cur[ei[q]] * inv, cur[ek[q]], val[q]);
+        val[q] = fma(-(cur[ei[q]] * cur[ek[q]]), inv, val[q]);  // the product does not wait for the reciprocal
         if (ek[q] == j + 1) nxt[ei[q]] = val[q];
       }
     }
     __syncthreads();
   }
   // L[i][k] = value / sqrt(pivot_k), L[k][k] = sqrt(pivot_k); zero above the diagonal
+#pragma unroll
   for (int e = tid; e < kT * kT; e += 256) D[(e >> 6) * kTP + (e & 63)] = 0.0, Xs[(e >> 6) * kTP + (e & 63)] = 0.0;
   __syncthreads();
 #pragma unroll
@@ -274,26 +281,37 @@ chol_panel_kernel(double *__restrict__ S, int rp, int p, double *__restrict__ X,
     }
   }
   __syncthreads();
-  // doubling: for every super-block [d, d + 2h): T = L21 X11, then X21 = -X22 T
-  for (int h = 8; h < kT; h *= 2) {
+  // doubling: for every super-block [d, d + 2h): T = L21 X11, then X21 = -X22 T.  A dot product
+  // runs as four interleaved partial sums: a dependent chain of double-precision operations
+  // is what these few hundred threads wait on.
+  for (int h = 8, hs = 3; h < kT; h *= 2, ++hs) {
     const int elems = (kT / (2 * h)) * h * h;
     for (int e = tid; e < elems; e += 256) {
-      const int z = e / (h * h), a = (e / h) % h, b = e % h, d = 2 * h * z;
-      double sum = 0.0;
-      for (int k = b; k < h; ++k) sum = fma(D[(d + h + a) * kTP + d + k], Xs[(d + k) * kTP + d + b], sum);
-      As[(d + h + a) * kTP + d + b] = sum;
+      const int z = e >> (2 * hs), a = (e >> hs) & (h - 1), b = e & (h - 1), d = 2 * h * z;
+      const double *lrow = D + (d + h + a) * kTP + d, *xcol = Xs + d * kTP + d + b;
+      double s4[4] = {0.0, 0.0, 0.0, 0.0};
+      for (int k = 0; k < h; k += 4) {  // X11 is lower triangular: the terms with k < b are stored zeros
+#pragma unroll
+        for (int u = 0; u < 4; ++u) s4[u] = fma(lrow[k + u], xcol[(k + u) * kTP], s4[u]);
+      }
+      As[(d + h + a) * kTP + d + b] = (s4[0] + s4[1]) + (s4[2] + s4[3]);
     }
     __syncthreads();
     for (int e = tid; e < elems; e += 256) {
-      const int z = e / (h * h), a = (e / h) % h, b = e % h, d = 2 * h * z;
-      double sum = 0.0;
-      for (int k = 0; k <= a; ++k) sum = fma(Xs[(d + h + a) * kTP + d + h + k], As[(d + h + k) * kTP + d + b], sum);
-      Xs[(d + h + a) * kTP + d + b] = -sum;
+      const int z = e >> (2 * hs), a = (e >> hs) & (h - 1), b = e & (h - 1), d = 2 * h * z;
+      const double *xrow = Xs + (d + h + a) * kTP + d + h, *tcol = As + (d + h) * kTP + d + b;
+      double s4[4] = {0.0, 0.0, 0.0, 0.0};
+      for (int k = 0; k < h; k += 4) {  // X22 is lower triangular: the terms with k > a are stored zeros
+#pragma unroll
+        for (int u = 0; u < 4; ++u) s4[u] = fma(xrow[k + u], tcol[(k + u) * kTP], s4[u]);
+      }
+      Xs[(d + h + a) * kTP + d + b] = -((s4[0] + s4[1]) + (s4[2] + s4[3]));
     }
     __syncthreads();
   }
   if (blockIdx.x == 0) {
-    for (int e = tid; e < kT * kT; e += 256) {
+  #pragma unroll
+  for (int e = tid; e < kT * kT; e += 256) {
       const int i = e >> 6, j = e & 63;
       X[(d0 + i) * rp + d0 + j] = Xs[i * kTP + j];
     }
@@ -301,6 +319,7 @@ chol_panel_kernel(double *__restrict__ S, int rp, int p, double *__restrict__ X,
   }
   // ---- this CTA's block of the panel: L_ip = S_ip L_pp^-T
   const int64_t r0 = static_cast<int64_t>(p + blockIdx.x) * kT;
+#pragma unroll
   for (int e = tid; e < kT * kT; e += 256) {
     const int a = e >> 6, c = e & 63;
     As[c * kTP + a] = S[(r0 + a) * rp + d0 + c];
@@ -309,11 +328,11 @@ chol_panel_kernel(double *__restrict__ S, int rp, int p, double *__restrict__ X,
   __syncthreads();
   const int tx = tid & 15, ty = tid >> 4;
   double acc[4][4] = {};
-  tile_fma(acc, As, D, ty * 4, tx * 4, kT);  // sum_c S_ip[a][c] (L_pp^-1)[b][c]
+  tile_fma(acc, As, D, ty, tx, kT);  // sum_c S_ip[a][c] (L_pp^-1)[b][c]
 #pragma unroll
   for (int i = 0; i < 4; ++i)
 #pragma unroll
-    for (int j = 0; j < 4; ++j) S[(r0 + ty * 4 + i) * rp + d0 + tx * 4 + j] = acc[i][j];
+    for (int j = 0; j < 4; ++j) S[(r0 + ty + 16 * i) * rp + d0 + tx + 16 * j] = acc[i][j];
 }
 
 // Trailing update after panel p: S_ij -= L_ip L_jp^T for p < j <= i.
@@ -328,19 +347,20 @@ chol_update_kernel(double *__restrict__ S, int rp, int p) {
   const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
   double acc[4][4] = {};
   for (int half = 0; half < 2; ++half) {  // the panel's 64 columns, 32 at a time
+#pragma unroll
     for (int e = tid; e < kT * 32; e += 256) {
       const int a = e >> 5, c = e & 31;
       As[c * kTP + a] = S[(i0 + a) * rp + c0 + half * 32 + c];
       Bs[c * kTP + a] = S[(j0 + a) * rp + c0 + half * 32 + c];
     }
     __syncthreads();
-    tile_fma(acc, As, Bs, ty * 4, tx * 4, 32);
+    tile_fma(acc, As, Bs, ty, tx, 32);
     __syncthreads();
   }
 #pragma unroll
   for (int i = 0; i < 4; ++i)
 #pragma unroll
-    for (int j = 0; j < 4; ++j) S[(i0 + ty * 4 + i) * rp + j0 + tx * 4 + j] -= acc[i][j];
+    for (int j = 0; j < 4; ++j) S[(i0 + ty + 16 * i) * rp + j0 + tx + 16 * j] -= acc[i][j];
 }
 
 // One product of the inversion by doubling, for every diagonal super-block of
@@ -364,18 +384,20 @@ block_gemm_kernel(const double *__restrict__ L, double *__restrict__ X, double *
   const int64_t m2_row0 = second ? d0 + h : d0, m2_col0 = d0 + tj;
   double acc[4][4] = {};
   for (int k0 = 0; k0 < h; k0 += 32) {
+#pragma unroll
     for (int e = tid; e < kT * 32; e += 256) {
       const int a = e >> 5, c = e & 31;  // As[c][a] = M1[row a][k0 + c]
       const int64_t row = m1_row0 + a, col = m1_col0 + k0 + c;
       As[c * kTP + a] = (row < rp && col < rp) ? M1[row * rp + col] : 0.0;
     }
+#pragma unroll
     for (int e = tid; e < kT * 32; e += 256) {
       const int c = e >> 6, b = e & 63;  // Bs[c][b] = M2[k0 + c][column b]
       const int64_t row = m2_row0 + k0 + c, col = m2_col0 + b;
       Bs[c * kTP + b] = (row < rp && col < rp) ? M2[row * rp + col] : 0.0;
     }
     __syncthreads();
-    tile_fma(acc, As, Bs, ty * 4, tx * 4, 32);
+    tile_fma(acc, As, Bs, ty, tx, 32);
     __syncthreads();
   }
   double *dst = second ? X : T;
@@ -384,7 +406,7 @@ block_gemm_kernel(const double *__restrict__ L, double *__restrict__ X, double *
   for (int i = 0; i < 4; ++i)
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
-      const int64_t row = dr0 + ty * 4 + i, col = dc0 + tx * 4 + j;
+      const int64_t row = dr0 + ty + 16 * i, col = dc0 + tx + 16 * j;
       if (row < rp && col < rp) dst[row * rp + col] = second ? -acc[i][j] : acc[i][j];
     }
 }
