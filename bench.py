@@ -513,9 +513,11 @@ def merge_report(m, world, peaks):
 # DRAM read + write bytes of the forward/backward launches (u, y, v, dx, dB) of ONE attention-shaped
 # matrix, from the ncu capture summarised in profiles/ (None where no capture of the current kernels exists).
 NCU_TRAFFIC = {
-    4: {"bytes": 266.6e6,
-        "of": "sum of dram__bytes_read + dram__bytes_write over the five launches (u, y, v, dx, dB) of one 4096x4096 matrix, "
-              "r=1024, T=4096 (profiles/loqt_gemm_kernel_llama7b_attention.md); algorithmic bytes of the same launches 332.4e6"},
+    4: {"bytes": 285.3e6,
+        "of": "sum of dram__bytes_read + dram__bytes_write over the five product launches (u, y, v, dx, dB) of one 4096x4096 matrix, "
+              "r=1024, T=4096 (profiles/loqt_gemm_kernel_llama7b_attention.md); algorithmic bytes of the same launches 338.4e6"},
+    3: {"bytes": 215.1e6,
+        "of": "the same for one 2048x2048 matrix, r=512, T=8192 (profiles/loqt_gemm_kernel_llama1b_attention.md); algorithmic 293e6"},
 }
 
 
@@ -627,7 +629,7 @@ def run_ours(args, rank, world, local_rank):
             "merge_requant": merge_report(m, world, peaks),
             "gpu_launches": m["launches"],
             "clocks": m["clocks"],
-            "roofline_traffic": None,
+            "roofline_traffic": NCU_TRAFFIC.get(ci, {"bytes": None})["bytes"],
         }
     if not args.no_cpu_baseline and world == 1:
         result["cpu_baseline"] = cpu_baseline(cfg, args.seed)
