@@ -75,6 +75,28 @@ def test_projection_matches_the_oracle_subspace(case):
     assert abs(cap - cap_ref) <= 1e-5 * cap_ref and cap <= opt * (1 + 1e-6)
 
 
+def test_full_size_7b_attention_shape():
+    """The projection at the benchmark's size (4096 x 4096, r = 1024: sixteen 64-column panels, eight
+    128-wide tile rows, every level of the inversion by doubling), one round, against the oracle's iterate.
+    The spectrum is the planted one (2 .. 1, then 0.5 .. 0.05), so the tolerance is formed from those values
+    instead of a 4096 x 4096 SVD."""
+    out, inn, r, iters = 4096, 4096, 1024, 1
+    Gb, Om, Gd, Od = _inputs(53, out, inn, r)
+    ws = L.new_workspace(L.loqt_workspace_bytes(L.LOQT_OP_PROJECTION, out, inn, r, 0))
+    P = L.loqt_projection(Gd, Od, iters, ws=ws)
+    L.loqt_device_status(ws)
+    P = f32(P).astype(np.float64)
+    assert np.isfinite(P).all() and np.abs(P.T @ P - np.eye(r)).max() < 2e-6
+    Q = O.subspace_iteration(Gb, Om, iters)
+    sines = O.subspace_sines(Q, P)
+    cond0 = np.linalg.cond(Gb @ Om)
+    tol = 8.0 * (2.0 ** -22 * cond0 * 0.25 ** iters + (2.0 ** -17 + 2.0 ** -22) * 2.0)
+    print(f"projection {(out, inn, r, iters)}: max sine {sines.max():.3e} (tolerance {tol:.3e}, cond(G Omega) = {cond0:.1f})")
+    assert sines.max() <= tol
+    cap, cap_ref = np.linalg.norm(P.T @ Gb) ** 2, np.linalg.norm(Q.T @ Gb) ** 2
+    assert abs(cap - cap_ref) <= 1e-5 * cap_ref
+
+
 def test_converges_to_the_definition():
     # a wide spectral gap (tail 0.2): four rounds leave (0.2)^9 of the starting angle
     out, inn, r = 512, 640, 64
