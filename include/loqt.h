@@ -115,7 +115,11 @@ loqt_status loqt_linear_fwd(loqt_nf4_mat Wq, loqt_nf4_mat Pq, const void *B, int
  * W_q and P_q are frozen: no other gradient is produced.  dB is overwritten,
  * or added to when accumulate_dB != 0 (gradient accumulation).  The split-K
  * reduction of dB is done in a fixed order, so results are reproducible.
- * dx may be NULL to skip the input gradient.
+ * dx may be NULL to skip the input gradient.  ws: workspace of at least
+ * loqt_workspace_bytes(LOQT_OP_BWD, ...) bytes; besides s*v and the split-K
+ * partial sums it holds deq(P_q) as bf16 (out x roundup(r, 64)), written once
+ * per call so that the product for v need not dequantise P_q again for every
+ * 256 token rows.
  */
 loqt_status loqt_linear_bwd(loqt_nf4_mat Wq, loqt_nf4_mat Pq, const void *B, int64_t ldb, float s,
                             const void *x, int64_t ldx, const void *dy, int64_t lddy, int32_t T,
@@ -129,8 +133,8 @@ loqt_status loqt_linear_bwd(loqt_nf4_mat Wq, loqt_nf4_mat Pq, const void *B, int
  * operand of the tensor-core product, the sum is formed in fp32.  Each block of
  * W_q depends only on its own previous contents, so the update is in place.
  * Two launches: deq(P_q) is written once, as bf16, into the workspace
- * (loqt_workspace_bytes(LOQT_OP_MERGE, ...) bytes), then one product kernel
- * requantises W_q in its epilogue.
+ * (loqt_workspace_bytes(LOQT_OP_MERGE, ...) bytes), then the merge kernel forms
+ * the product and requantises W_q in its epilogue.
  */
 loqt_status loqt_merge_requant(loqt_nf4_mat Wq, loqt_nf4_mat Pq, const void *B, int64_t ldb,
                                float s, void *ws, size_t ws_bytes, void *stream);

@@ -509,24 +509,12 @@ loqt_status orthonormalise(const float *Y, int64_t ldy, int m, int r, float *qf,
   cursor += up256(sq);
   double *T = reinterpret_cast<double *>(cursor);
 
-  // Every kernel of the sequence asks for the same split of the SM's memory between shared
-  // memory and L1: a change of the split between two launches makes the second wait for
-  // the SMs to drain and switch over.
-  static bool attr_set = false;
-  if (!attr_set) {
-    bool ok = cudaFuncSetAttribute(chol_panel_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kPanelSmem)) == cudaSuccess &&
-              cudaFuncSetAttribute(gram_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kBigSmem)) == cudaSuccess &&
-              cudaFuncSetAttribute(apply_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kBigSmem)) == cudaSuccess;
-    const int carve = cudaSharedmemCarveoutMaxShared;
-    ok = ok && cudaFuncSetAttribute(chol_panel_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, carve) == cudaSuccess &&
-         cudaFuncSetAttribute(chol_update_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, carve) == cudaSuccess &&
-         cudaFuncSetAttribute(block_gemm_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, carve) == cudaSuccess &&
-         cudaFuncSetAttribute(gram_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, carve) == cudaSuccess &&
-         cudaFuncSetAttribute(gram_reduce_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, carve) == cudaSuccess &&
-         cudaFuncSetAttribute(apply_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, carve) == cudaSuccess;
-    if (!ok) return LOQT_ERR_CUDA;
-    attr_set = true;
-  }
+  // (function attributes belong to the current device's context: set on every call, as the
+  // product engine does, so that a process driving several GPUs is served on each)
+  if (cudaFuncSetAttribute(chol_panel_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kPanelSmem)) != cudaSuccess ||
+      cudaFuncSetAttribute(gram_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kBigSmem)) != cudaSuccess ||
+      cudaFuncSetAttribute(apply_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kBigSmem)) != cudaSuccess)
+    return LOQT_ERR_CUDA;
   int launches = 0;
   // S = Y^T Y
   int rows_per_split = (m + splits - 1) / splits;
