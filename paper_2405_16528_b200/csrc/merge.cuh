@@ -245,6 +245,22 @@ loqt_merge_kernel(const __grid_constant__ MergeBatch mb) {
       const MergeProblem &pr = mb.prob[pi];
       const uint32_t acc = tile & 1u;
       const uint32_t ph = (tile >> 1) & 1u;
+      // The old scales of this warp's blocks of the tile (one or two of the BN / 64 column
+      // blocks) are asked for now, before the wait for the accumulator: a scalar load per
+      // row from global memory is otherwise the longest stall of a block.  Nothing else
+      // writes these scales before this thread does.
+      float m_pre[BN / 64];
+      {
+        const int row_p = m_blk * kHM + q * 32 + lane;
+#pragma unroll
+        for (int jb = 0; jb < BN / 64; ++jb) {
+          const int c0 = n_blk * BN + jb * 64;
+          const bool mine = static_cast<int>((tile * (BN / 64) + jb) % kEpiGroups) == grp;
+          m_pre[jb] = (!kComp && mine && row_p < pr.M && c0 < pr.wq_ld)
+                          ? pr.wq_absmax[static_cast<int64_t>(row_p) * (pr.wq_ld >> 6) + (c0 >> 6)]
+                          : 0.0f;
+        }
+      }
       if (!(ok = ptx::mbar_wait(tfull_bar(acc), ph, abort_flag, mb.status))) break;
       // the tile's old codes (rows of BN / 2 bytes, TMA-swizzled: 16-byte chunk ^= row & 7
       // for 128-byte rows, (row >> 1) & 3 for 64-byte rows); the new ones replace them there
@@ -289,7 +305,9 @@ loqt_merge_kernel(const __grid_constant__ MergeBatch mb) {
                                  (live && c0 + 2 * e + 1 < pr.N) ? __ldg(wp + 2 * e + 1) : 0.0f);
           }
         } else {
-          if (live) Mold = *mp;  // in flight while the accumulator is read
+#pragma unroll
+          for (int k = 0; k < BN / 64; ++k)
+            if (k == jb) Mold = m_pre[k];
           ca = ld_shared_v4(a0);
           cb = ld_shared_v4(a1);
         }
