@@ -203,7 +203,7 @@ __device__ __forceinline__ double fast_rcp(double x) {
 // precision) is replaced by one and reported through the status word.
 //
 // The factorisation keeps the lower triangle in registers (its 2080 elements dealt
-// over the 256 threads, nine slots each) and passes only the current column through
+// over the 256 threads, nine slots each, column by column) and passes only the current column through
 // shared memory: step j subtracts col[i] col[k] / pivot_j from every element (i, k)
 // with k > j, and the owners of column j + 1 publish it for the next step - one
 // barrier per step.  The inverse of the factor is built by doubling: 8 x 8 diagonal
@@ -220,18 +220,31 @@ chol_panel_kernel(double *__restrict__ S, int rp, int p, double *__restrict__ X,
   const int64_t d0 = static_cast<int64_t>(p) * kT;
 
   // ---- factorisation
+  // Elements are numbered column by column (column k holds rows k .. 63), so that slot q of
+  // every thread lies in a narrow band of columns: an element (i, k) is touched only while
+  // j < k, and once the band of a slot is behind the current column the slot is skipped by
+  // all threads at once - on average four of the nine slots are live.
   constexpr int kSlots = 9, kLower = kT * (kT + 1) / 2;
+  auto column_of = [](int idx, int &i, int &k) {  // idx -> (row, column) in column-major packed order
+    int c = 0, first = 0;                         // first = number of the column's top element
+    while (first + (kT - c) <= idx) first += kT - c, ++c;
+    k = c;
+    i = c + (idx - first);
+  };
   double val[kSlots];
-  int ei[kSlots], ek[kSlots];
+  int ei[kSlots], ek[kSlots], last_col[kSlots];
 #pragma unroll
   for (int q = 0; q < kSlots; ++q) {
     const int idx = tid + 256 * q;
     int i = 0, k = 0;
-    if (idx < kLower) lower_tile(idx, i, k);
+    if (idx < kLower) column_of(idx, i, k);
     ei[q] = i;
     ek[q] = idx < kLower ? k : -1;  // -1: empty slot
     val[q] = idx < kLower ? S[(d0 + i) * rp + d0 + k] : 0.0;
     if (ek[q] == 0) col[0][i] = val[q];
+    int li, lk;
+    column_of(min(256 * q + 255, kLower - 1), li, lk);  // the same for every thread
+    last_col[q] = lk;
   }
   __syncthreads();
   for (int j = 0; j < kT; ++j) {
@@ -246,6 +259,7 @@ chol_panel_kernel(double *__restrict__ S, int rp, int p, double *__restrict__ X,
     const double inv = fast_rcp(piv);
 #pragma unroll
     for (int q = 0; q < kSlots; ++q) {
+      if (last_col[q] <= j) continue;  // uniform: the whole slot is done
       if (ek[q] > j) {
         val[q] = fma(-(cur[ei[q]] * cur[ek[q]]), inv, val[q]);  // the product does not wait for the reciprocal
         if (ek[q] == j + 1) nxt[ei[q]] = val[q];
