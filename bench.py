@@ -453,18 +453,49 @@ def measure_config(args, ci, rank, world, local_rank, dist, device, e2e=True):
             h2d += sh["hx"].numel() * 2 + sh["hdy"].numel() * 2
             d2h += sh["hdB"].numel() * 4
 
+        # Copies and kernels run on three streams: the activations of the next matrix arrive
+        # (copy stream, two staging slots per shape) while the current one is computed, and dB
+        # leaves (second copy stream, two dB buffers per shape) while the next one is computed.
+        main = torch.cuda.current_stream()
+        s_in, s_out = torch.cuda.Stream(device=device), torch.cuda.Stream(device=device)
+        for sh in shapes.values():
+            sh["slots"] = [
+                {"dxin": torch.empty_like(sh["dxin"]), "ddy": torch.empty_like(sh["ddy"]),
+                 "dB": torch.empty((cfg.r, sh["hdB"].shape[1]), dtype=torch.float32, device=device),
+                 "free": None, "drained": None}
+                for _ in range(2)]
+            sh["next"] = 0
+
         def e2e_step():
             for m in mats:
                 sh = shapes[(m["out"], m["in"])]
                 b = bufs[(m["out"], m["in"])]
-                sh["dxin"].copy_(sh["hx"], non_blocking=True)
-                sh["ddy"].copy_(sh["hdy"], non_blocking=True)
-                xin = sh["dxin"][:, : m["in"]]
-                dyin = sh["ddy"][:, : m["out"]]
+                slot = sh["slots"][sh["next"]]
+                sh["next"] ^= 1
+                with torch.cuda.stream(s_in):
+                    if slot["free"] is not None:
+                        s_in.wait_event(slot["free"])      # the kernels that last read this slot are done
+                    slot["dxin"].copy_(sh["hx"], non_blocking=True)
+                    slot["ddy"].copy_(sh["hdy"], non_blocking=True)
+                    arrived = torch.cuda.Event()
+                    arrived.record(s_in)
+                main.wait_event(arrived)
+                if slot["drained"] is not None:
+                    main.wait_event(slot["drained"])       # this slot's previous dB has left
+                xin = slot["dxin"][:, : m["in"]]
+                dyin = slot["ddy"][:, : m["out"]]
                 L.loqt_linear_fwd(m["Wq"], m["Pq"], m["B"], s, xin, y=b["y"], ws=ws)
-                L.loqt_linear_bwd(m["Wq"], m["Pq"], m["B"], s, xin, dyin, dx=b["dx"], dB=b["dB"], ws=ws)
-                sh["hdB"].copy_(b["dB"], non_blocking=True)
+                L.loqt_linear_bwd(m["Wq"], m["Pq"], m["B"], s, xin, dyin, dx=b["dx"], dB=slot["dB"], ws=ws)
+                slot["free"] = torch.cuda.Event()
+                slot["free"].record(main)
+                with torch.cuda.stream(s_out):
+                    s_out.wait_event(slot["free"])
+                    sh["hdB"].copy_(slot["dB"], non_blocking=True)
+                    slot["drained"] = torch.cuda.Event()
+                    slot["drained"].record(s_out)
             merge()
+            main.wait_stream(s_out)
+            main.wait_stream(s_in)
 
         e2e_step()
         sync()
@@ -605,7 +636,7 @@ def run_ours(args, rank, world, local_rank):
             "h2d_bytes_per_step": main["h2d"],
             "d2h_bytes_per_step": main["d2h"],
             "steps": main["e2e_steps"],
-            "region": "H2D of x and dy of every matrix from pinned memory, fwd, bwd, D2H of dB, then the merge of all matrices",
+            "region": "H2D of x and dy of every matrix from pinned memory, fwd, bwd, D2H of dB, then the merge of all matrices; copies on their own streams, overlapped with the kernels",
             "left_out": "y and dx are not copied back: they stay on the device for the neighbouring layers",
         },
         "configs": {},
