@@ -544,6 +544,28 @@ def subspace_iteration(G: np.ndarray, Omega: np.ndarray, iters: int) -> np.ndarr
     return Q
 
 
+def top_r_right_subspace(G: np.ndarray, r: int) -> np.ndarray:
+    """The right-side counterpart (Section 2.1: a matrix with more rows than columns is
+    projected from the right): the r right singular vectors of G with the largest singular
+    values, as the rows of an r x in matrix (numpy's SVD, float64)."""
+    _, _, Vt = np.linalg.svd(np.asarray(G, dtype=np.float64), full_matrices=False)
+    return Vt[:r, :]
+
+
+def subspace_iteration_right(G: np.ndarray, Omega: np.ndarray, iters: int) -> np.ndarray:
+    """Randomised subspace iteration for the right singular subspace:
+
+        Q = orth(G^T Omega);  repeat iters times:  Z = orth(G Q);  Q = orth(G^T Z)
+
+    Omega: out x r test matrix.  Returns Q^T, r x in with orthonormal rows."""
+    G = np.asarray(G, dtype=np.float64)
+    Q, _ = np.linalg.qr(G.T @ np.asarray(Omega, dtype=np.float64))
+    for _ in range(int(iters)):
+        Z, _ = np.linalg.qr(G @ Q)
+        Q, _ = np.linalg.qr(G.T @ Z)
+    return Q.T
+
+
 def subspace_sines(P: np.ndarray, Q: np.ndarray) -> np.ndarray:
     """Sines of the principal angles between the column spaces of P and Q (both
     with orthonormal columns): the singular values of (I - P P^T) Q."""

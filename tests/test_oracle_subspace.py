@@ -75,3 +75,23 @@ def test_iteration_matches_plain_power_iteration_for_rank_one():
     y /= np.linalg.norm(y)
     Q = O.subspace_iteration(G, w, 3)
     assert min(np.linalg.norm(Q - y), np.linalg.norm(Q + y)) < 1e-10
+
+
+def test_right_side_recovers_a_planted_right_subspace():
+    # G = U diag(s) V^T with known V: the top-r right subspace is span(V[:, :r]); the iteration converges to it
+    out, inn, r = 160, 96, 12
+    rng = np.random.default_rng(5)
+    U, _ = np.linalg.qr(rng.normal(size=(out, inn)))
+    V, _ = np.linalg.qr(rng.normal(size=(inn, inn)))
+    s = np.concatenate([np.linspace(2.0, 1.0, r), 0.3 * np.linspace(1.0, 0.1, inn - r)])
+    G = (U * s) @ V.T
+    Qd = O.top_r_right_subspace(G, r)
+    assert Qd.shape == (r, inn) and np.allclose(Qd @ Qd.T, np.eye(r), atol=1e-12)
+    assert np.max(O.subspace_sines(V[:, :r], Qd.T)) < 1e-10
+    # what the right-side variant needs of it: G Q^T Q keeps the energy of the r largest singular values
+    assert np.isclose(np.linalg.norm(G @ Qd.T) ** 2, np.sum(s[:r] ** 2), rtol=1e-12)
+    Omega = rng.normal(size=(out, r))
+    err = [np.max(O.subspace_sines(V[:, :r], O.subspace_iteration_right(G, Omega, q).T)) for q in range(5)]
+    assert all(err[q + 1] < 0.3 * err[q] for q in range(1, 4)) and err[4] < 1e-3
+    Q = O.subspace_iteration_right(G, Omega, 2)
+    assert Q.shape == (r, inn) and np.allclose(Q @ Q.T, np.eye(r), atol=1e-12)
