@@ -231,6 +231,21 @@ loqt_status loqt_projection(const float *G, int64_t ldg, int32_t out, int32_t in
                             void *ws, size_t ws_bytes, void *stream);
 
 /*
+ * The same for the right-side variant (Section 2.1, the one-sided projection of a
+ * matrix with more rows than columns: G Q with Q spanning the leading right
+ * singular vectors).  The iteration above runs on G^T:
+ *     Q = orth(G^T Omega);   repeat iters times:   Z = orth(G Q);   Q = orth(G^T Z)
+ *   Omega : bf16 [out][ldo], the out x r test matrix.
+ *   Q     : fp32 [r][ldq], receives the basis transposed, r x in with orthonormal
+ *           rows: the layout of the factor Q_q of loqt_linear_fwd_right.
+ * Everything else (G, limits, precisions, LOQT_ERR_NUMERIC, workspace) as for
+ * loqt_projection.
+ */
+loqt_status loqt_projection_right(const float *G, int64_t ldg, int32_t out, int32_t in, int32_t r,
+                                  const void *Omega, int64_t ldo, int32_t iters, float *Q,
+                                  int64_t ldq, void *ws, size_t ws_bytes, void *stream);
+
+/*
  * Error-compensated initialisation of a layer for a new projection P
  * (Section 2.5 "Compensating for Quantization Errors"; Algorithm 2, the loop over
  * compensation steps; appendix: B = P^+ (W - Q)).  Alternating minimisation of

@@ -28,7 +28,7 @@ EXPORTS = (
     "loqt_device_status", "loqt_launch_count", "loqt_status_string",
     "loqt_set_tile_override", "loqt_variant_launches", "loqt_selftest_wait_timeout",
     "loqt_scales_workspace_bytes", "loqt_scales_double_quantize", "loqt_scales_double_dequantize",
-    "loqt_nf4_dequantize_dq", "loqt_linear_fwd_dq", "loqt_linear_bwd_dq", "loqt_adam8_step", "loqt_projection",
+    "loqt_nf4_dequantize_dq", "loqt_linear_fwd_dq", "loqt_linear_bwd_dq", "loqt_adam8_step", "loqt_projection", "loqt_projection_right",
 )
 
 
@@ -98,6 +98,8 @@ def lib():
     L.loqt_full_gradient.restype = ctypes.c_int
     L.loqt_projection.argtypes = [vp, i64, i32, i32, i32, vp, i64, i32, vp, i64, vp, sz, vp]
     L.loqt_projection.restype = ctypes.c_int
+    L.loqt_projection_right.argtypes = L.loqt_projection.argtypes
+    L.loqt_projection_right.restype = ctypes.c_int
     L.loqt_adam_step.argtypes = [vp, i64, vp, i64, vp, vp, i64, i32, i32, loqt_adam_params, vp]
     L.loqt_adam_step.restype = ctypes.c_int
     L.loqt_merge_requant_many.argtypes = [i32, ctypes.POINTER(M), ctypes.POINTER(M), ctypes.POINTER(vp), ctypes.POINTER(i64), f32, vp, sz, vp]
@@ -357,6 +359,22 @@ def loqt_projection(G: torch.Tensor, Omega: torch.Tensor, iters: int, P: torch.T
                                  int(iters), _dev(P, torch.float32), P.stride(0), ws.data_ptr(), ws.numel(), _stream()),
            "loqt_projection")
     return P
+
+
+def loqt_projection_right(G: torch.Tensor, Omega: torch.Tensor, iters: int, Q: torch.Tensor | None = None,
+                          ws: torch.Tensor | None = None) -> torch.Tensor:
+    """Q (fp32 [r, in], orthonormal rows) spanning approximately the r leading right singular vectors of
+    G (fp32 [out, in]) by `iters` rounds of subspace iteration started from Omega (bf16 [out, r])."""
+    out, inn = G.shape
+    r = Omega.shape[1]
+    if Q is None:
+        Q = torch.empty((r, inn), dtype=torch.float32, device=G.device)
+    if ws is None:
+        ws = new_workspace(loqt_workspace_bytes(LOQT_OP_PROJECTION, out, inn, r, 0), G.device)
+    _check(lib().loqt_projection_right(_dev(G, torch.float32), G.stride(0), out, inn, r, _dev(Omega, torch.bfloat16),
+                                       Omega.stride(0), int(iters), _dev(Q, torch.float32), Q.stride(0), ws.data_ptr(),
+                                       ws.numel(), _stream()), "loqt_projection_right")
+    return Q
 
 
 def loqt_adam_step(B: torch.Tensor, dB: torch.Tensor, m: torch.Tensor, v: torch.Tensor, step: int, lr: float,

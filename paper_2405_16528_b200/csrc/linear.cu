@@ -859,13 +859,17 @@ static loqt_status projection_product(const void *gb, int64_t ldgb, bool transpo
   return launch(c, stm);
 }
 
-extern "C" loqt_status loqt_projection(const float *G, int64_t ldg, int32_t out, int32_t in, int32_t r, const void *Omega,
-                                       int64_t ldo, int32_t iters, float *P, int64_t ldp, void *ws, size_t ws_bytes,
-                                       void *stream) {
+// The iteration for either side.  Left (right == false): basis of the leading left singular
+// subspace, out x r, from an in x r test matrix.  Right: the same iteration on G^T - the
+// roles of G and G^T in the products are exchanged - from an out x r test matrix; the basis
+// (in x r) is stored transposed, r x in, the layout of the right-side variant's factor Q.
+static loqt_status projection_impl(bool right, const float *G, int64_t ldg, int32_t out, int32_t in, int32_t r, const void *Omega,
+                                   int64_t ldo, int32_t iters, float *basis, int64_t ld_basis, void *ws, size_t ws_bytes,
+                                   void *stream) {
   loqt_status st;
   if (out <= 0 || in <= 0 || r <= 0 || r > out || r > in || r > 4096 || iters < 0 || iters > 16) return LOQT_ERR_INVALID_ARG;
-  if (G == nullptr || P == nullptr || ldg < in || ldp < r) return LOQT_ERR_INVALID_ARG;
-  if ((reinterpret_cast<uintptr_t>(G) & 15u) != 0 || (reinterpret_cast<uintptr_t>(P) & 3u) != 0) return LOQT_ERR_ALIGNMENT;
+  if (G == nullptr || basis == nullptr || ldg < in || ld_basis < (right ? in : r)) return LOQT_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(G) & 15u) != 0 || (reinterpret_cast<uintptr_t>(basis) & 3u) != 0) return LOQT_ERR_ALIGNMENT;
   if ((st = check_bf16(Omega, ldo, r)) != LOQT_OK) return st;
   if ((st = check_ws(ws, ws_bytes, loqt_workspace_bytes(LOQT_OP_PROJECTION, out, in, r, 0))) != LOQT_OK) return st;
   if ((st = check_arch()) != LOQT_OK) return st;
@@ -880,19 +884,40 @@ extern "C" loqt_status loqt_projection(const float *G, int64_t ldg, int32_t out,
   void *lo = cursor;                                  cursor += align256(static_cast<size_t>(big) * ldr * 2);
   void *orth_ws = cursor;
 
+  // A = G for the left side, G^T for the right: rows m_a, columns k_a; `main` products are A (.),
+  // `back` products A^T (.)
+  const int m_a = right ? in : out, k_a = right ? out : in;
+  auto product = [&](bool back, const void *bhi, const void *blo, int64_t ldq) {
+    const bool transposed = back != right;  // whether bf16 G is read as G^T
+    return projection_product(gb, ldgb, transposed, back ? k_a : m_a, back ? m_a : k_a, r, bhi, blo, ldq, Y, ldr, status, stm);
+  };
   if ((st = convert_f32_bf16(G, ldg, gb, ldgb, out, in, stm)) != LOQT_OK) return st;
-  // Q = orth(G Omega)
-  if ((st = projection_product(gb, ldgb, false, out, in, r, Omega, nullptr, ldo, Y, ldr, status, stm)) != LOQT_OK) return st;
-  if ((st = orthonormalise(Y, ldr, out, r, iters == 0 ? P : nullptr, ldp, hi, lo, ldr, orth_ws, status, stm)) != LOQT_OK) return st;
+  // Q = orth(A Omega)
+  if ((st = product(false, Omega, nullptr, ldo)) != LOQT_OK) return st;
+  if ((st = orthonormalise(Y, ldr, m_a, r, iters == 0 ? basis : nullptr, ld_basis, right, hi, lo, ldr, orth_ws, status, stm)) != LOQT_OK)
+    return st;
   for (int it = 1; it <= iters; ++it) {
-    // Z = orth(G^T Q)
-    if ((st = projection_product(gb, ldgb, true, in, out, r, hi, lo, ldr, Y, ldr, status, stm)) != LOQT_OK) return st;
-    if ((st = orthonormalise(Y, ldr, in, r, nullptr, 0, hi, lo, ldr, orth_ws, status, stm)) != LOQT_OK) return st;
-    // Q = orth(G Z)
-    if ((st = projection_product(gb, ldgb, false, out, in, r, hi, lo, ldr, Y, ldr, status, stm)) != LOQT_OK) return st;
-    if ((st = orthonormalise(Y, ldr, out, r, it == iters ? P : nullptr, ldp, hi, lo, ldr, orth_ws, status, stm)) != LOQT_OK) return st;
+    // Z = orth(A^T Q)
+    if ((st = product(true, hi, lo, ldr)) != LOQT_OK) return st;
+    if ((st = orthonormalise(Y, ldr, k_a, r, nullptr, 0, false, hi, lo, ldr, orth_ws, status, stm)) != LOQT_OK) return st;
+    // Q = orth(A Z)
+    if ((st = product(false, hi, lo, ldr)) != LOQT_OK) return st;
+    if ((st = orthonormalise(Y, ldr, m_a, r, it == iters ? basis : nullptr, ld_basis, right, hi, lo, ldr, orth_ws, status, stm)) != LOQT_OK)
+      return st;
   }
   return LOQT_OK;
+}
+
+extern "C" loqt_status loqt_projection(const float *G, int64_t ldg, int32_t out, int32_t in, int32_t r, const void *Omega,
+                                       int64_t ldo, int32_t iters, float *P, int64_t ldp, void *ws, size_t ws_bytes,
+                                       void *stream) {
+  return projection_impl(false, G, ldg, out, in, r, Omega, ldo, iters, P, ldp, ws, ws_bytes, stream);
+}
+
+extern "C" loqt_status loqt_projection_right(const float *G, int64_t ldg, int32_t out, int32_t in, int32_t r, const void *Omega,
+                                             int64_t ldo, int32_t iters, float *Q, int64_t ldq, void *ws, size_t ws_bytes,
+                                             void *stream) {
+  return projection_impl(true, G, ldg, out, in, r, Omega, ldo, iters, Q, ldq, ws, ws_bytes, stream);
 }
 
 // ---------------------------------------------------------------------------

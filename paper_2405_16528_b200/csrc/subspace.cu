@@ -427,11 +427,12 @@ block_gemm_kernel(const double *__restrict__ L, double *__restrict__ X, double *
 
 // Q = Y X^T with X = L^-1 lower triangular: Q[a][j] = sum_(c <= j) Y[a][c] X[j][c].
 // 128 x 128 tiles; the tile of column block bj sums over the columns c < 128 (bj + 1).
-// Outputs (each optional): Q as fp32, and Q split into two bf16 matrices hi + lo
+// Outputs (each optional): Q as fp32 (m x r, or transposed, r x m, when qf_transposed), and Q split into two bf16 matrices hi + lo
 // (hi = bf16(Q), lo = bf16(Q - hi)), the form in which the next product consumes it.
 __global__ void __launch_bounds__(256)
 apply_kernel(const float *__restrict__ Y, int64_t ldy, int m, int r, int rp, const double *__restrict__ X,
-             float *__restrict__ qf, int64_t ldqf, __nv_bfloat16 *__restrict__ qhi, __nv_bfloat16 *__restrict__ qlo, int64_t ldqb) {
+             float *__restrict__ qf, int64_t ldqf, int qf_transposed, __nv_bfloat16 *__restrict__ qhi, __nv_bfloat16 *__restrict__ qlo,
+             int64_t ldqb) {
   extern __shared__ __align__(16) double smg[];
   const int bj = static_cast<int>(gridDim.y) - 1 - static_cast<int>(blockIdx.y);  // longest sums first
   const int64_t row0 = static_cast<int64_t>(blockIdx.x) * kG;
@@ -480,7 +481,7 @@ apply_kernel(const float *__restrict__ Y, int64_t ldy, int m, int r, int rp, con
       const int col = j0 + own8(tx, j);
       if (col >= r) continue;
       const float f = static_cast<float>(acc[i][j]);
-      if (qf != nullptr) qf[row * ldqf + col] = f;
+      if (qf != nullptr) qf[qf_transposed ? col * ldqf + row : row * ldqf + col] = f;
       if (qhi != nullptr) {
         const __nv_bfloat16 hi = __float2bfloat16_rn(f);
         qhi[row * ldqb + col] = hi;
@@ -511,7 +512,7 @@ size_t orth_workspace_bytes(int m, int r) {
   return up256(static_cast<size_t>(gram_splits(m, static_cast<int>(rp))) * sq) + 2 * up256(sq);  // Gram partials / L, X, T
 }
 
-loqt_status orthonormalise(const float *Y, int64_t ldy, int m, int r, float *qf, int64_t ldqf, void *qhi, void *qlo,
+loqt_status orthonormalise(const float *Y, int64_t ldy, int m, int r, float *qf, int64_t ldqf, bool qf_transposed, void *qhi, void *qlo,
                            int64_t ldqb, void *ws, uint32_t *status, cudaStream_t stream) {
   const int rp = (r + kT - 1) / kT * kT, nb = rp / kT;
   const int splits = gram_splits(m, rp);
@@ -558,7 +559,7 @@ loqt_status orthonormalise(const float *Y, int64_t ldy, int m, int r, float *qf,
     launches += 2;
   }
   // Q = Y X^T
-  apply_kernel<<<dim3((m + kG - 1) / kG, gb), 256, kBigSmem, stream>>>(Y, ldy, m, r, rp, X, qf, ldqf, static_cast<__nv_bfloat16 *>(qhi),
+  apply_kernel<<<dim3((m + kG - 1) / kG, gb), 256, kBigSmem, stream>>>(Y, ldy, m, r, rp, X, qf, ldqf, qf_transposed ? 1 : 0, static_cast<__nv_bfloat16 *>(qhi),
                                                                        static_cast<__nv_bfloat16 *>(qlo), ldqb);
   count_launch(launches + 1);
   return cudaGetLastError() == cudaSuccess ? LOQT_OK : LOQT_ERR_CUDA;

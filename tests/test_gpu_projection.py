@@ -136,3 +136,30 @@ def test_argument_checks():
         L.loqt_projection(Gd, Od[:, :32], 17)  # too many iterations
     with pytest.raises(L.LoqtError, match="workspace"):
         L.loqt_projection(Gd, Od[:, :32], 1, ws=L.new_workspace(512))
+
+
+@pytest.mark.parametrize("case", [(1376, 512, 40, 1), (640, 256, 96, 2), (2736, 1024, 256, 1)])
+def test_right_side_projection_matches_the_oracle_subspace(case):
+    """loqt_projection_right: the basis of the leading right singular subspace, stored r x in as the
+    right-side variant's factor Q is, against the oracle's iterate on the same Omega (out x r)."""
+    out, inn, r, iters = case
+    G = synth.lowrank_gradient(54, ("G", out, inn, r), out, inn, r)
+    Om = synth.normal(54, ("Omega", out, r), (out, r), 1.0, torch.bfloat16)
+    Gd = torch.zeros((out, (inn + 3) // 4 * 4), dtype=torch.float32, device="cuda")[:, :inn]
+    Gd.copy_(G)
+    Od = torch.zeros((out, (r + 7) // 8 * 8), dtype=torch.bfloat16, device="cuda")[:, :r]
+    Od.copy_(Om)
+    Gb, Omf = O.bf16_round(G.numpy()).astype(np.float64), f32(Om).astype(np.float64)
+    ws = L.new_workspace(L.loqt_workspace_bytes(L.LOQT_OP_PROJECTION, out, inn, r, 0))
+    Q = L.loqt_projection_right(Gd, Od, iters, ws=ws)
+    L.loqt_device_status(ws)
+    Q = f32(Q).astype(np.float64)
+    assert Q.shape == (r, inn) and np.isfinite(Q).all()
+    assert np.abs(Q @ Q.T - np.eye(r)).max() < 2e-6
+    Qo = O.subspace_iteration_right(Gb, Omf, iters)
+    sines = O.subspace_sines(Qo.T, Q.T)
+    tol, cond0 = _tolerance(Gb.T, Omf, r, iters)
+    print(f"right projection {case}: max sine {sines.max():.3e} (tolerance {tol:.3e}, cond(G^T Omega) = {cond0:.1f})")
+    assert sines.max() <= tol
+    cap, cap_ref = np.linalg.norm(Gb @ Q.T) ** 2, np.linalg.norm(Gb @ Qo.T) ** 2
+    assert abs(cap - cap_ref) <= 1e-5 * cap_ref
