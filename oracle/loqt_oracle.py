@@ -315,6 +315,32 @@ def loqt_backward_right(wq, qq, B, s, x, dy, shape):
     return dx, dB
 
 
+def loqt_compensate_right(W, Q, steps, B0=None):
+    """Error-compensated initialisation for the right-side variant (Section 2.5 and
+    Algorithm 2's loop, carried over to the right-side factorisation W = Q_w + B Q of
+    Section 2.1): alternating minimisation of || Q_w + B Q - W || for a fixed Q with
+    orthonormal rows,
+
+        B_0 = 0;  for c = 1..steps:  Q_c = q_NF4( W - B_{c-1} Q ),  B_c = ( W - deq(Q_c) ) Q^+
+
+    with Q^+ = Q^T.  Precisions as in loqt_compensate: W and W - B Q are 32-bit, Q, the
+    residual and B enter the products as 16-bit operands, sums in float64.
+    W: fp32 [out, in]; Q: fp32 [r, in].  Returns ((codes, absmax) of Q_steps, B_steps as
+    fp32 holding bf16 values [out, r])."""
+    W = np.asarray(W, dtype=np.float32)
+    out, inn = W.shape
+    Qb = bf16_round(np.asarray(Q, dtype=np.float32)).astype(np.float64)
+    W64 = W.astype(np.float64)
+    B = np.zeros((out, Qb.shape[0]), dtype=np.float32) if B0 is None else bf16_round(np.asarray(B0, dtype=np.float32))
+    q = None
+    for _ in range(int(steps)):
+        what = (W64 - B.astype(np.float64) @ Qb).astype(np.float32)
+        q = nf4_quantize(what)
+        resid = bf16_round((W - nf4_dequantize(q[0], q[1], inn)).astype(np.float32))
+        B = bf16_round((resid.astype(np.float64) @ Qb.T).astype(np.float32))
+    return q, B
+
+
 def loqt_merge_values_right(wq, qq, B, s, shape) -> np.ndarray:
     """fl32( deq32(W_q) + s * B @ Q_BF16 ): the quantiser's input at a merge."""
     out, inn, r = shape

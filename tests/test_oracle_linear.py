@@ -376,3 +376,35 @@ def test_right_merge_equals_the_dense_sum_built_entry_by_entry(shape):
     Q32 = np.array([[float(np.float32(qq[1][k, i // 64]) * lv[qq[0][k, i]]) for i in range(inn)] for k in range(r)])
     wrong = (O.nf4_dequantize(*wq, inn).astype(np.float64) + s * B.astype(np.float64) @ Q32).astype(np.float32)
     assert np.mean(wrong != vw) > 0.2
+
+
+def test_right_compensation_is_the_least_squares_fit_and_keeps_improving():
+    # B_1 = (W - deq(q(W))) Q^+ is the minimiser of || B Q - (W - Q_1) ||_F (numpy's least-squares
+    # routine on the transposed system), up to the 16-bit roundings of the operands and of B
+    rng = np.random.default_rng(81)
+    out, inn, r = 96, 160, 16
+    W = (0.02 * rng.normal(size=(out, inn))).astype(np.float32)
+    Qf, _ = np.linalg.qr(rng.normal(size=(inn, r)))
+    Q = Qf.T.astype(np.float32)                       # r x in, orthonormal rows
+    (c1, m1), B1 = O.loqt_compensate_right(W, Q, 1)
+    q0 = O.nf4_quantize(W)
+    assert np.array_equal(c1, q0[0]) and np.array_equal(m1, q0[1])
+    R = W.astype(np.float64) - O.nf4_dequantize(q0[0], q0[1], inn)
+    Bls = np.linalg.lstsq(Q.astype(np.float64).T, R.T, rcond=None)[0].T       # min || Q^T B^T - R^T ||
+    assert np.abs(B1 - Bls).max() <= 2.0 ** -7 * np.abs(Bls).max()
+    # the objective falls step by step, and the fit beats plain quantisation by about the share r / in
+    def err(q, B):
+        return np.linalg.norm(O.nf4_dequantize(q[0], q[1], inn) + B.astype(np.float64) @ O.bf16_round(Q) - W) ** 2
+    e0 = np.linalg.norm(R) ** 2
+    es = [err(*O.loqt_compensate_right(W, Q, c)) for c in (1, 2, 3, 5)]
+    assert es[0] < e0 and all(es[i + 1] <= es[i] * (1 + 1e-9) for i in range(3))
+    assert es[0] < (1 - 0.7 * r / inn) * e0
+    # weights that NF4 represents exactly need no correction
+    Wr = O.nf4_dequantize(q0[0], q0[1], inn)
+    (c, m), B = O.loqt_compensate_right(Wr, Q, 3)
+    assert np.array_equal(c, q0[0]) and np.array_equal(m, q0[1]) and not B.any()
+    # one step from a given state equals the definition written out with that B
+    B0 = O.bf16_round((1e-3 * rng.normal(size=(out, r))).astype(np.float32))
+    (c2, m2), _ = O.loqt_compensate_right(W, Q, 1, B0=B0)
+    ref = O.nf4_quantize((W.astype(np.float64) - B0.astype(np.float64) @ O.bf16_round(Q).astype(np.float64)).astype(np.float32))
+    assert np.array_equal(c2, ref[0]) and np.array_equal(m2, ref[1])
