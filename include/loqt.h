@@ -71,7 +71,8 @@ typedef struct {
 
 /* Operation selector for loqt_workspace_bytes(). */
 enum { LOQT_OP_FWD = 0, LOQT_OP_BWD = 1, LOQT_OP_MERGE = 2, LOQT_OP_MERGE_SPLIT = 3, LOQT_OP_COMPENSATE = 4, LOQT_OP_FULL_GRADIENT = 5,
-       LOQT_OP_FWD_RIGHT = 6, LOQT_OP_BWD_RIGHT = 7, LOQT_OP_MERGE_RIGHT = 8, LOQT_OP_PROJECTION = 9 };
+       LOQT_OP_FWD_RIGHT = 6, LOQT_OP_BWD_RIGHT = 7, LOQT_OP_MERGE_RIGHT = 8, LOQT_OP_PROJECTION = 9,
+       LOQT_OP_COMPENSATE_RIGHT = 10 };
 
 /*
  * q_NF4 (Section 5.1, first two displayed equations): per block M = max|w|,
@@ -262,6 +263,20 @@ loqt_status loqt_projection_right(const float *G, int64_t ldg, int32_t out, int3
 loqt_status loqt_compensated_init(const float *W, int64_t ldw, const float *P, int64_t ldp,
                                   int32_t steps, loqt_nf4_mat Wq, loqt_nf4_mat Pq, void *B,
                                   int64_t ldb, void *ws, size_t ws_bytes, void *stream);
+
+/*
+ * The same initialisation for the right-side variant W = deq(W_q) + s B deq(Q_q)
+ * (Section 2.5 carried over to the right-side factorisation of Section 2.1):
+ *     B_0 = 0;   for c = 1..steps:   Q_c = q_NF4( W - B_{c-1} Q ),   B_c = ( W - deq(Q_c) ) Q^T
+ *   W  : fp32 [out][ldw], 16-byte aligned, ldw % 4 == 0.
+ *   Q  : fp32 [r][ldq], orthonormal rows (from loqt_projection_right).
+ *   Wq : receives Q_steps;  Qq : receives q_NF4(Q) (r x in);  B : receives B_steps as bf16 [out][ldb].
+ * Precisions and limits as for loqt_compensated_init.  Workspace:
+ * loqt_workspace_bytes(LOQT_OP_COMPENSATE_RIGHT, out, in, r, 0).
+ */
+loqt_status loqt_compensated_init_right(const float *W, int64_t ldw, const float *Q, int64_t ldq,
+                                        int32_t steps, loqt_nf4_mat Wq, loqt_nf4_mat Qq, void *B,
+                                        int64_t ldb, void *ws, size_t ws_bytes, void *stream);
 
 /*
  * One optimiser step on the trainable factor (Algorithm 1, update line

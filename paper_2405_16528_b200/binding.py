@@ -17,7 +17,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libloqt.so")
 
 LOQT_OP_FWD, LOQT_OP_BWD, LOQT_OP_MERGE, LOQT_OP_MERGE_SPLIT, LOQT_OP_COMPENSATE, LOQT_OP_FULL_GRADIENT = 0, 1, 2, 3, 4, 5
-LOQT_OP_FWD_RIGHT, LOQT_OP_BWD_RIGHT, LOQT_OP_MERGE_RIGHT, LOQT_OP_PROJECTION = 6, 7, 8, 9
+LOQT_OP_FWD_RIGHT, LOQT_OP_BWD_RIGHT, LOQT_OP_MERGE_RIGHT, LOQT_OP_PROJECTION, LOQT_OP_COMPENSATE_RIGHT = 6, 7, 8, 9, 10
 BLOCK = 64
 
 EXPORTS = (
@@ -28,7 +28,7 @@ EXPORTS = (
     "loqt_device_status", "loqt_launch_count", "loqt_status_string",
     "loqt_set_tile_override", "loqt_variant_launches", "loqt_selftest_wait_timeout",
     "loqt_scales_workspace_bytes", "loqt_scales_double_quantize", "loqt_scales_double_dequantize",
-    "loqt_nf4_dequantize_dq", "loqt_linear_fwd_dq", "loqt_linear_bwd_dq", "loqt_adam8_step", "loqt_projection", "loqt_projection_right",
+    "loqt_nf4_dequantize_dq", "loqt_linear_fwd_dq", "loqt_linear_bwd_dq", "loqt_adam8_step", "loqt_projection", "loqt_projection_right", "loqt_compensated_init_right",
 )
 
 
@@ -89,6 +89,8 @@ def lib():
     L.loqt_nf4_requantize.argtypes = [vp, i64, f32, M, vp]
     L.loqt_compensated_init.argtypes = [vp, i64, vp, i64, i32, M, M, vp, i64, vp, sz, vp]
     L.loqt_compensated_init.restype = ctypes.c_int
+    L.loqt_compensated_init_right.argtypes = L.loqt_compensated_init.argtypes
+    L.loqt_compensated_init_right.restype = ctypes.c_int
     L.loqt_linear_fwd_right.argtypes = L.loqt_linear_fwd.argtypes
     L.loqt_linear_bwd_right.argtypes = L.loqt_linear_bwd.argtypes
     L.loqt_merge_requant_right.argtypes = L.loqt_merge_requant.argtypes
@@ -291,6 +293,22 @@ def loqt_compensated_init(W: torch.Tensor, P: torch.Tensor, steps: int, ws: torc
                                        _stream()), "loqt_compensated_init")
     loqt_device_status(ws)
     return Wq, Pq, B
+
+
+def loqt_compensated_init_right(W: torch.Tensor, Q: torch.Tensor, steps: int, ws: torch.Tensor | None = None):
+    """Right-side variant.  Returns (Wq, Qq, B): Q_steps, q_NF4(Q) (r x in) and the bf16 factor B_steps (out x r)."""
+    out, inn = W.shape
+    r = Q.shape[0]
+    Wq, Qq = NF4Tensor.empty(out, inn, W.device), NF4Tensor.empty(r, inn, W.device)
+    ldb = (r + 7) // 8 * 8
+    B = torch.empty((out, ldb), dtype=torch.bfloat16, device=W.device)[:, :r]
+    if ws is None:
+        ws = new_workspace(loqt_workspace_bytes(LOQT_OP_COMPENSATE_RIGHT, out, inn, r, 0), W.device)
+    _check(lib().loqt_compensated_init_right(_dev(W, torch.float32), W.stride(0), _dev(Q, torch.float32), Q.stride(0), int(steps),
+                                             Wq.view(), Qq.view(), B.data_ptr(), B.stride(0), ws.data_ptr(), ws.numel(),
+                                             _stream()), "loqt_compensated_init_right")
+    loqt_device_status(ws)
+    return Wq, Qq, B
 
 
 def loqt_linear_fwd_right(Wq: NF4Tensor, Qq: NF4Tensor, B: torch.Tensor, s: float, x: torch.Tensor) -> torch.Tensor:

@@ -340,6 +340,11 @@ extern "C" size_t loqt_workspace_bytes(int op, int32_t out, int32_t in, int32_t 
     db_splits(out, r, T > 0 ? T : 1, splits, kbps);
     if (splits > 1) total += align256(static_cast<size_t>(splits) * out * ((static_cast<size_t>(r) + 3) / 4 * 4) * 4);
   }
+  // right-side compensated initialisation: bf16 Q (r x roundup(in, 64)) and the bf16 residual (out x roundup(in, 64))
+  if (op == LOQT_OP_COMPENSATE_RIGHT) {
+    const size_t ld64 = (static_cast<size_t>(in > 0 ? in : 0) + 63) / 64 * 64;
+    total += align256(static_cast<size_t>(r > 0 ? r : 0) * ld64 * 2) + align256(static_cast<size_t>(out > 0 ? out : 0) * ld64 * 2);
+  }
   if (op == LOQT_OP_MERGE_RIGHT) total += align256(static_cast<size_t>(r > 0 ? r : 0) * ((static_cast<size_t>(in > 0 ? in : 0) + 63) / 64 * 64) * 2);
   // projection: bf16 G, one fp32 iterate, its hi + lo bf16 basis, and the orthonormalisation's scratch
   if (op == LOQT_OP_PROJECTION) {
@@ -978,6 +983,53 @@ extern "C" loqt_status loqt_compensated_init(const float *W, int64_t ldw, const 
       if ((st = gemm_tn_f32(phat, ldr, resid, ld64, r, in, out, b32, ld4, 0, partial, status, stm)) != LOQT_OK) return st;
       if ((st = convert_f32_bf16(b32, ld4, B, ldb, r, in, stm)) != LOQT_OK) return st;
     }
+  }
+  return LOQT_OK;
+}
+
+// The same for the right-side variant: W ~ Q_w + B Q with Q (r x in, orthonormal rows) fixed,
+//   Q_c = q_NF4(W - B_(c-1) Q),   B_c = (W - deq(Q_c)) Q^T.
+extern "C" loqt_status loqt_compensated_init_right(const float *W, int64_t ldw, const float *Q, int64_t ldq, int32_t steps,
+                                                   loqt_nf4_mat Wq, loqt_nf4_mat Qq, void *B, int64_t ldb, void *ws,
+                                                   size_t ws_bytes, void *stream) {
+  loqt_status st;
+  if ((st = validate_nf4(Wq)) != LOQT_OK) return st;
+  if ((st = validate_nf4(Qq)) != LOQT_OK) return st;
+  if (Qq.cols != Wq.cols || steps < 1 || steps > 16) return LOQT_ERR_INVALID_ARG;
+  const int out = Wq.rows, in = Wq.cols, r = Qq.rows;
+  if (W == nullptr || Q == nullptr || ldw < in || ldq < in) return LOQT_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(W) & 15u) != 0 || (ldw & 3) != 0 || (reinterpret_cast<uintptr_t>(Q) & 3u) != 0)
+    return LOQT_ERR_ALIGNMENT;
+  if ((st = check_bf16(B, ldb, r)) != LOQT_OK) return st;
+  if ((st = check_ws(ws, ws_bytes, loqt_workspace_bytes(LOQT_OP_COMPENSATE_RIGHT, out, in, r, 0))) != LOQT_OK) return st;
+  if ((st = check_arch()) != LOQT_OK) return st;
+  cudaStream_t stm = static_cast<cudaStream_t>(stream);
+  uint32_t *status = static_cast<uint32_t *>(ws);
+  const int64_t ld64 = (static_cast<int64_t>(in) + 63) / 64 * 64;
+  uint8_t *cursor = static_cast<uint8_t *>(ws) + 256;
+  void *qhat = cursor;   cursor += align256(static_cast<size_t>(r) * ld64 * 2);
+  void *resid = cursor;
+
+  // Q_q = q(Q); the products use bf16(Q), the unquantised projection
+  if ((st = loqt_nf4_quantize(Q, ldq, Qq, stream)) != LOQT_OK) return st;
+  if ((st = convert_f32_bf16(Q, ldq, qhat, ld64, r, in, stm)) != LOQT_OK) return st;
+  for (int c = 1; c <= steps; ++c) {
+    if (c == 1) {
+      if ((st = nf4_quantize_residual(W, ldw, W, ldw, Wq, resid, ld64, stm)) != LOQT_OK) return st;
+    } else {
+      // the product B Q (out x in; K = r) with the quantiser and the residual in its epilogue
+      MergeItem item{Wq, {B, ldb}, {qhat, ld64}, r, -1.0f};
+      item.w32 = W; item.ld_w32 = ldw; item.resid = resid; item.ld_resid = ld64;
+      if ((st = merge_batch(&item, 1, status, stm)) != LOQT_OK) return st;
+    }
+    // B_c = residual Q^T   (out x r; K = in; both operands K-major), rounded to bf16 in the epilogue
+    GemmCall g{};
+    g.p.M = out; g.p.N = r; g.p.num_segs = 1;
+    g.p.seg[0].K = in; g.p.seg[0].a_kind = OP_TMA_K; g.p.seg[0].b_kind = OP_TMA_K;
+    g.a[0] = {resid, ld64}; g.b[0] = {qhat, ld64};
+    g.p.splits = 1; g.p.kb_per_split = 0;
+    g.p.epi = EPI_BF16; g.p.out = B; g.p.ld_out = ldb; g.p.alpha = 1.0f; g.p.status = status;
+    if ((st = launch(g, stm)) != LOQT_OK) return st;
   }
   return LOQT_OK;
 }

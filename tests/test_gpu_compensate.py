@@ -111,3 +111,55 @@ def test_argument_errors():
         L.loqt_compensated_init(Wd, Pd, 0)
     with pytest.raises(L.LoqtError, match="workspace"):
         L.loqt_compensated_init(Wd, Pd, 1, ws=L.new_workspace(1024))
+
+
+# ---- right-side variant: W ~ Q_w + B Q, Q r x in with orthonormal rows
+RIGHT_SHAPES = [(256, 256, 32), (1376, 512, 96), (5461, 256, 40), (320, 640, 64)]
+
+
+def _inputs_right(seed, out, inn, r):
+    W = synth.normal(seed, ("W", out, inn), (out, inn), 0.02)
+    Q = synth.orthonormal(seed, ("Q", inn, r), inn, r).T.contiguous()
+    ld = (inn + 3) // 4 * 4
+    Wd = torch.zeros((out, ld), dtype=torch.float32, device="cuda")[:, :inn]
+    Wd.copy_(W)
+    return W.numpy(), Q.numpy(), Wd, Q.cuda()
+
+
+@pytest.mark.parametrize("shape", RIGHT_SHAPES)
+@pytest.mark.parametrize("steps", [1, 2, 4])
+def test_right_variant_each_step_from_the_previous_state(shape, steps):
+    out, inn, r = shape
+    W, Q, Wd, Qd = _inputs_right(45, out, inn, r)
+    if steps == 1:
+        (rc, rm), rB = O.loqt_compensate_right(W, Q, 1)
+    else:
+        _, _, B_prev = L.loqt_compensated_init_right(Wd, Qd, steps - 1)
+        (rc, rm), rB = O.loqt_compensate_right(W, Q, 1, B0=f32(B_prev))
+    Wq, Qq, B = L.loqt_compensated_init_right(Wd, Qd, steps)
+    c, m = from_dev_nf4(Wq)
+    qc, qm = from_dev_nf4(Qq)
+    oc, om = O.nf4_quantize(Q)
+    assert np.array_equal(qc, oc) and np.array_equal(qm, om)
+    diff = c[:, :inn] != rc[:, :inn]
+    if steps == 1:
+        assert not diff.any() and np.array_equal(m, rm)          # Q_1 = q(W): bit-exact
+    assert diff.mean() <= 1e-4, f"{diff.mean():.2e} of the codes differ"
+    assert np.all(np.abs(c[:, :inn].astype(int) - rc[:, :inn].astype(int))[diff] == 1)
+    assert np.all(c[:, inn:] == 7)
+    assert np.abs(m - rm).max() <= 2.0 ** -20 * np.abs(rm).max()
+    clean = ~diff.any(axis=1)                                    # rows without a flipped code
+    check_close(f32(B)[clean], rB[clean], f"B_{steps} {shape} (rows without a flipped code)")
+    Qb = O.bf16_round(Q).astype(np.float64)
+    resid = O.bf16_round((W - O.nf4_dequantize(c, m, inn)).astype(np.float32)).astype(np.float64)
+    check_close(f32(B), O.bf16_round((resid @ Qb.T).astype(np.float32)), f"B_{steps} {shape} (from the library's codes)")
+
+
+def test_right_variant_representable_weights_need_no_correction():
+    out, inn, r = 256, 320, 32
+    W, Q, Wd, Qd = _inputs_right(46, out, inn, r)
+    q0 = O.nf4_quantize(W)
+    Wd.copy_(torch.from_numpy(O.nf4_dequantize(q0[0], q0[1], inn)))
+    Wq, Qq, B = L.loqt_compensated_init_right(Wd, Qd, 3)
+    c, m = from_dev_nf4(Wq)
+    assert np.array_equal(c, q0[0]) and np.array_equal(m, q0[1]) and not f32(B).any()
