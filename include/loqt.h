@@ -176,7 +176,10 @@ loqt_status loqt_merge_requant_split(loqt_nf4_mat Wq, loqt_nf4_mat Pq, const voi
  *   merge     W_q <- q_NF4( deq(W_q) + s B deq(Q_q) )   in place
  * Arguments, precisions and error behaviour as for loqt_linear_fwd / _bwd /
  * loqt_merge_requant; workspaces from loqt_workspace_bytes(LOQT_OP_FWD_RIGHT /
- * LOQT_OP_BWD_RIGHT / LOQT_OP_MERGE_RIGHT, out, in, r, T).
+ * LOQT_OP_BWD_RIGHT / LOQT_OP_MERGE_RIGHT, out, in, r, T).  Forward and backward
+ * each keep, in their workspace, a bf16 copy of deq(Q_q) that they write once per
+ * call for the product x deq(Q_q)^T (the operand is the same rounding of the same
+ * values as the in-product dequantisation gives).
  */
 loqt_status loqt_linear_fwd_right(loqt_nf4_mat Wq, loqt_nf4_mat Qq, const void *B, int64_t ldb, float s,
                                   const void *x, int64_t ldx, int32_t T, void *y, int64_t ldy,

@@ -333,9 +333,11 @@ extern "C" size_t loqt_workspace_bytes(int op, int32_t out, int32_t in, int32_t 
   }
   // right-side variant: u (T x r) in forward; u, v (T x r) and the split-K partials of dB (out x r) in backward;
   // deq(Q_q) as bf16 (r x roundup(in, 64)) in the merge
-  if (op == LOQT_OP_FWD_RIGHT) total += align256(static_cast<size_t>(T > 0 ? T : 0) * ld_lowrank(r) * 2);
+  // (forward and backward also stage deq(Q_q) as bf16 for the product u = x Q-hat^T, which has N = r only)
+  const size_t qhat_bytes = align256(static_cast<size_t>(r > 0 ? r : 0) * ((static_cast<size_t>(in > 0 ? in : 0) + 63) / 64 * 64) * 2);
+  if (op == LOQT_OP_FWD_RIGHT) total += align256(static_cast<size_t>(T > 0 ? T : 0) * ld_lowrank(r) * 2) + qhat_bytes;
   if (op == LOQT_OP_BWD_RIGHT) {
-    total += 2 * align256(static_cast<size_t>(T > 0 ? T : 0) * ld_lowrank(r) * 2);
+    total += 2 * align256(static_cast<size_t>(T > 0 ? T : 0) * ld_lowrank(r) * 2) + qhat_bytes;
     int splits = 1, kbps = 1;
     db_splits(out, r, T > 0 ? T : 1, splits, kbps);
     if (splits > 1) total += align256(static_cast<size_t>(splits) * out * ((static_cast<size_t>(r) + 3) / 4 * 4) * 4);
@@ -719,13 +721,18 @@ static loqt_status check_layer_right(const loqt_nf4_mat &Wq, const loqt_nf4_mat 
   return check_bf16(B, ldb, Qq.rows);
 }
 
-// u = s * x deq(Q_q)^T   (T x r; K = in, Q_q blocks along K)
+// u = s * x deq(Q_q)^T   (T x r; K = in).  As for v in the left-side backward: with N = r only,
+// dequantising Q_q inside the product would repeat it for every 256 token rows, so the factor
+// is dequantised once into `qhat` (bf16 r x Qq.ld) and the product is a plain bf16 one.
 static loqt_status right_u(const loqt_nf4_mat &Qq, float s, const void *x, int64_t ldx, int T, void *u, int64_t ldu,
-                           uint32_t *status, cudaStream_t stm) {
+                           void *qhat, uint32_t *status, cudaStream_t stm) {
+  const StageItem stage{Qq, qhat, Qq.ld};
+  loqt_status st = nf4_dequantize_bf16_batch(&stage, 1, stm);
+  if (st != LOQT_OK) return st;
   GemmCall c{};
   c.p.M = T; c.p.N = Qq.rows; c.p.num_segs = 1;
-  c.p.seg[0].K = Qq.cols; c.p.seg[0].a_kind = OP_TMA_K; c.p.seg[0].b_kind = OP_NF4_K; c.p.seg[0].b_nf4 = nf4_src(Qq);
-  c.a[0] = {x, ldx};
+  c.p.seg[0].K = Qq.cols; c.p.seg[0].a_kind = OP_TMA_K; c.p.seg[0].b_kind = OP_TMA_K;
+  c.a[0] = {x, ldx}; c.b[0] = {qhat, Qq.ld};
   c.p.splits = 1;
   c.p.epi = EPI_BF16; c.p.out = u; c.p.ld_out = ldu; c.p.alpha = s; c.p.status = status;
   return launch(c, stm);
@@ -746,7 +753,8 @@ extern "C" loqt_status loqt_linear_fwd_right(loqt_nf4_mat Wq, loqt_nf4_mat Qq, c
   uint32_t *status = static_cast<uint32_t *>(ws);
   void *u = static_cast<uint8_t *>(ws) + 256;
   const int64_t ldu = ld_lowrank(r);
-  if ((st = right_u(Qq, s, x, ldx, T, u, ldu, status, stm)) != LOQT_OK) return st;
+  void *qhat = static_cast<uint8_t *>(u) + align256(static_cast<size_t>(T) * ldu * 2);
+  if ((st = right_u(Qq, s, x, ldx, T, u, ldu, qhat, status, stm)) != LOQT_OK) return st;
   // y = x deq(W_q)^T + u B^T    (K = in, then K = r; B is K-major over r)
   GemmCall c{};
   c.p.M = T; c.p.N = out; c.p.num_segs = 2;
@@ -779,10 +787,11 @@ extern "C" loqt_status loqt_linear_bwd_right(loqt_nf4_mat Wq, loqt_nf4_mat Qq, c
   const size_t tr_bytes = align256(static_cast<size_t>(T) * ldt * 2);
   void *u = static_cast<uint8_t *>(ws) + 256;
   void *v = static_cast<uint8_t *>(u) + tr_bytes;
-  float *partial = reinterpret_cast<float *>(static_cast<uint8_t *>(v) + tr_bytes);
+  void *qhat = static_cast<uint8_t *>(v) + tr_bytes;
+  float *partial = reinterpret_cast<float *>(static_cast<uint8_t *>(qhat) + align256(static_cast<size_t>(r) * Qq.ld * 2));
 
   // u = s * x deq(Q_q)^T, recomputed (the forward's copy is not kept)
-  if ((st = right_u(Qq, s, x, ldx, T, u, ldt, status, stm)) != LOQT_OK) return st;
+  if ((st = right_u(Qq, s, x, ldx, T, u, ldt, qhat, status, stm)) != LOQT_OK) return st;
   if (dx != nullptr) {
     // v = s * dy B             (T x r; K = out; B stored [K][N])
     GemmCall c1{};
