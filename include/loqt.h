@@ -6,7 +6,7 @@
  *     W_eff = deq(W_q) + s * deq(P_q) * B            (out x in)
  *
  * with W_q (out x in) and P_q (out x r) frozen and stored in NF4 (Section 5.1:
- * blocks of 64 weights, one fp32 scale M = max|w| per block, 16 levels), B
+ * 64-weight blocks, each with one fp32 scale M = max|w| per block, 16 levels), B
  * (r x in) the only trained matrix, kept in bf16, and s the adapter scale of
  * Algorithm 1's merge line.
  *
