@@ -107,7 +107,9 @@ struct TensorMaps {
 // variant without spends that shared memory on a deeper operand ring.
 // REQ: the merge kernel (requantising epilogue): two buffers hold the packed codes
 // of the output tiles' W_q blocks on their way from and to global memory.
-template <int BN, int MH, bool TWO, bool NF4, bool REQ = false>
+// EXTRA: bytes of further staging after the code buffers (the compensation step's
+// fp32 weights on their way to the epilogue warps, two mbarriers per warp with them).
+template <int BN, int MH, bool TWO, bool NF4, bool REQ = false, int EXTRA = 0>
 struct SmemLayout {
   static constexpr int kBM = MH * kHM;
   static constexpr int kBNL = TWO ? BN / 2 : BN;  // B rows staged by this CTA
@@ -124,15 +126,16 @@ struct SmemLayout {
   static constexpr int kWTileBytes = REQ ? kHM * (BN / 2) : 0;  // codes of 128 rows x BN columns of W_q
   static constexpr int kWBufs = REQ ? 2 : 0;
   static constexpr int stages_for(int s) {
-    return s * kStageBytes + (NF4 ? (s > 4 ? s : 4) * kCodeBytes : 0) + kWBufs * kWTileBytes <= 225 * 1024;
+    return s * kStageBytes + (NF4 ? (s > 4 ? s : 4) * kCodeBytes : 0) + kWBufs * kWTileBytes + EXTRA <= 225 * 1024;
   }
   static constexpr int kStages = (!NF4 && stages_for(7)) ? 7 : stages_for(6) ? 6 : stages_for(5) ? 5 : stages_for(4) ? 4 : stages_for(3) ? 3 : 2;
   static constexpr int kCodeStages = !NF4 ? 0 : (kStages > 4 ? kStages : 4);
   static constexpr int kCodeOffset = kStages * kStageBytes;
   static constexpr int kWOffset = kCodeOffset + kCodeStages * kCodeBytes;  // (a multiple of 1024)
-  static constexpr int kBarOffset = kWOffset + kWBufs * kWTileBytes;
-  // full[S], empty[S], cfull[C], cempty[C], tfull[2], tempty[2], drain, wfull[2], wdone[2]
-  static constexpr int kNumBars = 2 * kStages + 2 * kCodeStages + 5 + 2 * kWBufs;
+  static constexpr int kExtraOffset = kWOffset + kWBufs * kWTileBytes;  // (a multiple of 1024)
+  static constexpr int kBarOffset = kExtraOffset + EXTRA;
+  // full[S], empty[S], cfull[C], cempty[C], tfull[2], tempty[2], drain, wfull[2], wdone[2], extra[24]
+  static constexpr int kNumBars = 2 * kStages + 2 * kCodeStages + 5 + 2 * kWBufs + (EXTRA > 0 ? 24 : 0);
   static constexpr int kMiscOffset = kBarOffset + kNumBars * 8;
   static constexpr int kTablesOffset = kMiscOffset + 16;
   static constexpr int kTotal = kTablesOffset + static_cast<int>(sizeof(Nf4Tables));
@@ -143,6 +146,7 @@ struct SmemLayout {
   static_assert(kBM * 32 <= kCodeBytes && kBNL * 32 <= kCodeBytes, "code tile too large");
   static_assert(!TWO || BN == 256, "pairs run 256-wide tiles");
   static_assert(!REQ || (MH == 1 && !TWO && !NF4), "the merge runs single 128-row tiles fed by TMA");
+  static_assert(EXTRA % 1024 == 0, "the extra staging keeps the 1024-byte alignment of what follows");
 };
 
 // Shared-memory matrix descriptor (tcgen05), 128-byte swizzle.

@@ -576,11 +576,34 @@ struct MergeItem {
   int64_t ld_resid = 0;
 };
 
+// fp32 matrix [rows][ld] as a tensor map; box in elements x rows, 128-byte swizzle.
+static bool make_f32_map(CUtensorMap *map, const float *base, int64_t cols, int64_t rows, int64_t ld, int box_cols,
+                         int box_rows) {
+  EncodeTiledFn fn = encode_fn();
+  if (fn == nullptr) return false;
+  const cuuint64_t dims[2] = {static_cast<cuuint64_t>(cols), static_cast<cuuint64_t>(rows)};
+  const cuuint64_t strides[1] = {static_cast<cuuint64_t>(ld) * 4};
+  const cuuint32_t box[2] = {static_cast<cuuint32_t>(box_cols), static_cast<cuuint32_t>(box_rows)};
+  const cuuint32_t estr[2] = {1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<float *>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 template <int BN, bool COMP = false>
 static loqt_status launch_merge(const MergeItem *items, int n, uint32_t *status, cudaStream_t stream) {
-  using L = SmemLayout<BN, 1, false, false, true>;
+  using L = MergeLayout<BN, COMP>;
   MergeBatch mb;
   memset(&mb, 0, sizeof(mb));
+  if (COMP) {
+    // one matrix per launch; W by TMA (16-byte aligned rows), the residual by 16-byte stores
+    // that may run into the padding of its rows
+    const MergeItem &it = items[0];
+    if (n != 1 || (reinterpret_cast<uintptr_t>(it.w32) & 15u) != 0 || (it.ld_w32 & 3) != 0 ||
+        (reinterpret_cast<uintptr_t>(it.resid) & 15u) != 0 || (it.ld_resid & 7) != 0 || it.ld_resid < it.Wq.ld)
+      return LOQT_ERR_INVALID_ARG;
+    if (!make_f32_map(&mb.wmap, it.w32, it.Wq.cols, it.Wq.rows, it.ld_w32, 32, 32)) return LOQT_ERR_CUDA;
+  }
   int tiles = 0;
   for (int i = 0; i < n; ++i) {
     const MergeItem &it = items[i];

@@ -46,6 +46,7 @@ struct MergeBatch {
   CUtensorMap b[kMergeBatchMax];   // B, bf16 [K][N]: box 64 (N) x 64 (K), an MN-major operand
   CUtensorMap wq[kMergeBatchMax];  // packed codes of W_q as bytes [M][wq_ld / 2]: box BN / 2 x 128 rows
   MergeProblem prob[kMergeBatchMax];
+  CUtensorMap wmap;  // compensation mode (one matrix per launch): W, fp32 [M][ld_w32]: box 32 columns x 32 rows
   int count;
   int tiles;  // of all matrices together
   uint32_t *status;
@@ -58,10 +59,14 @@ struct MergeBatch {
 // the codes and scales of Q are written (nothing of W_q is read), and with them
 // the bf16 residual W - deq32(Q) that the next product P^T (W - Q) consumes.  The
 // corrected weights W - P B never exist in memory.
+constexpr int kCompStageBytes = 32 * 128;  // per epilogue warp: 32 rows x 32 fp32 columns of W
+template <int BN, bool kComp>
+using MergeLayout = SmemLayout<BN, 1, false, false, true, kComp ? 12 * kCompStageBytes : 0>;
+
 template <int BN, bool kComp = false>
 __global__ void __launch_bounds__(kNumThreads, 1)
 loqt_merge_kernel(const __grid_constant__ MergeBatch mb) {
-  using L = SmemLayout<BN, 1, false, false, true>;
+  using L = MergeLayout<BN, kComp>;
   constexpr int kStages = L::kStages;
   constexpr int kEpiGroups = 3;
   extern __shared__ uint8_t smem_raw[];
@@ -76,6 +81,9 @@ loqt_merge_kernel(const __grid_constant__ MergeBatch mb) {
   const uint32_t drain_bar = bar0 + 8u * (2 * kStages + 4);
   auto wfull_bar = [&](int b) { return bar0 + 8u * (2 * kStages + 5 + b); };
   auto wdone_bar = [&](int b) { return bar0 + 8u * (2 * kStages + 7 + b); };
+  // compensation mode, per epilogue warp: staging tile filled / staging tile read by every lane
+  auto stage_bar = [&](int w) { return bar0 + 8u * (2 * kStages + 9 + w); };
+  auto free_bar = [&](int w) { return bar0 + 8u * (2 * kStages + 21 + w); };
   volatile uint32_t *misc = reinterpret_cast<volatile uint32_t *>(smem_gen + L::kMiscOffset);
   volatile uint32_t *tmem_slot = misc;
   volatile uint32_t *abort_flag = misc + 1;
@@ -97,6 +105,11 @@ loqt_merge_kernel(const __grid_constant__ MergeBatch mb) {
       ptx::mbar_init(wdone_bar(a), 4 * kEpiGroups);  // every epilogue warp, once per tile
     }
     ptx::mbar_init(drain_bar, 1);
+    if (kComp)
+      for (int w = 0; w < 4 * kEpiGroups; ++w) {
+        ptx::mbar_init(stage_bar(w), 1);
+        ptx::mbar_init(free_bar(w), 32);
+      }
     *abort_flag = 0;
     ptx::fence_barrier_init();
   }
@@ -232,6 +245,175 @@ loqt_merge_kernel(const __grid_constant__ MergeBatch mb) {
       ptx::bulk_wait_group<0>();
     }
   }
+  // =========================================================== epilogue of the compensation step
+  else if (kComp) {
+    // One matrix per launch.  A thread's 64 weights W reach it through shared
+    // memory: each warp owns a 32-row x 32-column fp32 staging tile that its lane 0
+    // fills by TMA, half a block at a time (the second half while the first is
+    // in use, the next block's first half while this block is quantised), so no
+    // thread reads a 256-byte row segment of its own from global memory.  The
+    // block is walked twice - once for its maximum, once for codes and residual -
+    // and the accumulator is read from TMEM both times rather than kept: W, which
+    // the residual needs, stays in registers instead.
+    constexpr int NB = BN / 64;
+    const MergeProblem &pr = mb.prob[0];
+    const int q = warp & 3;
+    const int ew = warp - kEpiWarp0;
+    const int grp = ew >> 2;
+    const uint32_t wbuf = smem_base + L::kExtraOffset + static_cast<uint32_t>(ew) * kCompStageBytes;
+    const uint32_t wbar = stage_bar(ew), fbar = free_bar(ew);
+    const uint32_t w_lane = wbuf + static_cast<uint32_t>(lane) * 128u;
+    const uint32_t key = static_cast<uint32_t>(lane & 7);  // 128-byte swizzle: 16-byte chunk ^= row & 7
+    const float alpha = pr.alpha;
+    const float2 a2 = make_float2(alpha, alpha);
+    uint32_t loads = 0;  // staging loads waited for so far
+    bool ok = true;
+    // the outcome of a wait, made the same for all lanes (the warp-wide TMEM loads and
+    // barriers below need the warp whole)
+    auto wait = [&](uint32_t bar, uint32_t parity) {
+      return __all_sync(0xffffffffu, ptx::mbar_wait(bar, parity, abort_flag, mb.status)) != 0;
+    };
+    // half `half` of block `seq` of this CTA's sequence of blocks (tile seq / NB, block seq % NB)
+    auto fetch = [&](uint32_t seq, int half) {
+      if (lane != 0) return;
+      const int g = blockIdx.x + static_cast<int>(seq / NB) * static_cast<int>(gridDim.x);
+      if (g >= mb.tiles) return;
+      const int n_blk = g / pr.mt, m_blk = g - n_blk * pr.mt;
+      ptx::mbar_arrive_expect_tx(wbar, kCompStageBytes);
+      ptx::tma_load_2d(wbuf, &mb.wmap, wbar, n_blk * BN + static_cast<int>(seq % NB) * 64 + 32 * half,
+                       m_blk * kHM + q * 32);
+    };
+    auto take = [&](float2 *w) {  // 32 weights of this lane's row out of the staging tile
+#pragma unroll
+      for (uint32_t j = 0; j < 8; ++j) {
+        const uint4 t = ld_shared_v4(w_lane + ((j ^ key) << 4));
+        w[2 * j] = make_float2(__uint_as_float(t.x), __uint_as_float(t.y));
+        w[2 * j + 1] = make_float2(__uint_as_float(t.z), __uint_as_float(t.w));
+      }
+    };
+    {
+      uint32_t first = static_cast<uint32_t>(grp);
+      fetch(first, 0);
+    }
+    uint32_t tile = 0;
+    for (int g = blockIdx.x; ok && g < mb.tiles; g += gridDim.x, ++tile) {
+      const int n_blk = g / pr.mt, m_blk = g - n_blk * pr.mt;
+      const uint32_t acc = tile & 1u;
+      const uint32_t ph = (tile >> 1) & 1u;
+      if (!(ok = wait(tfull_bar(acc), ph))) break;
+      // the mover's signal that the store which last read this code buffer is done with it
+      if (!(ok = wait(wfull_bar(acc), ph))) break;
+      ptx::tc_fence_after();
+      const int row_t = q * 32 + lane;
+      const int row = m_blk * kHM + row_t;
+      const bool row_ok = row < pr.M;
+      const uint32_t t_row = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + acc * BN;
+      const uint32_t w_row = smem_base + L::kWOffset + acc * L::kWTileBytes + static_cast<uint32_t>(row_t) * (BN / 2);
+      const uint32_t w_key = (BN == 256) ? static_cast<uint32_t>(row_t & 7) : static_cast<uint32_t>((row_t >> 1) & 3);
+#pragma unroll 1
+      for (int jb = 0; jb < NB; ++jb) {
+        const uint32_t seq = tile * NB + jb;
+        if (static_cast<int>(seq % kEpiGroups) != grp) continue;
+        const int c0 = n_blk * BN + jb * 64;
+        const bool live = row_ok && c0 < pr.wq_ld;
+        const uint32_t a0 = w_row + (((2u * jb) ^ w_key) << 4), a1 = w_row + (((2u * jb + 1u) ^ w_key) << 4);
+        float2 W[32];
+        uint32_t d[32];
+        float mx[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+        // ---- first walk: the block maximum of W + alpha * delta
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+          if (!(ok = wait(wbar, loads & 1u))) break;
+          ++loads;
+          take(W + 16 * h);
+          // Every lane has its copy before the staging tile is filled again: the lanes' reads
+          // are ordered before their arrivals, the next copy is issued after the wait for them
+          // (program order alone does not keep a shared-memory read ahead of a bulk copy).
+          ptx::mbar_arrive(fbar);
+          if (lane == 0) ok = ptx::mbar_wait(fbar, (loads - 1u) & 1u, abort_flag, mb.status);
+          if (!(ok = __all_sync(0xffffffffu, ok) != 0)) break;
+          if (h == 0) fetch(seq, 1);
+          else fetch(seq + kEpiGroups, 0);
+          ptx::tmem_ld32(t_row + jb * 64 + 32 * h, d);
+          ptx::tmem_ld_wait();
+#pragma unroll
+          for (int e = 0; e < 16; ++e) {
+            const float2 v = __ffma2_rn(a2, make_float2(__uint_as_float(d[2 * e]), __uint_as_float(d[2 * e + 1])), W[16 * h + e]);
+            mx[e & 3] = fmaxf(mx[e & 3], fmaxf(fabsf(v.x), fabsf(v.y)));
+          }
+        }
+        if (!ok) break;
+        const float Mnew = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
+        const Nf4Divisor dv = nf4_divisor(Mnew);
+        uint32_t o[8];
+        __nv_bfloat16 *rp = pr.resid + static_cast<int64_t>(row) * pr.ld_resid + c0;
+        // ---- second walk: codes, and the residual bf16( W - fl32(Mnew * q[code]) ) with the
+        // two fp32 roundings of its definition (scalar intrinsics: a packed multiply and add
+        // may be contracted into one fused operation)
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+          ptx::tmem_ld32(t_row + jb * 64 + 32 * h, d);
+          ptx::tmem_ld_wait();
+          if (live) {
+            auto quantise_half = [&](auto exact) {
+#pragma unroll
+              for (int g8 = 0; g8 < 4; ++g8) {
+                uint32_t word = 0;
+#pragma unroll
+                for (int h2 = 0; h2 < 4; ++h2) {
+                  const int e = 4 * g8 + h2;
+                  const float2 v = __ffma2_rn(a2, make_float2(__uint_as_float(d[2 * e]), __uint_as_float(d[2 * e + 1])), W[16 * h + e]);
+                  word |= nf4_code2(tables, nf4_normalise2<decltype(exact)::value>(dv, v)) << (8 * h2);
+                }
+                o[4 * h + g8] = word;
+              }
+            };
+            if (!(Mnew > 0.0f)) {
+#pragma unroll
+              for (int g8 = 0; g8 < 4; ++g8) o[4 * h + g8] = kZeroWord;
+            } else if (dv.exact) {
+              quantise_half(std::true_type{});
+            } else {
+              quantise_half(std::false_type{});
+            }
+#pragma unroll
+            for (int g8 = 0; g8 < 4; ++g8) {
+              uint32_t pk[4];
+#pragma unroll
+              for (int h2 = 0; h2 < 4; ++h2) {
+                const uint32_t byte = (o[4 * h + g8] >> (8 * h2)) & 0xFFu;
+                const float2 w = W[16 * h + 4 * g8 + h2];
+                const float e_lo = __fsub_rn(w.x, __fmul_rn(Mnew, tables.level[byte & 15u]));
+                const float e_hi = __fsub_rn(w.y, __fmul_rn(Mnew, tables.level[byte >> 4]));
+                pk[h2] = pack_bf16x2(e_lo, e_hi);
+              }
+              reinterpret_cast<uint4 *>(rp)[4 * h + g8] = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+            }
+          }
+        }
+        if (live) {
+          st_shared_v4(a0, make_uint4(o[0], o[1], o[2], o[3]));
+          st_shared_v4(a1, make_uint4(o[4], o[5], o[6], o[7]));
+          pr.wq_absmax[static_cast<int64_t>(row) * (pr.wq_ld >> 6) + (c0 >> 6)] = Mnew;
+        }
+        __syncwarp();
+      }
+      if (!ok) break;
+      ptx::fence_proxy_async_smem();
+      ptx::tc_fence_before();
+      __syncwarp();
+      if (lane == 0) {
+        ptx::mbar_arrive(wdone_bar(acc));
+        ptx::mbar_arrive(tempty_bar(acc));
+      }
+    }
+    if (!ok && lane == 0) {
+      // a staging load may still be in flight: give it time to land before the shared memory is released
+      const uint64_t t0 = ptx::globaltimer_ns();
+      while (ptx::globaltimer_ns() - t0 < 200000ull) {
+      }
+    }
+  }
   // =========================================================== epilogue
   else {
     const int q = warp & 3;                   // TMEM lane quarter this warp may access
@@ -256,7 +438,7 @@ loqt_merge_kernel(const __grid_constant__ MergeBatch mb) {
         for (int jb = 0; jb < BN / 64; ++jb) {
           const int c0 = n_blk * BN + jb * 64;
           const bool mine = static_cast<int>((tile * (BN / 64) + jb) % kEpiGroups) == grp;
-          m_pre[jb] = (!kComp && mine && row_p < pr.M && c0 < pr.wq_ld)
+          m_pre[jb] = (mine && row_p < pr.M && c0 < pr.wq_ld)
                           ? pr.wq_absmax[static_cast<int64_t>(row_p) * (pr.wq_ld >> 6) + (c0 >> 6)]
                           : 0.0f;
         }
@@ -283,41 +465,19 @@ loqt_merge_kernel(const __grid_constant__ MergeBatch mb) {
         const uint32_t a0 = w_row + (((2u * jb) ^ w_key) << 4), a1 = w_row + (((2u * jb + 1u) ^ w_key) << 4);
         float Mold = 0.0f;
         uint4 ca = make_uint4(0, 0, 0, 0), cb = ca;
-        // compensation mode: this thread's 64 weights, read straight from global memory
-        // (256 contiguous bytes per thread; elements beyond the matrix read as zero)
-        float2 v[32], wk[32];
-        const float *wp = nullptr;
-        bool wide = false;
-        if (kComp) {
-          wp = pr.w32 + static_cast<int64_t>(row) * pr.ld_w32 + c0;
-          wide = live && c0 + 64 <= pr.N && (pr.ld_w32 & 3) == 0 && (reinterpret_cast<uintptr_t>(pr.w32) & 15u) == 0;
-          if (wide) {
+        float2 v[32];
 #pragma unroll
-            for (int e = 0; e < 16; ++e) {
-              const float4 t = __ldg(reinterpret_cast<const float4 *>(wp) + e);
-              v[2 * e] = make_float2(t.x, t.y);
-              v[2 * e + 1] = make_float2(t.z, t.w);
-            }
-          } else {
-#pragma unroll
-            for (int e = 0; e < 32; ++e)
-              v[e] = make_float2((live && c0 + 2 * e < pr.N) ? __ldg(wp + 2 * e) : 0.0f,
-                                 (live && c0 + 2 * e + 1 < pr.N) ? __ldg(wp + 2 * e + 1) : 0.0f);
-          }
-        } else {
-#pragma unroll
-          for (int k = 0; k < BN / 64; ++k)
-            if (k == jb) Mold = m_pre[k];
-          ca = ld_shared_v4(a0);
-          cb = ld_shared_v4(a1);
-        }
+        for (int k = 0; k < BN / 64; ++k)
+          if (k == jb) Mold = m_pre[k];
+        ca = ld_shared_v4(a0);
+        cb = ld_shared_v4(a1);
         uint32_t d0[32], d1[32];
         ptx::tmem_ld32(t_row + jb * 64, d0);
         ptx::tmem_ld32(t_row + jb * 64 + 32, d1);
         ptx::tmem_ld_wait();
         if (live) {
           const uint32_t w[8] = {ca.x, ca.y, ca.z, ca.w, cb.x, cb.y, cb.z, cb.w};
-          // v = deq32(old) + alpha * delta (compensation: W + alpha * delta), two elements
+          // v = deq32(old) + alpha * delta, two elements
           // per packed instruction; four running maxima keep the dependent chain of the
           // block maximum short
           float mx[4] = {0.0f, 0.0f, 0.0f, 0.0f};
@@ -326,15 +486,10 @@ loqt_merge_kernel(const __grid_constant__ MergeBatch mb) {
           for (int e = 0; e < 32; ++e) {
             const float2 delta = make_float2(__uint_as_float(e < 16 ? d0[2 * e] : d1[2 * e - 32]),
                                              __uint_as_float(e < 16 ? d0[2 * e + 1] : d1[2 * e - 31]));
-            if (kComp) {
-              wk[e] = v[e];  // W itself, for the residual
-              v[e] = __ffma2_rn(a2, delta, v[e]);
-            } else {
-              const uint32_t word = w[e >> 2];
-              const float2 lv = make_float2(tables.level[(word >> (8 * (e & 3))) & 15u],
-                                            tables.level[(word >> (8 * (e & 3) + 4)) & 15u]);
-              v[e] = __ffma2_rn(a2, delta, __fmul2_rn(m2, lv));
-            }
+            const uint32_t word = w[e >> 2];
+            const float2 lv = make_float2(tables.level[(word >> (8 * (e & 3))) & 15u],
+                                          tables.level[(word >> (8 * (e & 3) + 4)) & 15u]);
+            v[e] = __ffma2_rn(a2, delta, __fmul2_rn(m2, lv));
             mx[e & 3] = fmaxf(mx[e & 3], fmaxf(fabsf(v[e].x), fabsf(v[e].y)));
           }
           const float Mnew = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
@@ -361,36 +516,6 @@ loqt_merge_kernel(const __grid_constant__ MergeBatch mb) {
           st_shared_v4(a0, make_uint4(o[0], o[1], o[2], o[3]));
           st_shared_v4(a1, make_uint4(o[4], o[5], o[6], o[7]));
           *mp = Mnew;
-          if (kComp) {
-            // residual = bf16( W - fl32(Mnew * q[code]) ): two fp32 roundings, as the definition
-            // has them; W comes from the copy kept above (reading it again from global memory,
-            // one row segment per thread, costs more load/store-unit time than the spills do)
-            __nv_bfloat16 *rp = pr.resid + static_cast<int64_t>(row) * pr.ld_resid + c0;
-            const bool wide_out = wide && (pr.ld_resid & 7) == 0 && (reinterpret_cast<uintptr_t>(pr.resid) & 15u) == 0;
-#pragma unroll
-            for (int g8 = 0; g8 < 8; ++g8) {
-              const float2 wv[4] = {wk[4 * g8], wk[4 * g8 + 1], wk[4 * g8 + 2], wk[4 * g8 + 3]};
-              uint32_t pk[4];
-#pragma unroll
-              for (int h2 = 0; h2 < 4; ++h2) {
-                const uint32_t byte = (o[g8] >> (8 * h2)) & 0xFFu;
-                // scalar intrinsics: the packed multiply and add may be contracted into one fused operation
-                const float e_lo = __fsub_rn(wv[h2].x, __fmul_rn(Mnew, tables.level[byte & 15u]));
-                const float e_hi = __fsub_rn(wv[h2].y, __fmul_rn(Mnew, tables.level[byte >> 4]));
-                pk[h2] = pack_bf16x2(e_lo, e_hi);
-              }
-              if (wide_out) {
-                reinterpret_cast<uint4 *>(rp)[g8] = make_uint4(pk[0], pk[1], pk[2], pk[3]);
-              } else {
-#pragma unroll
-                for (int h2 = 0; h2 < 4; ++h2) {
-                  const int c = 8 * g8 + 2 * h2;
-                  if (c0 + c < pr.N) rp[c] = __ushort_as_bfloat16(static_cast<unsigned short>(pk[h2] & 0xFFFFu));
-                  if (c0 + c + 1 < pr.N) rp[c + 1] = __ushort_as_bfloat16(static_cast<unsigned short>(pk[h2] >> 16));
-                }
-              }
-            }
-          }
         }
         __syncwarp();
       }
