@@ -358,14 +358,15 @@ loqt_merge_kernel(const __grid_constant__ MergeBatch mb) {
             auto quantise_half = [&](auto exact) {
 #pragma unroll
               for (int g8 = 0; g8 < 4; ++g8) {
-                uint32_t word = 0;
-#pragma unroll
-                for (int h2 = 0; h2 < 4; ++h2) {
-                  const int e = 4 * g8 + h2;
+                auto code = [&](auto h2) {  // byte h2 of the word: columns 8 g8 + 2 h2, + 1 of this half
+                  constexpr int kH2 = decltype(h2)::value;
+                  const int e = 4 * g8 + kH2;
                   const float2 v = __ffma2_rn(a2, make_float2(__uint_as_float(d[2 * e]), __uint_as_float(d[2 * e + 1])), W[16 * h + e]);
-                  word |= nf4_code2(tables, nf4_normalise2<decltype(exact)::value>(dv, v)) << (8 * h2);
-                }
-                o[4 * h + g8] = word;
+                  return nf4_code2<kH2>(tables, nf4_normalise2<decltype(exact)::value>(dv, v));
+                };
+                using std::integral_constant;
+                o[4 * h + g8] = code(integral_constant<int, 0>{}) | code(integral_constant<int, 1>{}) |
+                                code(integral_constant<int, 2>{}) | code(integral_constant<int, 3>{});
               }
             };
             if (!(Mnew > 0.0f)) {
@@ -498,11 +499,11 @@ loqt_merge_kernel(const __grid_constant__ MergeBatch mb) {
           auto quantise_block = [&](auto exact) {
 #pragma unroll
             for (int g8 = 0; g8 < 8; ++g8) {
-              uint32_t word = 0;
-#pragma unroll
-              for (int h2 = 0; h2 < 4; ++h2)
-                word |= nf4_code2(tables, nf4_normalise2<decltype(exact)::value>(dv, v[4 * g8 + h2])) << (8 * h2);
-              o[g8] = word;
+              constexpr bool kE = decltype(exact)::value;
+              o[g8] = nf4_code2<0>(tables, nf4_normalise2<kE>(dv, v[4 * g8])) |
+                      nf4_code2<1>(tables, nf4_normalise2<kE>(dv, v[4 * g8 + 1])) |
+                      nf4_code2<2>(tables, nf4_normalise2<kE>(dv, v[4 * g8 + 2])) |
+                      nf4_code2<3>(tables, nf4_normalise2<kE>(dv, v[4 * g8 + 3]));
             }
           };
           if (!(Mnew > 0.0f)) {
