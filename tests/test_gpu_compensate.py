@@ -13,9 +13,10 @@ pytestmark = pytest.mark.gpu
 
 # (out, in, r): several tiles with ragged edges; 5461 is the paper's 1B MLP width; then
 # tiny and ragged cases: fewer rows than the 32 of an epilogue warp, a width below one
-# staging tile, widths that end inside the first and inside the second half of a block
+# staging tile, widths that end inside the first and inside the second half of a block;
+# last, more tiles than the GPU has SMs, so that a CTA walks several tiles (272 of 128 x 256)
 SHAPES = [(256, 256, 32), (384, 320, 64), (200, 136, 24), (640, 5461, 96), (1376, 512, 128),
-          (24, 40, 8), (72, 24, 16), (136, 100, 8), (520, 1065, 40)]
+          (24, 40, 8), (72, 24, 16), (136, 100, 8), (520, 1065, 40), (2176, 4000, 192)]
 
 
 def _inputs(seed, out, inn, r):
