@@ -118,7 +118,7 @@ def test_argument_errors():
 
 
 # ---- right-side variant: W ~ Q_w + B Q, Q r x in with orthonormal rows
-RIGHT_SHAPES = [(256, 256, 32), (1376, 512, 96), (5461, 256, 40), (320, 640, 64)]
+RIGHT_SHAPES = [(256, 256, 32), (1376, 512, 96), (5461, 256, 40), (320, 640, 64), (4000, 2176, 192)]  # the last: 288 tiles
 
 
 def _inputs_right(seed, out, inn, r):
