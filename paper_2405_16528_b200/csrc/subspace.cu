@@ -225,47 +225,72 @@ chol_panel_kernel(double *__restrict__ S, int rp, int p, double *__restrict__ X,
   // j < k, and once the band of a slot is behind the current column the slot is skipped by
   // all threads at once - on average four of the nine slots are live.
   constexpr int kSlots = 9, kLower = kT * (kT + 1) / 2;
-  auto column_of = [](int idx, int &i, int &k) {  // idx -> (row, column) in column-major packed order
-    int c = 0, first = 0;                         // first = number of the column's top element
-    while (first + (kT - c) <= idx) first += kT - c, ++c;
-    k = c;
-    i = c + (idx - first);
-  };
   double val[kSlots];
   int ei[kSlots], ek[kSlots], last_col[kSlots];
+  {
+    // idx -> (row, column) in column-major packed order; a thread's slots and the slots' last
+    // elements come in ascending order, so each of the two scans passes over the columns once
+    int c = 0, first = 0;    // column of the thread's current slot, number of its top element
+    int lc = 0, lfirst = 0;  // the same for the last element of the slot (equal in every thread)
 #pragma unroll
-  for (int q = 0; q < kSlots; ++q) {
-    const int idx = tid + 256 * q;
-    int i = 0, k = 0;
-    if (idx < kLower) column_of(idx, i, k);
-    ei[q] = i;
-    ek[q] = idx < kLower ? k : -1;  // -1: empty slot
-    val[q] = idx < kLower ? S[(d0 + i) * rp + d0 + k] : 0.0;
-    if (ek[q] == 0) col[0][i] = val[q];
-    int li, lk;
-    column_of(min(256 * q + 255, kLower - 1), li, lk);  // the same for every thread
-    last_col[q] = lk;
+    for (int q = 0; q < kSlots; ++q) {
+      const int idx = tid + 256 * q;
+      const bool have = idx < kLower;
+      while (have && first + (kT - c) <= idx) first += kT - c, ++c;
+      ei[q] = have ? c + (idx - first) : 0;
+      ek[q] = have ? c : -1;  // -1: empty slot
+      val[q] = have ? S[(d0 + ei[q]) * rp + d0 + c] : 0.0;
+      if (ek[q] == 0) col[0][ei[q]] = val[q];
+      const int lidx = min(256 * q + 255, kLower - 1);
+      while (lfirst + (kT - lc) <= lidx) lfirst += kT - lc, ++lc;
+      last_col[q] = lc;
+    }
   }
   __syncthreads();
-  for (int j = 0; j < kT; ++j) {
+  // Step j with slots kFirst .. 8 live.  Nothing in it branches on a thread's own elements:
+  // both factors of every live slot are read, the products and the fused updates follow as
+  // independent chains, and a slot outside the trailing block keeps its value by a select -
+  // with a branch per slot the chains of a thread's slots ran one after the other, which
+  // was most of the panel's time.
+  auto step = [&](auto first_c, int j) {
+    constexpr int kFirst = decltype(first_c)::value;
     const double *cur = col[j & 1];
     double *nxt = col[(j + 1) & 1];
     double piv = cur[j];
-    if (!(piv > 0.0)) {
+    if (!(piv > 0.0)) {  // (the same in every thread)
       if (tid == 0) atomicOr(status, kErrNumeric);
       piv = 1.0;
     }
     if (tid == 0) pivot[j] = piv;
     const double inv = fast_rcp(piv);
+    double prod[kSlots];
 #pragma unroll
-    for (int q = 0; q < kSlots; ++q) {
-      if (last_col[q] <= j) continue;  // uniform: the whole slot is done
-      if (ek[q] > j) {
-        val[q] = fma(-(cur[ei[q]] * cur[ek[q]]), inv, val[q]);  // the product does not wait for the reciprocal
-        if (ek[q] == j + 1) nxt[ei[q]] = val[q];
-      }
+    for (int q = kFirst; q < kSlots; ++q) prod[q] = cur[ei[q]] * cur[max(ek[q], 0)];  // does not wait for the reciprocal
+#pragma unroll
+    for (int q = kFirst; q < kSlots; ++q) {
+      const double upd = fma(-prod[q], inv, val[q]);
+      val[q] = (ek[q] > j) ? upd : val[q];
+      if (ek[q] == j + 1) nxt[ei[q]] = val[q];
     }
     __syncthreads();
+  };
+  {
+    int j = 0;
+    auto run = [&](auto first_c) {  // the steps during which slot kFirst is the first live one
+      constexpr int kFirst = decltype(first_c)::value;
+      const int end = kFirst < kSlots ? min(last_col[kFirst < kSlots ? kFirst : 0], kT) : kT;
+      for (; j < end; ++j) step(first_c, j);
+    };
+    run(std::integral_constant<int, 0>{});
+    run(std::integral_constant<int, 1>{});
+    run(std::integral_constant<int, 2>{});
+    run(std::integral_constant<int, 3>{});
+    run(std::integral_constant<int, 4>{});
+    run(std::integral_constant<int, 5>{});
+    run(std::integral_constant<int, 6>{});
+    run(std::integral_constant<int, 7>{});
+    run(std::integral_constant<int, 8>{});
+    run(std::integral_constant<int, 9>{});  // the last columns: pivots only
   }
   // L[i][k] = value / sqrt(pivot_k), L[k][k] = sqrt(pivot_k); zero above the diagonal
 #pragma unroll
@@ -295,34 +320,45 @@ chol_panel_kernel(double *__restrict__ S, int rp, int p, double *__restrict__ X,
     }
   }
   __syncthreads();
-  // doubling: for every super-block [d, d + 2h): T = L21 X11, then X21 = -X22 T.  A dot product
-  // runs as four interleaved partial sums: a dependent chain of double-precision operations
-  // is what these few hundred threads wait on.
-  for (int h = 8, hs = 3; h < kT; h *= 2, ++hs) {
-    const int elems = (kT / (2 * h)) * h * h;
-    for (int e = tid; e < elems; e += 256) {
-      const int z = e >> (2 * hs), a = (e >> hs) & (h - 1), b = e & (h - 1), d = 2 * h * z;
-      const double *lrow = D + (d + h + a) * kTP + d, *xcol = Xs + d * kTP + d + b;
-      double s4[4] = {0.0, 0.0, 0.0, 0.0};
-      for (int k = 0; k < h; k += 4) {  // X11 is lower triangular: the terms with k < b are stored zeros
+  // doubling: for every super-block [d, d + 2h): T = L21 X11, then X21 = -X22 T.  A thread
+  // has h / 8 elements of each product; their dot products advance together, each as four
+  // interleaved partial sums: a dependent chain of double-precision operations is what
+  // these few hundred threads wait on, so the chains run side by side, not one after another.
+  auto level = [&](auto h_c) {
+    constexpr int h = decltype(h_c)::value, hs = (h == 8) ? 3 : (h == 16) ? 4 : 5;
+    constexpr int kE = h / 8;  // elements per thread: (kT / (2 h)) h h / 256
+    auto products = [&](const double *left, int left_col, const double *right, int right_row, double *out, double sign) {
+      // out[d + h + a][d + b] = sign * sum_k left[d + h + a][d + left_col + k] right[d + right_row + k][d + b]
+      const double *lp[kE], *rp_[kE];
+      double *op[kE];
+      double s4[kE][4];
 #pragma unroll
-        for (int u = 0; u < 4; ++u) s4[u] = fma(lrow[k + u], xcol[(k + u) * kTP], s4[u]);
-      }
-      As[(d + h + a) * kTP + d + b] = (s4[0] + s4[1]) + (s4[2] + s4[3]);
-    }
-    __syncthreads();
-    for (int e = tid; e < elems; e += 256) {
-      const int z = e >> (2 * hs), a = (e >> hs) & (h - 1), b = e & (h - 1), d = 2 * h * z;
-      const double *xrow = Xs + (d + h + a) * kTP + d + h, *tcol = As + (d + h) * kTP + d + b;
-      double s4[4] = {0.0, 0.0, 0.0, 0.0};
-      for (int k = 0; k < h; k += 4) {  // X22 is lower triangular: the terms with k > a are stored zeros
+      for (int i = 0; i < kE; ++i) {
+        const int e = tid + 256 * i;
+        const int z = e >> (2 * hs), a = (e >> hs) & (h - 1), b = e & (h - 1), d = 2 * h * z;
+        lp[i] = left + (d + h + a) * kTP + d + left_col;
+        rp_[i] = right + (d + right_row) * kTP + d + b;
+        op[i] = out + (d + h + a) * kTP + d + b;
 #pragma unroll
-        for (int u = 0; u < 4; ++u) s4[u] = fma(xrow[k + u], tcol[(k + u) * kTP], s4[u]);
+        for (int u = 0; u < 4; ++u) s4[i][u] = 0.0;
       }
-      Xs[(d + h + a) * kTP + d + b] = -((s4[0] + s4[1]) + (s4[2] + s4[3]));
-    }
+      for (int k = 0; k < h; k += 4) {  // (the triangular factors' stored zeros are multiplied through)
+#pragma unroll
+        for (int u = 0; u < 4; ++u)
+#pragma unroll
+          for (int i = 0; i < kE; ++i) s4[i][u] = fma(lp[i][k + u], rp_[i][(k + u) * kTP], s4[i][u]);
+      }
+#pragma unroll
+      for (int i = 0; i < kE; ++i) *op[i] = sign * ((s4[i][0] + s4[i][1]) + (s4[i][2] + s4[i][3]));
+    };
+    products(D, 0, Xs, 0, As, 1.0);    // T = L21 X11
     __syncthreads();
-  }
+    products(Xs, h, As, h, Xs, -1.0);  // X21 = -X22 T
+    __syncthreads();
+  };
+  level(std::integral_constant<int, 8>{});
+  level(std::integral_constant<int, 16>{});
+  level(std::integral_constant<int, 32>{});
   if (blockIdx.x == 0) {
   #pragma unroll
   for (int e = tid; e < kT * kT; e += 256) {
