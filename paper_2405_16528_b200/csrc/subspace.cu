@@ -395,13 +395,30 @@ chol_update_kernel(double *__restrict__ S, int rp, int p) {
   const int64_t i0 = static_cast<int64_t>(p + 1 + ti) * kT, j0 = static_cast<int64_t>(p + 1 + tj) * kT;
   const int64_t c0 = static_cast<int64_t>(p) * kT;
   const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
-  double acc[4][4] = {};
-  for (int half = 0; half < 2; ++half) {  // the panel's 64 columns, 32 at a time
+  // Everything the CTA reads from global memory is asked for at once - both halves of the two
+  // panel blocks (the panel's 64 columns go through shared memory 32 at a time) and the tile
+  // of S itself - so that one memory latency is waited for, not three.
+  double ra[2][8], rb[2][8], cur[4][4];
 #pragma unroll
-    for (int e = tid; e < kT * 32; e += 256) {
-      const int a = e >> 5, c = e & 31;
-      As[c * kTP + a] = S[(i0 + a) * rp + c0 + half * 32 + c];
-      Bs[c * kTP + a] = S[(j0 + a) * rp + c0 + half * 32 + c];
+  for (int half = 0; half < 2; ++half)
+#pragma unroll
+    for (int q = 0; q < 8; ++q) {
+      const int e = tid + 256 * q, a = e >> 5, c = e & 31;
+      ra[half][q] = S[(i0 + a) * rp + c0 + half * 32 + c];
+      rb[half][q] = S[(j0 + a) * rp + c0 + half * 32 + c];
+    }
+#pragma unroll
+  for (int i = 0; i < 4; ++i)
+#pragma unroll
+    for (int j = 0; j < 4; ++j) cur[i][j] = S[(i0 + ty + 16 * i) * rp + j0 + tx + 16 * j];
+  double acc[4][4] = {};
+#pragma unroll
+  for (int half = 0; half < 2; ++half) {
+#pragma unroll
+    for (int q = 0; q < 8; ++q) {
+      const int e = tid + 256 * q, a = e >> 5, c = e & 31;
+      As[c * kTP + a] = ra[half][q];
+      Bs[c * kTP + a] = rb[half][q];
     }
     __syncthreads();
     tile_fma(acc, As, Bs, ty, tx, 32);
@@ -410,7 +427,7 @@ chol_update_kernel(double *__restrict__ S, int rp, int p) {
 #pragma unroll
   for (int i = 0; i < 4; ++i)
 #pragma unroll
-    for (int j = 0; j < 4; ++j) S[(i0 + ty + 16 * i) * rp + j0 + tx + 16 * j] -= acc[i][j];
+    for (int j = 0; j < 4; ++j) S[(i0 + ty + 16 * i) * rp + j0 + tx + 16 * j] = cur[i][j] - acc[i][j];
 }
 
 // One product of the inversion by doubling, for every diagonal super-block of
@@ -433,20 +450,38 @@ block_gemm_kernel(const double *__restrict__ L, double *__restrict__ X, double *
   const int64_t m1_row0 = d0 + h + ti, m1_col0 = second ? d0 + h : d0;
   const int64_t m2_row0 = second ? d0 + h : d0, m2_col0 = d0 + tj;
   double acc[4][4] = {};
-  for (int k0 = 0; k0 < h; k0 += 32) {
+  // X is lower triangular: in the first product the rows of A above the column tile are zero,
+  // in the second the columns of B right of the row tile are - those k are passed over (the
+  // sums lose terms that are exactly zero).  The next 32 columns are on their way from global
+  // memory into registers while the current ones are multiplied.
+  const int k_lo = second ? 0 : tj, k_hi = second ? min(h, ti + kT) : h;
+  double ra[8], rb[8];
+  auto fetch = [&](int k0) {
 #pragma unroll
-    for (int e = tid; e < kT * 32; e += 256) {
-      const int a = e >> 5, c = e & 31;  // As[c][a] = M1[row a][k0 + c]
-      const int64_t row = m1_row0 + a, col = m1_col0 + k0 + c;
-      As[c * kTP + a] = (row < rp && col < rp) ? M1[row * rp + col] : 0.0;
+    for (int q = 0; q < 8; ++q) {
+      const int e = tid + 256 * q;
+      {
+        const int a = e >> 5, c = e & 31;  // As[c][a] = M1[row a][k0 + c]
+        const int64_t row = m1_row0 + a, col = m1_col0 + k0 + c;
+        ra[q] = (row < rp && col < rp) ? M1[row * rp + col] : 0.0;
+      }
+      {
+        const int c = e >> 6, b = e & 63;  // Bs[c][b] = M2[k0 + c][column b]
+        const int64_t row = m2_row0 + k0 + c, col = m2_col0 + b;
+        rb[q] = (row < rp && col < rp) ? M2[row * rp + col] : 0.0;
+      }
     }
+  };
+  fetch(k_lo);
+  for (int k0 = k_lo; k0 < k_hi; k0 += 32) {
 #pragma unroll
-    for (int e = tid; e < kT * 32; e += 256) {
-      const int c = e >> 6, b = e & 63;  // Bs[c][b] = M2[k0 + c][column b]
-      const int64_t row = m2_row0 + k0 + c, col = m2_col0 + b;
-      Bs[c * kTP + b] = (row < rp && col < rp) ? M2[row * rp + col] : 0.0;
+    for (int q = 0; q < 8; ++q) {
+      const int e = tid + 256 * q;
+      As[(e & 31) * kTP + (e >> 5)] = ra[q];
+      Bs[(e >> 6) * kTP + (e & 63)] = rb[q];
     }
     __syncthreads();
+    if (k0 + 32 < k_hi) fetch(k0 + 32);
     tile_fma(acc, As, Bs, ty, tx, 32);
     __syncthreads();
   }
