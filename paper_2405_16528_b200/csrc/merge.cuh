@@ -352,6 +352,7 @@ loqt_merge_kernel(const __grid_constant__ MergeBatch mb) {
         // may be contracted into one fused operation)
 #pragma unroll
         for (int h = 0; h < 2; ++h) {
+          __syncwarp();  // the lanes' paths below differ (live rows, kind of division): whole again for the TMEM load
           ptx::tmem_ld32(t_row + jb * 64 + 32 * h, d);
           ptx::tmem_ld_wait();
           if (live) {

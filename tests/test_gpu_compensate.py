@@ -108,6 +108,25 @@ def test_representable_weights_need_no_correction():
     assert np.array_equal(c, q0[0]) and np.array_equal(m, q0[1]) and not f32(B).any()
 
 
+def test_rows_of_very_different_scale_share_a_warp():
+    # Block scales beyond 2^+-60 take the IEEE division, the others the division by
+    # reciprocal, and all-zero rows neither: here the three kinds sit in neighbouring rows,
+    # so the lanes of one epilogue warp part ways inside a block.  The weights are
+    # representable (scaling a row by a power of two keeps them so), which makes the
+    # expected result exact: the codes and scales of q(W), B = 0.
+    out, inn, r = 256, 320, 32
+    W, P, Wd, Pd = _inputs(47, out, inn, r)
+    q0 = O.nf4_quantize(W)
+    k = np.array([0, 70, -70, 0, 65, -65, 0, 0])[np.arange(out) % 8]
+    Wr = (O.nf4_dequantize(q0[0], q0[1], inn) * (2.0 ** k)[:, None]).astype(np.float32)
+    Wr[np.arange(out) % 16 == 5] = 0.0
+    ref_c, ref_m = O.nf4_quantize(Wr)
+    Wd.copy_(torch.from_numpy(Wr))
+    Wq, Pq, B = L.loqt_compensated_init(Wd, Pd, 3)
+    c, m = from_dev_nf4(Wq)
+    assert np.array_equal(c, ref_c) and np.array_equal(m, ref_m) and not f32(B).any()
+
+
 def test_argument_errors():
     out, inn, r = 256, 256, 32
     W, P, Wd, Pd = _inputs(43, out, inn, r)

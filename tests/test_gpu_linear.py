@@ -140,6 +140,24 @@ def test_merge_zero_B_leaves_weights_untouched():
     assert torch.equal(before.codes, d["Wq"].codes) and torch.equal(before.absmax, d["Wq"].absmax)
 
 
+def test_merge_zero_B_with_rows_of_very_different_scale():
+    # Scales beyond 2^+-60 take the IEEE division in the requantising epilogue, the others the
+    # division by reciprocal, all-zero blocks neither; with the three kinds in neighbouring
+    # rows the lanes of one epilogue warp part ways inside a block.  A merge with B = 0 must
+    # still hand back every code and scale as it found them.
+    out, inn, r = 256, 320, 32
+    h, d = _setup(14, out, inn, r, 8)
+    Wq = d["Wq"]
+    k = torch.tensor([0, 70, -70, 0, 65, -65, 0, 0], dtype=torch.float32, device="cuda")[torch.arange(out, device="cuda") % 8]
+    Wq.absmax.mul_(torch.exp2(k)[:, None])
+    zero = torch.arange(out, device="cuda") % 16 == 5
+    Wq.absmax[zero] = 0.0
+    Wq.codes[zero] = 0x77
+    before = Wq.clone()
+    L.loqt_merge_requant(Wq, d["Pq"], torch.zeros_like(d["B"]), 1.0)
+    assert torch.equal(before.codes, Wq.codes) and torch.equal(before.absmax, Wq.absmax)
+
+
 def test_merge_many_matches_single():
     # 18 matrices of mixed shapes (ragged and not, several ranks) through one call: the batched launch walks
     # the tiles of all of them as one sequence and must leave every matrix exactly as a merge of its own does;
